@@ -1,0 +1,557 @@
+#!/usr/bin/env python
+"""Benchmark of the SBP boxing sweep (and, at one GPU, of the sharded operators).
+
+    python bench.py --gpus N --steps K --warmup W [--impl reference]
+
+One step = the seven boxing transforms of the bandwidth-sweep workload (logical bf16
+[8192, 8192], k = 4): P(sum)->B, P(sum)->S(0), P(sum)->S(1), S(0)->B, S(0)->S(1), S(1)->S(0),
+B->S(1), each reading every input local tensor once and writing every output local tensor
+once.  value = algorithmic bytes of a step / device time of a step.  With N > 1 every rank
+runs its own replica of the sweep (no collective on the data path; weak scaling).
+
+Prints one JSON line (rank 0).  --impl reference times the CPU oracle instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import sbp_datagen as dg  # noqa: E402
+
+METRIC = "boxing/embedding/softmax HBM GB/s and sharded MatMul TFLOP/s vs B200 peak"
+SWEEP_SHAPE = (8192, 8192)
+SWEEP_K = 4
+SEED = 1002
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+NOMINAL_HBM_GBS = 8000.0
+NOMINAL_BF16_TFLOPS = 2250.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS,
+            "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------ clocks
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while a timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.lines = []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._pump, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            parts = [p.strip() for p in ln.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------ workload
+
+TRANSFORMS = [
+    # name, source kind, destination signature, algorithmic bytes in units of |T|
+    ("P(sum)->B", "P", "B", 8),
+    ("P(sum)->S(0)", "P", "S0", 5),
+    ("P(sum)->S(1)", "P", "S1", 5),
+    ("S(0)->B", "S0", "B", 5),
+    ("S(0)->S(1)", "S0", "S1", 2),
+    ("S(1)->S(0)", "S1", "S0", 2),
+    ("B->S(1)", "B", "S1", 2),
+]
+
+
+def t_bytes():
+    return SWEEP_SHAPE[0] * SWEEP_SHAPE[1] * 2
+
+
+def step_bytes():
+    return sum(t[3] for t in TRANSFORMS) * t_bytes()
+
+
+def build_sweep(sbp, device):
+    """Device-resident sources and destinations of the seven transforms."""
+    k, shape, bf16 = SWEEP_K, SWEEP_SHAPE, torch.bfloat16
+    sig = {"P": sbp.P_SUM, "B": sbp.B, "S0": sbp.S(0), "S1": sbp.S(1)}
+    T = dg.normal(SEED, 0, shape, 0.0, 1.0, bf16, device)
+    n0, n1 = shape
+    src = {
+        "P": sbp.SbpTensor(shape, bf16, sbp.P_SUM, [dg.normal(SEED, 10 + r, shape, 0.0, 1.0, bf16, device) for r in range(k)]),
+        "S0": sbp.SbpTensor(shape, bf16, sbp.S(0), [T[r * n0 // k:(r + 1) * n0 // k].contiguous() for r in range(k)]),
+        "S1": sbp.SbpTensor(shape, bf16, sbp.S(1), [T[:, r * n1 // k:(r + 1) * n1 // k].contiguous() for r in range(k)]),
+        "B": sbp.SbpTensor(shape, bf16, sbp.B, [T.clone() for _ in range(k)]),
+    }
+    work = []
+    for name, s, d, units in TRANSFORMS:
+        dst = sbp.empty_global(shape, bf16, sig[d], k, device=device)
+        work.append((name, src[s], dst, units * t_bytes()))
+    return T, src, work
+
+
+def run_sweep(sbp, work, events=None):
+    for i, (_, s, d, _) in enumerate(work):
+        if events is not None:
+            events[i][0].record()
+        sbp.sbp_boxing(s, d)
+        if events is not None:
+            events[i][1].record()
+
+
+
+# ------------------------------------------------------------------------------ ncu traffic
+
+# DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/.
+# None = not captured for the kernel as it stands.
+NCU_TRAFFIC = {}
+
+
+def ncu_traffic(name):
+    return NCU_TRAFFIC.get(name)
+
+
+# ------------------------------------------------------------------------------ end to end
+
+def e2e_sweep(sbp, src, work, device, steps, dist):
+    """The sweep through sbp_boxing_host: pinned host buffers in, pinned host buffers out,
+    host->device and device->host copies inside the timed region."""
+    host_src = {}
+    for key, g in src.items():
+        host_src[key] = sbp.SbpTensor(g.shape, g.dtype, g.sig, [t.cpu().pin_memory() for t in g.locals])
+    host_dst = {}
+    jobs = []
+    h2d = d2h = 0
+    ws_bytes = 0
+    key_of = {id(g): key for key, g in src.items()}
+    for name, s, d, _ in work:
+        hs = host_src[key_of[id(s)]]
+        dk = repr(d.sig)
+        if dk not in host_dst:
+            host_dst[dk] = sbp.SbpTensor(d.shape, d.dtype, d.sig,
+                                         [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in d.locals])
+        hd = host_dst[dk]
+        jobs.append((hs, hd))
+        h2d += sum(t.numel() * t.element_size() for t in hs.locals)
+        d2h += sum(t.numel() * t.element_size() for t in hd.locals)
+        ws_bytes = max(ws_bytes, sbp.sbp_boxing_host_workspace_bytes(hs, hd))
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device=device)
+
+    def one_step():
+        for hs, hd in jobs:
+            sbp.sbp_boxing_host(hs, hd, ws)
+
+    one_step()
+    torch.cuda.synchronize()
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0 = time.perf_counter()
+    start.record()
+    for _ in range(steps):
+        one_step()
+    end.record()
+    torch.cuda.synchronize()
+    wall = time.perf_counter() - t0
+    if dist is not None:
+        dist.barrier()
+    ms = max(start.elapsed_time(end), wall * 1e3)
+    if dist is not None:
+        t = torch.tensor([ms], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    ms /= steps
+    # spot check: the last transform's result on the host equals the device-resident run
+    ref = work[-1][2].locals[0].cpu()
+    if not torch.equal(ref, jobs[-1][1].locals[0]):
+        raise RuntimeError("end-to-end result differs from the device-resident result")
+    return {"value": step_bytes() / (ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms, "steps": steps,
+            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+
+# ------------------------------------------------------------------------------ operator sections
+
+_FLUSH = None
+
+
+def _flush_l2(device):
+    global _FLUSH
+    if _FLUSH is None:
+        _FLUSH = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    _FLUSH.fill_(1)
+
+
+def time_op(fn, device, iters=10, warmup=3):
+    """Average and best device time (ms) of fn(), L2 flushed between iterations."""
+    for _ in range(warmup):
+        fn()
+    torch.cuda.synchronize()
+    ms = []
+    for _ in range(iters):
+        _flush_l2(device)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        torch.cuda.synchronize()
+        ms.append(a.elapsed_time(b))
+    return sum(ms) / len(ms), min(ms)
+
+
+def _hbm_entry(name, nbytes, avg, best, peaks, extra=None):
+    gbs = nbytes / (avg * 1e-3) / 1e9
+    e = {"op": name, "bound": "hbm", "bytes": nbytes, "ms": avg, "best_ms": best, "achieved": gbs, "unit": "GB/s",
+         "peak": peaks["hbm_gbs"], "frac_measured": gbs / peaks["hbm_gbs"], "frac_nominal": gbs / NOMINAL_HBM_GBS,
+         "traffic": ncu_traffic(name)}
+    if extra:
+        e.update(extra)
+    return e
+
+
+def _tensor_entry(name, flops, avg, best, peaks, extra=None):
+    tf = flops / (avg * 1e-3) / 1e12
+    e = {"op": name, "bound": "tensor", "flops": flops, "ms": avg, "best_ms": best, "achieved": tf, "unit": "TFLOP/s",
+         "peak": peaks["bf16_tflops"], "frac_measured": tf / peaks["bf16_tflops"],
+         "frac_sustained": tf / peaks["bf16_tflops_sustained"], "frac_nominal": tf / NOMINAL_BF16_TFLOPS}
+    if extra:
+        e.update(extra)
+    return e
+
+
+def section_embedding(sbp, device, peaks):
+    """Row-split embedding: fp32 table [2^24, 128] S(0) over k = 8, ids int64 [65536, 26] Zipf(1.05)."""
+    k, rows, dim = 8, 1 << 24, 128
+    ids = dg.zipf_ids(1005, 1, (65536, 26), rows, 1.05, device)
+    table = sbp.SbpTensor((rows, dim), torch.float32, sbp.S(0),
+                          [dg.uniform(1005, 100 + r, (rows // k, dim), -0.05, 0.05, torch.float32, device) for r in range(k)])
+    idt = sbp.SbpTensor((65536, 26), torch.int64, sbp.B, [ids] * k)
+    out_b = sbp.empty_global((65536, 26, dim), torch.float32, sbp.B, k, device=device)
+    out_1 = sbp.empty_global((65536, 26, dim), torch.float32, sbp.B, k, device=device, alias_replicas=True)
+    n = 65536 * 26
+    row_b = dim * 4
+    unique = int(torch.unique(ids).numel())
+    res = []
+    avg, best = time_op(lambda: sbp.sbp_embedding(table, idt, out_b), device)
+    res.append(_hbm_entry("embedding fused gather -> B (8 replicas written)", n * 8 + n * row_b + k * n * row_b, avg, best, peaks,
+                          {"unique_rows": unique, "lookups": n}))
+    avg, best = time_op(lambda: sbp.sbp_embedding(table, idt, out_1), device)
+    res.append(_hbm_entry("embedding fused gather -> B (replicas aliased, 1 write)", n * 8 + 2 * n * row_b, avg, best, peaks,
+                          {"unique_rows": unique, "lookups": n}))
+    del out_1
+    out_p = sbp.empty_global((65536, 26, dim), torch.float32, sbp.P_SUM, k, device=device)
+
+    def unfused():
+        sbp.sbp_embedding(table, idt, out_p)
+        sbp.sbp_boxing(out_p, out_b)
+    avg, best = time_op(unfused, device, iters=5)
+    res.append(_hbm_entry("embedding unfused: gather -> P(sum), then P(sum) -> B", k * n * 8 + n * row_b + 3 * k * n * row_b,
+                          avg, best, peaks))
+    return res
+
+
+def section_softmax(sbp, device, peaks):
+    """Class-split softmax cross entropy on materialised bf16 logits [512, 2^20], S(1) over k = 8."""
+    k, rows, classes = 8, 512, 1 << 20
+    sigma = (512 ** 0.5) * 0.01
+    logits = sbp.SbpTensor((rows, classes), torch.bfloat16, sbp.S(1),
+                           [dg.normal(1004, 10 + r, (rows, classes // k), 0.0, sigma, torch.bfloat16, device) for r in range(k)])
+    labels = dg.integers(1004, 1, (rows,), 0, classes, device)
+    lab = sbp.SbpTensor((rows,), torch.int64, sbp.B, [labels] * k)
+    loss = sbp.empty_global((rows,), torch.float32, sbp.B, k, device=device)
+    ws = torch.empty(sbp.sbp_softmax_xent_workspace_bytes(logits), dtype=torch.uint8, device=device)
+    avg, best = time_op(lambda: sbp.sbp_softmax_xent(logits, lab, loss, None, None, ws), device)
+    return [_hbm_entry("softmax-xent on bf16 logits (partial + combine)", rows * classes * 2 + rows * 8, avg, best, peaks,
+                       {"loss_mean": float(loss.locals[0].mean().item())})]
+
+
+def section_mlp(sbp, device, peaks):
+    """Megatron-style MLP: X[8192,4096] B, W1[4096,16384] S(1), GeLU, W2[16384,4096] S(0), k = 8."""
+    k, M, H, F = 8, 8192, 4096, 16384
+    bf16 = torch.bfloat16
+    X = dg.normal(1003, 0, (M, H), 0.0, 1.0, bf16, device)
+    x = sbp.SbpTensor((M, H), bf16, sbp.B, [X] * k)
+    w1 = sbp.SbpTensor((H, F), bf16, sbp.S(1), [dg.normal(1003, 10 + r, (H, F // k), 0.0, 0.02, bf16, device) for r in range(k)])
+    w2 = sbp.SbpTensor((F, H), bf16, sbp.S(0), [dg.normal(1003, 30 + r, (F // k, H), 0.0, 0.02, bf16, device) for r in range(k)])
+    h = sbp.empty_global((M, F), bf16, sbp.S(1), k, device=device)
+    y_p = sbp.empty_global((M, H), bf16, sbp.P_SUM, k, device=device)
+    y_b = sbp.empty_global((M, H), bf16, sbp.B, k, device=device)
+    ws = torch.empty(max(1, sbp.sbp_matmul_workspace_bytes(h, w2, y_b), sbp.sbp_matmul_workspace_bytes(x, w1, h)),
+                     dtype=torch.uint8, device=device)
+    flops = 2.0 * M * H * F
+    res = []
+    avg, best = time_op(lambda: sbp.sbp_matmul(x, w1, h, sbp.SBP_EPILOGUE_GELU, ws), device, iters=5)
+    res.append(_tensor_entry("MLP GEMM1 (B,S(1))->S(1) + GeLU", flops, avg, best, peaks))
+    avg, best = time_op(lambda: sbp.sbp_matmul(h, w2, y_p, 0, ws), device, iters=5)
+    res.append(_tensor_entry("MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials", flops, avg, best, peaks))
+    avg, best = time_op(lambda: sbp.sbp_boxing(y_p, y_b), device)
+    res.append(_hbm_entry("MLP P(sum)->B of the bf16 partials", 2 * k * M * H * 2, avg, best, peaks))
+    avg, best = time_op(lambda: sbp.sbp_matmul(h, w2, y_b, 0, ws), device, iters=5)
+    res.append(_tensor_entry("MLP GEMM2 fused (S(1),S(0))->B", flops, avg, best, peaks))
+    return res
+
+
+def section_classifier_gemm(sbp, device, peaks):
+    """Classifier logits: F[512,512] B x W[512, 2^20] S(1) over k = 8 -> bf16 logits S(1)."""
+    k, rows, feat, classes = 8, 512, 512, 1 << 20
+    bf16 = torch.bfloat16
+    Fm = dg.normal(1004, 0, (rows, feat), 0.0, 1.0, bf16, device)
+    f = sbp.SbpTensor((rows, feat), bf16, sbp.B, [Fm] * k)
+    w = sbp.SbpTensor((feat, classes), bf16, sbp.S(1),
+                      [dg.normal(1004, 40 + r, (feat, classes // k), 0.0, 0.01, bf16, device) for r in range(k)])
+    z = sbp.empty_global((rows, classes), bf16, sbp.S(1), k, device=device)
+    ws = torch.empty(max(1, sbp.sbp_matmul_workspace_bytes(f, w, z)), dtype=torch.uint8, device=device)
+    avg, best = time_op(lambda: sbp.sbp_matmul(f, w, z, 0, ws), device, iters=5)
+    e = _tensor_entry("classifier GEMM (B,S(1))->S(1), bf16 logits", 2.0 * rows * feat * classes, avg, best, peaks)
+    nbytes = feat * classes * 2 + rows * classes * 2 + rows * feat * 2
+    e["hbm_gbs"] = nbytes / (avg * 1e-3) / 1e9
+    e["hbm_frac_measured"] = e["hbm_gbs"] / peaks["hbm_gbs"]
+    return [e]
+
+
+def run_operator_sections(sbp, device, peaks):
+    out = []
+    for fn in (section_softmax, section_classifier_gemm, section_mlp, section_embedding):
+        try:
+            out.extend(fn(sbp, device, peaks))
+        except sbp.SbpError as e:            # an operator this build cannot run is reported, not hidden
+            out.append({"op": fn.__name__, "error": str(e)})
+        torch.cuda.empty_cache()
+    return out
+
+
+# ------------------------------------------------------------------------------ CPU baseline (oracle)
+
+def oracle_sweep_sample(rows: int):
+    """Times the CPU oracle, as it stands, on the first `rows` rows of the sweep workload.
+    Returns (bytes processed, seconds, threads used)."""
+    import numpy as np
+    from oracle import sbp_oracle as O
+    k = SWEEP_K
+    shape = (rows, SWEEP_SHAPE[1])
+    T = dg.normal(SEED, 0, shape, 0.0, 1.0, torch.bfloat16).float().numpy()
+    P = [dg.normal(SEED, 10 + r, shape, 0.0, 1.0, torch.bfloat16).float().numpy() for r in range(k)]
+    srcs = {"P": (P, O.PSUM), "S0": (O.to_locals(T, O.S0, k), O.S0), "S1": (O.to_locals(T, O.S1, k), O.S1),
+            "B": (O.to_locals(T, O.B, k), O.B)}
+    dsts = {"B": O.B, "S0": O.S0, "S1": O.S1}
+    nbytes = 0
+    t0 = time.perf_counter()
+    for _, s, d, units in TRANSFORMS:
+        loc, sg = srcs[s]
+        out = O.boxing(loc, sg, dsts[d], "bf16")
+        assert len(out) == k
+        nbytes += units * rows * SWEEP_SHAPE[1] * 2
+    return nbytes, time.perf_counter() - t0, 1
+
+
+# ------------------------------------------------------------------------------ main
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-ops", action="store_true", help="skip the sharded-operator sections (N = 1 only)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--copy-engine", type=int, default=0)
+    return ap.parse_args()
+
+
+def reference_arm(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    rows = 256
+    for _ in range(max(args.warmup, 0)):
+        oracle_sweep_sample(64)
+    total_b, total_s = 0, 0.0
+    for _ in range(args.steps):
+        b, s, cores = oracle_sweep_sample(rows)
+        total_b += b
+        total_s += s
+    value = total_b / total_s / 1e9
+    sample = f"first {rows} of {SWEEP_SHAPE[0]} rows of every local tensor, all 7 transforms, per step"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_s / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "boxing sweep bf16 [8192,8192] k=4, 7 transforms (CPU oracle on a row sample)"},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(line))
+    return 0
+
+
+def main():
+    args = parse()
+    if args.impl == "reference":
+        return reference_arm(args)
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the library has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=device)
+
+    import paper_2110_15032_b200 as sbp
+    sbp.load_library()
+    sbp.sbp_boxing_set_copy_engine(args.copy_engine)
+    peaks = measured_peaks()
+
+    T, src, work = build_sweep(sbp, device)
+    for _ in range(max(args.warmup, 3)):
+        run_sweep(sbp, work)
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    events = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in work]
+              for _ in range(args.steps)]
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    barrier()
+    launches0 = sbp.sbp_launch_count()
+    start, end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    start.record()
+    for s in range(args.steps):
+        run_sweep(sbp, work, events[s])
+    end.record()
+    barrier()
+    launches = sbp.sbp_launch_count() - launches0
+    clocks = sampler.stop() if rank == 0 else None
+    sbp.sbp_check_device_errors()
+    ms_total = start.elapsed_time(end)
+    if dist is not None:
+        t = torch.tensor([ms_total], device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    ms_step = ms_total / args.steps
+    value = world * step_bytes() / (ms_step * 1e-3) / 1e9
+
+    per = []
+    for i, (name, _, _, nbytes) in enumerate(work):
+        ms = [events[s][i][0].elapsed_time(events[s][i][1]) for s in range(args.steps)]
+        avg = sum(ms) / len(ms)
+        per.append({"transform": name, "bytes": nbytes, "ms": avg, "best_ms": min(ms),
+                    "gbs": nbytes / (avg * 1e-3) / 1e9,
+                    "frac_measured": nbytes / (avg * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                    "frac_nominal": nbytes / (avg * 1e-3) / 1e9 / NOMINAL_HBM_GBS})
+    dom = max(per, key=lambda p: p["ms"])
+    roofline = {"bound": "hbm", "kernel": "box_tile_kernel (" + dom["transform"] + ")",
+                "achieved": dom["gbs"], "peak": peaks["hbm_gbs"], "peak_source": peaks["source"],
+                "unit": "GB/s", "frac": dom["gbs"] / peaks["hbm_gbs"], "traffic": ncu_traffic(dom["transform"])}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": "boxing sweep: logical bf16 [8192,8192] N(0,1), k=4, 7 transforms per step",
+                   "parallelism": f"replicas x{world}" if world > 1 else "1 GPU, k=4 logical shards",
+                   "l2": "inputs larger than L2: a step streams 3.4 GB through distinct buffers between repeats",
+                   "copy_engine": args.copy_engine},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "transforms": per,
+    }
+
+    if rank == 0:
+        line["clocks"] = clocks
+
+    # end-to-end: the same sweep through the host-buffer entry point, copies inside the region
+    e2e = e2e_sweep(sbp, src, work, device, args.e2e_steps, dist)
+    e2e["value"] *= world
+    line["e2e"] = e2e
+
+    if rank == 0 and world == 1:
+        if not args.no_cpu_baseline:
+            rows = 1024
+            nbytes, secs, cores = oracle_sweep_sample(rows)
+            line["cpu_baseline"] = {"value": nbytes / secs / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
+                                    "sample": f"first {rows} of {SWEEP_SHAPE[0]} rows of every local tensor, "
+                                              f"all 7 transforms once ({secs:.1f} s)"}
+        if not args.no_ops:
+            del T, src, work
+            torch.cuda.empty_cache()
+            line["ops"] = run_operator_sections(sbp, device, peaks)
+    if rank == 0:
+        print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -1,0 +1,219 @@
+/*
+ * sbp.h -- C ABI of the B200 (sm_100a) SBP library.
+ *
+ * SBP is the paper's abstraction (Section 3.1) for how a *global* (logical) tensor maps
+ * onto the *local* tensors of the k devices of a placement:
+ *     S(i)   split along axis i in a balanced manner,
+ *     B      broadcast: every local tensor is an exact copy of the global tensor,
+ *     P(op)  partial-value: every local tensor has the global shape and the global tensor
+ *            is the element-wise reduction (sum or max) over the local tensors.
+ * In this library the k "devices" of a placement are k logical shards that all live in
+ * ONE GPU's memory; there is no inter-GPU traffic.
+ *
+ * General conventions (hold for every entry point unless it says otherwise)
+ *   - All pointers inside an sbp_tensor are DEVICE pointers owned by the caller.  Every
+ *     local tensor is dense row-major with the local shape given by sbp_local_shape().
+ *   - The library allocates no device memory and frees none.  Scratch memory, where an
+ *     operation needs it, is passed in by the caller ("ws", "ws_bytes"); its required
+ *     size comes from the matching *_workspace_bytes() query.
+ *   - Work is enqueued on `cuda_stream` (a cudaStream_t passed as void*; NULL = the
+ *     legacy default stream) and the call returns without waiting for it.
+ *   - All argument checking happens on the host before anything is launched; when a
+ *     call returns anything other than SBP_OK nothing has been written.
+ *   - Source and destination buffers must not overlap.
+ *   - Balanced split of an axis of length n over k shards: shard r holds
+ *     ceil(n/k) elements if r < n mod k, else floor(n/k), contiguous, in rank order.
+ *   - 16-byte aligned pointers and row segments take the 128-bit vector path; anything
+ *     else takes an element-wise path with identical results.
+ *   - sbp_last_error() returns a thread-local, human readable detail for the last
+ *     non-OK status returned on the calling thread.
+ */
+#ifndef SBP_H_
+#define SBP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SBP_OK = 0,
+  SBP_ERR_INVALID_ARG = 1, /* null pointer, bad rank, k out of range, ...                */
+  SBP_ERR_SHAPE = 2,       /* logical shapes of the operands do not fit together         */
+  SBP_ERR_DTYPE = 3,       /* dtype not supported by this operation                      */
+  SBP_ERR_SIGNATURE = 4,   /* SBP signatures are not a valid combination                 */
+  SBP_ERR_UNSUPPORTED = 5, /* valid request that this build does not implement           */
+  SBP_ERR_ALIGNMENT = 6,   /* a pointer is not aligned to its element size               */
+  SBP_ERR_WORKSPACE = 7,   /* workspace missing or too small                             */
+  SBP_ERR_CUDA = 8,        /* a CUDA runtime / driver call failed (no device, launch...) */
+  SBP_ERR_TIMEOUT = 9      /* a bounded device-side wait expired                         */
+} sbp_status;
+
+typedef enum { SBP_F32 = 0, SBP_BF16 = 1, SBP_I64 = 2 } sbp_dtype;
+
+typedef enum {
+  SBP_SPLIT = 0,
+  SBP_BROADCAST = 1,
+  SBP_PARTIAL_SUM = 2,
+  SBP_PARTIAL_MAX = 3
+} sbp_kind;
+
+/* One SBP signature.  `axis` is read only when kind == SBP_SPLIT. */
+typedef struct {
+  int32_t kind; /* sbp_kind */
+  int32_t axis;
+} sbp_sig;
+
+#define SBP_MAX_DIMS 4
+#define SBP_MAX_K 16
+#define SBP_MAX_PDIMS 2
+
+/*
+ * A global tensor together with its placement, signature and local tensors
+ * (Section 3: "a global tensor is mapped to multiple local tensors"; Section 3.4: a
+ * tensor carries a placement and an sbp attribute).  Plain data; the caller owns it.
+ *
+ *   shape[0..ndim)   LOGICAL (global) shape, 1 <= ndim <= SBP_MAX_DIMS.
+ *   pdims, pshape    placement hierarchy; k = product of pshape[0..pdims).  The paper's
+ *                    multi-dimensional SBP (Section 3.3) needs pdims == 2; this build
+ *                    implements pdims == 1 and answers SBP_ERR_UNSUPPORTED otherwise.
+ *   sbp[p]           one signature per placement axis.
+ *   local[r]         device pointer of shard r's local tensor, r in [0, k).  For a B
+ *                    tensor the k replicas may all be the same pointer; a kernel then
+ *                    writes that buffer once.
+ */
+typedef struct {
+  int32_t ndim;
+  int32_t dtype; /* sbp_dtype */
+  int64_t shape[SBP_MAX_DIMS];
+  int32_t pdims;
+  int32_t pshape[SBP_MAX_PDIMS];
+  sbp_sig sbp[SBP_MAX_PDIMS];
+  void* local[SBP_MAX_K];
+} sbp_tensor;
+
+/* ---------------------------------------------------------------- descriptors, rules */
+
+const char* sbp_status_string(sbp_status s);
+const char* sbp_last_error(void);
+
+/* Number of kernels this library has launched from the calling process so far (all
+ * threads).  Lets a harness count launches inside a timed region. */
+uint64_t sbp_launch_count(void);
+
+/* Local shape of shard r under t's signature (Section 3.1).  Host only, no CUDA. */
+sbp_status sbp_local_shape(const sbp_tensor* t, int32_t r, int64_t out_shape[SBP_MAX_DIMS]);
+
+/* Table 1 ("Valid SBP signatures for MatMul"): signature of Y = XW from those of X and
+ * W, or SBP_ERR_SIGNATURE when the pair is not one of the table's six rows. */
+sbp_status sbp_matmul_infer(sbp_sig x, sbp_sig w, sbp_sig* y);
+
+/* ---------------------------------------------------------------- boxing (Section 3.2)
+ *
+ * A boxing op re-arranges or transforms the local tensors of a global tensor so that
+ * the same global tensor is seen under another signature (Section 3.2; Table 2, column
+ * "same" placement).  src and dst must agree in logical shape, dtype and k.
+ *
+ *   src            dst        the collective it stands for (Table 2)
+ *   P(sum)         B          all-reduce       out_j[e] = round(sum_r in_r[e])
+ *   P(sum)         S(i)       reduce-scatter   out_r    = slice_r,i(sum_r' in_r')
+ *   P(max)         B / S(i)   same with max; exact
+ *   S(i)           B          all-gather       out_j    = concat_i(in_0 .. in_{k-1})
+ *   S(i)           S(j)       all2all (i!=j);  plain copy when i == j
+ *   B              S(i)       local slice of the shard's own replica
+ *   B              B          copy of the shard's own replica
+ *   P(op)          P(op)      copy
+ * Anything else (S->P, B->P, P(sum)<->P(max)) returns SBP_ERR_UNSUPPORTED.
+ *
+ * P(sum) arithmetic: an fp32 accumulator starts as shard 0, shards 1..k-1 are added in
+ * rank order with plain IEEE adds, and the result is rounded once (nearest even) to the
+ * storage dtype.  P(max): acc = shard 0; shard r replaces acc only when strictly greater.
+ * Reductions accept SBP_F32 and SBP_BF16; pure data movement accepts every dtype.
+ */
+sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream);
+
+/* Same transform, but every local[] pointer of src_host and dst_host is a HOST pointer
+ * (pinned memory recommended).  The source local tensors are copied to the device
+ * workspace, transformed there and the destination local tensors copied back, all
+ * enqueued on cuda_stream.  dev_ws must hold sbp_boxing_host_workspace_bytes() bytes. */
+size_t sbp_boxing_host_workspace_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_host);
+sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, void* dev_ws,
+                           size_t dev_ws_bytes, void* cuda_stream);
+
+/* Kernels of this library bound every device-side wait.  When one expires the kernel sets a
+ * device flag and returns; this call (which synchronises with the device) reads and clears
+ * the flag: SBP_ERR_TIMEOUT if a wait expired since the last call, else SBP_OK. */
+sbp_status sbp_check_device_errors(void);
+
+/* Selects the copy engine of the pure data-movement transforms: 0 = choose (default),
+ * 1 = 128-bit load/store kernel, 2 = bulk asynchronous copies staged through shared
+ * memory (needs 16-byte aligned segments, else falls back to 1).  Process-wide. */
+void sbp_boxing_set_copy_engine(int32_t engine);
+
+/* ---------------------------------------------------------------- MatMul (Table 1)
+ *
+ * Y = XW on the local tensors, under the signatures the descriptors carry:
+ *   (S(0),B)->S(0)   (B,S(1))->S(1)   (S(1),S(0))->P(sum)
+ *   (P(sum),B)->P(sum)   (B,P(sum))->P(sum)   (B,B)->B
+ * y->sbp must be the signature Table 1 deduces, or -- for rows whose deduced signature is
+ * P(sum) -- B or S(i): the partial products are then reduced in rank order inside the
+ * kernel's accumulator and Y is written directly in that signature (the boxing op of
+ * Section 3.2 fused into the producer).  Any other request is SBP_ERR_SIGNATURE; call
+ * sbp_boxing afterwards instead.
+ *
+ * x: [M,K], w: [K,N], y: [M,N] logical, all 2-D, same dtype for x and w:
+ *   SBP_F32  : fp32 FMA accumulation, y SBP_F32.
+ *   SBP_BF16 : bf16 operands, fp32 accumulation on the tensor cores, y SBP_BF16 or SBP_F32.
+ * flags: SBP_EPILOGUE_GELU applies GeLU(v) = v/2 (1 + erf(v/sqrt 2)) to the fp32
+ * accumulator before the store; only where Y is S or B (GeLU is not linear, so it cannot
+ * be applied to partial values).
+ * ws: scratch for the tensor-core path (see sbp_matmul_workspace_bytes; may be NULL when
+ * that returns 0).
+ */
+#define SBP_EPILOGUE_GELU 1u
+size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y);
+sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, uint32_t flags,
+                      void* ws, size_t ws_bytes, void* cuda_stream);
+
+/* ---------------------------------------------------------------- split softmax cross entropy
+ *
+ * Section 6.3 (classifier weight S(1) => logits S(1)): the softmax has two reductions,
+ * max and sum, each done locally per shard first and then across shards
+ * (P(max)->B, P(sum)->B); the loss is the sparse cross entropy of the label's column.
+ *
+ *   logits  [rows, classes]  S(1), SBP_BF16 or SBP_F32
+ *   labels  [rows]           B, SBP_I64, each in [0, classes)
+ *   loss    [rows]           B, SBP_F32:  log(sum_j exp(z_ij - m_i)) + m_i - z_i,label_i
+ *   row_max [rows]           B, SBP_F32, optional (NULL): m_i = max_j z_ij
+ *   row_sum [rows]           B, SBP_F32, optional (NULL): sum_j exp(z_ij - m_i)
+ * ws holds the per-shard partial max / exp-sum / label-logit vectors.
+ * A label outside [0, classes) contributes a label logit of 0.
+ */
+size_t sbp_softmax_xent_workspace_bytes(const sbp_tensor* logits);
+sbp_status sbp_softmax_xent(const sbp_tensor* logits, const sbp_tensor* labels, sbp_tensor* loss,
+                            sbp_tensor* row_max, sbp_tensor* row_sum, void* ws, size_t ws_bytes,
+                            void* cuda_stream);
+
+/* ---------------------------------------------------------------- row-split embedding
+ *
+ * Section 6.3 (embedding table S(0), "splitting the vocabulary IDs"):
+ *   table [rows, dim]   S(0), SBP_F32 or SBP_BF16
+ *   ids   [...]         B, SBP_I64, 1 <= ndim <= 3
+ *   out   [..., dim]    P(sum): shard r writes table row id where id falls in its own row
+ *                       range and zeros elsewhere (the k outputs sum to the lookup);
+ *                       or B: the lookup itself, written to every replica -- the
+ *                       P(sum)->B boxing fused into the gather (exactly one shard
+ *                       contributes to a row, so the sum is that row; a -0.0 entry is
+ *                       written as +0.0 when k > 1, as x + 0 would give).
+ * An id outside [0, rows) produces a zero row and, when oob_count is not NULL, adds 1 to
+ * the device int32 it points to (the caller zeroes it).
+ */
+sbp_status sbp_embedding(const sbp_tensor* table, const sbp_tensor* ids, sbp_tensor* out,
+                         int32_t* oob_count, void* cuda_stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SBP_H_ */

@@ -1,0 +1,15 @@
+"""B200 (sm_100a) SBP library: boxing transforms between SBP signatures and the sharded
+operators they feed, over k logical shards resident in one GPU's memory.
+
+This package is a thin ctypes binding over the C ABI declared in include/sbp.h.  It
+marshals arguments only -- every step runs in the library's CUDA kernels -- and it fails
+loudly when the compiled library is missing: there is no CPU or PyTorch fallback.
+"""
+from .binding import (  # noqa: F401
+    B, P_MAX, P_SUM, S, Sig, SbpError, SbpTensor,
+    empty_global, lib_path, load_library,
+    sbp_boxing, sbp_boxing_host, sbp_boxing_host_workspace_bytes, sbp_boxing_set_copy_engine,
+    sbp_check_device_errors, sbp_embedding, sbp_launch_count, sbp_local_shape, sbp_matmul,
+    sbp_matmul_infer, sbp_matmul_workspace_bytes, sbp_softmax_xent,
+    sbp_softmax_xent_workspace_bytes, SBP_EPILOGUE_GELU,
+)

@@ -1,0 +1,248 @@
+"""ctypes binding of include/sbp.h.  Argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+import torch
+
+SBP_MAX_DIMS = 4
+SBP_MAX_K = 16
+SBP_MAX_PDIMS = 2
+SBP_EPILOGUE_GELU = 1
+
+SBP_SPLIT, SBP_BROADCAST, SBP_PARTIAL_SUM, SBP_PARTIAL_MAX = 0, 1, 2, 3
+_DTYPES = {torch.float32: 0, torch.bfloat16: 1, torch.int64: 2}
+
+
+class _Sig(C.Structure):
+    _fields_ = [("kind", C.c_int32), ("axis", C.c_int32)]
+
+
+class _Tensor(C.Structure):
+    _fields_ = [
+        ("ndim", C.c_int32),
+        ("dtype", C.c_int32),
+        ("shape", C.c_int64 * SBP_MAX_DIMS),
+        ("pdims", C.c_int32),
+        ("pshape", C.c_int32 * SBP_MAX_PDIMS),
+        ("sbp", _Sig * SBP_MAX_PDIMS),
+        ("local", C.c_void_p * SBP_MAX_K),
+    ]
+
+
+@dataclass(frozen=True)
+class Sig:
+    """One SBP signature: S(axis), B, P_SUM or P_MAX (the paper's Section 3.1)."""
+    kind: int
+    axis: int = 0
+
+    def __repr__(self):
+        return {SBP_SPLIT: f"S({self.axis})", SBP_BROADCAST: "B",
+                SBP_PARTIAL_SUM: "P(sum)", SBP_PARTIAL_MAX: "P(max)"}[self.kind]
+
+    def _c(self) -> _Sig:
+        return _Sig(self.kind, self.axis)
+
+
+def S(axis: int) -> Sig:
+    return Sig(SBP_SPLIT, int(axis))
+
+
+B = Sig(SBP_BROADCAST)
+P_SUM = Sig(SBP_PARTIAL_SUM)
+P_MAX = Sig(SBP_PARTIAL_MAX)
+
+
+class SbpError(RuntimeError):
+    def __init__(self, status: int, name: str, detail: str):
+        super().__init__(f"{name}: {detail}")
+        self.status = status
+        self.name = name
+
+
+_LIB = None
+
+
+def lib_path() -> str:
+    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsbp_b200.so")
+
+
+def load_library():
+    """Loads libsbp_b200.so.  Raises if it has not been built: there is no fallback."""
+    global _LIB
+    if _LIB is not None:
+        return _LIB
+    path = lib_path()
+    if not os.path.exists(path):
+        raise RuntimeError(
+            f"{path} is missing: build it with `python -m paper_2110_15032_b200.build` "
+            "(nvcc, sm_100a).  This package has no CPU or PyTorch fallback.")
+    lib = C.CDLL(path)
+    T = C.POINTER(_Tensor)
+    lib.sbp_status_string.restype = C.c_char_p
+    lib.sbp_status_string.argtypes = [C.c_int]
+    lib.sbp_last_error.restype = C.c_char_p
+    lib.sbp_launch_count.restype = C.c_uint64
+    lib.sbp_local_shape.argtypes = [T, C.c_int32, C.POINTER(C.c_int64)]
+    lib.sbp_matmul_infer.argtypes = [_Sig, _Sig, C.POINTER(_Sig)]
+    lib.sbp_boxing.argtypes = [T, T, C.c_void_p]
+    lib.sbp_boxing_host_workspace_bytes.restype = C.c_size_t
+    lib.sbp_boxing_host_workspace_bytes.argtypes = [T, T]
+    lib.sbp_boxing_host.argtypes = [T, T, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sbp_boxing_set_copy_engine.argtypes = [C.c_int32]
+    lib.sbp_boxing_set_copy_engine.restype = None
+    lib.sbp_check_device_errors.argtypes = []
+    lib.sbp_matmul_workspace_bytes.restype = C.c_size_t
+    lib.sbp_matmul_workspace_bytes.argtypes = [T, T, T]
+    lib.sbp_matmul.argtypes = [T, T, T, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sbp_softmax_xent_workspace_bytes.restype = C.c_size_t
+    lib.sbp_softmax_xent_workspace_bytes.argtypes = [T]
+    lib.sbp_softmax_xent.argtypes = [T, T, T, T, T, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sbp_embedding.argtypes = [T, T, T, C.c_void_p, C.c_void_p]
+    _LIB = lib
+    return lib
+
+
+def _check(status: int):
+    if status != 0:
+        lib = load_library()
+        raise SbpError(status, lib.sbp_status_string(status).decode(), lib.sbp_last_error().decode())
+
+
+class SbpTensor:
+    """A global tensor = logical shape + dtype + signature + the k local tensors.
+
+    `locals` are torch tensors used purely as memory (device memory for every entry
+    point except sbp_boxing_host, which takes host tensors).  Each must be contiguous.
+    """
+
+    def __init__(self, shape: Sequence[int], dtype: torch.dtype, sig: Sig, locals: Sequence[torch.Tensor]):
+        self.shape = tuple(int(s) for s in shape)
+        self.dtype = dtype
+        self.sig = sig
+        self.locals: List[torch.Tensor] = list(locals)
+        self.k = len(self.locals)
+        for t in self.locals:
+            if not t.is_contiguous():
+                raise ValueError("local tensors must be contiguous")
+            if t.dtype != dtype:
+                raise ValueError("local tensor dtype differs from the descriptor's")
+
+    def _c(self) -> _Tensor:
+        d = _Tensor()
+        d.ndim = len(self.shape)
+        d.dtype = _DTYPES[self.dtype]
+        for i, s in enumerate(self.shape):
+            d.shape[i] = s
+        d.pdims = 1
+        d.pshape[0] = self.k
+        d.pshape[1] = 1
+        d.sbp[0] = self.sig._c()
+        for r, t in enumerate(self.locals):
+            d.local[r] = t.data_ptr()
+        return d
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream)
+
+
+def sbp_local_shape(shape, sig: Sig, k: int, r: int, dtype=torch.float32):
+    d = _Tensor()
+    d.ndim = len(shape)
+    d.dtype = _DTYPES[dtype]
+    for i, s in enumerate(shape):
+        d.shape[i] = int(s)
+    d.pdims = 1
+    d.pshape[0] = k
+    d.sbp[0] = sig._c()
+    out = (C.c_int64 * SBP_MAX_DIMS)()
+    _check(load_library().sbp_local_shape(C.byref(d), r, out))
+    return tuple(out[i] for i in range(len(shape)))
+
+
+def empty_global(shape, dtype, sig: Sig, k: int, device="cuda", alias_replicas: bool = False) -> SbpTensor:
+    """Allocates (torch.empty) the k local tensors of a global tensor."""
+    locs = []
+    for r in range(k):
+        if alias_replicas and sig.kind == SBP_BROADCAST and r > 0:
+            locs.append(locs[0])
+        else:
+            locs.append(torch.empty(sbp_local_shape(shape, sig, k, r, dtype), dtype=dtype, device=device))
+    return SbpTensor(shape, dtype, sig, locs)
+
+
+def sbp_matmul_infer(x: Sig, w: Sig) -> Sig:
+    out = _Sig()
+    _check(load_library().sbp_matmul_infer(x._c(), w._c(), C.byref(out)))
+    return Sig(out.kind, out.axis if out.kind == SBP_SPLIT else 0)
+
+
+def sbp_launch_count() -> int:
+    return int(load_library().sbp_launch_count())
+
+
+def sbp_check_device_errors() -> None:
+    _check(load_library().sbp_check_device_errors())
+
+
+def sbp_boxing_set_copy_engine(engine: int) -> None:
+    load_library().sbp_boxing_set_copy_engine(int(engine))
+
+
+def sbp_boxing(src: SbpTensor, dst: SbpTensor, stream=None) -> None:
+    a, b = src._c(), dst._c()
+    _check(load_library().sbp_boxing(C.byref(a), C.byref(b), _stream_ptr(stream)))
+
+
+def sbp_boxing_host_workspace_bytes(src_host: SbpTensor, dst_host: SbpTensor) -> int:
+    a, b = src_host._c(), dst_host._c()
+    return int(load_library().sbp_boxing_host_workspace_bytes(C.byref(a), C.byref(b)))
+
+
+def sbp_boxing_host(src_host: SbpTensor, dst_host: SbpTensor, dev_ws: torch.Tensor, stream=None) -> None:
+    a, b = src_host._c(), dst_host._c()
+    _check(load_library().sbp_boxing_host(C.byref(a), C.byref(b), C.c_void_p(dev_ws.data_ptr()),
+                                          dev_ws.numel() * dev_ws.element_size(), _stream_ptr(stream)))
+
+
+def sbp_matmul_workspace_bytes(x: SbpTensor, w: SbpTensor, y: SbpTensor) -> int:
+    a, b, c = x._c(), w._c(), y._c()
+    return int(load_library().sbp_matmul_workspace_bytes(C.byref(a), C.byref(b), C.byref(c)))
+
+
+def sbp_matmul(x: SbpTensor, w: SbpTensor, y: SbpTensor, flags: int = 0,
+               ws: Optional[torch.Tensor] = None, stream=None) -> None:
+    a, b, c = x._c(), w._c(), y._c()
+    wp = C.c_void_p(ws.data_ptr()) if ws is not None else C.c_void_p(0)
+    wb = ws.numel() * ws.element_size() if ws is not None else 0
+    _check(load_library().sbp_matmul(C.byref(a), C.byref(b), C.byref(c), flags, wp, wb, _stream_ptr(stream)))
+
+
+def sbp_softmax_xent_workspace_bytes(logits: SbpTensor) -> int:
+    a = logits._c()
+    return int(load_library().sbp_softmax_xent_workspace_bytes(C.byref(a)))
+
+
+def sbp_softmax_xent(logits: SbpTensor, labels: SbpTensor, loss: SbpTensor,
+                     row_max: Optional[SbpTensor], row_sum: Optional[SbpTensor],
+                     ws: torch.Tensor, stream=None) -> None:
+    a, b, c = logits._c(), labels._c(), loss._c()
+    m = row_max._c() if row_max is not None else None
+    s = row_sum._c() if row_sum is not None else None
+    _check(load_library().sbp_softmax_xent(
+        C.byref(a), C.byref(b), C.byref(c),
+        C.byref(m) if m is not None else None, C.byref(s) if s is not None else None,
+        C.c_void_p(ws.data_ptr()), ws.numel() * ws.element_size(), _stream_ptr(stream)))
+
+
+def sbp_embedding(table: SbpTensor, ids: SbpTensor, out: SbpTensor,
+                  oob_count: Optional[torch.Tensor] = None, stream=None) -> None:
+    a, b, c = table._c(), ids._c(), out._c()
+    oob = C.c_void_p(oob_count.data_ptr()) if oob_count is not None else C.c_void_p(0)
+    _check(load_library().sbp_embedding(C.byref(a), C.byref(b), C.byref(c), oob, _stream_ptr(stream)))

@@ -1,0 +1,506 @@
+// Boxing transforms between SBP signatures on k shards held in one GPU's memory
+// (Section 3.2, Table 2 "same placement" column).
+//
+// Every transform is expressed on one canonical 5-D view of the logical tensor,
+//     [A][Na][M][Nb][C],
+// where at most the axes Na and Nb are restricted by a split signature (on the source
+// side, the destination side, or both) and C is the contiguous tail.  A *task* is one
+// (source shard, destination shard) pair; the elements it moves are the intersection of
+// the two shards' regions: A * la * M contiguous segments of lb * C elements.  Tasks are
+// cut into tiles of J*256 vectors (rows = segments, columns = vectors inside a segment);
+// one CTA moves one tile, each thread J vectors with all loads issued before the stores.
+//
+//   data movement  S(i)->S(j), S(i)->B (one read, k writes), B->S(i), copies
+//   reduction      P(sum)/P(max) -> B (k reads, k writes) or -> S(i) (k reads, 1 write);
+//                  fp32 accumulator, shards added in rank order, one rounding at the end
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <atomic>
+
+#include "boxing_params.h"
+#include "sbp_internal.h"
+
+namespace sbp {
+
+enum BoxOp : int { OP_COPY = 0, OP_SUM_F32, OP_SUM_BF16, OP_MAX_F32, OP_MAX_BF16 };
+
+// ------------------------------------------------------------------ element arithmetic
+
+// fp32 lanes carried by one vector of type V
+template <typename V>
+struct AccF32 {
+  static constexpr int N = sizeof(V) / 4;
+  float v[N];
+  __device__ void load(const V& x) {
+    const float* f = reinterpret_cast<const float*>(&x);
+#pragma unroll
+    for (int i = 0; i < N; ++i) v[i] = f[i];
+  }
+  __device__ V store() const {
+    V out;
+    float* f = reinterpret_cast<float*>(&out);
+#pragma unroll
+    for (int i = 0; i < N; ++i) f[i] = v[i];
+    return out;
+  }
+};
+
+template <typename V>
+struct AccBF16 {
+  static constexpr int N = sizeof(V) / 2;
+  float v[N];
+  __device__ void load(const V& x) {
+    const __nv_bfloat16* h = reinterpret_cast<const __nv_bfloat16*>(&x);
+#pragma unroll
+    for (int i = 0; i < N; ++i) v[i] = __bfloat162float(h[i]);
+  }
+  __device__ V store() const {
+    V out;
+    __nv_bfloat16* h = reinterpret_cast<__nv_bfloat16*>(&out);
+#pragma unroll
+    for (int i = 0; i < N; ++i) h[i] = __float2bfloat16_rn(v[i]);   // the single rounding
+    return out;
+  }
+};
+
+template <int OP, typename V>
+struct Lanes {
+  using type = AccF32<V>;
+};
+template <typename V>
+struct Lanes<OP_SUM_BF16, V> {
+  using type = AccBF16<V>;
+};
+template <typename V>
+struct Lanes<OP_MAX_BF16, V> {
+  using type = AccBF16<V>;
+};
+
+template <int OP, typename L>
+__device__ __forceinline__ void combine(L& acc, const L& x) {
+#pragma unroll
+  for (int i = 0; i < L::N; ++i) {
+    if (OP == OP_SUM_F32 || OP == OP_SUM_BF16)
+      acc.v[i] = __fadd_rn(acc.v[i], x.v[i]);          // plain IEEE add, never contracted
+    else
+      acc.v[i] = (x.v[i] > acc.v[i]) ? x.v[i] : acc.v[i];   // first wins on ties
+  }
+}
+
+template <typename V>
+__device__ __forceinline__ V ld_stream(const V* p) {
+  return *p;
+}
+template <>
+__device__ __forceinline__ uint4 ld_stream<uint4>(const uint4* p) {
+  uint4 r;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "l"(p));
+  return r;
+}
+
+// ------------------------------------------------------------------ the tile kernel
+
+struct TaskGeom {
+  long long nseg, seg_vecs;   // segments in the task, vectors per segment
+  long long la;
+  long long Na_s, aoff_s, Nb_s, boff_s;
+  long long Na_d, aoff_d, Nb_d, boff_d;
+};
+
+__device__ __forceinline__ void task_geometry(const BoxParams& p, int s, int d, int vbytes, TaskGeom* g) {
+  long long a0 = 0, la = p.Na, b0 = 0, lb = p.Nb;
+  if (p.src_a) split_range(p.Na, p.k, s, (int64_t*)&a0, (int64_t*)&la);
+  else if (p.dst_a) split_range(p.Na, p.k, d, (int64_t*)&a0, (int64_t*)&la);
+  if (p.src_b) split_range(p.Nb, p.k, s, (int64_t*)&b0, (int64_t*)&lb);
+  else if (p.dst_b) split_range(p.Nb, p.k, d, (int64_t*)&b0, (int64_t*)&lb);
+  g->la = la;
+  g->nseg = p.A * la * p.M;
+  g->seg_vecs = lb * p.C * p.esz / vbytes;
+  g->Na_s = p.src_a ? la : p.Na;  g->aoff_s = p.src_a ? 0 : a0;
+  g->Nb_s = p.src_b ? lb : p.Nb;  g->boff_s = p.src_b ? 0 : b0;
+  g->Na_d = p.dst_a ? la : p.Na;  g->aoff_d = p.dst_a ? 0 : a0;
+  g->Nb_d = p.dst_b ? lb : p.Nb;  g->boff_d = p.dst_b ? 0 : b0;
+}
+
+// V: vector type moved by one thread access.  OP: BoxOp.  J: vectors per thread.
+// KT: compile-time number of source shards of a reduction (0 = read p.k at run time).
+template <typename V, int OP, int J, int KT>
+__global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ BoxParams p) {
+  const long long u = blockIdx.x;
+  const int t = (int)(u / p.tiles_per_task);
+  const long long rem = u - (long long)t * p.tiles_per_task;
+  const long long row_tile = rem / p.col_tiles;
+  const long long col_tile = rem - row_tile * p.col_tiles;
+
+  int s = t, d = t;
+  if (p.mode == MODE_PAIRS) { s = t / p.k; d = t - s * p.k; }
+  else if (p.mode == MODE_REDUCE_B) { s = 0; d = 0; }
+
+  TaskGeom g;
+  task_geometry(p, s, d, (int)sizeof(V), &g);
+  const long long seg0 = row_tile * p.rows_per_tile;
+  if (seg0 >= g.nseg) return;
+  const long long col0 = col_tile << p.cv_log2;
+  if (col0 >= g.seg_vecs) return;
+
+  const long long cs = p.C * p.esz;   // bytes per unit step of the Nb axis
+  const bool flat = (p.A == 1 && p.M == 1);
+
+  long long so[J], dofs[J];
+  bool ok[J];
+#pragma unroll
+  for (int j = 0; j < J; ++j) {
+    const int f = threadIdx.x + j * 256;
+    const long long seg = seg0 + (f >> p.cv_log2);
+    const long long col = col0 + (f & ((1 << p.cv_log2) - 1));
+    ok[j] = seg < g.nseg && col < g.seg_vecs;
+    long long x = 0, ia = seg, m = 0;
+    if (!flat) {
+      const long long q = seg / p.M;
+      m = seg - q * p.M;
+      x = q / g.la;
+      ia = q - x * g.la;
+    }
+    so[j] = ((((x * g.Na_s + g.aoff_s + ia) * p.M + m) * g.Nb_s + g.boff_s) * cs) / (long long)sizeof(V) + col;
+    dofs[j] = ((((x * g.Na_d + g.aoff_d + ia) * p.M + m) * g.Nb_d + g.boff_d) * cs) / (long long)sizeof(V) + col;
+  }
+
+  V val[J];
+  if constexpr (OP == OP_COPY) {
+    const V* sp = reinterpret_cast<const V*>(p.src[s]);
+#pragma unroll
+    for (int j = 0; j < J; ++j)
+      if (ok[j]) val[j] = ld_stream(sp + so[j]);
+  } else {
+    using L = typename Lanes<OP, V>::type;
+    const int kk = KT ? KT : p.k;
+    if constexpr (KT != 0) {
+      V raw[J][KT ? KT : 1];
+#pragma unroll
+      for (int j = 0; j < J; ++j)
+#pragma unroll
+        for (int r = 0; r < (KT ? KT : 1); ++r)
+          if (ok[j]) raw[j][r] = ld_stream(reinterpret_cast<const V*>(p.src[r]) + so[j]);
+#pragma unroll
+      for (int j = 0; j < J; ++j) {
+        if (!ok[j]) continue;
+        L acc;
+        acc.load(raw[j][0]);
+#pragma unroll
+        for (int r = 1; r < (KT ? KT : 1); ++r) {
+          L x;
+          x.load(raw[j][r]);
+          combine<OP>(acc, x);
+        }
+        val[j] = acc.store();
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < J; ++j) {
+        if (!ok[j]) continue;
+        L acc;
+        acc.load(ld_stream(reinterpret_cast<const V*>(p.src[0]) + so[j]));
+        for (int r = 1; r < kk; ++r) {
+          L x;
+          x.load(ld_stream(reinterpret_cast<const V*>(p.src[r]) + so[j]));
+          combine<OP>(acc, x);
+        }
+        val[j] = acc.store();
+      }
+    }
+  }
+
+  if (p.mode == MODE_GATHER || p.mode == MODE_REDUCE_B) {
+    for (int r = 0; r < p.n_dst; ++r) {
+      V* dp = reinterpret_cast<V*>(p.dst[r]);
+#pragma unroll
+      for (int j = 0; j < J; ++j)
+        if (ok[j]) dp[dofs[j]] = val[j];
+    }
+  } else {
+    V* dp = reinterpret_cast<V*>(p.dst[d]);
+#pragma unroll
+    for (int j = 0; j < J; ++j)
+      if (ok[j]) dp[dofs[j]] = val[j];
+  }
+}
+
+// ------------------------------------------------------------------ host side
+
+static std::atomic<int> g_copy_engine{0};
+
+struct Plan {
+  BoxParams p;
+  int op;
+  int vbytes;
+  int ntasks;
+  long long grid;
+};
+
+static int pick_vector_bytes(const BoxParams& p, const sbp_tensor* src, const sbp_tensor* dst, int k) {
+  for (int vb = 16; vb > p.esz; vb >>= 1) {
+    bool ok = true;
+    for (int r = 0; r < k && ok; ++r) {
+      ok = ok && reinterpret_cast<uintptr_t>(src->local[r]) % vb == 0;
+      ok = ok && reinterpret_cast<uintptr_t>(dst->local[r]) % vb == 0;
+      int64_t st, ln;
+      if (p.src_b || p.dst_b) {
+        split_range(p.Nb, k, r, &st, &ln);
+        ok = ok && (st * p.C * p.esz) % vb == 0 && (ln * p.C * p.esz) % vb == 0;
+      }
+    }
+    ok = ok && (p.Nb * p.C * p.esz) % vb == 0;
+    if (ok) return vb;
+  }
+  return p.esz;
+}
+
+template <typename V, int OP, int J>
+static void launch_k(const Plan& pl, cudaStream_t st) {
+  dim3 grid((unsigned)pl.grid), block(256);
+  if (OP == OP_COPY) {
+    box_tile_kernel<V, OP, J, 0><<<grid, block, 0, st>>>(pl.p);
+    return;
+  }
+  switch (pl.p.k) {
+    case 1: box_tile_kernel<V, OP, J, 1><<<grid, block, 0, st>>>(pl.p); break;
+    case 2: box_tile_kernel<V, OP, J, 2><<<grid, block, 0, st>>>(pl.p); break;
+    case 4: box_tile_kernel<V, OP, J, 4><<<grid, block, 0, st>>>(pl.p); break;
+    case 8: box_tile_kernel<V, OP, J, 8><<<grid, block, 0, st>>>(pl.p); break;
+    default: box_tile_kernel<V, OP, J, 0><<<grid, block, 0, st>>>(pl.p); break;
+  }
+}
+
+template <int OP, int J>
+static void launch_v(const Plan& pl, cudaStream_t st) {
+  switch (pl.vbytes) {
+    case 16: launch_k<uint4, OP, J>(pl, st); break;
+    case 8: launch_k<uint2, OP, J>(pl, st); break;
+    case 4: launch_k<uint32_t, OP, J>(pl, st); break;
+    default: launch_k<uint16_t, OP, J>(pl, st); break;
+  }
+}
+
+// 2-byte vectors cannot carry an fp32 lane, 8-byte+ copies of int64 never use 2/4.
+template <int OP, int J>
+static void launch_v_f32(const Plan& pl, cudaStream_t st) {
+  switch (pl.vbytes) {
+    case 16: launch_k<uint4, OP, J>(pl, st); break;
+    case 8: launch_k<uint2, OP, J>(pl, st); break;
+    default: launch_k<uint32_t, OP, J>(pl, st); break;
+  }
+}
+
+constexpr int kJCopy = 4;
+constexpr int kJReduce = 2;
+
+static sbp_status make_plan(const sbp_tensor* src, const sbp_tensor* dst, Plan* pl) {
+  const int k = placement_k(src);
+  const sbp_sig ss = src->sbp[0], ds = dst->sbp[0];
+  BoxParams& p = pl->p;
+  p = BoxParams{};
+  p.k = k;
+  p.esz = elem_size(src->dtype);
+  const bool src_p = ss.kind == SBP_PARTIAL_SUM || ss.kind == SBP_PARTIAL_MAX;
+  const bool dst_p = ds.kind == SBP_PARTIAL_SUM || ds.kind == SBP_PARTIAL_MAX;
+
+  pl->op = OP_COPY;
+  if (src_p && dst_p) {
+    if (ss.kind != ds.kind)
+      return fail(SBP_ERR_UNSUPPORTED, "boxing between P(sum) and P(max) has no meaning");
+    p.mode = MODE_DIAG;
+  } else if (dst_p) {
+    return fail(SBP_ERR_UNSUPPORTED, "boxing S->P / B->P is not implemented");
+  } else if (src_p) {
+    if (src->dtype == SBP_I64) return fail(SBP_ERR_DTYPE, "partial-value reduction needs F32 or BF16");
+    const bool bf = src->dtype == SBP_BF16;
+    pl->op = ss.kind == SBP_PARTIAL_SUM ? (bf ? OP_SUM_BF16 : OP_SUM_F32) : (bf ? OP_MAX_BF16 : OP_MAX_F32);
+    p.mode = ds.kind == SBP_BROADCAST ? MODE_REDUCE_B : MODE_REDUCE_S;
+  } else if (ss.kind == SBP_SPLIT && ds.kind == SBP_BROADCAST) {
+    p.mode = MODE_GATHER;
+  } else if (ss.kind == SBP_SPLIT && ds.kind == SBP_SPLIT && ss.axis != ds.axis) {
+    p.mode = MODE_PAIRS;
+  } else {
+    p.mode = MODE_DIAG;   // S(i)->S(i), B->S(i), B->B
+  }
+
+  // canonical 5-D view
+  const int sa = ss.kind == SBP_SPLIT ? ss.axis : -1;
+  const int da = ds.kind == SBP_SPLIT ? ds.axis : -1;
+  auto prod = [&](int lo, int hi) {
+    long long v = 1;
+    for (int d = lo; d < hi; ++d) v *= src->shape[d];
+    return v;
+  };
+  p.A = p.Na = p.M = p.Nb = 1;
+  if (sa < 0 && da < 0) {
+    p.C = prod(0, src->ndim);
+  } else if (sa < 0 || da < 0 || sa == da) {
+    const int ax = sa >= 0 ? sa : da;
+    p.A = prod(0, ax);
+    p.Nb = src->shape[ax];
+    p.C = prod(ax + 1, src->ndim);
+    p.src_b = sa >= 0;
+    p.dst_b = da >= 0;
+  } else {
+    const int lo = std::min(sa, da), hi = std::max(sa, da);
+    p.A = prod(0, lo);
+    p.Na = src->shape[lo];
+    p.M = prod(lo + 1, hi);
+    p.Nb = src->shape[hi];
+    p.C = prod(hi + 1, src->ndim);
+    p.src_a = sa == lo;  p.dst_a = da == lo;
+    p.src_b = sa == hi;  p.dst_b = da == hi;
+  }
+
+  for (int r = 0; r < k; ++r) {
+    p.src[r] = static_cast<const char*>(src->local[r]);
+    p.dst[r] = static_cast<char*>(dst->local[r]);
+  }
+  pl->vbytes = pick_vector_bytes(p, src, dst, k);
+  if (pl->op != OP_COPY && pl->vbytes < 4 && src->dtype == SBP_F32) pl->vbytes = 4;
+
+  // distinct destination buffers for the one-read-many-writes modes
+  p.n_dst = 0;
+  if (p.mode == MODE_GATHER || p.mode == MODE_REDUCE_B) {
+    char* uniq[SBP_MAX_K];
+    for (int r = 0; r < k; ++r) {
+      bool seen = false;
+      for (int q = 0; q < p.n_dst; ++q) seen = seen || uniq[q] == p.dst[r];
+      if (!seen) uniq[p.n_dst++] = p.dst[r];
+    }
+    for (int q = 0; q < p.n_dst; ++q) p.dst[q] = uniq[q];
+  }
+
+  // tiling: the largest segment / segment count over shards bounds the per-task grid
+  const long long la_max = (p.src_a || p.dst_a) ? (p.Na + k - 1) / k : p.Na;
+  const long long lb_max = (p.src_b || p.dst_b) ? (p.Nb + k - 1) / k : p.Nb;
+  const long long nseg_max = p.A * la_max * p.M;
+  const long long seg_vecs_max = lb_max * p.C * p.esz / pl->vbytes;
+  const int J = pl->op == OP_COPY ? kJCopy : kJReduce;
+  const int tile_vecs = J * 256;
+  int cv_log2 = 0;
+  while ((1 << cv_log2) < tile_vecs && (1LL << cv_log2) < seg_vecs_max) ++cv_log2;
+  p.cv_log2 = cv_log2;
+  p.rows_per_tile = tile_vecs >> cv_log2;
+  p.col_tiles = std::max(1LL, (seg_vecs_max + (1LL << cv_log2) - 1) >> cv_log2);
+  const long long row_tiles = std::max(1LL, (nseg_max + p.rows_per_tile - 1) / p.rows_per_tile);
+  p.tiles_per_task = p.col_tiles * row_tiles;
+  pl->ntasks = p.mode == MODE_PAIRS ? k * k : (p.mode == MODE_REDUCE_B ? 1 : k);
+  pl->grid = p.tiles_per_task * pl->ntasks;
+  if (pl->grid > 0x7fffffffLL) return fail(SBP_ERR_UNSUPPORTED, "tensor too large for one launch");
+  return SBP_OK;
+}
+
+// Bulk-copy engine (defined in boxing_bulk.cu); returns false when it does not apply.
+bool launch_bulk_copy(const BoxParams& p, int ntasks, cudaStream_t st);
+
+static sbp_status check_pair(const sbp_tensor* src, const sbp_tensor* dst, bool need_ptrs) {
+  sbp_status st = check_tensor(src, "src", need_ptrs);
+  if (st != SBP_OK) return st;
+  st = check_tensor(dst, "dst", need_ptrs);
+  if (st != SBP_OK) return st;
+  if (src->ndim != dst->ndim) return fail(SBP_ERR_SHAPE, "src and dst differ in rank");
+  for (int d = 0; d < src->ndim; ++d)
+    if (src->shape[d] != dst->shape[d]) return fail(SBP_ERR_SHAPE, "src and dst differ on axis %d", d);
+  if (src->dtype != dst->dtype) return fail(SBP_ERR_DTYPE, "src and dst differ in dtype");
+  if (placement_k(src) != placement_k(dst)) return fail(SBP_ERR_INVALID_ARG, "src and dst differ in k");
+  return SBP_OK;
+}
+
+}  // namespace sbp
+
+using namespace sbp;
+
+extern "C" {
+
+void sbp_boxing_set_copy_engine(int32_t engine) { g_copy_engine.store(engine); }
+
+sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream) {
+  sbp_status st = check_pair(src, dst, true);
+  if (st != SBP_OK) return st;
+  Plan pl;
+  st = make_plan(src, dst, &pl);
+  if (st != SBP_OK) return st;
+  if (numel(src) == 0) return SBP_OK;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+  bool done = false;
+  if (pl.op == OP_COPY && g_copy_engine.load() == 2 && pl.vbytes == 16)
+    done = launch_bulk_copy(pl.p, pl.ntasks, stream);
+  if (!done) {
+    switch (pl.op) {
+      case OP_COPY: launch_v<OP_COPY, kJCopy>(pl, stream); break;
+      case OP_SUM_F32: launch_v_f32<OP_SUM_F32, kJReduce>(pl, stream); break;
+      case OP_MAX_F32: launch_v_f32<OP_MAX_F32, kJReduce>(pl, stream); break;
+      case OP_SUM_BF16: launch_v<OP_SUM_BF16, kJReduce>(pl, stream); break;
+      case OP_MAX_BF16: launch_v<OP_MAX_BF16, kJReduce>(pl, stream); break;
+    }
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "boxing launch");
+  count_launch();
+  return SBP_OK;
+}
+
+static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
+
+size_t sbp_boxing_host_workspace_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_host) {
+  if (check_pair(src_host, dst_host, false) != SBP_OK) return 0;
+  const int k = placement_k(src_host);
+  size_t total = 0;
+  for (int r = 0; r < k; ++r) {
+    total += align256((size_t)local_numel(src_host, r) * elem_size(src_host->dtype));
+    total += align256((size_t)local_numel(dst_host, r) * elem_size(dst_host->dtype));
+  }
+  return total;
+}
+
+sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, void* dev_ws, size_t dev_ws_bytes,
+                           void* cuda_stream) {
+  sbp_status st = check_pair(src_host, dst_host, true);
+  if (st != SBP_OK) return st;
+  const size_t need = sbp_boxing_host_workspace_bytes(src_host, dst_host);
+  if (need > 0 && (!dev_ws || dev_ws_bytes < need))
+    return fail(SBP_ERR_WORKSPACE, "device workspace of %zu bytes needed, %zu given", need, dev_ws_bytes);
+  if (reinterpret_cast<uintptr_t>(dev_ws) % 256 != 0)
+    return fail(SBP_ERR_ALIGNMENT, "device workspace must be 256-byte aligned");
+  const int k = placement_k(src_host);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  sbp_tensor s = *src_host, d = *dst_host;
+  char* cur = static_cast<char*>(dev_ws);
+  const int esz = elem_size(src_host->dtype);
+  for (int r = 0; r < k; ++r) {
+    s.local[r] = cur;
+    cur += align256((size_t)local_numel(src_host, r) * esz);
+  }
+  // Destination replicas that alias on the host alias on the device as well.
+  for (int r = 0; r < k; ++r) {
+    d.local[r] = nullptr;
+    for (int q = 0; q < r; ++q)
+      if (dst_host->local[q] == dst_host->local[r]) d.local[r] = d.local[q];
+    if (!d.local[r]) {
+      d.local[r] = cur;
+      cur += align256((size_t)local_numel(dst_host, r) * esz);
+    }
+  }
+  for (int r = 0; r < k; ++r) {
+    const size_t bytes = (size_t)local_numel(src_host, r) * esz;
+    if (bytes) SBP_CUDA_TRY(cudaMemcpyAsync(s.local[r], src_host->local[r], bytes, cudaMemcpyHostToDevice, stream));
+  }
+  st = sbp_boxing(&s, &d, cuda_stream);
+  if (st != SBP_OK) return st;
+  for (int r = 0; r < k; ++r) {
+    bool dup = false;
+    for (int q = 0; q < r; ++q) dup = dup || dst_host->local[q] == dst_host->local[r];
+    const size_t bytes = (size_t)local_numel(dst_host, r) * esz;
+    if (!dup && bytes)
+      SBP_CUDA_TRY(cudaMemcpyAsync(dst_host->local[r], d.local[r], bytes, cudaMemcpyDeviceToHost, stream));
+  }
+  return SBP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,255 @@
+// Bulk-copy engine for the pure data-movement boxing transforms (S(i)->S(j), S(i)->B,
+// B->S(i)): the copy engine of the SM moves whole row segments global -> shared -> global
+// (cp.async.bulk), so no register file traffic and one issuing thread per CTA.
+//
+// A persistent grid of small CTAs walks the same (task, segment rows, column chunk) tiles
+// as the load/store kernel.  Each CTA owns a ring of kStages shared-memory buffers: the
+// loads of tile i + kStages - 1 are in flight while tile i is being stored.  A tile is
+// filled by one bulk load per segment (all signalling one mbarrier with the tile's byte
+// count) and drained by one bulk store per segment per destination replica.
+//
+// Every wait is bounded.  If a wait expires the CTA records it in a device flag that
+// sbp_check_device_errors() reports as SBP_ERR_TIMEOUT, drains its stores and returns.
+#include <cuda_runtime.h>
+
+#include "boxing_params.h"
+#include "sbp_internal.h"
+
+namespace sbp {
+
+__device__ int g_bulk_timeout_flag = 0;
+
+constexpr int kStages = 4;
+constexpr int kStageBytes = 16 * 1024;
+constexpr int kCtasPerSm = 3;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+
+struct BulkParams {
+  BoxParams b;
+  long long row_tiles, col_tiles;   // tiling of one task for this engine
+  long long tiles_per_task;
+  int rows_per_tile;                // segments per tile
+  long long chunk_bytes;            // column chunk of a segment (multiple of 16)
+  long long total_tiles;
+};
+
+__device__ __forceinline__ unsigned smem_u32(const void* p) {
+  return (unsigned)__cvta_generic_to_shared(p);
+}
+
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+// Waits for the phase with the given parity; gives up after kWaitLimitNs.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
+  const unsigned long long t0 = global_ns();
+  for (;;) {
+    unsigned done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    if (done) return true;
+    if (global_ns() - t0 > kWaitLimitNs) return false;
+  }
+}
+
+// One tile of one task: which shards, which segments, where they sit on both sides.
+struct BulkTile {
+  int s, d;
+  long long rows, bytes;      // segments in the tile, bytes of each segment piece
+  long long seg0, cb;         // first segment, byte offset of the column chunk
+  long long la;
+  long long Na_s, aoff_s, Nb_s, boff_s;
+  long long Na_d, aoff_d, Nb_d, boff_d;
+};
+
+__device__ __forceinline__ BulkTile bulk_tile(const BulkParams& q, long long u) {
+  const BoxParams& p = q.b;
+  BulkTile g;
+  const int t = (int)(u / q.tiles_per_task);
+  const long long rem = u - (long long)t * q.tiles_per_task;
+  const long long row_tile = rem / q.col_tiles, col_tile = rem - row_tile * q.col_tiles;
+  g.s = t;
+  g.d = t;
+  if (p.mode == MODE_PAIRS) { g.s = t / p.k; g.d = t - g.s * p.k; }
+  long long a0 = 0, la = p.Na, b0 = 0, lb = p.Nb;
+  if (p.src_a) split_range(p.Na, p.k, g.s, (int64_t*)&a0, (int64_t*)&la);
+  else if (p.dst_a) split_range(p.Na, p.k, g.d, (int64_t*)&a0, (int64_t*)&la);
+  if (p.src_b) split_range(p.Nb, p.k, g.s, (int64_t*)&b0, (int64_t*)&lb);
+  else if (p.dst_b) split_range(p.Nb, p.k, g.d, (int64_t*)&b0, (int64_t*)&lb);
+  const long long nseg = p.A * la * p.M, seg_bytes = lb * p.C * p.esz;
+  g.seg0 = row_tile * q.rows_per_tile;
+  g.cb = col_tile * q.chunk_bytes;
+  g.rows = nseg - g.seg0 < q.rows_per_tile ? nseg - g.seg0 : q.rows_per_tile;
+  g.bytes = seg_bytes - g.cb < q.chunk_bytes ? seg_bytes - g.cb : q.chunk_bytes;
+  g.la = la;
+  g.Na_s = p.src_a ? la : p.Na;  g.aoff_s = p.src_a ? 0 : a0;
+  g.Nb_s = p.src_b ? lb : p.Nb;  g.boff_s = p.src_b ? 0 : b0;
+  g.Na_d = p.dst_a ? la : p.Na;  g.aoff_d = p.dst_a ? 0 : a0;
+  g.Nb_d = p.dst_b ? lb : p.Nb;  g.boff_d = p.dst_b ? 0 : b0;
+  return g;
+}
+
+// Byte offsets of the start of segment `seg` inside the source and destination buffers.
+__device__ __forceinline__ void seg_offsets(const BoxParams& p, const BulkTile& g, long long seg, long long* so,
+                                            long long* dofs) {
+  const long long cs = p.C * p.esz;
+  long long x = 0, ia = seg, m = 0;
+  if (!(p.A == 1 && p.M == 1)) {
+    const long long q = seg / p.M;
+    m = seg - q * p.M;
+    x = q / g.la;
+    ia = q - x * g.la;
+  }
+  *so = (((x * g.Na_s + g.aoff_s + ia) * p.M + m) * g.Nb_s + g.boff_s) * cs;
+  *dofs = (((x * g.Na_d + g.aoff_d + ia) * p.M + m) * g.Nb_d + g.boff_d) * cs;
+}
+
+__global__ void __launch_bounds__(32) box_bulk_kernel(const __grid_constant__ BulkParams q) {
+  extern __shared__ __align__(128) unsigned char smem[];
+  __shared__ __align__(8) unsigned long long bars[kStages];
+  if (threadIdx.x != 0) return;
+  const BoxParams& p = q.b;
+
+  for (int i = 0; i < kStages; ++i)
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[i])) : "memory");
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+
+  const long long first = blockIdx.x, stride = gridDim.x;
+  const long long n_mine = first < q.total_tiles ? (q.total_tiles - first + stride - 1) / stride : 0;
+  bool timed_out = false;
+
+  // Loads of my tile number `it` into its ring slot: one bulk copy per segment.
+  auto issue_loads = [&](long long it) {
+    const BulkTile g = bulk_tile(q, first + it * stride);
+    const int slot = (int)(it % kStages);
+    const unsigned bar = smem_u32(&bars[slot]);
+    if (g.rows <= 0 || g.bytes <= 0) {   // tile outside an uneven shard: complete the phase empty
+      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+      return;
+    }
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
+                 "r"((unsigned)(g.rows * g.bytes))
+                 : "memory");
+    unsigned char* buf = smem + (size_t)slot * kStageBytes;
+    for (long long r = 0; r < g.rows; ++r) {
+      long long so, dofs;
+      seg_offsets(p, g, g.seg0 + r, &so, &dofs);
+      asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
+                       smem_u32(buf + r * g.bytes)),
+                   "l"(p.src[g.s] + so + g.cb), "r"((unsigned)g.bytes), "r"(bar)
+                   : "memory");
+    }
+  };
+
+  // Stores of my tile number `it` out of its ring slot, once per destination replica.
+  auto issue_stores = [&](long long it) {
+    const BulkTile g = bulk_tile(q, first + it * stride);
+    const int slot = (int)(it % kStages);
+    if (g.rows > 0 && g.bytes > 0) {
+      unsigned char* buf = smem + (size_t)slot * kStageBytes;
+      const int nd = p.mode == MODE_GATHER ? p.n_dst : 1;
+      for (long long r = 0; r < g.rows; ++r) {
+        long long so, dofs;
+        seg_offsets(p, g, g.seg0 + r, &so, &dofs);
+        for (int j = 0; j < nd; ++j) {
+          char* base = p.mode == MODE_GATHER ? p.dst[j] : p.dst[g.d];
+          asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(base + dofs + g.cb),
+                       "r"(smem_u32(buf + r * g.bytes)), "r"((unsigned)g.bytes)
+                       : "memory");
+        }
+      }
+    }
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+  };
+
+  const long long prologue = n_mine < kStages - 1 ? n_mine : kStages - 1;
+  for (long long it = 0; it < prologue; ++it) issue_loads(it);
+
+  for (long long it = 0; it < n_mine; ++it) {
+    const int slot = (int)(it % kStages);
+    const unsigned parity = (unsigned)((it / kStages) & 1);
+    if (!mbar_wait(smem_u32(&bars[slot]), parity)) {
+      timed_out = true;
+      break;
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    issue_stores(it);
+    // The slot that tile it + kStages - 1 will use was last drained by tile it - 1:
+    // wait until every store group except the newest has finished reading shared memory.
+    const long long nxt = it + kStages - 1;
+    if (nxt < n_mine) {
+      asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+      issue_loads(nxt);
+    }
+  }
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  if (timed_out) atomicExch(&g_bulk_timeout_flag, 1);
+}
+
+bool launch_bulk_copy(const BoxParams& p, int ntasks, cudaStream_t st) {
+  if (p.mode != MODE_PAIRS && p.mode != MODE_DIAG && p.mode != MODE_GATHER) return false;
+  const int k = p.k;
+  const long long la_max = (p.src_a || p.dst_a) ? (p.Na + k - 1) / k : p.Na;
+  const long long lb_max = (p.src_b || p.dst_b) ? (p.Nb + k - 1) / k : p.Nb;
+  const long long nseg_max = p.A * la_max * p.M;
+  const long long seg_bytes_max = lb_max * p.C * p.esz;
+  if (seg_bytes_max < 512) return false;   // too many tiny descriptors: the vector kernel is better
+  BulkParams q;
+  q.b = p;
+  if (seg_bytes_max >= kStageBytes) {
+    q.rows_per_tile = 1;
+    q.chunk_bytes = kStageBytes;
+  } else {
+    q.rows_per_tile = (int)(kStageBytes / seg_bytes_max);
+    q.chunk_bytes = seg_bytes_max;
+  }
+  q.col_tiles = (seg_bytes_max + q.chunk_bytes - 1) / q.chunk_bytes;
+  q.row_tiles = (nseg_max + q.rows_per_tile - 1) / q.rows_per_tile;
+  q.tiles_per_task = q.col_tiles * q.row_tiles;
+  q.total_tiles = q.tiles_per_task * ntasks;
+  if (q.total_tiles <= 0) return false;
+
+  static int sm_count = 0;
+  static bool attr_set = false;
+  const size_t smem = (size_t)kStages * kStageBytes;
+  if (!attr_set) {
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return false;
+    if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+    if (cudaFuncSetAttribute(box_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
+        cudaSuccess)
+      return false;
+    attr_set = true;
+  }
+  long long grid = (long long)sm_count * kCtasPerSm;
+  if (grid > q.total_tiles) grid = q.total_tiles;
+  box_bulk_kernel<<<(unsigned)grid, 32, smem, st>>>(q);
+  return true;
+}
+
+sbp_status read_and_clear_bulk_timeout(bool* timed_out) {
+  int flag = 0, zero = 0;
+  SBP_CUDA_TRY(cudaMemcpyFromSymbol(&flag, g_bulk_timeout_flag, sizeof(int)));
+  if (flag) SBP_CUDA_TRY(cudaMemcpyToSymbol(g_bulk_timeout_flag, &zero, sizeof(int)));
+  *timed_out = flag != 0;
+  return SBP_OK;
+}
+
+}  // namespace sbp
+
+extern "C" sbp_status sbp_check_device_errors(void) {
+  bool timed_out = false;
+  sbp_status st = sbp::read_and_clear_bulk_timeout(&timed_out);
+  if (st != SBP_OK) return st;
+  if (timed_out) return sbp::fail(SBP_ERR_TIMEOUT, "a bulk-copy boxing kernel gave up waiting for its loads");
+  return SBP_OK;
+}

@@ -1,0 +1,30 @@
+// Parameter block shared by the two boxing copy engines (host + device, this library only).
+#pragma once
+
+#include "sbp.h"
+
+namespace sbp {
+
+enum BoxMode : int {
+  MODE_PAIRS = 0,      // task t: source shard t / k, destination shard t % k
+  MODE_DIAG = 1,       // task t: source shard t, destination shard t
+  MODE_GATHER = 2,     // task t: source shard t, every destination replica
+  MODE_REDUCE_S = 3,   // task t: all sources, destination shard t
+  MODE_REDUCE_B = 4    // one task: all sources, every destination replica
+};
+
+// The logical tensor is viewed as [A][Na][M][Nb][C] (elements); src_a/src_b/dst_a/dst_b say
+// which side's split signature restricts the axes Na and Nb.
+struct BoxParams {
+  const char* src[SBP_MAX_K];
+  char* dst[SBP_MAX_K];
+  long long A, Na, M, Nb, C;
+  long long tiles_per_task, col_tiles;
+  int k, esz, mode;
+  int src_a, src_b, dst_a, dst_b;
+  int n_dst;                        // distinct destination buffers (GATHER / REDUCE_B)
+  int cv_log2;                      // tile width in vectors, log2
+  int rows_per_tile;
+};
+
+}  // namespace sbp

@@ -1,0 +1,218 @@
+// Row-split embedding lookup (Section 6.3: table S(0), "splitting the vocabulary IDs").
+//
+//   unfused: shard r writes out_r[l,:] = table_r[id_l - start_r,:] when id_l lies in its own
+//            row range and zeros otherwise; the k outputs form a P(sum) tensor.
+//   fused:   the P(sum) -> B boxing folded into the gather.  Exactly one shard contributes
+//            to a lookup, so the sum over shards is that shard's row; the kernel finds the
+//            owning shard from the id, reads the row once and writes every B replica.
+//
+// One thread moves one 16-byte piece of a row (or one element on the unaligned path) for J
+// lookups; all id loads, then all row loads, are issued before the first store.
+#include <cuda_bf16.h>
+
+#include "sbp_internal.h"
+
+namespace sbp {
+
+struct EmbParams {
+  const char* table[SBP_MAX_K];
+  const long long* ids[SBP_MAX_K];
+  char* out[SBP_MAX_K];
+  long long rows;         // logical table rows
+  long long n_lookups;
+  long long vpr;          // vectors per row
+  int vpr_log2;           // >= 0 when vpr is a power of two, else -1
+  int k, esz;
+  int n_dst;              // fused: distinct replicas
+  int canon_neg_zero;     // fused and k > 1: write -0.0 as +0.0 (what x + 0 gives)
+  int* oob;
+};
+
+__host__ __device__ inline int owner_of_row(long long id, long long rows, int k, long long* start) {
+  const long long base = rows / k, rem = rows % k;
+  const long long big = rem * (base + 1);
+  int r;
+  if (id < big) {
+    r = (int)(id / (base + 1));
+    *start = r * (base + 1);
+  } else {
+    r = (int)(rem + (id - big) / base);
+    *start = big + (r - rem) * base;
+  }
+  return r;
+}
+
+template <typename V>
+__device__ __forceinline__ V zero_vec() {
+  V z;
+  unsigned char* b = reinterpret_cast<unsigned char*>(&z);
+#pragma unroll
+  for (int i = 0; i < (int)sizeof(V); ++i) b[i] = 0;
+  return z;
+}
+
+// Replaces every -0.0 lane by +0.0.  ESZ = 4 (fp32) or 2 (bf16).
+template <typename V, int ESZ>
+__device__ __forceinline__ V canon(V v) {
+  if (ESZ == 4) {
+    uint32_t* w = reinterpret_cast<uint32_t*>(&v);
+#pragma unroll
+    for (int i = 0; i < (int)(sizeof(V) / 4); ++i)
+      if (w[i] == 0x80000000u) w[i] = 0;
+  } else {
+    uint16_t* h = reinterpret_cast<uint16_t*>(&v);
+#pragma unroll
+    for (int i = 0; i < (int)(sizeof(V) / 2); ++i)
+      if (h[i] == 0x8000u) h[i] = 0;
+  }
+  return v;
+}
+
+template <typename V, int ESZ, int J, bool FUSED>
+__global__ void __launch_bounds__(256) embedding_kernel(const __grid_constant__ EmbParams p) {
+  const long long total = p.n_lookups * p.vpr;
+  const long long stride = (long long)gridDim.x * 256;
+  const long long base = (long long)blockIdx.x * 256 + threadIdx.x;
+  const int shard = FUSED ? 0 : blockIdx.y;
+
+  long long item[J], look[J], col[J], id[J];
+  bool ok[J];
+#pragma unroll
+  for (int j = 0; j < J; ++j) {
+    item[j] = base + j * stride;
+    ok[j] = item[j] < total;
+    if (p.vpr_log2 >= 0) {
+      look[j] = item[j] >> p.vpr_log2;
+      col[j] = item[j] & (p.vpr - 1);
+    } else {
+      look[j] = item[j] / p.vpr;
+      col[j] = item[j] - look[j] * p.vpr;
+    }
+  }
+#pragma unroll
+  for (int j = 0; j < J; ++j) id[j] = ok[j] ? __ldg(p.ids[shard] + look[j]) : 0;
+
+  V val[J];
+#pragma unroll
+  for (int j = 0; j < J; ++j) {
+    val[j] = zero_vec<V>();
+    if (!ok[j]) continue;
+    const bool in_table = id[j] >= 0 && id[j] < p.rows;
+    if (!in_table) {
+      if (p.oob && col[j] == 0 && shard == 0) atomicAdd(p.oob, 1);
+      continue;
+    }
+    long long start;
+    const int r = owner_of_row(id[j], p.rows, p.k, &start);
+    if (FUSED || r == shard)
+      val[j] = __ldg(reinterpret_cast<const V*>(p.table[r]) + (id[j] - start) * p.vpr + col[j]);
+  }
+
+  if (FUSED) {
+    for (int q = 0; q < p.n_dst; ++q) {
+      V* o = reinterpret_cast<V*>(p.out[q]);
+#pragma unroll
+      for (int j = 0; j < J; ++j)
+        if (ok[j]) o[item[j]] = p.canon_neg_zero ? canon<V, ESZ>(val[j]) : val[j];
+    }
+  } else {
+    V* o = reinterpret_cast<V*>(p.out[shard]);
+#pragma unroll
+    for (int j = 0; j < J; ++j)
+      if (ok[j]) o[item[j]] = val[j];
+  }
+}
+
+template <typename V, int ESZ>
+static void launch_emb(const EmbParams& p, bool fused, cudaStream_t st) {
+  constexpr int J = 4;
+  const long long total = p.n_lookups * p.vpr;
+  long long blocks = (total + 256LL * J - 1) / (256LL * J);
+  if (blocks < 1) blocks = 1;
+  if (fused) {
+    embedding_kernel<V, ESZ, J, true><<<dim3((unsigned)blocks), 256, 0, st>>>(p);
+  } else {
+    embedding_kernel<V, ESZ, J, false><<<dim3((unsigned)blocks, p.k), 256, 0, st>>>(p);
+  }
+}
+
+}  // namespace sbp
+
+using namespace sbp;
+
+extern "C" sbp_status sbp_embedding(const sbp_tensor* table, const sbp_tensor* ids, sbp_tensor* out,
+                                    int32_t* oob_count, void* cuda_stream) {
+  sbp_status st = check_tensor(table, "table", true);
+  if (st != SBP_OK) return st;
+  st = check_tensor(ids, "ids", true);
+  if (st != SBP_OK) return st;
+  st = check_tensor(out, "out", true);
+  if (st != SBP_OK) return st;
+  if (table->ndim != 2) return fail(SBP_ERR_SHAPE, "table must be [rows, dim]");
+  if (table->dtype != SBP_F32 && table->dtype != SBP_BF16) return fail(SBP_ERR_DTYPE, "table must be F32 or BF16");
+  if (out->dtype != table->dtype) return fail(SBP_ERR_DTYPE, "out and table differ in dtype");
+  if (ids->dtype != SBP_I64) return fail(SBP_ERR_DTYPE, "ids must be I64");
+  if (ids->ndim > 3) return fail(SBP_ERR_SHAPE, "ids rank %d > 3", ids->ndim);
+  if (out->ndim != ids->ndim + 1) return fail(SBP_ERR_SHAPE, "out rank must be ids rank + 1");
+  for (int d = 0; d < ids->ndim; ++d)
+    if (out->shape[d] != ids->shape[d]) return fail(SBP_ERR_SHAPE, "out and ids differ on axis %d", d);
+  if (out->shape[out->ndim - 1] != table->shape[1]) return fail(SBP_ERR_SHAPE, "out's last axis must equal dim");
+  const int k = placement_k(table);
+  if (placement_k(ids) != k || placement_k(out) != k) return fail(SBP_ERR_INVALID_ARG, "operands differ in k");
+  if (!(table->sbp[0].kind == SBP_SPLIT && table->sbp[0].axis == 0))
+    return fail(table->sbp[0].kind == SBP_SPLIT ? SBP_ERR_UNSUPPORTED : SBP_ERR_SIGNATURE,
+                "table must be S(0) (a table split along the hidden axis is not implemented)");
+  if (ids->sbp[0].kind != SBP_BROADCAST) return fail(SBP_ERR_SIGNATURE, "ids must be B");
+  const bool fused = out->sbp[0].kind == SBP_BROADCAST;
+  if (!fused && out->sbp[0].kind != SBP_PARTIAL_SUM)
+    return fail(SBP_ERR_SIGNATURE, "out must be P(sum) (unfused) or B (boxing fused into the gather)");
+  const long long n_lookups = numel(ids);
+  if (n_lookups == 0 || table->shape[1] == 0) return SBP_OK;
+
+  EmbParams p{};
+  p.k = k;
+  p.esz = elem_size(table->dtype);
+  p.rows = table->shape[0];
+  p.n_lookups = n_lookups;
+  p.oob = oob_count;
+  const long long row_bytes = table->shape[1] * p.esz;
+  int vb = 16;
+  for (; vb > p.esz; vb >>= 1) {
+    bool ok = row_bytes % vb == 0;
+    for (int r = 0; r < k && ok; ++r)
+      ok = reinterpret_cast<uintptr_t>(table->local[r]) % vb == 0 && reinterpret_cast<uintptr_t>(out->local[r]) % vb == 0;
+    if (ok) break;
+  }
+  p.vpr = row_bytes / vb;
+  p.vpr_log2 = -1;
+  for (int b = 0; b < 40; ++b)
+    if ((1LL << b) == p.vpr) p.vpr_log2 = b;
+  for (int r = 0; r < k; ++r) {
+    p.table[r] = static_cast<const char*>(table->local[r]);
+    p.ids[r] = static_cast<const long long*>(ids->local[r]);
+    p.out[r] = static_cast<char*>(out->local[r]);
+  }
+  if (fused) {
+    p.canon_neg_zero = k > 1;
+    char* uniq[SBP_MAX_K];
+    for (int r = 0; r < k; ++r) {
+      bool seen = false;
+      for (int q = 0; q < p.n_dst; ++q) seen = seen || uniq[q] == p.out[r];
+      if (!seen) uniq[p.n_dst++] = p.out[r];
+    }
+    for (int q = 0; q < p.n_dst; ++q) p.out[q] = uniq[q];
+  }
+  if ((n_lookups * p.vpr + 1023) / 1024 > 0x7fffffffLL) return fail(SBP_ERR_UNSUPPORTED, "too many lookups for one launch");
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const bool f32 = table->dtype == SBP_F32;
+  switch (vb) {
+    case 16: f32 ? launch_emb<uint4, 4>(p, fused, stream) : launch_emb<uint4, 2>(p, fused, stream); break;
+    case 8: f32 ? launch_emb<uint2, 4>(p, fused, stream) : launch_emb<uint2, 2>(p, fused, stream); break;
+    case 4: f32 ? launch_emb<uint32_t, 4>(p, fused, stream) : launch_emb<uint32_t, 2>(p, fused, stream); break;
+    default: launch_emb<uint16_t, 2>(p, fused, stream); break;
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "embedding launch");
+  count_launch();
+  return SBP_OK;
+}

@@ -1,0 +1,259 @@
+// MatMul under the SBP signatures of Table 1: signature rule -> grouped-GEMM plan -> kernel.
+//
+// Two kernels execute a plan:
+//   * the tensor-core kernel (matmul_tc.cu): bf16 operands, fp32 accumulation in tensor
+//     memory, TMA-fed tiles; taken whenever the shapes meet its alignment rules;
+//   * the FMA kernel in this file: fp32 operands (and bf16 operands whose shapes the tensor
+//     core kernel cannot take), fp32 accumulation with fused multiply-adds, k ascending.
+#include <cuda_bf16.h>
+
+#include "matmul_plan.h"
+#include "sbp_internal.h"
+
+namespace sbp {
+
+// Defined in matmul_tc.cu.  Returns SBP_ERR_UNSUPPORTED (without touching the error text)
+// when the plan does not meet the tensor-core kernel's rules; the caller then falls back
+// to the FMA kernel.
+sbp_status launch_matmul_tc(const MatmulPlan& plan, void* ws, size_t ws_bytes, cudaStream_t st, bool* taken);
+size_t matmul_tc_workspace_bytes(const MatmulPlan& plan);
+
+__device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f)); }
+
+template <typename T>
+__device__ __forceinline__ float ld_f32(const T* p);
+template <>
+__device__ __forceinline__ float ld_f32<float>(const float* p) { return *p; }
+template <>
+__device__ __forceinline__ float ld_f32<__nv_bfloat16>(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+
+template <typename T>
+__device__ __forceinline__ void st_out(T* p, float v);
+template <>
+__device__ __forceinline__ void st_out<float>(float* p, float v) { *p = v; }
+template <>
+__device__ __forceinline__ void st_out<__nv_bfloat16>(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+constexpr int BM = 64, BN = 64, BK = 16;
+
+template <typename TI, typename TO>
+__global__ void __launch_bounds__(256) matmul_fma_kernel(const __grid_constant__ MatmulPlan p) {
+  const int g = blockIdx.z;
+  const long long M = p.m[g], N = p.n[g];
+  const long long m0 = (long long)blockIdx.y * BM, n0 = (long long)blockIdx.x * BN;
+  if (m0 >= M || n0 >= N) return;
+  __shared__ float As[BK][BM + 1];
+  __shared__ float Bs[BK][BN + 1];
+  const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+  float acc[4][4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) acc[i][j] = 0.f;
+
+  const int s_lo = p.chain ? 0 : g, s_hi = p.chain ? p.nseg : g + 1;
+  for (int s = s_lo; s < s_hi; ++s) {
+    const TI* A = static_cast<const TI*>(p.a[s]) + (p.row_off[g] + m0) * p.lda[s];
+    const TI* Bm = static_cast<const TI*>(p.b[s]) + p.col_off[g] + n0;
+    const long long K = p.kseg[s];
+    for (long long k0 = 0; k0 < K; k0 += BK) {
+      for (int e = threadIdx.x; e < BM * BK; e += 256) {
+        const int r = e / BK, c = e % BK;
+        As[c][r] = (m0 + r < M && k0 + c < K) ? ld_f32<TI>(A + (long long)r * p.lda[s] + k0 + c) : 0.f;
+      }
+      for (int e = threadIdx.x; e < BK * BN; e += 256) {
+        const int r = e / BN, c = e % BN;
+        Bs[r][c] = (k0 + r < K && n0 + c < N) ? ld_f32<TI>(Bm + (k0 + r) * p.ldb[s] + c) : 0.f;
+      }
+      __syncthreads();
+#pragma unroll
+      for (int kk = 0; kk < BK; ++kk) {
+        float a[4], b[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) a[i] = As[kk][ty * 4 + i];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) b[j] = Bs[kk][tx * 4 + j];
+#pragma unroll
+        for (int i = 0; i < 4; ++i)
+#pragma unroll
+          for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+      }
+      __syncthreads();
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const long long r = m0 + ty * 4 + i;
+    if (r >= M) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const long long c = n0 + tx * 4 + j;
+      if (c >= N) continue;
+      float v = acc[i][j];
+      if (p.gelu) v = gelu_erf(v);
+      st_out<TO>(static_cast<TO*>(p.y[g]) + r * p.ldy[g] + c, v);
+      if (g == 0)
+        for (int q = 0; q < p.n_rep; ++q) st_out<TO>(static_cast<TO*>(p.y_rep[q]) + r * p.ldy[g] + c, v);
+    }
+  }
+}
+
+static sbp_status launch_fma(const MatmulPlan& p, cudaStream_t st) {
+  long long mmax = 0, nmax = 0;
+  for (int g = 0; g < p.ngroups; ++g) {
+    mmax = p.m[g] > mmax ? p.m[g] : mmax;
+    nmax = p.n[g] > nmax ? p.n[g] : nmax;
+  }
+  if (mmax == 0 || nmax == 0) return SBP_OK;
+  const long long gx = (nmax + BN - 1) / BN, gy = (mmax + BM - 1) / BM;
+  if (gx > 0x7fffffffLL || gy > 65535) return fail(SBP_ERR_UNSUPPORTED, "matrix too large for the FMA kernel");
+  dim3 grid((unsigned)gx, (unsigned)gy, (unsigned)p.ngroups);
+  if (p.in_dtype == SBP_F32 && p.out_dtype == SBP_F32)
+    matmul_fma_kernel<float, float><<<grid, 256, 0, st>>>(p);
+  else if (p.in_dtype == SBP_BF16 && p.out_dtype == SBP_BF16)
+    matmul_fma_kernel<__nv_bfloat16, __nv_bfloat16><<<grid, 256, 0, st>>>(p);
+  else if (p.in_dtype == SBP_BF16 && p.out_dtype == SBP_F32)
+    matmul_fma_kernel<__nv_bfloat16, float><<<grid, 256, 0, st>>>(p);
+  else
+    return fail(SBP_ERR_DTYPE, "F32 operands need an F32 result");
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "matmul launch");
+  count_launch();
+  return SBP_OK;
+}
+
+static bool is_s(sbp_sig s, int ax) { return s.kind == SBP_SPLIT && s.axis == ax; }
+static bool is_b(sbp_sig s) { return s.kind == SBP_BROADCAST; }
+static bool is_p(sbp_sig s) { return s.kind == SBP_PARTIAL_SUM; }
+
+// Validates the three descriptors and fills the plan.  need_ptrs = false for size queries.
+static sbp_status build_plan(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y, uint32_t flags,
+                             bool need_ptrs, MatmulPlan* plan) {
+  sbp_status st = check_tensor(x, "x", need_ptrs);
+  if (st != SBP_OK) return st;
+  st = check_tensor(w, "w", need_ptrs);
+  if (st != SBP_OK) return st;
+  st = check_tensor(y, "y", need_ptrs);
+  if (st != SBP_OK) return st;
+  if (x->ndim != 2 || w->ndim != 2 || y->ndim != 2) return fail(SBP_ERR_SHAPE, "x, w and y must be 2-D");
+  const long long M = x->shape[0], K = x->shape[1], N = w->shape[1];
+  if (w->shape[0] != K) return fail(SBP_ERR_SHAPE, "x is [%lld,%lld] but w has %lld rows", M, K, (long long)w->shape[0]);
+  if (y->shape[0] != M || y->shape[1] != N) return fail(SBP_ERR_SHAPE, "y must be [%lld,%lld]", M, N);
+  if (x->dtype != w->dtype) return fail(SBP_ERR_DTYPE, "x and w differ in dtype");
+  if (x->dtype != SBP_F32 && x->dtype != SBP_BF16) return fail(SBP_ERR_DTYPE, "operands must be F32 or BF16");
+  if (y->dtype != SBP_F32 && y->dtype != SBP_BF16) return fail(SBP_ERR_DTYPE, "y must be F32 or BF16");
+  if (x->dtype == SBP_F32 && y->dtype != SBP_F32) return fail(SBP_ERR_DTYPE, "F32 operands need an F32 result");
+  const int k = placement_k(x);
+  if (placement_k(w) != k || placement_k(y) != k) return fail(SBP_ERR_INVALID_ARG, "operands differ in k");
+
+  const sbp_sig xs = x->sbp[0], ws = w->sbp[0], ys = y->sbp[0];
+  sbp_sig natural;
+  st = sbp_matmul_infer(xs, ws, &natural);
+  if (st != SBP_OK) return st;
+  const bool fused = is_p(natural) && !is_p(ys);
+  if (!fused && !same_sig(natural, ys))
+    return fail(SBP_ERR_SIGNATURE, "y's signature is neither the one Table 1 deduces nor a fusable boxing of it");
+  if (fused && !(is_b(ys) || ys.kind == SBP_SPLIT))
+    return fail(SBP_ERR_SIGNATURE, "a P(sum) product can be written directly only as B or S(i)");
+  if ((flags & SBP_EPILOGUE_GELU) && is_p(natural) && !fused)
+    return fail(SBP_ERR_SIGNATURE, "GeLU is not linear: it cannot be applied to partial values");
+  if (flags & ~SBP_EPILOGUE_GELU) return fail(SBP_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
+
+  MatmulPlan& p = *plan;
+  p = MatmulPlan{};
+  p.gelu = (flags & SBP_EPILOGUE_GELU) ? 1 : 0;
+  p.in_dtype = x->dtype;
+  p.out_dtype = y->dtype;
+
+  auto range = [&](long long n, int r, long long* start, long long* len) {
+    int64_t s_, l_;
+    split_range(n, k, r, &s_, &l_);
+    *start = s_;
+    *len = l_;
+  };
+  // K-segments = the local operands of each shard
+  for (int r = 0; r < k; ++r) {
+    long long st_, ln;
+    p.a[r] = x->local[r];
+    p.b[r] = w->local[r];
+    p.lda[r] = K;
+    p.ldb[r] = N;
+    p.kseg[r] = K;
+    if (is_s(xs, 1)) { range(K, r, &st_, &ln); p.lda[r] = ln; p.kseg[r] = ln; }
+    if (is_s(ws, 1)) { range(N, r, &st_, &ln); p.ldb[r] = ln; }
+  }
+  p.nseg = k;
+
+  auto set_replicas = [&]() {   // one group, stored to every distinct B replica
+    p.ngroups = 1;
+    p.m[0] = M; p.n[0] = N; p.ldy[0] = N;
+    void* uniq[SBP_MAX_K];
+    int nu = 0;
+    for (int r = 0; r < k; ++r) {
+      bool seen = false;
+      for (int q = 0; q < nu; ++q) seen = seen || uniq[q] == y->local[r];
+      if (!seen) uniq[nu++] = y->local[r];
+    }
+    p.y[0] = uniq[0];
+    p.n_rep = nu - 1;
+    for (int q = 1; q < nu; ++q) p.y_rep[q - 1] = uniq[q];
+  };
+
+  if (!fused) {
+    p.chain = 0;
+    if (is_b(natural)) {
+      p.nseg = 1;
+      set_replicas();
+    } else {
+      p.ngroups = k;
+      for (int g = 0; g < k; ++g) {
+        long long st_, ln;
+        p.m[g] = M; p.n[g] = N; p.ldy[g] = N;
+        if (is_s(natural, 0)) { range(M, g, &st_, &ln); p.m[g] = ln; }
+        if (is_s(natural, 1)) { range(N, g, &st_, &ln); p.n[g] = ln; p.ldy[g] = ln; }
+        p.y[g] = y->local[g];
+      }
+    }
+  } else {
+    p.chain = 1;
+    if (is_b(ys)) {
+      set_replicas();
+    } else {
+      p.ngroups = k;
+      for (int g = 0; g < k; ++g) {
+        long long st_, ln;
+        p.m[g] = M; p.n[g] = N; p.ldy[g] = N;
+        if (ys.axis == 0) { range(M, g, &st_, &ln); p.m[g] = ln; p.row_off[g] = st_; }
+        else { range(N, g, &st_, &ln); p.n[g] = ln; p.col_off[g] = st_; p.ldy[g] = ln; }
+        p.y[g] = y->local[g];
+      }
+    }
+  }
+  return SBP_OK;
+}
+
+}  // namespace sbp
+
+using namespace sbp;
+
+extern "C" {
+
+size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y) {
+  MatmulPlan plan;
+  if (build_plan(x, w, y, 0, false, &plan) != SBP_OK) return 0;
+  return matmul_tc_workspace_bytes(plan);
+}
+
+sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, uint32_t flags, void* ws,
+                      size_t ws_bytes, void* cuda_stream) {
+  MatmulPlan plan;
+  sbp_status st = build_plan(x, w, y, flags, true, &plan);
+  if (st != SBP_OK) return st;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  bool taken = false;
+  st = launch_matmul_tc(plan, ws, ws_bytes, stream, &taken);
+  if (taken) return st;
+  return launch_fma(plan, stream);
+}
+
+}  // extern "C"

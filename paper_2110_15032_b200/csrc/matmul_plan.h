@@ -1,0 +1,37 @@
+// Grouped-GEMM plan shared by the MatMul kernels of this library (host + device).
+//
+// Every MatMul signature of Table 1 -- and every fused "P(sum) result written directly as
+// B or S(i)" variant -- is a list of independent output groups; a group's result is the sum
+// over one or more K-segments, taken in segment order:
+//
+//   Y_g[M_g, N_g] = sum_{s in segs(g)}  A_s[row_off_g : row_off_g + M_g, 0 : K_s]
+//                                     * B_s[0 : K_s, col_off_g : col_off_g + N_g]
+//
+//   unfused (chain == 0): segs(g) = {g}       one local product per shard
+//   fused   (chain == 1): segs(g) = {0..nseg-1}  the partial products of all shards are
+//                                              accumulated in rank order in the accumulator
+#pragma once
+
+#include <cstdint>
+
+#include "sbp.h"
+
+namespace sbp {
+
+struct MatmulPlan {
+  // per K-segment (= per source shard)
+  const void* a[SBP_MAX_K];
+  const void* b[SBP_MAX_K];
+  long long lda[SBP_MAX_K], ldb[SBP_MAX_K], kseg[SBP_MAX_K];
+  // per output group
+  long long m[SBP_MAX_K], n[SBP_MAX_K], row_off[SBP_MAX_K], col_off[SBP_MAX_K], ldy[SBP_MAX_K];
+  void* y[SBP_MAX_K];
+  // extra destinations of group 0 when one result is stored to several B replicas
+  void* y_rep[SBP_MAX_K];
+  int n_rep;
+  int ngroups, nseg, chain;
+  int gelu;
+  int in_dtype, out_dtype;   // sbp_dtype
+};
+
+}  // namespace sbp

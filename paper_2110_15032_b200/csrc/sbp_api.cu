@@ -1,0 +1,132 @@
+// Descriptor checks, the MatMul signature rule (Table 1) and error reporting.
+#include <atomic>
+#include <cstring>
+
+#include "sbp_internal.h"
+
+namespace sbp {
+
+static thread_local char g_err[512] = "";
+static std::atomic<uint64_t> g_launches{0};
+
+sbp_status fail(sbp_status s, const char* fmt, ...) {
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(g_err, sizeof(g_err), fmt, ap);
+  va_end(ap);
+  return s;
+}
+
+void count_launch(uint64_t n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+sbp_status cuda_fail(cudaError_t e, const char* what) {
+  return fail(SBP_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
+}
+
+sbp_status check_tensor(const sbp_tensor* t, const char* name, bool need_ptrs) {
+  if (!t) return fail(SBP_ERR_INVALID_ARG, "%s: null descriptor", name);
+  if (t->ndim < 1 || t->ndim > SBP_MAX_DIMS)
+    return fail(SBP_ERR_INVALID_ARG, "%s: ndim %d outside [1,%d]", name, t->ndim, SBP_MAX_DIMS);
+  if (elem_size(t->dtype) == 0) return fail(SBP_ERR_DTYPE, "%s: unknown dtype %d", name, t->dtype);
+  for (int d = 0; d < t->ndim; ++d)
+    if (t->shape[d] < 0) return fail(SBP_ERR_SHAPE, "%s: negative extent on axis %d", name, d);
+  if (t->pdims < 1 || t->pdims > SBP_MAX_PDIMS)
+    return fail(SBP_ERR_INVALID_ARG, "%s: pdims %d outside [1,%d]", name, t->pdims, SBP_MAX_PDIMS);
+  for (int p = 0; p < t->pdims; ++p)
+    if (t->pshape[p] < 1) return fail(SBP_ERR_INVALID_ARG, "%s: placement extent < 1", name);
+  int k = placement_k(t);
+  if (k > SBP_MAX_K) return fail(SBP_ERR_INVALID_ARG, "%s: k = %d exceeds %d", name, k, SBP_MAX_K);
+  if (t->pdims != 1)
+    return fail(SBP_ERR_UNSUPPORTED, "%s: multi-dimensional SBP (pdims = %d) is not implemented", name,
+                t->pdims);
+  sbp_sig s = t->sbp[0];
+  if (s.kind < SBP_SPLIT || s.kind > SBP_PARTIAL_MAX)
+    return fail(SBP_ERR_SIGNATURE, "%s: unknown sbp kind %d", name, s.kind);
+  if (s.kind == SBP_SPLIT && (s.axis < 0 || s.axis >= t->ndim))
+    return fail(SBP_ERR_SIGNATURE, "%s: split axis %d outside [0,%d)", name, s.axis, t->ndim);
+  if (need_ptrs) {
+    for (int r = 0; r < k; ++r) {
+      if (!t->local[r] && local_numel(t, r) > 0)
+        return fail(SBP_ERR_INVALID_ARG, "%s: local[%d] is null", name, r);
+      if (reinterpret_cast<uintptr_t>(t->local[r]) % elem_size(t->dtype) != 0)
+        return fail(SBP_ERR_ALIGNMENT, "%s: local[%d] is not aligned to its element size", name, r);
+    }
+  }
+  return SBP_OK;
+}
+
+int64_t local_numel(const sbp_tensor* t, int r) {
+  int k = placement_k(t);
+  int64_t n = 1;
+  for (int d = 0; d < t->ndim; ++d) {
+    int64_t e = t->shape[d];
+    if (t->sbp[0].kind == SBP_SPLIT && t->sbp[0].axis == d) {
+      int64_t st;
+      split_range(t->shape[d], k, r, &st, &e);
+    }
+    n *= e;
+  }
+  return n;
+}
+
+}  // namespace sbp
+
+using namespace sbp;
+
+extern "C" {
+
+const char* sbp_status_string(sbp_status s) {
+  switch (s) {
+    case SBP_OK: return "SBP_OK";
+    case SBP_ERR_INVALID_ARG: return "SBP_ERR_INVALID_ARG";
+    case SBP_ERR_SHAPE: return "SBP_ERR_SHAPE";
+    case SBP_ERR_DTYPE: return "SBP_ERR_DTYPE";
+    case SBP_ERR_SIGNATURE: return "SBP_ERR_SIGNATURE";
+    case SBP_ERR_UNSUPPORTED: return "SBP_ERR_UNSUPPORTED";
+    case SBP_ERR_ALIGNMENT: return "SBP_ERR_ALIGNMENT";
+    case SBP_ERR_WORKSPACE: return "SBP_ERR_WORKSPACE";
+    case SBP_ERR_CUDA: return "SBP_ERR_CUDA";
+    case SBP_ERR_TIMEOUT: return "SBP_ERR_TIMEOUT";
+  }
+  return "SBP_ERR_?";
+}
+
+const char* sbp_last_error(void) { return g_err; }
+
+uint64_t sbp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+sbp_status sbp_local_shape(const sbp_tensor* t, int32_t r, int64_t out_shape[SBP_MAX_DIMS]) {
+  sbp_status st = check_tensor(t, "t", false);
+  if (st != SBP_OK) return st;
+  if (!out_shape) return fail(SBP_ERR_INVALID_ARG, "out_shape is null");
+  int k = placement_k(t);
+  if (r < 0 || r >= k) return fail(SBP_ERR_INVALID_ARG, "shard %d outside [0,%d)", r, k);
+  for (int d = 0; d < SBP_MAX_DIMS; ++d) out_shape[d] = d < t->ndim ? t->shape[d] : 1;
+  if (t->sbp[0].kind == SBP_SPLIT) {
+    int64_t start, len;
+    split_range(t->shape[t->sbp[0].axis], k, r, &start, &len);
+    out_shape[t->sbp[0].axis] = len;
+  }
+  return SBP_OK;
+}
+
+sbp_status sbp_matmul_infer(sbp_sig x, sbp_sig w, sbp_sig* y) {
+  if (!y) return fail(SBP_ERR_INVALID_ARG, "y is null");
+  auto is_s = [](sbp_sig s, int ax) { return s.kind == SBP_SPLIT && s.axis == ax; };
+  auto is_b = [](sbp_sig s) { return s.kind == SBP_BROADCAST; };
+  auto is_p = [](sbp_sig s) { return s.kind == SBP_PARTIAL_SUM; };
+  sbp_sig out = {SBP_BROADCAST, 0};
+  if (is_s(x, 0) && is_b(w)) out = {SBP_SPLIT, 0};            // data parallelism
+  else if (is_b(x) && is_s(w, 1)) out = {SBP_SPLIT, 1};       // model parallelism
+  else if (is_s(x, 1) && is_s(w, 0)) out = {SBP_PARTIAL_SUM, 0};
+  else if (is_p(x) && is_b(w)) out = {SBP_PARTIAL_SUM, 0};
+  else if (is_b(x) && is_p(w)) out = {SBP_PARTIAL_SUM, 0};
+  else if (is_b(x) && is_b(w)) out = {SBP_BROADCAST, 0};
+  else
+    return fail(SBP_ERR_SIGNATURE, "(kind %d axis %d) x (kind %d axis %d) is not a valid MatMul signature",
+                x.kind, x.axis, w.kind, w.axis);
+  *y = out;
+  return SBP_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,65 @@
+// Internal helpers shared by the library's translation units (host side only).
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <cstdarg>
+#include <cstdint>
+#include <cstdio>
+
+#include "sbp.h"
+
+namespace sbp {
+
+// Records the detail string returned by sbp_last_error() and passes the status through.
+sbp_status fail(sbp_status s, const char* fmt, ...);
+void count_launch(uint64_t n = 1);
+
+inline int elem_size(int32_t dtype) {
+  switch (dtype) {
+    case SBP_F32: return 4;
+    case SBP_BF16: return 2;
+    case SBP_I64: return 8;
+    default: return 0;
+  }
+}
+
+// Balanced split (Section 3.1): start and length of shard r's piece of an axis of length n.
+__host__ __device__ inline void split_range(int64_t n, int k, int r, int64_t* start, int64_t* len) {
+  int64_t base = n / k, rem = n % k;
+  *len = base + (r < rem ? 1 : 0);
+  *start = r * base + (r < rem ? r : rem);
+}
+
+inline int placement_k(const sbp_tensor* t) {
+  int k = 1;
+  for (int p = 0; p < t->pdims; ++p) k *= t->pshape[p];
+  return k;
+}
+
+inline bool same_sig(sbp_sig a, sbp_sig b) {
+  return a.kind == b.kind && (a.kind != SBP_SPLIT || a.axis == b.axis);
+}
+
+// Full validation of a descriptor (rank, dtype, placement, signature, pointers).
+// need_ptrs: every local[r], r < k, must be non-null and aligned to the element size.
+sbp_status check_tensor(const sbp_tensor* t, const char* name, bool need_ptrs);
+
+inline int64_t numel(const sbp_tensor* t) {
+  int64_t n = 1;
+  for (int d = 0; d < t->ndim; ++d) n *= t->shape[d];
+  return n;
+}
+
+// Elements of shard r's local tensor.
+int64_t local_numel(const sbp_tensor* t, int r);
+
+sbp_status cuda_fail(cudaError_t e, const char* what);
+
+#define SBP_CUDA_TRY(expr)                                   \
+  do {                                                       \
+    cudaError_t _e = (expr);                                 \
+    if (_e != cudaSuccess) return ::sbp::cuda_fail(_e, #expr); \
+  } while (0)
+
+}  // namespace sbp

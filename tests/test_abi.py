@@ -1,0 +1,184 @@
+"""CPU-side checks of the C ABI: the library loads, exports every declared symbol, and its
+host logic (local shapes, the MatMul signature rule, argument validation) is right.
+No kernel is launched here."""
+import ctypes as C
+import os
+import re
+
+import pytest
+import torch
+from conftest import ROOT, read_golden
+
+import paper_2110_15032_b200 as sbp
+from paper_2110_15032_b200 import binding
+from oracle import sbp_oracle as O
+
+
+@pytest.fixture(scope="module")
+def lib():
+    from paper_2110_15032_b200.build import build
+    build()
+    return sbp.load_library()
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "sbp.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(sbp_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(lib):
+    names = _declared_functions()
+    assert len(names) >= 15
+    for n in names:
+        assert hasattr(lib, n), f"{n} is declared in include/sbp.h but not exported"
+
+
+def test_struct_layout_matches_header(lib):
+    # ndim,dtype (8) + shape (32) + pdims (4) + pshape (8) + sbp (16) + pad (4) + local (128)
+    assert C.sizeof(binding._Tensor) == 8 + 32 + 4 + 8 + 16 + 4 + 128
+    assert binding._Tensor.local.offset % 8 == 0
+
+
+def test_status_strings(lib):
+    assert lib.sbp_status_string(0) == b"SBP_OK"
+    assert lib.sbp_status_string(4) == b"SBP_ERR_SIGNATURE"
+    assert lib.sbp_status_string(9) == b"SBP_ERR_TIMEOUT"
+
+
+@pytest.mark.parametrize("shape", [(64, 96), (7, 10), (5, 3, 9), (2, 3, 4, 5), (3,)])
+@pytest.mark.parametrize("k", [1, 2, 3, 4, 8, 16])
+def test_local_shape_matches_oracle_split(lib, shape, k):
+    for axis in range(len(shape)):
+        parts = O.balanced_split(shape[axis], k)
+        for r in range(k):
+            want = list(shape)
+            want[axis] = parts[r][1]
+            assert sbp.sbp_local_shape(shape, sbp.S(axis), k, r) == tuple(want)
+    for sig in (sbp.B, sbp.P_SUM, sbp.P_MAX):
+        assert sbp.sbp_local_shape(shape, sig, k, k - 1) == tuple(shape)
+
+
+def test_local_shape_rejects_bad_descriptors(lib):
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_local_shape((4, 4), sbp.S(2), 2, 0)
+    assert e.value.name == "SBP_ERR_SIGNATURE"
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_local_shape((4, 4), sbp.S(0), 2, 2)
+    assert e.value.name == "SBP_ERR_INVALID_ARG"
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_local_shape((4, 4), sbp.S(0), 17, 0)
+    assert e.value.name == "SBP_ERR_INVALID_ARG"
+
+
+def _sig(tok):
+    return {"S(0)": sbp.S(0), "S(1)": sbp.S(1), "B": sbp.B, "P(sum)": sbp.P_SUM}[tok]
+
+
+def test_matmul_infer_is_table1(lib):
+    valid = {(_sig(a), _sig(b)): _sig(c) for a, b, c in read_golden("table1_matmul_sbp.txt")}
+    sigs = [sbp.S(0), sbp.S(1), sbp.B, sbp.P_SUM, sbp.P_MAX]
+    rejected = 0
+    for xs in sigs:
+        for ws in sigs:
+            if (xs, ws) in valid:
+                assert sbp.sbp_matmul_infer(xs, ws) == valid[(xs, ws)]
+            else:
+                with pytest.raises(sbp.SbpError) as e:
+                    sbp.sbp_matmul_infer(xs, ws)
+                assert e.value.name == "SBP_ERR_SIGNATURE"
+                rejected += 1
+    assert rejected == 25 - 6
+
+
+def _host_tensor(shape, dtype, sig, k):
+    locs = [torch.zeros(sbp.sbp_local_shape(shape, sig, k, r, dtype), dtype=dtype) for r in range(k)]
+    return sbp.SbpTensor(shape, dtype, sig, locs)
+
+
+def _status(fn, *a):
+    try:
+        fn(*a)
+    except sbp.SbpError as e:
+        return e.name
+    return "SBP_OK"
+
+
+def test_boxing_validation_happens_before_any_launch(lib):
+    """Bad requests are refused on the host (so this runs without a GPU) and write nothing."""
+    stream = C.c_void_p(0)
+
+    def boxing(src, dst):
+        a, b = src._c(), dst._c()
+        binding._check(lib.sbp_boxing(C.byref(a), C.byref(b), stream))
+
+    f32, bf16, i64 = torch.float32, torch.bfloat16, torch.int64
+    src = _host_tensor((8, 8), f32, sbp.S(0), 2)
+    assert _status(boxing, src, _host_tensor((8, 9), f32, sbp.B, 2)) == "SBP_ERR_SHAPE"
+    assert _status(boxing, src, _host_tensor((8, 8), bf16, sbp.B, 2)) == "SBP_ERR_DTYPE"
+    assert _status(boxing, src, _host_tensor((8, 8), f32, sbp.B, 4)) == "SBP_ERR_INVALID_ARG"
+    assert _status(boxing, src, _host_tensor((8, 8), f32, sbp.P_SUM, 2)) == "SBP_ERR_UNSUPPORTED"
+    assert _status(boxing, _host_tensor((8, 8), f32, sbp.P_SUM, 2),
+                   _host_tensor((8, 8), f32, sbp.P_MAX, 2)) == "SBP_ERR_UNSUPPORTED"
+    assert _status(boxing, _host_tensor((8, 8), i64, sbp.P_SUM, 2),
+                   _host_tensor((8, 8), i64, sbp.B, 2)) == "SBP_ERR_DTYPE"
+    d = src._c()
+    d.pdims = 2
+    d.pshape[0], d.pshape[1] = 2, 1
+    b = _host_tensor((8, 8), f32, sbp.B, 2)._c()
+    assert lib.sbp_boxing(C.byref(d), C.byref(b), stream) == 5          # multi-dimensional SBP: unsupported
+    d = src._c()
+    d.local[1] = None
+    assert lib.sbp_boxing(C.byref(d), C.byref(b), stream) == 1          # null local tensor
+
+
+def test_matmul_validation(lib):
+    f32 = torch.float32
+
+    def mm(x, w, y, flags=0):
+        a, b, c = x._c(), w._c(), y._c()
+        binding._check(lib.sbp_matmul(C.byref(a), C.byref(b), C.byref(c), flags, None, 0, None))
+
+    k = 2
+    x = _host_tensor((8, 6), f32, sbp.S(0), k)
+    assert _status(mm, x, _host_tensor((6, 4), f32, sbp.S(0), k), _host_tensor((8, 4), f32, sbp.S(0), k)) == "SBP_ERR_SIGNATURE"
+    assert _status(mm, x, _host_tensor((5, 4), f32, sbp.B, k), _host_tensor((8, 4), f32, sbp.S(0), k)) == "SBP_ERR_SHAPE"
+    assert _status(mm, x, _host_tensor((6, 4), f32, sbp.B, k), _host_tensor((8, 4), f32, sbp.B, k)) == "SBP_ERR_SIGNATURE"
+    xs1 = _host_tensor((8, 6), f32, sbp.S(1), k)
+    ws0 = _host_tensor((6, 4), f32, sbp.S(0), k)
+    assert _status(mm, xs1, ws0, _host_tensor((8, 4), f32, sbp.P_SUM, k), sbp.SBP_EPILOGUE_GELU) == "SBP_ERR_SIGNATURE"
+    assert _status(mm, xs1, ws0, _host_tensor((8, 4), f32, sbp.P_MAX, k)) == "SBP_ERR_SIGNATURE"
+    assert _status(mm, xs1, ws0, _host_tensor((8, 4), torch.bfloat16, sbp.P_SUM, k)) == "SBP_ERR_DTYPE"
+
+
+def test_softmax_and_embedding_validation(lib):
+    f32, i64 = torch.float32, torch.int64
+    k = 2
+
+    def xent(logits, labels, loss):
+        a, b, c = logits._c(), labels._c(), loss._c()
+        binding._check(lib.sbp_softmax_xent(C.byref(a), C.byref(b), C.byref(c), None, None, None, 0, None))
+
+    labels = _host_tensor((4,), i64, sbp.B, k)
+    loss = _host_tensor((4,), f32, sbp.B, k)
+    assert _status(xent, _host_tensor((4, 10), f32, sbp.S(0), k), labels, loss) == "SBP_ERR_SIGNATURE"
+    assert _status(xent, _host_tensor((4, 10), f32, sbp.S(1), k), _host_tensor((5,), i64, sbp.B, k), loss) == "SBP_ERR_SHAPE"
+    assert _status(xent, _host_tensor((4, 10), f32, sbp.S(1), k), labels, loss) == "SBP_ERR_WORKSPACE"
+    assert sbp.sbp_softmax_xent_workspace_bytes(_host_tensor((4, 10), f32, sbp.S(1), k)) >= 3 * k * 4 * 4
+
+    def emb(table, ids, out):
+        a, b, c = table._c(), ids._c(), out._c()
+        binding._check(lib.sbp_embedding(C.byref(a), C.byref(b), C.byref(c), None, None))
+
+    ids = _host_tensor((3, 2), i64, sbp.B, k)
+    assert _status(emb, _host_tensor((10, 4), f32, sbp.S(1), k), ids, _host_tensor((3, 2, 4), f32, sbp.B, k)) == "SBP_ERR_UNSUPPORTED"
+    assert _status(emb, _host_tensor((10, 4), f32, sbp.B, k), ids, _host_tensor((3, 2, 4), f32, sbp.B, k)) == "SBP_ERR_SIGNATURE"
+    assert _status(emb, _host_tensor((10, 4), f32, sbp.S(0), k), ids, _host_tensor((3, 2, 5), f32, sbp.B, k)) == "SBP_ERR_SHAPE"
+    assert _status(emb, _host_tensor((10, 4), f32, sbp.S(0), k), ids, _host_tensor((3, 2, 4), f32, sbp.S(0), k)) == "SBP_ERR_SIGNATURE"
+
+
+def test_missing_library_fails_loudly(monkeypatch, tmp_path):
+    monkeypatch.setattr(binding, "_LIB", None)
+    monkeypatch.setattr(binding, "lib_path", lambda: str(tmp_path / "libsbp_b200.so"))
+    with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
+        binding.load_library()

@@ -1,0 +1,203 @@
+"""Parity of the CUDA boxing kernels against the CPU oracle (Section 3.2, Table 2).
+
+Pure data movement must be bit-exact.  P(sum) reductions follow the same fixed-order fp32
+rule on both sides and are expected bit-equal; the asserted bar is 1e-6 relative plus an
+fp64 cross-check that is safe under cancellation.  P(max) is exact."""
+import numpy as np
+import pytest
+import torch
+from helpers import bits, make_global, np_bits, osig, split_cpu, storage_of, to_np
+
+import paper_2110_15032_b200 as sbp
+import sbp_datagen as dg
+from oracle import sbp_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+F32, BF16, I64 = torch.float32, torch.bfloat16, torch.int64
+
+
+def _source_locals(shape, dtype, sig, k, seed):
+    """CPU local tensors of a seeded global tensor under `sig`."""
+    if sig.kind in (2, 3):      # P: k independent shards
+        return [dg.normal(seed, r, shape, 0.0, 1.0, dtype) for r in range(k)]
+    if dtype == I64:
+        T = dg.integers(seed, 0, shape, -(1 << 40), 1 << 40)
+    else:
+        T = dg.normal(seed, 0, shape, 0.0, 1.0, dtype)
+    return split_cpu(T, sig, k)
+
+
+def _oracle_boxing(src_cpu, dtype, src_sig, dst_sig):
+    if dtype == I64:
+        arrs = [t.numpy() for t in src_cpu]
+    else:
+        arrs = [to_np(t) for t in src_cpu]
+    return O.boxing(arrs, osig(src_sig), osig(dst_sig), storage_of(dtype) if dtype != I64 else "f32")
+
+
+def _run(shape, dtype, src_sig, dst_sig, k, seed=1, engine=0, alias=False, offset_elems=0):
+    src_cpu = _source_locals(shape, dtype, src_sig, k, seed)
+    want = _oracle_boxing(src_cpu, dtype, src_sig, dst_sig)
+    if offset_elems:
+        # place every local tensor at an odd element offset inside a larger buffer
+        def shifted(t):
+            buf = torch.zeros(t.numel() + offset_elems + 8, dtype=t.dtype, device="cuda")
+            v = buf[offset_elems:offset_elems + t.numel()].view(t.shape)
+            v.copy_(t)
+            return v
+        src = sbp.SbpTensor(shape, dtype, src_sig, [shifted(t) for t in src_cpu])
+    else:
+        src = make_global(src_cpu, shape, dtype, src_sig)
+    dst = sbp.empty_global(shape, dtype, dst_sig, k, alias_replicas=alias)
+    for t in dst.locals:
+        t.view(torch.uint8).fill_(0xAB)
+    sbp.sbp_boxing_set_copy_engine(engine)
+    try:
+        sbp.sbp_boxing(src, dst)
+        torch.cuda.synchronize()
+        sbp.sbp_check_device_errors()
+    finally:
+        sbp.sbp_boxing_set_copy_engine(0)
+    assert len(want) == k
+    for r in range(k):
+        got = dst.locals[r]
+        assert tuple(got.shape) == tuple(want[r].shape), (r, got.shape, want[r].shape)
+        assert np.array_equal(bits(got), np_bits(want[r], dtype)), f"shard {r} differs"
+    return src_cpu, dst
+
+
+MOVES = [(sbp.S(0), sbp.B), (sbp.S(1), sbp.B), (sbp.S(0), sbp.S(1)), (sbp.S(1), sbp.S(0)),
+         (sbp.B, sbp.S(0)), (sbp.B, sbp.S(1)), (sbp.S(0), sbp.S(0)), (sbp.B, sbp.B)]
+REDUCES = [(sbp.P_SUM, sbp.B), (sbp.P_SUM, sbp.S(0)), (sbp.P_SUM, sbp.S(1)),
+           (sbp.P_MAX, sbp.B), (sbp.P_MAX, sbp.S(1)), (sbp.P_SUM, sbp.P_SUM)]
+
+
+@pytest.mark.parametrize("src_sig,dst_sig", MOVES + REDUCES)
+@pytest.mark.parametrize("k", [1, 2, 3, 4, 8])
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_boxing_2d_aligned_and_ragged(src_sig, dst_sig, k, dtype):
+    _run((64, 96), dtype, src_sig, dst_sig, k)           # config-1 result shape, aligned
+    _run((67, 101), dtype, src_sig, dst_sig, k)          # nothing divides: element-wise path
+    _run((130, 520), dtype, src_sig, dst_sig, k)         # several tiles and a ragged tail
+
+
+@pytest.mark.parametrize("src_sig,dst_sig", MOVES)
+def test_boxing_int64_moves(src_sig, dst_sig):
+    _run((33, 40), I64, src_sig, dst_sig, 4)
+
+
+@pytest.mark.parametrize("shape", [(6, 10, 16), (3, 5, 7, 8), (4, 9, 10), (40,)])
+@pytest.mark.parametrize("k", [2, 3, 4])
+def test_boxing_nd_every_axis_pair(shape, k):
+    nd = len(shape)
+    for i in range(nd):
+        _run(shape, F32, sbp.S(i), sbp.B, k)
+        _run(shape, BF16, sbp.B, sbp.S(i), k)
+        _run(shape, F32, sbp.P_SUM, sbp.S(i), k)
+        for j in range(nd):
+            if i != j:
+                _run(shape, F32, sbp.S(i), sbp.S(j), k)
+
+
+@pytest.mark.parametrize("src_sig,dst_sig", MOVES[:6])
+@pytest.mark.parametrize("k", [2, 4])
+def test_bulk_copy_engine_matches(src_sig, dst_sig, k):
+    _run((512, 1024), BF16, src_sig, dst_sig, k, engine=2)     # 512 B .. 2 KiB segments
+    _run((384, 8192), F32, src_sig, dst_sig, k, engine=2)      # segments above one stage
+    _run((250, 1000), F32, src_sig, dst_sig, k, engine=2)      # uneven shards where k = 4 leaves a tail
+    _run((67, 101), F32, src_sig, dst_sig, k, engine=2)        # unaligned: falls back to load/store
+
+
+def test_boxing_larger_than_one_wave():
+    _run((2048, 3072), BF16, sbp.P_SUM, sbp.B, 4)
+    _run((2048, 3072), BF16, sbp.S(0), sbp.S(1), 4)
+    _run((2048, 3072), BF16, sbp.S(0), sbp.S(1), 4, engine=2)
+    _run((2048, 3072), BF16, sbp.S(0), sbp.B, 4, engine=2)
+
+
+def test_boxing_unaligned_pointers_and_aliased_replicas():
+    _run((64, 96), F32, sbp.S(0), sbp.B, 2, offset_elems=1)
+    _run((64, 96), BF16, sbp.P_SUM, sbp.B, 4, offset_elems=3)
+    _run((64, 96), BF16, sbp.S(0), sbp.S(1), 4, offset_elems=1)
+    _, dst = _run((64, 96), F32, sbp.P_SUM, sbp.B, 4, alias=True)
+    assert all(t.data_ptr() == dst.locals[0].data_ptr() for t in dst.locals)
+    _run((64, 96), BF16, sbp.S(1), sbp.B, 4, alias=True)
+
+
+def test_boxing_degenerate_shapes():
+    _run((3, 96), F32, sbp.S(0), sbp.B, 4)          # a shard with no rows
+    _run((3, 96), F32, sbp.S(0), sbp.S(1), 4)
+    _run((3, 5), F32, sbp.P_SUM, sbp.S(0), 8)
+    _run((0, 16), F32, sbp.S(0), sbp.B, 2)          # empty tensor: nothing launched
+    _run((1, 1), BF16, sbp.P_MAX, sbp.B, 2)
+
+
+def test_psum_tolerance_and_fp64_cross_check():
+    """The stated bar: fixed-order fp32 reductions within 1e-6 relative of the oracle's, and
+    within one storage ulp / 1e-6 * sum|in| of the fp64 sum."""
+    k, shape = 4, (256, 512)
+    for dtype in (F32, BF16):
+        src_cpu = [dg.normal(77, r, shape, 0.0, 1.0, dtype) for r in range(k)]
+        src = make_global(src_cpu, shape, dtype, sbp.P_SUM)
+        dst = sbp.empty_global(shape, dtype, sbp.B, k)
+        sbp.sbp_boxing(src, dst)
+        torch.cuda.synchronize()
+        arrs = [to_np(t) for t in src_cpu]
+        ref32 = O.reduce_sum_fixed_order(arrs, storage_of(dtype)).astype(np.float64)
+        ref64 = O.reduce_sum_fp64(arrs)
+        mag = sum(np.abs(a.astype(np.float64)) for a in arrs)
+        for t in dst.locals:
+            got = to_np(t).astype(np.float64)
+            assert np.all(np.abs(got - ref32) <= 1e-6 * np.abs(ref32))
+            ulp = 2.0 ** -8 * np.maximum(np.abs(ref64), 2.0 ** -126) if dtype == BF16 else 0.0
+            assert np.all(np.abs(got - ref64) <= 1e-6 * mag + ulp)
+
+
+def test_pmax_sign_of_zero_and_ties():
+    a = torch.tensor([[0.0, -0.0, 1.0, -2.0]], dtype=F32)
+    b = torch.tensor([[-0.0, 0.0, 1.0, -1.0]], dtype=F32)
+    src = make_global([a, b], (1, 4), F32, sbp.P_MAX)
+    dst = sbp.empty_global((1, 4), F32, sbp.B, 2)
+    sbp.sbp_boxing(src, dst)
+    torch.cuda.synchronize()
+    want = O.reduce_max_fixed_order([a.numpy(), b.numpy()])
+    assert np.array_equal(bits(dst.locals[0]), np_bits(want, F32))
+    assert np.signbit(want[0, 1]) and not np.signbit(want[0, 0])
+
+
+def test_round_trips_on_device():
+    """S(0)->S(1)->S(0), S(i)->B->S(i) and B->S(i)->B return the input bits."""
+    k, shape = 4, (96, 160)
+    T = dg.normal(5, 0, shape, 0, 1, BF16)
+    s0 = make_global(split_cpu(T, sbp.S(0), k), shape, BF16, sbp.S(0))
+    s1 = sbp.empty_global(shape, BF16, sbp.S(1), k)
+    back = sbp.empty_global(shape, BF16, sbp.S(0), k)
+    rep = sbp.empty_global(shape, BF16, sbp.B, k)
+    sbp.sbp_boxing(s0, s1)
+    sbp.sbp_boxing(s1, back)
+    sbp.sbp_boxing(s1, rep)
+    torch.cuda.synchronize()
+    for a, b in zip(s0.locals, back.locals):
+        assert torch.equal(a, b)
+    for r in rep.locals:
+        assert np.array_equal(bits(r), bits(T))
+
+
+def test_host_buffer_entry_point():
+    k, shape = 4, (128, 256)
+    src_cpu = [dg.normal(9, r, shape, 0, 1, BF16).pin_memory() for r in range(k)]
+    src = sbp.SbpTensor(shape, BF16, sbp.P_SUM, src_cpu)
+    dst_cpu = [torch.empty(sbp.sbp_local_shape(shape, sbp.S(1), k, r, BF16), dtype=BF16).pin_memory() for r in range(k)]
+    dst = sbp.SbpTensor(shape, BF16, sbp.S(1), dst_cpu)
+    need = sbp.sbp_boxing_host_workspace_bytes(src, dst)
+    assert need >= (k + 1) * 128 * 256 * 2
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    sbp.sbp_boxing_host(src, dst, ws)
+    torch.cuda.synchronize()
+    want = O.boxing([to_np(t) for t in src_cpu], O.PSUM, O.S1, "bf16")
+    for r in range(k):
+        assert np.array_equal(bits(dst_cpu[r]), np_bits(want[r], BF16))
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_boxing_host(src, dst, ws[:1024])
+    assert e.value.name == "SBP_ERR_WORKSPACE"

@@ -1,0 +1,323 @@
+"""Parity of the sharded operators (Table 1 MatMul, class-split softmax cross entropy,
+row-split embedding) against the CPU oracle.
+
+Tolerances.  bf16-input / fp32-accumulate MatMul and softmax: |gpu - ref| <= 1e-3 + 2e-2 |ref|
+against the fp64 oracle.  fp32 FMA MatMul: |gpu - ref| <= 4 sqrt(K) 2^-24 (|X||W|)_ij (rounding
+of a K-term fp32 dot product).  Embedding and every index result: bit-exact."""
+import math
+
+import numpy as np
+import pytest
+import torch
+from helpers import assert_close, bits, make_global, np_bits, osig, split_cpu, to_np
+
+import paper_2110_15032_b200 as sbp
+import sbp_datagen as dg
+from oracle import sbp_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+F32, BF16, I64 = torch.float32, torch.bfloat16, torch.int64
+
+TABLE1 = [(sbp.S(0), sbp.B), (sbp.B, sbp.S(1)), (sbp.S(1), sbp.S(0)),
+          (sbp.P_SUM, sbp.B), (sbp.B, sbp.P_SUM), (sbp.B, sbp.B)]
+
+
+def _shard_operand(T, sig, k, seed, tid, dtype):
+    """CPU local tensors of logical T under sig.  For P(sum): k-1 seeded shards plus the
+    remainder, so that the fixed-order sum of the shards is the logical operand."""
+    if sig.kind == 2:
+        parts = [dg.uniform(seed, tid + r, T.shape, -1.0, 1.0, dtype) for r in range(k - 1)]
+        acc = T.to(torch.float64)
+        for p_ in parts:
+            acc = acc - p_.to(torch.float64)
+        parts.append(acc.to(dtype))
+        return parts
+    return split_cpu(T, sig, k)
+
+
+def _matmul_case(M, K, N, k, dtype, xs, ws, ys=None, flags=0, out_dtype=None, seed=1001):
+    out_dtype = out_dtype or dtype
+    X = dg.uniform(seed, 0, (M, K), -1.0, 1.0, dtype)
+    W = dg.uniform(seed, 1, (K, N), -1.0, 1.0, dtype)
+    xl = _shard_operand(X, xs, k, seed, 10, dtype)
+    wl = _shard_operand(W, ws, k, seed, 40, dtype)
+    natural = sbp.sbp_matmul_infer(xs, ws)
+    ys = ys or natural
+    x = make_global(xl, (M, K), dtype, xs)
+    w = make_global(wl, (K, N), dtype, ws)
+    y = sbp.empty_global((M, N), out_dtype, ys, k)
+    for t in y.locals:
+        t.view(torch.uint8).fill_(0x7F)
+    nbytes = sbp.sbp_matmul_workspace_bytes(x, w, y)
+    wsbuf = torch.empty(max(nbytes, 1), dtype=torch.uint8, device="cuda")
+    sbp.sbp_matmul(x, w, y, flags, wsbuf)
+    torch.cuda.synchronize()
+    sbp.sbp_check_device_errors()
+
+    y_sig, y_locals, Y = O.matmul_locals([to_np(t) for t in xl], osig(xs), [to_np(t) for t in wl], osig(ws))
+    assert osig(natural) == y_sig
+    if flags & sbp.SBP_EPILOGUE_GELU:
+        Y = O.gelu(Y)
+        y_locals = [O.gelu(a) for a in y_locals]
+    if ys != natural:                       # fused boxing: the logical product in the requested signature
+        want = O.to_locals(Y, osig(ys), k)
+    else:
+        want = y_locals
+    if dtype == F32:
+        # fp32 FMA dot products: |err| <= lambda sqrt(K) u (|X||W|)_ij  (probabilistic bound on
+        # recursive summation, lambda = 4, u = 2^-24); the abs-products come from the oracle.
+        _, abs_locals, Yabs = O.matmul_locals([np.abs(to_np(t)) for t in xl], osig(xs),
+                                              [np.abs(to_np(t)) for t in wl], osig(ws))
+        abs_want = O.to_locals(Yabs, osig(ys), k) if ys != natural else abs_locals
+        coef = 4.0 * math.sqrt(max(K, 1)) * 2.0 ** -24
+    for r in range(k):
+        assert tuple(y.locals[r].shape) == tuple(want[r].shape)
+        if dtype == F32:
+            err = np.abs(to_np(y.locals[r]).astype(np.float64) - want[r])
+            assert np.all(err <= coef * abs_want[r] + 1e-30), f"{xs}x{ws}->{ys} shard {r}: {err.max()}"
+        else:
+            assert_close(to_np(y.locals[r]), want[r], 2e-2, 1e-3, f"{xs}x{ws}->{ys} shard {r}")
+    rtol, atol = (1e-4, 1e-4) if dtype == F32 else (2e-2, 1e-3)
+    # SBP invariant on the device result: the locals reproduce the logical product
+    got = [to_np(t).astype(np.float64) for t in y.locals]
+    if ys.kind == 2:
+        # each partial carries its own rounding, so the bound scales with sum_r |Y_r|, not |Y|
+        mag = sum(np.abs(a) for a in want)
+        assert np.all(np.abs(O.reduce_sum_fp64(got) - Y) <= k * atol + rtol * mag), "sum of partials"
+    elif ys.kind == 1:
+        assert all(np.array_equal(got[0], g) for g in got)
+    return y
+
+
+@pytest.mark.parametrize("xs,ws", TABLE1)
+def test_config1_all_six_signatures_fp32(xs, ws):
+    """Tiny SBP correctness config: A[64,128] * B[128,96], uniform[-1,1], k = 2."""
+    _matmul_case(64, 128, 96, 2, F32, xs, ws)
+
+
+@pytest.mark.parametrize("xs,ws", TABLE1)
+@pytest.mark.parametrize("k", [1, 3, 4])
+def test_matmul_signatures_ragged_fp32(xs, ws, k):
+    _matmul_case(70, 45, 83, k, F32, xs, ws)
+
+
+@pytest.mark.parametrize("xs,ws", TABLE1)
+def test_matmul_signatures_bf16_small(xs, ws):
+    _matmul_case(70, 45, 83, 3, BF16, xs, ws)            # shapes the tensor-core path cannot take
+    _matmul_case(256, 256, 256, 2, BF16, xs, ws)
+
+
+@pytest.mark.parametrize("ys", [sbp.B, sbp.S(0), sbp.S(1)])
+@pytest.mark.parametrize("xs,ws", [(sbp.S(1), sbp.S(0)), (sbp.P_SUM, sbp.B), (sbp.B, sbp.P_SUM)])
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_matmul_fused_output_boxing(xs, ws, ys, dtype):
+    _matmul_case(64, 128, 96, 2, dtype, xs, ws, ys=ys)
+    _matmul_case(70, 45, 83, 3, dtype, xs, ws, ys=ys)
+
+
+def test_matmul_gelu_epilogue_and_f32_out():
+    _matmul_case(64, 128, 96, 2, F32, sbp.B, sbp.S(1), flags=sbp.SBP_EPILOGUE_GELU)
+    _matmul_case(64, 128, 96, 2, BF16, sbp.B, sbp.S(1), flags=sbp.SBP_EPILOGUE_GELU)
+    _matmul_case(64, 128, 96, 2, BF16, sbp.S(1), sbp.S(0), ys=sbp.B, flags=sbp.SBP_EPILOGUE_GELU)
+    _matmul_case(64, 128, 96, 2, BF16, sbp.S(1), sbp.S(0), out_dtype=F32)
+
+
+def test_matmul_exact_on_small_integers_and_permutation():
+    """Integer-valued operands: every product and sum is exact in fp32, so every signature
+    must equal the logical product exactly; a permutation matrix as W permutes columns."""
+    M, K, N, k = 32, 64, 48, 4
+    X = dg.small_integers(3, 0, (M, K), -4, 5, F32)
+    W = dg.small_integers(3, 1, (K, N), -4, 5, F32)
+    Y = O.matmul_logical(X.numpy(), W.numpy())
+    for xs, ws in [(sbp.S(0), sbp.B), (sbp.B, sbp.S(1)), (sbp.S(1), sbp.S(0)), (sbp.B, sbp.B)]:
+        for dtype in (F32, BF16):
+            x = make_global(split_cpu(X.to(dtype), xs, k), (M, K), dtype, xs)
+            w = make_global(split_cpu(W.to(dtype), ws, k), (K, N), dtype, ws)
+            ys = sbp.sbp_matmul_infer(xs, ws)
+            y = sbp.empty_global((M, N), F32, ys, k)
+            sbp.sbp_matmul(x, w, y)
+            torch.cuda.synchronize()
+            got = [to_np(t).astype(np.float64) for t in y.locals]
+            full = O.reduce_sum_fp64(got) if ys.kind == 2 else O.from_locals(got, osig(ys))
+            assert np.array_equal(full, Y)
+    perm = torch.randperm(K, generator=torch.Generator().manual_seed(0))
+    Pm = torch.zeros(K, K)
+    Pm[perm, torch.arange(K)] = 1.0
+    x = make_global(split_cpu(X, sbp.S(0), k), (M, K), F32, sbp.S(0))
+    w = make_global(split_cpu(Pm, sbp.B, k), (K, K), F32, sbp.B)
+    y = sbp.empty_global((M, K), F32, sbp.S(0), k)
+    sbp.sbp_matmul(x, w, y)
+    torch.cuda.synchronize()
+    assert np.array_equal(O.from_locals([to_np(t) for t in y.locals], O.S0), X[:, perm].numpy())
+
+
+def test_config1_chain_matmul_then_boxing():
+    """Config 1 end to end: the six products, then P->B, P->S(0), S(0)->B, S(0)->S(1), B->S(1)
+    on the results; and the Y = U V W deferred-reduction chain of Section 3.3."""
+    M, K, N, k = 64, 128, 96, 2
+    y_p = _matmul_case(M, K, N, k, F32, sbp.S(1), sbp.S(0))
+    y_s0 = _matmul_case(M, K, N, k, F32, sbp.S(0), sbp.B)
+    y_b = _matmul_case(M, K, N, k, F32, sbp.B, sbp.B)
+    for src, dst_sig in [(y_p, sbp.B), (y_p, sbp.S(0)), (y_s0, sbp.B), (y_s0, sbp.S(1)), (y_b, sbp.S(1))]:
+        dst = sbp.empty_global((M, N), F32, dst_sig, k)
+        sbp.sbp_boxing(src, dst)
+        torch.cuda.synchronize()
+        want = O.boxing([to_np(t) for t in src.locals], osig(src.sig), osig(dst_sig), "f32")
+        for r in range(k):
+            assert np.array_equal(bits(dst.locals[r]), np_bits(want[r], F32))
+    # U:S(1) V:S(0) W:B  ->  (UV):P(sum), (UV)W:P(sum) without boxing in between, then P->B
+    U = dg.uniform(1001, 5, (M, K), -1, 1, F32)
+    V = dg.uniform(1001, 6, (K, N), -1, 1, F32)
+    Wm = dg.uniform(1001, 7, (N, 40), -1, 1, F32)
+    u = make_global(split_cpu(U, sbp.S(1), k), (M, K), F32, sbp.S(1))
+    v = make_global(split_cpu(V, sbp.S(0), k), (K, N), F32, sbp.S(0))
+    wm = make_global(split_cpu(Wm, sbp.B, k), (N, 40), F32, sbp.B)
+    uv = sbp.empty_global((M, N), F32, sbp.P_SUM, k)
+    uvw = sbp.empty_global((M, 40), F32, sbp.P_SUM, k)
+    out = sbp.empty_global((M, 40), F32, sbp.B, k)
+    sbp.sbp_matmul(u, v, uv)
+    sbp.sbp_matmul(uv, wm, uvw)
+    sbp.sbp_boxing(uvw, out)
+    torch.cuda.synchronize()
+    want = O.matmul_logical(O.matmul_logical(U.numpy(), V.numpy()), Wm.numpy())
+    for t in out.locals:
+        assert_close(to_np(t), want, 1e-4, 1e-4, "UVW chain")
+
+
+# ------------------------------------------------------------------ softmax cross entropy
+
+def _xent_case(rows, classes, k, dtype, sigma=1.0, seed=1004, alias=False, with_stats=True, labels=None):
+    Z = dg.normal(seed, 0, (rows, classes), 0.0, sigma, dtype)
+    if labels is None:
+        labels = dg.integers(seed, 1, (rows,), 0, classes)
+    logits = make_global(split_cpu(Z, sbp.S(1), k), (rows, classes), dtype, sbp.S(1))
+    lab = make_global([labels] * k, (rows,), I64, sbp.B)
+    loss = sbp.empty_global((rows,), F32, sbp.B, k, alias_replicas=alias)
+    rmax = sbp.empty_global((rows,), F32, sbp.B, k) if with_stats else None
+    rsum = sbp.empty_global((rows,), F32, sbp.B, k) if with_stats else None
+    ws = torch.empty(sbp.sbp_softmax_xent_workspace_bytes(logits), dtype=torch.uint8, device="cuda")
+    sbp.sbp_softmax_xent(logits, lab, loss, rmax, rsum, ws)
+    torch.cuda.synchronize()
+    m, Ssum, ref = O.softmax_xent_logical(to_np(Z), labels.numpy())
+    for t in loss.locals:
+        assert_close(to_np(t), ref, 2e-2, 1e-3, "loss")
+    if with_stats:
+        for t in rmax.locals:
+            assert np.array_equal(to_np(t).astype(np.float64), m)          # the max is exact
+        for t in rsum.locals:
+            assert_close(to_np(t), Ssum, 2e-2, 1e-3, "row_sum")
+    return to_np(loss.locals[0]), ref
+
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+@pytest.mark.parametrize("k", [1, 2, 4, 8])
+def test_softmax_xent_parity(dtype, k):
+    _xent_case(16, 4096, k, dtype)
+    _xent_case(5, 1000, k, dtype)                    # ragged: element-wise path
+    _xent_case(3, 70000, k, dtype, sigma=0.226)      # several column chunks per shard
+
+
+def test_softmax_xent_tight_accuracy_and_shard_invariance():
+    """fp32 partial sums of exp: far inside the stated tolerance, and independent of k."""
+    ref_losses = []
+    for k in (1, 2, 4, 8):
+        got, ref = _xent_case(8, 32768, k, BF16, sigma=0.226, seed=55)
+        assert np.all(np.abs(got - ref) <= 2e-5 * np.abs(ref))
+        ref_losses.append(got)
+    for g in ref_losses[1:]:
+        assert np.all(np.abs(g - ref_losses[0]) <= 1e-6 * np.abs(ref_losses[0]) + 1e-6)
+
+
+def test_softmax_xent_closed_forms_and_edges():
+    rows, classes, k = 4, 512, 4
+    Z = torch.full((rows, classes), 2.5, dtype=BF16)
+    labels = torch.tensor([0, 127, 128, 511])
+    logits = make_global(split_cpu(Z, sbp.S(1), k), (rows, classes), BF16, sbp.S(1))
+    lab = make_global([labels] * k, (rows,), I64, sbp.B)
+    loss = sbp.empty_global((rows,), F32, sbp.B, k)
+    rsum = sbp.empty_global((rows,), F32, sbp.B, k)
+    ws = torch.empty(sbp.sbp_softmax_xent_workspace_bytes(logits), dtype=torch.uint8, device="cuda")
+    sbp.sbp_softmax_xent(logits, lab, loss, None, rsum, ws)
+    torch.cuda.synchronize()
+    assert np.allclose(to_np(loss.locals[0]), math.log(classes), rtol=1e-6)        # all-equal logits: ln C
+    assert np.allclose(to_np(rsum.locals[0]), classes, rtol=1e-6)
+    # labels on shard boundaries, first and last class; aliasing of replicas; no stats
+    lab_edge = torch.tensor([0, 1023, 1024, 4095, 2047, 2048, 3071, 3072])
+    _xent_case(8, 4096, 4, BF16, labels=lab_edge, alias=True, with_stats=False)
+    # k > classes: some shards hold no class at all
+    _xent_case(4, 3, 4, F32)
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_softmax_xent(logits, lab, loss, None, rsum, ws[:16])
+    assert e.value.name == "SBP_ERR_WORKSPACE"
+
+
+# ------------------------------------------------------------------ embedding
+
+def _emb_case(rows, dim, ids, k, dtype, fused, alias=False, table=None):
+    if table is None:
+        table = dg.uniform(1005, 0, (rows, dim), -0.05, 0.05, dtype)
+    tab = make_global(split_cpu(table, sbp.S(0), k), (rows, dim), dtype, sbp.S(0))
+    idt = make_global([ids] * k, tuple(ids.shape), I64, sbp.B)
+    out_shape = tuple(ids.shape) + (dim,)
+    out = sbp.empty_global(out_shape, dtype, sbp.B if fused else sbp.P_SUM, k, alias_replicas=alias)
+    for t in out.locals:
+        t.view(torch.uint8).fill_(0x5A)
+    oob = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sbp.sbp_embedding(tab, idt, out, oob)
+    torch.cuda.synchronize()
+    tnp = to_np(table)
+    if fused:
+        want = O.embedding_logical(tnp, ids.numpy())
+        if k > 1:
+            want = want + np.float32(0.0)        # what P(sum)->B of the partials gives for -0.0
+        for t in out.locals:
+            assert np.array_equal(bits(t), np_bits(want, dtype))
+    else:
+        parts = O.embedding_partials(O.to_locals(tnp, O.S0, k), ids.numpy())
+        for r in range(k):
+            assert np.array_equal(bits(out.locals[r]), np_bits(parts[r], dtype)), f"shard {r}"
+    return out, int(oob.item())
+
+
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("k", [1, 2, 3, 8])
+@pytest.mark.parametrize("dtype,dim", [(F32, 128), (F32, 33), (BF16, 64), (BF16, 7)])
+def test_embedding_parity(fused, k, dtype, dim):
+    rows = 1000
+    ids = dg.zipf_ids(1005, 1, (97, 26), 1024).clamp_(max=rows - 1)
+    _emb_case(rows, dim, ids, k, dtype, fused)
+
+
+def test_embedding_closed_forms_and_edges():
+    rows, dim, k = 256, 128, 4
+    ids = torch.arange(rows).reshape(rows, 1)
+    out, _ = _emb_case(rows, dim, ids, k, F32, True)
+    table = dg.uniform(1005, 0, (rows, dim), -0.05, 0.05, F32)
+    assert np.array_equal(to_np(out.locals[0]).reshape(rows, dim), table.numpy())    # arange ids: the table itself
+    ids1 = torch.full((16, 2), 70)                                                   # all in shard 1
+    outp, _ = _emb_case(rows, dim, ids1, k, F32, False)
+    assert all(not outp.locals[r].any().item() for r in (0, 2, 3)) and outp.locals[1].any().item()
+    bad = torch.tensor([[-1, rows, 5, 1 << 40]])
+    _, oob = _emb_case(rows, dim, bad, k, F32, True)
+    assert oob == 3
+    _, oob = _emb_case(rows, dim, bad, k, F32, False)
+    assert oob == 3
+    _emb_case(rows, dim, ids1, k, F32, True, alias=True)
+    _emb_case(3, 16, torch.tensor([0, 1, 2, 2, 0]), 8, F32, False)                   # k > rows
+    _emb_case(3, 16, torch.tensor([0, 1, 2, 2, 0]), 8, F32, True)
+
+
+def test_embedding_fused_equals_unfused_plus_boxing_with_negative_zero():
+    rows, dim, k = 64, 32, 4
+    table = dg.uniform(1005, 9, (rows, dim), -0.05, 0.05, F32)
+    table[5, 3] = -0.0
+    table[40, 0] = -0.0
+    ids = torch.tensor([[5, 40, 7], [63, 5, 0]])
+    fused, _ = _emb_case(rows, dim, ids, k, F32, True, table=table)
+    parts, _ = _emb_case(rows, dim, ids, k, F32, False, table=table)
+    boxed = sbp.empty_global(tuple(ids.shape) + (dim,), F32, sbp.B, k)
+    sbp.sbp_boxing(parts, boxed)
+    torch.cuda.synchronize()
+    for a, b in zip(fused.locals, boxed.locals):
+        assert np.array_equal(bits(a), bits(b))

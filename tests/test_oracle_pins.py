@@ -489,3 +489,11 @@ def test_pins_catch_planted_mistakes(monkeypatch):
         mp.setattr(O, "gelu", lambda x: 0.5 * np.asarray(x) * (1 + np.tanh(0.79788456 * (x + 0.044715 * x ** 3))))
         with pytest.raises(AssertionError):
             test_gelu_closed_forms()
+
+
+def test_boxing_p_to_p_keeps_each_partial():
+    # Table 2: P -> P on the same devices moves nothing, so each device keeps its partial.
+    loc = [dg.normal(23, r, (3, 5), 0, 1).numpy() for r in range(3)]
+    out = O.boxing(loc, PSUM, PSUM)
+    assert all(np.array_equal(a, b) and a is not b for a, b in zip(out, loc))
+    assert O.table2_same_placement_cost(PSUM, PSUM, 3, 60) == 0

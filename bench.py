@@ -407,13 +407,15 @@ def oracle_sweep_sample(rows: int):
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-ops", action="store_true", help="skip the sharded-operator sections (N = 1 only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--copy-engine", type=int, default=0)
+    ap.add_argument("--rows", type=int, default=SWEEP_SHAPE[0],
+                    help="rows of the logical sweep tensor (smaller = a profiling-sized case, not the benchmark)")
     return ap.parse_args()
 
 
@@ -445,6 +447,8 @@ def reference_arm(args):
 
 def main():
     args = parse()
+    global SWEEP_SHAPE
+    SWEEP_SHAPE = (args.rows, SWEEP_SHAPE[1])
     if args.impl == "reference":
         return reference_arm(args)
 
@@ -518,7 +522,7 @@ def main():
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": "boxing sweep: logical bf16 [8192,8192] N(0,1), k=4, 7 transforms per step",
+        "config": {"workload": f"boxing sweep: logical bf16 [{SWEEP_SHAPE[0]},{SWEEP_SHAPE[1]}] N(0,1), k=4, 7 transforms per step",
                    "parallelism": f"replicas x{world}" if world > 1 else "1 GPU, k=4 logical shards",
                    "l2": "inputs larger than L2: a step streams 3.4 GB through distinct buffers between repeats",
                    "copy_engine": args.copy_engine},
@@ -531,13 +535,16 @@ def main():
         line["clocks"] = clocks
 
     # end-to-end: the same sweep through the host-buffer entry point, copies inside the region
-    e2e = e2e_sweep(sbp, src, work, device, args.e2e_steps, dist)
-    e2e["value"] *= world
-    line["e2e"] = e2e
+    if args.e2e_steps > 0:
+        e2e = e2e_sweep(sbp, src, work, device, args.e2e_steps, dist)
+        e2e["value"] *= world
+        line["e2e"] = e2e
+    else:
+        line["e2e"] = None
 
     if rank == 0 and world == 1:
         if not args.no_cpu_baseline:
-            rows = 1024
+            rows = min(4096, SWEEP_SHAPE[0])
             nbytes, secs, cores = oracle_sweep_sample(rows)
             line["cpu_baseline"] = {"value": nbytes / secs / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
                                     "sample": f"first {rows} of {SWEEP_SHAPE[0]} rows of every local tensor, "

@@ -338,9 +338,16 @@ static sbp_status make_plan(const sbp_tensor* src, const sbp_tensor* dst, Plan* 
   p.A = p.Na = p.M = p.Nb = 1;
   if (sa < 0 && da < 0) {
     p.C = prod(0, src->ndim);
-  } else if (sa < 0 || da < 0 || sa == da) {
+  } else if (sa >= 0 && sa == da) {
+    // Same split on both sides: shard r's local tensor is copied whole, and a local tensor
+    // is one contiguous run of len_r * (all other extents) elements on both sides.
+    p.Nb = src->shape[sa];
+    p.C = prod(0, sa) * prod(sa + 1, src->ndim);
+    p.src_b = p.dst_b = 1;
+  } else if (sa < 0 || da < 0) {
+    // One restricted axis: [1][Na = outer (unrestricted)][1][Nb = n_ax][C].
     const int ax = sa >= 0 ? sa : da;
-    p.A = prod(0, ax);
+    p.Na = prod(0, ax);
     p.Nb = src->shape[ax];
     p.C = prod(ax + 1, src->ndim);
     p.src_b = sa >= 0;
@@ -429,7 +436,11 @@ sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream)
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
   bool done = false;
-  if (pl.op == OP_COPY && g_copy_engine.load() == 2 && pl.vbytes == 16)
+  // Default choice, from measurement on B200: the bulk engine wins where one read feeds one
+  // write (re-layouts and slices); the load/store kernel wins where one read feeds k writes.
+  const int engine = g_copy_engine.load();
+  const bool want_bulk = engine == 2 || (engine == 0 && pl.p.mode != MODE_GATHER);
+  if (pl.op == OP_COPY && want_bulk && pl.vbytes == 16)
     done = launch_bulk_copy(pl.p, pl.ntasks, stream);
   if (!done) {
     switch (pl.op) {

@@ -16,13 +16,15 @@
 #include <cuda_bf16.h>
 
 #include <cfloat>
+#include <cmath>
 
 #include "sbp_internal.h"
 
 namespace sbp {
 
 constexpr int kThreads = 256;
-constexpr int kLoadsPerThread = 8;
+constexpr int kLoadsPerThread = 8;    // vectors per thread per chunk
+constexpr int kMaxChunksPerCta = 8;   // a CTA walks up to this many chunks of one row
 
 struct XentParams {
   const char* logits[SBP_MAX_K];
@@ -32,7 +34,8 @@ struct XentParams {
   float* part_t;
   long long rows, classes;
   int k, nsplit;
-  long long chunk;   // elements per column chunk
+  long long chunk;   // elements per chunk (kThreads * kLoadsPerThread * VEC)
+  long long span;    // elements per CTA (chunk * chunks per CTA)
 };
 
 struct XentCombineParams {
@@ -47,60 +50,146 @@ struct XentCombineParams {
   int parts;
 };
 
-template <typename T>
-__device__ __forceinline__ float to_f32(T v);
-template <>
-__device__ __forceinline__ float to_f32<float>(float v) { return v; }
-template <>
-__device__ __forceinline__ float to_f32<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+constexpr float kLog2e = 1.4426950408889634f;
 
+__device__ __forceinline__ float ex2(float x) {
+  float y;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+  return y;
+}
+
+// (m, s) <- merge with (m2, s2), where s is a sum of exp(z - m).  A piece with no elements
+// carries (m = -inf, s = 0) and must not produce inf - inf.
 __device__ __forceinline__ void merge(float& m, float& s, float m2, float s2) {
   const float mm = fmaxf(m, m2);
-  // exp(-inf - finite) = 0; a piece with no elements carries (m = -inf, s = 0).
-  const float a = (m == -INFINITY) ? 0.f : s * __expf(m - mm);
-  const float b = (m2 == -INFINITY) ? 0.f : s2 * __expf(m2 - mm);
+  const float a = (m == -INFINITY) ? 0.f : s * ex2((m - mm) * kLog2e);
+  const float b = (m2 == -INFINITY) ? 0.f : s2 * ex2((m2 - mm) * kLog2e);
   s = a + b;
   m = mm;
 }
 
-// T: element type.  VEC: elements per load (16 bytes / sizeof(T), or 1 on the unaligned path).
-template <typename T, int VEC>
+// ---- chunk policies: how one thread loads, maxes and exp-sums its kLoadsPerThread vectors
+
+// bf16, 8 elements per 16-byte load; max on packed pairs, exp in fp32.
+struct ChunkBF16x8 {
+  using T = __nv_bfloat16;
+  static constexpr int VEC = 8;
+  uint4 raw[kLoadsPerThread];
+  __device__ __forceinline__ void load(const T* z, long long n, int tid) {
+#pragma unroll
+    for (int u = 0; u < kLoadsPerThread; ++u) {
+      const long long e0 = ((long long)u * kThreads + tid) * VEC;
+      if (e0 < n) {
+        asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                     : "=r"(raw[u].x), "=r"(raw[u].y), "=r"(raw[u].z), "=r"(raw[u].w)
+                     : "l"(z + e0));
+      } else {
+        raw[u] = make_uint4(0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u, 0xFF80FF80u);   // -inf, -inf
+      }
+    }
+  }
+  __device__ __forceinline__ float max() const {
+    __nv_bfloat162 mx = *reinterpret_cast<const __nv_bfloat162*>(&raw[0].x);
+#pragma unroll
+    for (int u = 0; u < kLoadsPerThread; ++u) {
+      const uint32_t* w = reinterpret_cast<const uint32_t*>(&raw[u]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) mx = __hmax2(mx, *reinterpret_cast<const __nv_bfloat162*>(&w[i]));
+    }
+    return fmaxf(__low2float(mx), __high2float(mx));
+  }
+  // sum of 2^(z*log2e + neg_m_l2e) over the thread's elements
+  __device__ __forceinline__ float expsum(float neg_m_l2e) const {
+    float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+    for (int u = 0; u < kLoadsPerThread; ++u) {
+      const uint32_t* w = reinterpret_cast<const uint32_t*>(&raw[u]);
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const float lo = __uint_as_float(w[i] << 16);
+        const float hi = __uint_as_float(w[i] & 0xffff0000u);
+        s0 += ex2(fmaf(lo, kLog2e, neg_m_l2e));
+        s1 += ex2(fmaf(hi, kLog2e, neg_m_l2e));
+      }
+    }
+    return s0 + s1;
+  }
+};
+
+// Generic policy: element type TT, V elements per load (V * sizeof(TT) is 16 or sizeof(TT)).
+template <typename TT, int V>
+struct ChunkGeneric {
+  using T = TT;
+  static constexpr int VEC = V;
+  struct alignas(sizeof(TT) * V) Pack { TT e[V]; };
+  Pack raw[kLoadsPerThread];
+  bool ok[kLoadsPerThread];
+  __device__ __forceinline__ static float f32(float v) { return v; }
+  __device__ __forceinline__ static float f32(__nv_bfloat16 v) { return __bfloat162float(v); }
+  __device__ __forceinline__ void load(const T* z, long long n, int tid) {
+#pragma unroll
+    for (int u = 0; u < kLoadsPerThread; ++u) {
+      const long long e0 = ((long long)u * kThreads + tid) * VEC;
+      ok[u] = e0 < n;
+      if (ok[u]) raw[u] = *reinterpret_cast<const Pack*>(z + e0);
+    }
+  }
+  __device__ __forceinline__ float max() const {
+    float m = -INFINITY;
+#pragma unroll
+    for (int u = 0; u < kLoadsPerThread; ++u)
+      if (ok[u]) {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) m = fmaxf(m, f32(raw[u].e[i]));
+      }
+    return m;
+  }
+  __device__ __forceinline__ float expsum(float neg_m_l2e) const {
+    float s = 0.f;
+#pragma unroll
+    for (int u = 0; u < kLoadsPerThread; ++u)
+      if (ok[u]) {
+#pragma unroll
+        for (int i = 0; i < VEC; ++i) s += ex2(fmaf(f32(raw[u].e[i]), kLog2e, neg_m_l2e));
+      }
+    return s;
+  }
+};
+
+// One CTA per (row, shard, column span).  Each thread keeps a running (m, s) over the chunks
+// of its span -- the loads of the next chunk are issued before the current one is reduced --
+// and the CTA merges the 256 pairs with a fixed tree.
+template <typename Chunk>
 __global__ void __launch_bounds__(kThreads) xent_partial_kernel(const __grid_constant__ XentParams p) {
+  using T = typename Chunk::T;
   const long long row = blockIdx.x;
   const int split = blockIdx.y;
   const int shard = blockIdx.z;
   long long c_start, c_len;
   split_range(p.classes, p.k, shard, (int64_t*)&c_start, (int64_t*)&c_len);
-  const long long c0 = (long long)split * p.chunk;
-  long long n = c_len - c0;
-  if (n > p.chunk) n = p.chunk;
+  const long long c0 = (long long)split * p.span;
+  long long n = c_len - c0;       // elements of this CTA's span (may be <= 0 on uneven shards)
+  if (n > p.span) n = p.span;
   const int part = shard * p.nsplit + split;
-
   const T* z = reinterpret_cast<const T*>(p.logits[shard]) + row * c_len + c0;
+  const int tid = threadIdx.x;
 
-  struct alignas(sizeof(T) * VEC) Pack { T e[VEC]; };
-  Pack raw[kLoadsPerThread];
-  bool ok[kLoadsPerThread];
-#pragma unroll
-  for (int u = 0; u < kLoadsPerThread; ++u) {
-    const long long e0 = ((long long)u * kThreads + threadIdx.x) * VEC;
-    ok[u] = e0 < n;   // n is a multiple of VEC on the vector path
-    if (ok[u]) raw[u] = *reinterpret_cast<const Pack*>(z + e0);
+  float m = -INFINITY, s = 0.f;
+  Chunk cur, nxt;
+  if (n > 0) cur.load(z, n, tid);
+  for (long long off = 0; off < n; off += p.chunk) {
+    const bool more = off + p.chunk < n;
+    if (more) nxt.load(z + off + p.chunk, n - off - p.chunk, tid);
+    const float cm = cur.max();
+    if (cm != -INFINITY) {
+      const float mm = fmaxf(m, cm);
+      const float neg = -mm * kLog2e;
+      const float carried = (m == -INFINITY) ? 0.f : s * ex2(fmaf(m, kLog2e, neg));
+      s = carried + cur.expsum(neg);
+      m = mm;
+    }
+    if (more) cur = nxt;
   }
-  float m = -INFINITY;
-#pragma unroll
-  for (int u = 0; u < kLoadsPerThread; ++u)
-    if (ok[u]) {
-#pragma unroll
-      for (int i = 0; i < VEC; ++i) m = fmaxf(m, to_f32<T>(raw[u].e[i]));
-    }
-  float s = 0.f;
-#pragma unroll
-  for (int u = 0; u < kLoadsPerThread; ++u)
-    if (ok[u]) {
-#pragma unroll
-      for (int i = 0; i < VEC; ++i) s += __expf(to_f32<T>(raw[u].e[i]) - m);
-    }
 
 #pragma unroll
   for (int off = 16; off > 0; off >>= 1) {
@@ -109,18 +198,18 @@ __global__ void __launch_bounds__(kThreads) xent_partial_kernel(const __grid_con
     merge(m, s, m2, s2);
   }
   __shared__ float sm[kThreads / 32], ss[kThreads / 32];
-  if ((threadIdx.x & 31) == 0) {
-    sm[threadIdx.x >> 5] = m;
-    ss[threadIdx.x >> 5] = s;
+  if ((tid & 31) == 0) {
+    sm[tid >> 5] = m;
+    ss[tid >> 5] = s;
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
+  if (tid == 0) {
     float mm = sm[0], sv = ss[0];
 #pragma unroll
     for (int w = 1; w < kThreads / 32; ++w) merge(mm, sv, sm[w], ss[w]);
     float t = 0.f;
     const long long y = p.labels[row] - c_start - c0;
-    if (y >= 0 && y < n) t = to_f32<T>(z[y]);
+    if (y >= 0 && y < n) t = static_cast<float>(z[y]);
     p.part_m[(long long)part * p.rows + row] = mm;
     p.part_s[(long long)part * p.rows + row] = sv;
     p.part_t[(long long)part * p.rows + row] = t;
@@ -144,12 +233,23 @@ __global__ void __launch_bounds__(128) xent_combine_kernel(const __grid_constant
   for (int j = 0; j < p.n_sum; ++j) p.row_sum[j][row] = S;
 }
 
-static int nsplit_for(const sbp_tensor* logits, int vec) {
+// Elements of one CTA's column span, and how many spans cover the widest shard.
+static void tiling_for(const sbp_tensor* logits, int vec, long long* chunk, long long* span, int* nsplit) {
   const int k = placement_k(logits);
   const long long c_max = (logits->shape[1] + k - 1) / k;
-  const long long chunk = (long long)kThreads * kLoadsPerThread * vec;
-  long long ns = (c_max + chunk - 1) / chunk;
-  return (int)(ns < 1 ? 1 : ns);
+  *chunk = (long long)kThreads * kLoadsPerThread * vec;
+  long long chunks = (c_max + *chunk - 1) / *chunk;
+  if (chunks < 1) chunks = 1;
+  const long long per_cta = chunks < kMaxChunksPerCta ? chunks : kMaxChunksPerCta;
+  *span = *chunk * per_cta;
+  *nsplit = (int)((chunks + per_cta - 1) / per_cta);
+}
+
+static int nsplit_for(const sbp_tensor* logits, int vec) {
+  long long chunk, span;
+  int ns;
+  tiling_for(logits, vec, &chunk, &span, &ns);
+  return ns;
 }
 
 // Elements per load: 16 bytes worth when every shard's rows are 16-byte aligned, else 1.
@@ -193,18 +293,10 @@ extern "C" {
 
 size_t sbp_softmax_xent_workspace_bytes(const sbp_tensor* logits) {
   if (check_tensor(logits, "logits", false) != SBP_OK || logits->ndim != 2) return 0;
-  // sized for the unaligned path as well, so the answer does not depend on pointer values
+  // sized for the element-wise path as well, so the answer does not depend on pointer values
   const int k = placement_k(logits);
-  const int esz = elem_size(logits->dtype);
-  bool vec_ok = true;
-  for (int r = 0; r < k; ++r) {
-    int64_t st, ln;
-    split_range(logits->shape[1], k, r, &st, &ln);
-    vec_ok = vec_ok && (ln * esz) % 16 == 0;
-  }
   const int ns = nsplit_for(logits, 1);
-  const int ns_vec = nsplit_for(logits, 16 / esz);
-  (void)vec_ok;
+  const int ns_vec = nsplit_for(logits, 16 / elem_size(logits->dtype));
   const size_t parts = (size_t)k * (size_t)(ns > ns_vec ? ns : ns_vec);
   return 3 * parts * (size_t)logits->shape[0] * sizeof(float);
 }
@@ -251,16 +343,19 @@ sbp_status sbp_softmax_xent(const sbp_tensor* logits, const sbp_tensor* labels, 
   p.classes = classes;
   p.k = k;
   p.nsplit = nsplit;
-  p.chunk = (long long)kThreads * kLoadsPerThread * vec;
+  {
+    int ns;
+    tiling_for(logits, vec, &p.chunk, &p.span, &ns);
+  }
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   dim3 grid((unsigned)rows, (unsigned)nsplit, (unsigned)k);
   if (logits->dtype == SBP_BF16) {
-    if (vec > 1) xent_partial_kernel<__nv_bfloat16, 8><<<grid, kThreads, 0, stream>>>(p);
-    else xent_partial_kernel<__nv_bfloat16, 1><<<grid, kThreads, 0, stream>>>(p);
+    if (vec > 1) xent_partial_kernel<ChunkBF16x8><<<grid, kThreads, 0, stream>>>(p);
+    else xent_partial_kernel<ChunkGeneric<__nv_bfloat16, 1>><<<grid, kThreads, 0, stream>>>(p);
   } else {
-    if (vec > 1) xent_partial_kernel<float, 4><<<grid, kThreads, 0, stream>>>(p);
-    else xent_partial_kernel<float, 1><<<grid, kThreads, 0, stream>>>(p);
+    if (vec > 1) xent_partial_kernel<ChunkGeneric<float, 4>><<<grid, kThreads, 0, stream>>>(p);
+    else xent_partial_kernel<ChunkGeneric<float, 1>><<<grid, kThreads, 0, stream>>>(p);
   }
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e, "softmax partial launch");

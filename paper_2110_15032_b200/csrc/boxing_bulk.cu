@@ -245,11 +245,3 @@ sbp_status read_and_clear_bulk_timeout(bool* timed_out) {
 }
 
 }  // namespace sbp
-
-extern "C" sbp_status sbp_check_device_errors(void) {
-  bool timed_out = false;
-  sbp_status st = sbp::read_and_clear_bulk_timeout(&timed_out);
-  if (st != SBP_OK) return st;
-  if (timed_out) return sbp::fail(SBP_ERR_TIMEOUT, "a bulk-copy boxing kernel gave up waiting for its loads");
-  return SBP_OK;
-}

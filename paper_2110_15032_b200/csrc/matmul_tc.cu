@@ -1,14 +1,524 @@
-// Tensor-core MatMul kernel (placeholder until the tcgen05 kernel lands in this file).
+// Tensor-core MatMul for sm_100a: bf16 operands, fp32 accumulation in tensor memory.
+//
+// One persistent CTA per SM walks the (group, m-tile, n-tile) list of a grouped-GEMM plan
+// (matmul_plan.h).  Tile = 128 x 256 outputs, K-block = 64.  Six warps, three roles:
+//
+//   warp 0  producer   TMA loads of the A tile [128 x 64] (K-major) and the B tile [64 x 256]
+//                      (N-major, four 64-column boxes) into a kStages-deep shared-memory ring
+//   warp 1  MMA        one thread issues tcgen05.mma (M128 N256 K16, four per K-block) into one
+//                      of two 256-column accumulators in tensor memory; tcgen05.commit frees
+//                      the ring slot and, after the last K-block, publishes the accumulator
+//   warps 2-5 epilogue each warp drains its own 32 lanes of the accumulator (tcgen05.ld),
+//                      applies GeLU when asked, rounds to the output type, stages 32 x 128-byte
+//                      slabs in shared memory and writes them with TMA stores -- once per
+//                      destination replica -- while the MMA warp already fills the other
+//                      accumulator
+//
+// A fused "P(sum) product written as B / S(i)" plan simply chains the K-blocks of all shards'
+// operands, in rank order, into the same accumulator: the partial products are never stored.
+//
+// Every wait is bounded in time.  A wait that expires raises a flag that
+// sbp_check_device_errors() reports; the CTA then stops issuing work, waits (bounded) for the
+// loads it still has in flight, frees its tensor memory and returns.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <mutex>
+
 #include "matmul_plan.h"
 #include "sbp_internal.h"
 
 namespace sbp {
 
+constexpr int BM = 128, BN = 256, BK = 64;
+constexpr int kStages = 4;
+constexpr int kStageA = BM * BK * 2;              // 16 KiB
+constexpr int kStageB = BK * BN * 2;              // 32 KiB
+constexpr int kStageBytes = kStageA + kStageB;    // 48 KiB
+constexpr int kSlabBytes = 32 * 128;              // one epilogue slab: 32 rows x 128 bytes
+constexpr int kEpiBytes = 4 * 2 * kSlabBytes;     // 4 warps x 2 buffers
+constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024;   // + alignment slack
+constexpr int kThreadsTc = 192;
+constexpr int kTmemCols = 512;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+__device__ int g_tc_timeout_flag = 0;
+
+struct TcParams {
+  CUtensorMap map_a[SBP_MAX_K];
+  CUtensorMap map_b[SBP_MAX_K];
+  CUtensorMap map_y[SBP_MAX_K];
+  CUtensorMap map_rep[SBP_MAX_K];
+  long long m[SBP_MAX_K], n[SBP_MAX_K], row_off[SBP_MAX_K], col_off[SBP_MAX_K];
+  int kblocks[SBP_MAX_K];       // per segment
+  int tile_begin[SBP_MAX_K + 1];   // prefix sum of tiles per group
+  int tiles_m[SBP_MAX_K];
+  int ngroups, nseg, chain, gelu, n_rep;
+  int out_f32;
+  int total_tiles;
+};
+
+// ------------------------------------------------------------------ PTX helpers
+
+__device__ __forceinline__ unsigned smem_addr(const void* p) { return (unsigned)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ unsigned long long now_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+
+__device__ __forceinline__ void mbar_init(unsigned bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+
+__device__ __forceinline__ bool mbar_try(unsigned bar, unsigned parity) {
+  unsigned done;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(done)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return done != 0;
+}
+
+// Bounded wait.  Returns false (and raises the abort flag) when the limit expires.
+__device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity, volatile int* abort_flag) {
+  if (mbar_try(bar, parity)) return true;
+  const unsigned long long t0 = now_ns();
+  for (;;) {
+    if (mbar_try(bar, parity)) return true;
+    if (*abort_flag) return false;
+    if (now_ns() - t0 > kWaitLimitNs) {
+      *abort_flag = 1;
+      atomicExch(&g_tc_timeout_flag, 1);
+      return false;
+    }
+  }
+}
+
+__device__ __forceinline__ void mbar_expect_tx(unsigned bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+
+__device__ __forceinline__ void mbar_arrive(unsigned bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int x, int y, unsigned bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "l"(map), "r"(x), "r"(y), "r"(bar)
+      : "memory");
+}
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, unsigned src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(map), "r"(x),
+               "r"(y), "r"(src)
+               : "memory");
+}
+
+__device__ __forceinline__ void umma_bf16(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
+                                          unsigned idesc, unsigned accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+      : "memory");
+}
+
+// Arrives on an mbarrier once every tcgen05 operation issued so far by this thread is done.
+__device__ __forceinline__ void umma_commit(unsigned bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
+  unsigned* r = reinterpret_cast<unsigned*>(v);
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.
+__device__ __forceinline__ unsigned long long smem_desc(unsigned addr, unsigned lbo, unsigned sbo) {
+  unsigned long long d = 0;
+  d |= (unsigned long long)((addr & 0x3FFFF) >> 4);
+  d |= (unsigned long long)(lbo >> 4) << 16;
+  d |= (unsigned long long)(sbo >> 4) << 32;
+  d |= 1ull << 46;   // descriptor version of this architecture
+  d |= 2ull << 61;   // 128-byte swizzle
+  return d;
+}
+
+// Instruction descriptor: D fp32, A and B bf16, A K-major, B N-major, M = 128, N = 256.
+constexpr unsigned kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((BN >> 3) << 17) |
+                            ((BM >> 4) << 24);
+
+__device__ __forceinline__ float gelu_erf_tc(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f)); }
+
+struct TileCoord {
+  int g, m0, n0;
+};
+
+__device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
+  int g = 0;
+  while (g + 1 < p.ngroups && tile >= p.tile_begin[g + 1]) ++g;
+  const int local = tile - p.tile_begin[g];
+  const int nt = local / p.tiles_m[g], mt = local - nt * p.tiles_m[g];   // m fastest
+  return TileCoord{g, mt * BM, nt * BN};
+}
+
+// ------------------------------------------------------------------ the kernel
+
+__global__ void __launch_bounds__(kThreadsTc, 1) matmul_tc_kernel(const __grid_constant__ TcParams p) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ __align__(8) unsigned long long bar_full[kStages], bar_empty[kStages], bar_acc_full[2], bar_acc_empty[2];
+  __shared__ unsigned tmem_base_slot;
+  __shared__ int abort_flag_s;
+  volatile int* abort_flag = &abort_flag_s;
+
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  unsigned char* epi = smem + kStages * kStageBytes;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    abort_flag_s = 0;
+    for (int i = 0; i < kStages; ++i) {
+      mbar_init(smem_addr(&bar_full[i]), 1);
+      mbar_init(smem_addr(&bar_empty[i]), 1);
+    }
+    for (int i = 0; i < 2; ++i) {
+      mbar_init(smem_addr(&bar_acc_full[i]), 1);
+      mbar_init(smem_addr(&bar_acc_empty[i]), 4);
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&tmem_base_slot)),
+                 "r"(kTmemCols)
+                 : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const unsigned tmem_base = tmem_base_slot;
+
+  const int first = blockIdx.x, stride = gridDim.x;
+
+  if (warp == 0) {
+    // ------------------------------------------------ producer
+    if (lane == 0) {
+      long long kb_iter = 0;
+      for (int tile = first; tile < p.total_tiles && !*abort_flag; tile += stride) {
+        const TileCoord tc = tile_coord(p, tile);
+        const int s_lo = p.chain ? 0 : tc.g, s_hi = p.chain ? p.nseg : tc.g + 1;
+        for (int s = s_lo; s < s_hi; ++s) {
+          for (int kb = 0; kb < p.kblocks[s]; ++kb, ++kb_iter) {
+            const int slot = (int)(kb_iter % kStages);
+            const unsigned parity = (unsigned)(((kb_iter / kStages) & 1) ^ 1);
+            if (!mbar_wait(smem_addr(&bar_empty[slot]), parity, abort_flag)) goto producer_done;
+            const unsigned full = smem_addr(&bar_full[slot]);
+            mbar_expect_tx(full, kStageBytes);
+            unsigned char* sa = smem + slot * kStageBytes;
+            unsigned char* sb = sa + kStageA;
+            tma_load_2d(smem_addr(sa), &p.map_a[s], kb * BK, (int)p.row_off[tc.g] + tc.m0, full);
+#pragma unroll
+            for (int c = 0; c < BN / 64; ++c)
+              tma_load_2d(smem_addr(sb + c * (BK * 128)), &p.map_b[s], (int)p.col_off[tc.g] + tc.n0 + c * 64, kb * BK, full);
+          }
+        }
+      }
+    producer_done:
+      if (*abort_flag) {
+        // give the loads still in flight a bounded chance to land before the CTA goes away
+        const long long issued = kb_iter;
+        for (long long i = issued > kStages ? issued - kStages : 0; i < issued; ++i) {
+          const unsigned long long t0 = now_ns();
+          while (!mbar_try(smem_addr(&bar_full[i % kStages]), (unsigned)((i / kStages) & 1)) && now_ns() - t0 < 100000000ull) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      long long kb_iter = 0;
+      int tile_iter = 0;
+      for (int tile = first; tile < p.total_tiles && !*abort_flag; tile += stride, ++tile_iter) {
+        const TileCoord tc = tile_coord(p, tile);
+        const int acc = tile_iter & 1;
+        if (!mbar_wait(smem_addr(&bar_acc_empty[acc]), (unsigned)(((tile_iter >> 1) & 1) ^ 1), abort_flag)) break;
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const unsigned d_tmem = tmem_base + acc * BN;
+        const int s_lo = p.chain ? 0 : tc.g, s_hi = p.chain ? p.nseg : tc.g + 1;
+        unsigned accumulate = 0;
+        bool ok = true;
+        for (int s = s_lo; s < s_hi && ok; ++s) {
+          for (int kb = 0; kb < p.kblocks[s]; ++kb, ++kb_iter) {
+            const int slot = (int)(kb_iter % kStages);
+            if (!mbar_wait(smem_addr(&bar_full[slot]), (unsigned)((kb_iter / kStages) & 1), abort_flag)) {
+              ok = false;
+              break;
+            }
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const unsigned sa = smem_addr(smem + slot * kStageBytes);
+            const unsigned sb = sa + kStageA;
+#pragma unroll
+            for (int kk = 0; kk < BK / 16; ++kk) {
+              // A: K-major, rows of 128 bytes, 8-row groups 1024 bytes apart; 16 K-elements = 32 bytes
+              const unsigned long long da = smem_desc(sa + kk * 32, 16, 1024);
+              // B: N-major, 64-column chunks BK*128 bytes apart, 8-row K groups 1024 bytes apart;
+              //    16 K-rows = 2048 bytes
+              const unsigned long long db = smem_desc(sb + kk * 2048, BK * 128, 1024);
+              umma_bf16(d_tmem, da, db, kIdesc, accumulate);
+              accumulate = 1;
+            }
+            umma_commit(smem_addr(&bar_empty[slot]));   // slot reusable once these MMAs have read it
+          }
+        }
+        if (!ok) break;
+        umma_commit(smem_addr(&bar_acc_full[acc]));      // accumulator complete
+      }
+    }
+  } else {
+    // ------------------------------------------------ epilogue (warps 2..5)
+    const int q = warp & 3;                       // the 32 tensor-memory lanes this warp may read
+    unsigned char* my_epi = epi + (warp - 2) * 2 * kSlabBytes;
+    const int cols_per_slab = p.out_f32 ? 32 : 64;
+    const int nslabs = BN / cols_per_slab;
+    int tile_iter = 0;
+    unsigned slab_iter = 0;
+    for (int tile = first; tile < p.total_tiles; tile += stride, ++tile_iter) {
+      if (*abort_flag) break;
+      const TileCoord tc = tile_coord(p, tile);
+      const int acc = tile_iter & 1;
+      bool ok = true;
+      if (lane == 0) ok = mbar_wait(smem_addr(&bar_acc_full[acc]), (unsigned)((tile_iter >> 1) & 1), abort_flag);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) break;
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const long long Mg = p.m[tc.g], Ng = p.n[tc.g];
+      const int row0 = tc.m0 + q * 32;
+      const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * BN;
+      for (int sl = 0; sl < nslabs; ++sl) {
+        const int col0 = tc.n0 + sl * cols_per_slab;
+        const bool live = row0 < Mg && col0 < Ng;   // warp-uniform
+        float v[64];
+        if (live) {
+          tmem_ld32(taddr + sl * cols_per_slab, v);
+          if (!p.out_f32) tmem_ld32(taddr + sl * cols_per_slab + 32, v + 32);
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+          unsigned char* buf = my_epi + (slab_iter & 1) * kSlabBytes;
+          // the store that last used this buffer must have finished reading it
+          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          __syncwarp();
+          unsigned char* rowp = buf + lane * 128;
+          if (p.out_f32) {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              float4 o;
+              o.x = v[4 * c + 0]; o.y = v[4 * c + 1]; o.z = v[4 * c + 2]; o.w = v[4 * c + 3];
+              if (p.gelu) { o.x = gelu_erf_tc(o.x); o.y = gelu_erf_tc(o.y); o.z = gelu_erf_tc(o.z); o.w = gelu_erf_tc(o.w); }
+              *reinterpret_cast<float4*>(rowp + ((c ^ (lane & 7)) << 4)) = o;
+            }
+          } else {
+#pragma unroll
+            for (int c = 0; c < 8; ++c) {
+              float f[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) f[e] = p.gelu ? gelu_erf_tc(v[8 * c + e]) : v[8 * c + e];
+              uint4 o;
+              __nv_bfloat162 h;
+              h = __floats2bfloat162_rn(f[0], f[1]); o.x = *reinterpret_cast<unsigned*>(&h);
+              h = __floats2bfloat162_rn(f[2], f[3]); o.y = *reinterpret_cast<unsigned*>(&h);
+              h = __floats2bfloat162_rn(f[4], f[5]); o.z = *reinterpret_cast<unsigned*>(&h);
+              h = __floats2bfloat162_rn(f[6], f[7]); o.w = *reinterpret_cast<unsigned*>(&h);
+              *reinterpret_cast<uint4*>(rowp + ((c ^ (lane & 7)) << 4)) = o;
+            }
+          }
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&p.map_y[tc.g], col0, row0, smem_addr(buf));
+            if (tc.g == 0)
+              for (int r = 0; r < p.n_rep; ++r) tma_store_2d(&p.map_rep[r], col0, row0, smem_addr(buf));
+            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+          }
+          ++slab_iter;
+        }
+      }
+      asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(smem_addr(&bar_acc_empty[acc]));
+    }
+    if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  }
+
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    __syncwarp();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(ptr);
+  });
+  return fn;
+}
+
+// 2-D row-major tensor [rows, cols] with leading dimension ld (elements), box [box_rows, box_cols].
+static bool make_map(CUtensorMap* map, const void* base, int esz, long long rows, long long cols, long long ld,
+                     int box_rows, int box_cols) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)ld * esz};
+  cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUtensorMapDataType dt = esz == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
+  return fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
+         CUDA_SUCCESS;
+}
+
 size_t matmul_tc_workspace_bytes(const MatmulPlan&) { return 0; }
 
-sbp_status launch_matmul_tc(const MatmulPlan&, void*, size_t, cudaStream_t, bool* taken) {
+static bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
+
+sbp_status launch_matmul_tc(const MatmulPlan& plan, void*, size_t, cudaStream_t st, bool* taken) {
   *taken = false;
-  return SBP_ERR_UNSUPPORTED;
+  if (plan.in_dtype != SBP_BF16) return SBP_ERR_UNSUPPORTED;
+  const int oesz = plan.out_dtype == SBP_F32 ? 4 : 2;
+
+  // the rules of the TMA path: 16-byte aligned bases, leading dimensions and column offsets
+  for (int s = 0; s < plan.nseg; ++s) {
+    const bool used = plan.chain || s < plan.ngroups;
+    if (!used) continue;
+    if (plan.kseg[s] > 0 && (!aligned16(plan.a[s]) || !aligned16(plan.b[s]))) return SBP_ERR_UNSUPPORTED;
+    if (plan.lda[s] % 8 != 0 || plan.ldb[s] % 8 != 0) return SBP_ERR_UNSUPPORTED;
+    if (plan.lda[s] == 0 || plan.ldb[s] == 0) return SBP_ERR_UNSUPPORTED;
+  }
+  long long ktotal_chain = 0;
+  for (int s = 0; s < plan.nseg; ++s) ktotal_chain += plan.kseg[s];
+  for (int g = 0; g < plan.ngroups; ++g) {
+    if (plan.m[g] == 0 || plan.n[g] == 0) continue;
+    if (!aligned16(plan.y[g]) || (plan.ldy[g] * oesz) % 16 != 0) return SBP_ERR_UNSUPPORTED;
+    if (plan.col_off[g] % 8 != 0) return SBP_ERR_UNSUPPORTED;
+    const long long kg = plan.chain ? ktotal_chain : plan.kseg[g];
+    if (kg == 0) return SBP_ERR_UNSUPPORTED;   // an all-zero result: left to the FMA kernel
+    if (plan.m[g] > 0x7fffffffLL || plan.n[g] > 0x7fffffffLL) return SBP_ERR_UNSUPPORTED;
+  }
+  for (int r = 0; r < plan.n_rep; ++r)
+    if (!aligned16(plan.y_rep[r])) return SBP_ERR_UNSUPPORTED;
+  if (!encode_fn()) return SBP_ERR_UNSUPPORTED;
+
+  static TcParams p;          // large; filled under a lock and copied by value at launch
+  static std::mutex mu;
+  std::lock_guard<std::mutex> lock(mu);
+  p.ngroups = plan.ngroups;
+  p.nseg = plan.nseg;
+  p.chain = plan.chain;
+  p.gelu = plan.gelu;
+  p.n_rep = plan.n_rep;
+  p.out_f32 = plan.out_dtype == SBP_F32;
+
+  for (int s = 0; s < plan.nseg; ++s) {
+    p.kblocks[s] = (int)((plan.kseg[s] + BK - 1) / BK);
+    const bool used = plan.chain || s < plan.ngroups;
+    if (!used || plan.kseg[s] == 0) continue;
+    long long rows_a = 0, cols_b = 0;
+    if (plan.chain) {
+      for (int g = 0; g < plan.ngroups; ++g) {
+        rows_a = std::max(rows_a, plan.row_off[g] + plan.m[g]);
+        cols_b = std::max(cols_b, plan.col_off[g] + plan.n[g]);
+      }
+    } else {
+      rows_a = plan.m[s];
+      cols_b = plan.n[s];
+    }
+    if (rows_a == 0 || cols_b == 0) { p.kblocks[s] = plan.chain ? p.kblocks[s] : 0; continue; }
+    if (!make_map(&p.map_a[s], plan.a[s], 2, rows_a, plan.kseg[s], plan.lda[s], BM, BK))
+      return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for operand x of shard %d", s);
+    if (!make_map(&p.map_b[s], plan.b[s], 2, plan.kseg[s], cols_b, plan.ldb[s], BK, 64))
+      return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for operand w of shard %d", s);
+  }
+  int tiles = 0;
+  const int box_cols = p.out_f32 ? 32 : 64;
+  for (int g = 0; g < plan.ngroups; ++g) {
+    p.m[g] = plan.m[g];
+    p.n[g] = plan.n[g];
+    p.row_off[g] = plan.row_off[g];
+    p.col_off[g] = plan.col_off[g];
+    p.tile_begin[g] = tiles;
+    const long long tm = (plan.m[g] + BM - 1) / BM, tn = (plan.n[g] + BN - 1) / BN;
+    p.tiles_m[g] = (int)std::max(1LL, tm);
+    if (plan.m[g] > 0 && plan.n[g] > 0) {
+      if (tm * tn + tiles > 0x3fffffffLL) return SBP_ERR_UNSUPPORTED;
+      tiles += (int)(tm * tn);
+      if (!make_map(&p.map_y[g], plan.y[g], oesz, plan.m[g], plan.n[g], plan.ldy[g], 32, box_cols))
+        return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for the result of group %d", g);
+    }
+  }
+  p.tile_begin[plan.ngroups] = tiles;
+  for (int g = plan.ngroups + 1; g <= SBP_MAX_K; ++g) p.tile_begin[g] = tiles;
+  p.total_tiles = tiles;
+  for (int r = 0; r < plan.n_rep; ++r)
+    if (!make_map(&p.map_rep[r], plan.y_rep[r], oesz, plan.m[0], plan.n[0], plan.ldy[0], 32, box_cols))
+      return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for a result replica");
+  *taken = true;
+  if (tiles == 0) return SBP_OK;
+
+  static int sm_count = 0;
+  if (sm_count == 0) {
+    int dev = 0;
+    SBP_CUDA_TRY(cudaGetDevice(&dev));
+    SBP_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+    SBP_CUDA_TRY(cudaFuncSetAttribute(matmul_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+  }
+  const int grid = tiles < sm_count ? tiles : sm_count;
+  matmul_tc_kernel<<<grid, kThreadsTc, kSmemBytes, st>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "tensor-core matmul launch");
+  count_launch();
+  return SBP_OK;
+}
+
+sbp_status read_and_clear_tc_timeout(bool* timed_out) {
+  int flag = 0, zero = 0;
+  SBP_CUDA_TRY(cudaMemcpyFromSymbol(&flag, g_tc_timeout_flag, sizeof(int)));
+  if (flag) SBP_CUDA_TRY(cudaMemcpyToSymbol(g_tc_timeout_flag, &zero, sizeof(int)));
+  *timed_out = flag != 0;
+  return SBP_OK;
 }
 
 }  // namespace sbp

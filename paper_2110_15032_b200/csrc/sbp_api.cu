@@ -69,6 +69,10 @@ int64_t local_numel(const sbp_tensor* t, int r) {
   return n;
 }
 
+// Defined next to the kernels that own the flags.
+sbp_status read_and_clear_bulk_timeout(bool* timed_out);
+sbp_status read_and_clear_tc_timeout(bool* timed_out);
+
 }  // namespace sbp
 
 using namespace sbp;
@@ -94,6 +98,17 @@ const char* sbp_status_string(sbp_status s) {
 const char* sbp_last_error(void) { return g_err; }
 
 uint64_t sbp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+sbp_status sbp_check_device_errors(void) {
+  bool bulk = false, tc = false;
+  sbp_status st = read_and_clear_bulk_timeout(&bulk);
+  if (st != SBP_OK) return st;
+  st = read_and_clear_tc_timeout(&tc);
+  if (st != SBP_OK) return st;
+  if (bulk) return fail(SBP_ERR_TIMEOUT, "a bulk-copy boxing kernel gave up waiting for its loads");
+  if (tc) return fail(SBP_ERR_TIMEOUT, "the tensor-core matmul kernel gave up waiting on one of its barriers");
+  return SBP_OK;
+}
 
 sbp_status sbp_local_shape(const sbp_tensor* t, int32_t r, int64_t out_shape[SBP_MAX_DIMS]) {
   sbp_status st = check_tensor(t, "t", false);

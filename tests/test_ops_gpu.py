@@ -321,3 +321,78 @@ def test_embedding_fused_equals_unfused_plus_boxing_with_negative_zero():
     torch.cuda.synchronize()
     for a, b in zip(fused.locals, boxed.locals):
         assert np.array_equal(bits(a), bits(b))
+
+
+# ------------------------------------------------------------------ tensor-core MatMul path
+
+@pytest.mark.parametrize("xs,ws", TABLE1)
+@pytest.mark.parametrize("k", [2, 3])
+def test_matmul_tensor_core_multi_tile_ragged(xs, ws, k):
+    """Shapes that span several 128 x 256 tiles and 64-deep K-blocks, with ragged edges in
+    every dimension (all leading dimensions stay multiples of 8 elements)."""
+    _matmul_case(392, 336, 528, k, BF16, xs, ws, seed=2001)
+
+
+@pytest.mark.parametrize("ys", [sbp.B, sbp.S(0), sbp.S(1)])
+@pytest.mark.parametrize("xs,ws", [(sbp.S(1), sbp.S(0)), (sbp.P_SUM, sbp.B)])
+def test_matmul_tensor_core_fused_boxing(xs, ws, ys):
+    _matmul_case(392, 336, 528, 4, BF16, xs, ws, ys=ys, seed=2002)
+    _matmul_case(256, 1024, 512, 8, BF16, xs, ws, ys=ys, seed=2003, out_dtype=F32)
+
+
+def test_matmul_tensor_core_gelu_and_many_tiles():
+    # more tiles than SMs, so every CTA walks several tiles and both accumulators
+    _matmul_case(2048, 256, 4096, 8, BF16, sbp.B, sbp.S(1), flags=sbp.SBP_EPILOGUE_GELU, seed=2004)
+    _matmul_case(2048, 512, 2048, 4, BF16, sbp.S(0), sbp.B, seed=2005)
+    _matmul_case(1024, 2048, 1024, 8, BF16, sbp.S(1), sbp.S(0), seed=2006)
+
+
+def test_mlp_block_small_against_oracle():
+    """The Megatron-style block at reduced size: B x S(1) -> S(1) with GeLU, S(1) x S(0) ->
+    P(sum) written directly as B.  Hidden state is stored as bf16 between the products."""
+    k, M, H, Fd = 8, 512, 256, 1024
+    X = dg.normal(1003, 0, (M, H), 0.0, 1.0, BF16)
+    W1 = dg.normal(1003, 1, (H, Fd), 0.0, 0.02, BF16)
+    W2 = dg.normal(1003, 2, (Fd, H), 0.0, 0.02, BF16)
+    x = make_global(split_cpu(X, sbp.B, k), (M, H), BF16, sbp.B)
+    w1 = make_global(split_cpu(W1, sbp.S(1), k), (H, Fd), BF16, sbp.S(1))
+    w2 = make_global(split_cpu(W2, sbp.S(0), k), (Fd, H), BF16, sbp.S(0))
+    h = sbp.empty_global((M, Fd), BF16, sbp.S(1), k)
+    y = sbp.empty_global((M, H), BF16, sbp.B, k)
+    sbp.sbp_matmul(x, w1, h, sbp.SBP_EPILOGUE_GELU)
+    sbp.sbp_matmul(h, w2, y)
+    torch.cuda.synchronize()
+    sbp.sbp_check_device_errors()
+    want = O.mlp_logical(to_np(X), to_np(W1), to_np(W2))
+    for t in y.locals:
+        assert_close(to_np(t), want, 2e-2, 1e-3, "MLP block")
+    # the unfused route (fp32 partials, then P(sum) -> B) gives the same values
+    yp = sbp.empty_global((M, H), F32, sbp.P_SUM, k)
+    yb = sbp.empty_global((M, H), F32, sbp.B, k)
+    sbp.sbp_matmul(h, w2, yp)
+    sbp.sbp_boxing(yp, yb)
+    torch.cuda.synchronize()
+    assert_close(to_np(yb.locals[0]), want, 2e-2, 1e-3, "MLP block, unfused")
+
+
+def test_classifier_chain_small_against_oracle():
+    """Features B x classifier weight S(1) -> bf16 logits S(1) -> split softmax cross entropy."""
+    k, rows, feat, classes = 8, 64, 512, 16384
+    Fm = dg.normal(1004, 0, (rows, feat), 0.0, 1.0, BF16)
+    W = dg.normal(1004, 2, (feat, classes), 0.0, 0.01, BF16)
+    labels = dg.integers(1004, 1, (rows,), 0, classes)
+    f = make_global(split_cpu(Fm, sbp.B, k), (rows, feat), BF16, sbp.B)
+    w = make_global(split_cpu(W, sbp.S(1), k), (feat, classes), BF16, sbp.S(1))
+    z = sbp.empty_global((rows, classes), BF16, sbp.S(1), k)
+    lab = make_global([labels] * k, (rows,), I64, sbp.B)
+    loss = sbp.empty_global((rows,), F32, sbp.B, k)
+    ws = torch.empty(sbp.sbp_softmax_xent_workspace_bytes(z), dtype=torch.uint8, device="cuda")
+    sbp.sbp_matmul(f, w, z)
+    sbp.sbp_softmax_xent(z, lab, loss, None, None, ws)
+    torch.cuda.synchronize()
+    Z = O.matmul_logical(to_np(Fm), to_np(W))
+    _, _, ref = O.softmax_xent_logical(Z, labels.numpy())
+    assert_close(to_np(loss.locals[0]), ref, 2e-2, 1e-3, "classifier chain loss")
+    zl = O.to_locals(Z, O.S1, k)
+    for r in range(k):
+        assert_close(to_np(z.locals[r]), zl[r], 2e-2, 1e-3, f"logits shard {r}")

@@ -196,6 +196,29 @@ sbp_status sbp_softmax_xent(const sbp_tensor* logits, const sbp_tensor* labels, 
                             sbp_tensor* row_max, sbp_tensor* row_sum, void* ws, size_t ws_bytes,
                             void* cuda_stream);
 
+/* Variant of sbp_softmax_xent for callers that have no device workspace to give and may not
+ * create one.  (The paper has no counterpart; this exists for programs that embed the library
+ * under constraints the paper does not discuss.)  Typical cases: a plug-in that runs inside
+ * someone else's memory plan, where every device byte was handed out up front and a fresh
+ * allocation would either fail or stall the device; or a latency-critical path that must not
+ * enter the allocator.  Same arguments, results and checks as sbp_softmax_xent, minus
+ * ws / ws_bytes: the per-shard partial vectors go into an array that is part of the library.
+ *
+ *   - The array is SBP_SOFTMAX_XENT_STATIC_SCRATCH_BYTES large and every GPU that loads the
+ *     library holds it until the process ends.  A shape whose partials need more is refused
+ *     with SBP_ERR_WORKSPACE and nothing is launched; use sbp_softmax_xent for those.
+ *   - The call allocates nothing on the device and frees nothing.
+ *   - The first call on each device looks up the array's device address (that device must be
+ *     current, as it must for the launch anyway).  Make that first call ahead of any stream
+ *     capture.
+ *   - All calls share the one array, and it keeps whatever the previous call left there.
+ *     Nothing in it has to start at zero: each call overwrites every entry it later reads.
+ *     Two calls that overlap on the GPU (different streams, no ordering between them) race on
+ *     it and may both produce wrong results; keep calls ordered. */
+#define SBP_SOFTMAX_XENT_STATIC_SCRATCH_BYTES (3u * 1024u * 1024u)
+sbp_status sbp_softmax_xent_static(const sbp_tensor* logits, const sbp_tensor* labels, sbp_tensor* loss,
+                                   sbp_tensor* row_max, sbp_tensor* row_sum, void* cuda_stream);
+
 /* ---------------------------------------------------------------- row-split embedding
  *
  * Section 6.3 (embedding table S(0), "splitting the vocabulary IDs"):

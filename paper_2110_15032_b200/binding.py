@@ -101,6 +101,7 @@ def load_library():
     lib.sbp_softmax_xent_workspace_bytes.restype = C.c_size_t
     lib.sbp_softmax_xent_workspace_bytes.argtypes = [T]
     lib.sbp_softmax_xent.argtypes = [T, T, T, T, T, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sbp_softmax_xent_static.argtypes = [T, T, T, T, T, C.c_void_p]
     lib.sbp_embedding.argtypes = [T, T, T, C.c_void_p, C.c_void_p]
     _LIB = lib
     return lib
@@ -239,6 +240,21 @@ def sbp_softmax_xent(logits: SbpTensor, labels: SbpTensor, loss: SbpTensor,
         C.byref(a), C.byref(b), C.byref(c),
         C.byref(m) if m is not None else None, C.byref(s) if s is not None else None,
         C.c_void_p(ws.data_ptr()), ws.numel() * ws.element_size(), _stream_ptr(stream)))
+
+
+def sbp_softmax_xent_static(logits: SbpTensor, labels: SbpTensor, loss: SbpTensor,
+                            row_max: Optional[SbpTensor] = None, row_sum: Optional[SbpTensor] = None,
+                            stream=None) -> None:
+    """sbp_softmax_xent without a workspace argument: the partial vectors live in an array
+    built into the library, for callers that cannot allocate device memory.  See
+    include/sbp.h for the size limit and the sharing rules."""
+    a, b, c = logits._c(), labels._c(), loss._c()
+    m = row_max._c() if row_max is not None else None
+    s = row_sum._c() if row_sum is not None else None
+    _check(load_library().sbp_softmax_xent_static(
+        C.byref(a), C.byref(b), C.byref(c),
+        C.byref(m) if m is not None else None, C.byref(s) if s is not None else None,
+        _stream_ptr(stream)))
 
 
 def sbp_embedding(table: SbpTensor, ids: SbpTensor, out: SbpTensor,

@@ -18,6 +18,8 @@
 #include <cfloat>
 #include <cmath>
 
+#include <mutex>
+
 #include "sbp_internal.h"
 
 namespace sbp {
@@ -377,3 +379,48 @@ sbp_status sbp_softmax_xent(const sbp_tensor* logits, const sbp_tensor* labels, 
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------ built-in scratch variant
+//
+// Scratch for callers that cannot hand in a workspace.  It lives in the library's image, so
+// every GPU that loads the library carries these 3 MiB until the process exits.
+namespace sbp {
+constexpr size_t kStaticScratchBytes = SBP_SOFTMAX_XENT_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) float g_xent_static_scratch[kStaticScratchBytes / sizeof(float)];
+constexpr int kMaxDevices = 64;
+}  // namespace sbp
+
+extern "C" sbp_status sbp_softmax_xent_static(const sbp_tensor* logits, const sbp_tensor* labels, sbp_tensor* loss,
+                                              sbp_tensor* row_max, sbp_tensor* row_sum, void* cuda_stream) {
+  // Size check first, so that an oversized request is refused before anything else happens.
+  sbp_status st = check_tensor(logits, "logits", true);
+  if (st != SBP_OK) return st;
+  if (logits->ndim != 2) return fail(SBP_ERR_SHAPE, "logits must be [rows, classes]");
+  const size_t need =
+      3 * (size_t)placement_k(logits) * (size_t)nsplit_for(logits, pick_vec(logits)) * (size_t)logits->shape[0] * sizeof(float);
+  if (need > kStaticScratchBytes)
+    return fail(SBP_ERR_WORKSPACE,
+                "this shape needs %zu bytes of scratch but the built-in array holds %zu; call sbp_softmax_xent "
+                "with a workspace of your own instead",
+                need, kStaticScratchBytes);
+
+  // In host code the array's name is only a handle; its device address has to be looked up,
+  // once per device, while that device is current.
+  static float* dev_ptr[kMaxDevices] = {};
+  static std::mutex mu;
+  int dev = 0;
+  SBP_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return fail(SBP_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
+  float* scratch = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(mu);
+    if (!dev_ptr[dev]) {
+      void* ptr = nullptr;
+      SBP_CUDA_TRY(cudaGetSymbolAddress(&ptr, g_xent_static_scratch));
+      dev_ptr[dev] = static_cast<float*>(ptr);
+    }
+    scratch = dev_ptr[dev];
+  }
+  return sbp_softmax_xent(logits, labels, loss, row_max, row_sum, scratch, kStaticScratchBytes, cuda_stream);
+}
+

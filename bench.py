@@ -214,12 +214,7 @@ def e2e_sweep(sbp, src, work, device, steps, dist):
     wall = time.perf_counter() - t0
     if dist is not None:
         dist.barrier()
-    ms = max(start.elapsed_time(end), wall * 1e3)
-    if dist is not None:
-        t = torch.tensor([ms], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    ms /= steps
+    ms = max_over_ranks(max(start.elapsed_time(end), wall * 1e3), dist, device) / steps
     # spot check: the last transform's result on the host equals the device-resident run
     ref = work[-1][2].locals[0].cpu()
     if not torch.equal(ref, jobs[-1][1].locals[0]):
@@ -402,6 +397,23 @@ def oracle_sweep_sample(rows: int):
     return nbytes, time.perf_counter() - t0, 1
 
 
+# ------------------------------------------------------------------------------ ranks
+
+def max_over_ranks(ms: float, dist, device) -> float:
+    """Slowest rank's time: what a multi-rank number is computed from."""
+    if dist is None:
+        return ms
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(world: int, ms_step: float) -> float:
+    """Every rank runs its own replica of the sweep (no collective on the data path), so the
+    job moves world x step_bytes() in the slowest rank's step time."""
+    return world * step_bytes() / (ms_step * 1e-3) / 1e9
+
+
 # ------------------------------------------------------------------------------ main
 
 def parse():
@@ -497,13 +509,9 @@ def main():
     launches = sbp.sbp_launch_count() - launches0
     clocks = sampler.stop() if rank == 0 else None
     sbp.sbp_check_device_errors()
-    ms_total = start.elapsed_time(end)
-    if dist is not None:
-        t = torch.tensor([ms_total], device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(start.elapsed_time(end), dist, device)
     ms_step = ms_total / args.steps
-    value = world * step_bytes() / (ms_step * 1e-3) / 1e9
+    value = whole_job_gbs(world, ms_step)
 
     per = []
     for i, (name, _, _, nbytes) in enumerate(work):

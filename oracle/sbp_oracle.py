@@ -71,6 +71,23 @@ def to_locals(T, sig, k):
     raise ValueError("to_locals is not defined for a partial-value signature")
 
 
+def locate(shape, sig, k, index):
+    """Where global element `index` (a tuple) lives under S(i) or B: a list of
+    (shard, local index) pairs -- one pair for S(i), k pairs for B (Section 3.1)."""
+    index = tuple(int(v) for v in index)
+    if sig[0] == "B":
+        return [(r, index) for r in range(k)]
+    if sig[0] == "S":
+        ax = sig[1]
+        for r, (start, ln) in enumerate(balanced_split(shape[ax], k)):
+            if start <= index[ax] < start + ln:
+                loc = list(index)
+                loc[ax] = index[ax] - start
+                return [(r, tuple(loc))]
+        raise IndexError(index)
+    raise ValueError("locate is not defined for a partial-value signature")
+
+
 def round_to_bf16(x32):
     """float32 -> nearest bf16 (ties to even), returned as float32.  Finite inputs."""
     x32 = np.ascontiguousarray(x32, dtype=np.float32)

@@ -1,0 +1,221 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times.
+
+The oracle cannot redo these sizes whole in seconds, so each case checks sampled outputs that
+the oracle computes one by one from the same seeded inputs (the needed input elements are
+copied off the device; no expected value comes from the CUDA path), plus properties that hold
+at any size (replicas equal, round trips return the input bits)."""
+import numpy as np
+import pytest
+import torch
+from helpers import assert_close, bits, np_bits, osig, to_np
+
+import bench
+import paper_2110_15032_b200 as sbp
+import sbp_datagen as dg
+from oracle import sbp_oracle as O
+
+pytestmark = pytest.mark.gpu
+
+F32, BF16, I64 = torch.float32, torch.bfloat16, torch.int64
+DEV = "cuda"
+
+
+def _sample_indices(shape, k, n, seed):
+    """Random logical indices plus the corners and every shard boundary of both axes."""
+    rng = np.random.default_rng(seed)
+    idx = {(int(rng.integers(shape[0])), int(rng.integers(shape[1]))) for _ in range(n)}
+    edges0 = {0, shape[0] - 1} | {s for s, _ in O.balanced_split(shape[0], k)} | {s + l - 1 for s, l in O.balanced_split(shape[0], k) if l}
+    edges1 = {0, shape[1] - 1} | {s for s, _ in O.balanced_split(shape[1], k)} | {s + l - 1 for s, l in O.balanced_split(shape[1], k) if l}
+    idx |= {(i, j) for i in edges0 for j in edges1}
+    return sorted(idx)
+
+
+def _gather(global_tensor, shard_local_pairs):
+    """Values at [(shard, local index)] of an SbpTensor, as exact float32 / int numpy."""
+    out = []
+    by_shard = {}
+    for pos, (r, li) in enumerate(shard_local_pairs):
+        by_shard.setdefault(r, []).append((pos, li))
+    vals = [None] * len(shard_local_pairs)
+    for r, items in by_shard.items():
+        ii = torch.tensor([li for _, li in items], device=global_tensor.locals[r].device)
+        got = global_tensor.locals[r][tuple(ii[:, d] for d in range(ii.shape[1]))]
+        got = to_np(got)
+        for (pos, _), v in zip(items, got):
+            vals[pos] = v
+    return np.array(vals)
+
+
+def test_config2_boxing_sweep_full_size_sampled():
+    k, shape = bench.SWEEP_K, (8192, 8192)
+    T, src, work = bench.build_sweep(sbp, torch.device(DEV))
+    bench.run_sweep(sbp, work)
+    torch.cuda.synchronize()
+    sbp.sbp_check_device_errors()
+    samples = _sample_indices(shape, k, 3000, 7)
+    for name, s, d, _ in work:
+        # logical value of every sample, by the oracle, from the source local tensors
+        if s.sig.kind == 2:
+            per_shard = [_gather(s, [(r, ix) for ix in samples]) for r in range(k)]
+            logical = O.reduce_sum_fixed_order(per_shard, "bf16")
+        else:
+            logical = _gather(s, [O.locate(shape, osig(s.sig), k, ix)[0] for ix in samples])
+        pairs, expect = [], []
+        for ix, v in zip(samples, logical):
+            for pr in O.locate(shape, osig(d.sig), k, ix):
+                pairs.append(pr)
+                expect.append(v)
+        got = _gather(d, pairs)
+        assert np.array_equal(np_bits(got, BF16), np_bits(np.array(expect), BF16)), name
+    # any-size properties: B replicas identical; S(0)->S(1)->S(0) returns the input bits
+    by_name = {w[0]: w for w in work}
+    for nm in ("P(sum)->B", "S(0)->B"):
+        reps = by_name[nm][2].locals
+        assert all(torch.equal(reps[0], r) for r in reps[1:]), nm
+    assert torch.equal(by_name["S(0)->B"][2].locals[0], T)
+    back = sbp.empty_global(shape, BF16, sbp.S(0), k)
+    sbp.sbp_boxing(by_name["S(0)->S(1)"][2], back)
+    torch.cuda.synchronize()
+    assert all(torch.equal(a, b) for a, b in zip(back.locals, src["S0"].locals))
+
+
+def test_config3_mlp_full_size_sampled_rows():
+    k, M, H, Fd = 8, 8192, 4096, 16384
+    dev = torch.device(DEV)
+    X = dg.normal(1003, 0, (M, H), 0.0, 1.0, BF16, dev)
+    w1l = [dg.normal(1003, 10 + r, (H, Fd // k), 0.0, 0.02, BF16, dev) for r in range(k)]
+    w2l = [dg.normal(1003, 30 + r, (Fd // k, H), 0.0, 0.02, BF16, dev) for r in range(k)]
+    x = sbp.SbpTensor((M, H), BF16, sbp.B, [X] * k)
+    w1 = sbp.SbpTensor((H, Fd), BF16, sbp.S(1), w1l)
+    w2 = sbp.SbpTensor((Fd, H), BF16, sbp.S(0), w2l)
+    h = sbp.empty_global((M, Fd), BF16, sbp.S(1), k)
+    y = sbp.empty_global((M, H), BF16, sbp.B, k)
+    sbp.sbp_matmul(x, w1, h, sbp.SBP_EPILOGUE_GELU)
+    sbp.sbp_matmul(h, w2, y)
+    torch.cuda.synchronize()
+    sbp.sbp_check_device_errors()
+    rows = [0, 127, 128, 4095, 8191]
+    W1 = O.from_locals([to_np(t) for t in w1l], O.S1)
+    W2 = O.from_locals([to_np(t) for t in w2l], O.S0)
+    Xs = to_np(X[rows])
+    Hs = O.gelu(O.matmul_logical(Xs, W1))
+    want = O.matmul_logical(Hs, W2)
+    # first product + GeLU: one rounding, the stated tolerance applies as it stands
+    hl = O.to_locals(Hs, O.S1, k)
+    for r in (0, 3, 7):
+        assert_close(to_np(h.locals[r][rows]), hl[r], 2e-2, 1e-3, f"hidden shard {r}")
+    # whole block: the hidden state is stored as bf16 (unit roundoff 2^-8) between the products,
+    # which perturbs Y_ij by a sum of 16384 independent terms of standard deviation
+    # <= (2^-8 / sqrt 3) |G_if W2_fj|.  That noise does not shrink with |Y_ij|, so on top of the
+    # stated tolerance the test allows 2^-6 sqrt(sum_f G_if^2 W2_fj^2)  (about 7 sigma).
+    noise = 2.0 ** -6 * np.sqrt(O.matmul_logical(Hs ** 2, W2.astype(np.float64) ** 2))
+    for t in (y.locals[0], y.locals[k - 1]):
+        err = np.abs(to_np(t[rows]).astype(np.float64) - want)
+        assert np.all(err <= 1e-3 + 2e-2 * np.abs(want) + noise), float((err - noise).max())
+    assert all(torch.equal(y.locals[0], t) for t in y.locals[1:])
+    # second product on its own, seeded bf16 input in place of the hidden state: the stated
+    # tolerance as it stands, for the fused (S(1),S(0)) -> B route and for fp32 partials + boxing
+    del h, y
+    hs = [dg.normal(1003, 50 + r, (M, Fd // k), 0.0, 1.0, BF16, dev) for r in range(k)]
+    hin = sbp.SbpTensor((M, Fd), BF16, sbp.S(1), hs)
+    yb = sbp.empty_global((M, H), BF16, sbp.B, k)
+    sbp.sbp_matmul(hin, w2, yb)
+    torch.cuda.synchronize()
+    Hin = O.from_locals([to_np(t[rows]) for t in hs], O.S1)
+    want2 = O.matmul_logical(Hin, W2)
+    assert_close(to_np(yb.locals[k - 1][rows]), want2, 2e-2, 1e-3, "second product, fused to B")
+    yp = sbp.empty_global((M, H), F32, sbp.P_SUM, k)
+    sbp.sbp_matmul(hin, w2, yp)
+    torch.cuda.synchronize()
+    _, parts, _ = O.matmul_locals(O.to_locals(Hin, O.S1, k), O.S1, O.to_locals(W2, O.S0, k), O.S0)
+    for r in (0, 6):
+        assert_close(to_np(yp.locals[r][rows]), parts[r], 2e-2, 1e-3, f"partial product {r}")
+    sbp.sbp_check_device_errors()
+
+
+def test_config4_softmax_and_classifier_full_size_sampled_rows():
+    k, rows, feat, classes = 8, 512, 512, 1 << 20
+    dev = torch.device(DEV)
+    sigma = (512 ** 0.5) * 0.01
+    labels = dg.integers(1004, 1, (rows,), 0, classes, dev)
+    lab = sbp.SbpTensor((rows,), I64, sbp.B, [labels] * k)
+    # (a) the softmax kernel on seeded logits, exactly as bench.py streams them
+    zl = [dg.normal(1004, 10 + r, (rows, classes // k), 0.0, sigma, BF16, dev) for r in range(k)]
+    logits = sbp.SbpTensor((rows, classes), BF16, sbp.S(1), zl)
+    loss = sbp.empty_global((rows,), F32, sbp.B, k)
+    rmax = sbp.empty_global((rows,), F32, sbp.B, k)
+    rsum = sbp.empty_global((rows,), F32, sbp.B, k)
+    ws = torch.empty(sbp.sbp_softmax_xent_workspace_bytes(logits), dtype=torch.uint8, device=dev)
+    sbp.sbp_softmax_xent(logits, lab, loss, rmax, rsum, ws)
+    torch.cuda.synchronize()
+    pick = [0, 1, 255, 256, 511]
+    Z = O.from_locals([to_np(t[pick]) for t in zl], O.S1)
+    m, S, ref = O.softmax_xent_logical(Z, labels[pick].cpu().numpy())
+    assert_close(to_np(loss.locals[0][pick]), ref, 2e-2, 1e-3, "loss")
+    assert np.array_equal(to_np(rmax.locals[k - 1][pick]).astype(np.float64), m)
+    assert_close(to_np(rsum.locals[0][pick]), S, 2e-2, 1e-3, "row_sum")
+    assert np.all(np.abs(to_np(loss.locals[0][pick]) - ref) <= 1e-4 * np.abs(ref))      # in fact far tighter
+    del zl, logits
+    # (b) the classifier product feeding it: F (B) x W (S(1)) -> bf16 logits S(1), then the loss
+    Fm = dg.normal(1004, 0, (rows, feat), 0.0, 1.0, BF16, dev)
+    wl = [dg.normal(1004, 40 + r, (feat, classes // k), 0.0, 0.01, BF16, dev) for r in range(k)]
+    f = sbp.SbpTensor((rows, feat), BF16, sbp.B, [Fm] * k)
+    w = sbp.SbpTensor((feat, classes), BF16, sbp.S(1), wl)
+    z = sbp.empty_global((rows, classes), BF16, sbp.S(1), k)
+    sbp.sbp_matmul(f, w, z)
+    sbp.sbp_softmax_xent(z, lab, loss, None, None, ws)
+    torch.cuda.synchronize()
+    sbp.sbp_check_device_errors()
+    pick = [3, 300]
+    Fs = to_np(Fm[pick])
+    Zs = []
+    for r in range(k):
+        Zr = O.matmul_logical(Fs, to_np(wl[r]))
+        assert_close(to_np(z.locals[r][pick]), Zr, 2e-2, 1e-3, f"logits shard {r}")
+        Zs.append(Zr)
+    _, _, ref = O.softmax_xent_logical(O.from_locals(Zs, O.S1), labels[pick].cpu().numpy())
+    assert_close(to_np(loss.locals[0][pick]), ref, 2e-2, 1e-3, "chain loss")
+
+
+def test_config5_embedding_full_size_sampled_lookups():
+    k, rows, dim = 8, 1 << 24, 128
+    dev = torch.device(DEV)
+    ids = dg.zipf_ids(1005, 1, (65536, 26), rows, 1.05, dev)
+    tl = [dg.uniform(1005, 100 + r, (rows // k, dim), -0.05, 0.05, F32, dev) for r in range(k)]
+    table = sbp.SbpTensor((rows, dim), F32, sbp.S(0), tl)
+    idt = sbp.SbpTensor((65536, 26), I64, sbp.B, [ids] * k)
+    out_b = sbp.empty_global((65536, 26, dim), F32, sbp.B, k)
+    oob = torch.zeros(1, dtype=torch.int32, device=dev)
+    sbp.sbp_embedding(table, idt, out_b, oob)
+    torch.cuda.synchronize()
+    assert int(oob.item()) == 0
+    rng = np.random.default_rng(5)
+    picks = [(int(rng.integers(65536)), int(rng.integers(26))) for _ in range(4096)] + [(0, 0), (65535, 25)]
+    idv = ids.cpu().numpy()
+    # expected rows by the oracle's own lookup on the sampled table rows
+    need = sorted({int(idv[b, f]) for b, f in picks})
+    row_of = {g: i for i, g in enumerate(need)}
+    pairs = [O.locate((rows, dim), O.S0, k, (g, 0))[0] for g in need]
+    sub = np.stack([to_np(tl[r][li[0]]) for r, li in pairs])             # [len(need), dim]
+    sub_ids = np.array([[row_of[int(idv[b, f])] for b, f in picks]])
+    want = O.embedding_logical(sub, sub_ids)[0] + np.float32(0.0)
+    bi = torch.tensor([b for b, _ in picks], device=dev)
+    fi = torch.tensor([f for _, f in picks], device=dev)
+    for t in (out_b.locals[0], out_b.locals[k - 1]):
+        assert np.array_equal(bits(t[bi, fi]), np_bits(want, F32))
+    assert all(torch.equal(out_b.locals[0], t) for t in out_b.locals[1:])
+    # unfused: P(sum) shards, then boxing, equals the fused result bit for bit
+    del out_b.locals[1:]
+    fused0 = out_b.locals[0]
+    out_p = sbp.empty_global((65536, 26, dim), F32, sbp.P_SUM, k)
+    sbp.sbp_embedding(table, idt, out_p)
+    torch.cuda.synchronize()
+    owner = np.array([O.locate((rows, dim), O.S0, k, (int(idv[b, f]), 0))[0][0] for b, f in picks])
+    for r in (0, 5):
+        got = to_np(out_p.locals[r][bi, fi])
+        exp = np.where((owner == r)[:, None], O.embedding_logical(sub, sub_ids)[0], np.float32(0.0))
+        assert np.array_equal(np_bits(got, F32), np_bits(exp, F32))
+    boxed = sbp.SbpTensor((65536, 26, dim), F32, sbp.B, [torch.empty_like(fused0)] * k)
+    sbp.sbp_boxing(out_p, boxed)
+    torch.cuda.synchronize()
+    assert torch.equal(boxed.locals[0], fused0)

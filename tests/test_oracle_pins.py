@@ -497,3 +497,15 @@ def test_boxing_p_to_p_keeps_each_partial():
     out = O.boxing(loc, PSUM, PSUM)
     assert all(np.array_equal(a, b) and a is not b for a, b in zip(out, loc))
     assert O.table2_same_placement_cost(PSUM, PSUM, 3, 60) == 0
+
+
+@pytest.mark.parametrize("shape,k", [((5, 7), 3), ((4, 6, 5), 4), ((9,), 2)])
+def test_locate_agrees_with_to_locals(shape, k):
+    T = np.arange(int(np.prod(shape)), dtype=np.float32).reshape(shape)
+    for axis in range(len(shape)):
+        loc = O.to_locals(T, O.S(axis), k)
+        for idx in itertools.product(*[range(s) for s in shape]):
+            (r, li), = O.locate(shape, O.S(axis), k, idx)
+            assert loc[r][li] == T[idx]
+    pairs = O.locate(shape, B, k, (0,) * len(shape))
+    assert [r for r, _ in pairs] == list(range(k)) and all(li == (0,) * len(shape) for _, li in pairs)

@@ -362,9 +362,11 @@ def section_classifier_gemm(sbp, device, peaks):
     return [e]
 
 
-def run_operator_sections(sbp, device, peaks):
+def run_operator_sections(sbp, device, peaks, which="softmax,classifier,mlp,embedding"):
     out = []
-    for fn in (section_softmax, section_classifier_gemm, section_mlp, section_embedding):
+    table = {"softmax": section_softmax, "classifier": section_classifier_gemm, "mlp": section_mlp,
+             "embedding": section_embedding}
+    for fn in [table[w.strip()] for w in which.split(",") if w.strip()]:
         try:
             out.extend(fn(sbp, device, peaks))
         except sbp.SbpError as e:            # an operator this build cannot run is reported, not hidden
@@ -424,6 +426,8 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-ops", action="store_true", help="skip the sharded-operator sections (N = 1 only)")
+    ap.add_argument("--ops", default="softmax,classifier,mlp,embedding",
+                    help="comma-separated operator sections to run: softmax, classifier, mlp, embedding")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--copy-engine", type=int, default=0)
     ap.add_argument("--rows", type=int, default=SWEEP_SHAPE[0],
@@ -560,7 +564,7 @@ def main():
         if not args.no_ops:
             del T, src, work
             torch.cuda.empty_cache()
-            line["ops"] = run_operator_sections(sbp, device, peaks)
+            line["ops"] = run_operator_sections(sbp, device, peaks, args.ops)
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

@@ -130,8 +130,10 @@ __device__ __forceinline__ void task_geometry(const BoxParams& p, int s, int d, 
 template <typename V, int OP, int J, int KT>
 __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ BoxParams p) {
   const long long u = blockIdx.x;
-  const int t = (int)(u / p.tiles_per_task);
-  const long long rem = u - (long long)t * p.tiles_per_task;
+  // Task index varies fastest: CTAs that run together then touch the same rows of every shard
+  // (whole DRAM pages) instead of one column stripe of one shard.
+  const long long rem = u / p.ntasks;
+  const int t = (int)(u - rem * p.ntasks);
   const long long row_tile = rem / p.col_tiles;
   const long long col_tile = rem - row_tile * p.col_tiles;
 
@@ -397,6 +399,7 @@ static sbp_status make_plan(const sbp_tensor* src, const sbp_tensor* dst, Plan* 
   const long long row_tiles = std::max(1LL, (nseg_max + p.rows_per_tile - 1) / p.rows_per_tile);
   p.tiles_per_task = p.col_tiles * row_tiles;
   pl->ntasks = p.mode == MODE_PAIRS ? k * k : (p.mode == MODE_REDUCE_B ? 1 : k);
+  p.ntasks = pl->ntasks;
   pl->grid = p.tiles_per_task * pl->ntasks;
   if (pl->grid > 0x7fffffffLL) return fail(SBP_ERR_UNSUPPORTED, "tensor too large for one launch");
   return SBP_OK;

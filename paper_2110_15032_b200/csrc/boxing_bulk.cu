@@ -73,8 +73,8 @@ struct BulkTile {
 __device__ __forceinline__ BulkTile bulk_tile(const BulkParams& q, long long u) {
   const BoxParams& p = q.b;
   BulkTile g;
-  const int t = (int)(u / q.tiles_per_task);
-  const long long rem = u - (long long)t * q.tiles_per_task;
+  const long long rem = u / p.ntasks;            // task index varies fastest (see boxing.cu)
+  const int t = (int)(u - rem * p.ntasks);
   const long long row_tile = rem / q.col_tiles, col_tile = rem - row_tile * q.col_tiles;
   g.s = t;
   g.d = t;

@@ -25,6 +25,7 @@ struct BoxParams {
   int n_dst;                        // distinct destination buffers (GATHER / REDUCE_B)
   int cv_log2;                      // tile width in vectors, log2
   int rows_per_tile;
+  int ntasks;                       // tasks of the transform; tiles are dealt task-fastest
 };
 
 }  // namespace sbp

@@ -1,25 +1,31 @@
 // Tensor-core MatMul for sm_100a: bf16 operands, fp32 accumulation in tensor memory.
 //
-// One persistent CTA per SM walks the (group, m-tile, n-tile) list of a grouped-GEMM plan
-// (matmul_plan.h).  Tile = 128 x 256 outputs, K-block = 64.  Six warps, three roles:
+// Pairs of CTAs (a cluster of two SMs) walk the (group, m-tile, n-tile) list of a grouped-GEMM
+// plan (matmul_plan.h).  A pair owns one 256 x 256 output tile at a time: CTA r of the pair
+// holds rows 128 r .. 128 r + 127 of the A tile, columns 128 r .. 128 r + 127 of the B tile and
+// rows 128 r .. of the accumulator in its own tensor memory; one tcgen05.mma.cta_group::2
+// instruction, issued by the pair's first CTA, multiplies across both.  Per CTA and 64-deep
+// K-block that is 16 KiB of A and 16 KiB of B through TMA for 2 x 128 x 256 x 64 MACs, two
+// thirds of what two independent 128 x 256 CTAs would pull from L2.
 //
-//   warp 0  producer   TMA loads of the A tile [128 x 64] (K-major) and the B tile [64 x 256]
-//                      (N-major, four 64-column boxes) into a kStages-deep shared-memory ring
-//   warp 1  MMA        one thread issues tcgen05.mma (M128 N256 K16, four per K-block) into one
-//                      of two 256-column accumulators in tensor memory; tcgen05.commit frees
-//                      the ring slot and, after the last K-block, publishes the accumulator
-//   warps 2-5 epilogue each warp drains its own 32 lanes of the accumulator (tcgen05.ld),
-//                      applies GeLU when asked, rounds to the output type, stages 32 x 128-byte
-//                      slabs in shared memory and writes them with TMA stores -- once per
-//                      destination replica -- while the MMA warp already fills the other
-//                      accumulator
+//   warp 0     producer   TMA loads of this CTA's A and B halves into a kStages-deep ring; the
+//                         transaction bytes of both CTAs land on the first CTA's "full" barrier
+//   warp 1     MMA        (first CTA only) one thread issues four M256 N256 K16 MMAs per K-block
+//                         into one of two 256-column accumulators; tcgen05.commit, delivered to
+//                         both CTAs, frees the ring slot / publishes the accumulator
+//   warps 2-9  epilogue   warp w drains lanes 32 (w mod 4) .. +31, columns 128 ((w-2)/4) .. +127
+//                         of its CTA's accumulator (tcgen05.ld), applies GeLU when asked, rounds
+//                         to the output type, stages 32 x 128-byte slabs in swizzled shared memory
+//                         and writes them with TMA stores, once per destination replica, while
+//                         the next tile's MMAs fill the other accumulator
 //
 // A fused "P(sum) product written as B / S(i)" plan simply chains the K-blocks of all shards'
 // operands, in rank order, into the same accumulator: the partial products are never stored.
 //
 // Every wait is bounded in time.  A wait that expires raises a flag that
 // sbp_check_device_errors() reports; the CTA then stops issuing work, waits (bounded) for the
-// loads it still has in flight, frees its tensor memory and returns.
+// loads it still has in flight, meets its partner at the closing cluster barrier, frees its
+// tensor memory and returns.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -32,15 +38,17 @@
 
 namespace sbp {
 
-constexpr int BM = 128, BN = 256, BK = 64;
-constexpr int kStages = 4;
-constexpr int kStageA = BM * BK * 2;              // 16 KiB
-constexpr int kStageB = BK * BN * 2;              // 32 KiB
-constexpr int kStageBytes = kStageA + kStageB;    // 48 KiB
+constexpr int BM = 256, BN = 256, BK = 64;      // tile of a CTA pair
+constexpr int BMH = BM / 2, BNH = BN / 2;       // what one CTA of the pair loads
+constexpr int kStages = 5;
+constexpr int kStageA = BMH * BK * 2;             // 16 KiB
+constexpr int kStageB = BK * BNH * 2;             // 16 KiB
+constexpr int kStageBytes = kStageA + kStageB;    // 32 KiB per CTA
+constexpr int kEpiWarps = 8;
 constexpr int kSlabBytes = 32 * 128;              // one epilogue slab: 32 rows x 128 bytes
-constexpr int kEpiBytes = 4 * 2 * kSlabBytes;     // 4 warps x 2 buffers
+constexpr int kEpiBytes = kEpiWarps * 2 * kSlabBytes;
 constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024;   // + alignment slack
-constexpr int kThreadsTc = 192;
+constexpr int kThreadsTc = 32 * (2 + kEpiWarps);
 constexpr int kTmemCols = 512;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
@@ -109,9 +117,34 @@ __device__ __forceinline__ void mbar_arrive(unsigned bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 
+// Address of the same shared-memory object in CTA `rank` of this cluster.
+__device__ __forceinline__ unsigned map_to_cta(unsigned addr, unsigned rank) {
+  unsigned r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+
+// Arrive on an mbarrier that may live in the partner CTA (cluster-space address).
+__device__ __forceinline__ void mbar_arrive_cluster(unsigned cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+
+__device__ __forceinline__ unsigned cluster_ctarank() {
+  unsigned r;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+  return r;
+}
+
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+
+// TMA load into this CTA's shared memory; the byte count is credited to `bar`, which may be the
+// partner CTA's barrier (pair form of the instruction; no multicast).
 __device__ __forceinline__ void tma_load_2d(unsigned dst, const CUtensorMap* map, int x, int y, unsigned bar) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
+      "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(dst),
       "l"(map), "r"(x), "r"(y), "r"(bar)
       : "memory");
 }
@@ -122,19 +155,24 @@ __device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int 
                : "memory");
 }
 
+// One MMA across the CTA pair: D[256 x 256] (+)= A[256 x 16] * B[16 x 256].
 __device__ __forceinline__ void umma_bf16(unsigned d_tmem, unsigned long long a_desc, unsigned long long b_desc,
                                           unsigned idesc, unsigned accumulate) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
       "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
       : "memory");
 }
 
-// Arrives on an mbarrier once every tcgen05 operation issued so far by this thread is done.
-__device__ __forceinline__ void umma_commit(unsigned bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+// Arrives on the barrier at this offset in BOTH CTAs of the pair once every tcgen05 operation
+// issued so far by this thread is done.
+__device__ __forceinline__ void umma_commit_pair(unsigned bar) {
+  const unsigned short mask = 3;
+  asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;" ::"r"(bar),
+               "h"(mask)
+               : "memory");
 }
 
 __device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
@@ -162,11 +200,27 @@ __device__ __forceinline__ unsigned long long smem_desc(unsigned addr, unsigned 
   return d;
 }
 
-// Instruction descriptor: D fp32, A and B bf16, A K-major, B N-major, M = 128, N = 256.
+// Instruction descriptor: D fp32, A and B bf16, A K-major, B N-major, M = 256 (pair), N = 256.
 constexpr unsigned kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((BN >> 3) << 17) |
                             ((BM >> 4) << 24);
 
-__device__ __forceinline__ float gelu_erf_tc(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f)); }
+// erf by the rational approximation 7.1.26 of Abramowitz & Stegun (|error| <= 1.5e-7), which is
+// far below the rounding of the bf16 / fp32 store that follows and costs two special-function
+// operations where erff costs a long polynomial.
+__device__ __forceinline__ float erf_as(float x) {
+  const float ax = fabsf(x);
+  const float t = __frcp_rn(fmaf(0.3275911f, ax, 1.0f));
+  float poly = fmaf(1.061405429f, t, -1.453152027f);
+  poly = fmaf(poly, t, 1.421413741f);
+  poly = fmaf(poly, t, -0.284496736f);
+  poly = fmaf(poly, t, 0.254829592f);
+  poly *= t;
+  float e;
+  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(-ax * ax * 1.4426950408889634f));
+  return copysignf(fmaf(-poly, e, 1.0f), x);
+}
+
+__device__ __forceinline__ float gelu_erf_tc(float v) { return 0.5f * v * (1.0f + erf_as(v * 0.70710678118654752440f)); }
 
 struct TileCoord {
   int g, m0, n0;
@@ -182,7 +236,8 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
 
 // ------------------------------------------------------------------ the kernel
 
-__global__ void __launch_bounds__(kThreadsTc, 1) matmul_tc_kernel(const __grid_constant__ TcParams p) {
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
+    matmul_tc_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ __align__(8) unsigned long long bar_full[kStages], bar_empty[kStages], bar_acc_full[2], bar_acc_empty[2];
   __shared__ unsigned tmem_base_slot;
@@ -192,35 +247,37 @@ __global__ void __launch_bounds__(kThreadsTc, 1) matmul_tc_kernel(const __grid_c
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   unsigned char* epi = smem + kStages * kStageBytes;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned rank = cluster_ctarank();     // 0 = the CTA that issues the pair's MMAs
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
     for (int i = 0; i < kStages; ++i) {
-      mbar_init(smem_addr(&bar_full[i]), 1);
-      mbar_init(smem_addr(&bar_empty[i]), 1);
+      mbar_init(smem_addr(&bar_full[i]), 1);      // used in CTA 0 only: one arrive + both CTAs' bytes
+      mbar_init(smem_addr(&bar_empty[i]), 1);     // one commit per use, delivered to both CTAs
     }
     for (int i = 0; i < 2; ++i) {
       mbar_init(smem_addr(&bar_acc_full[i]), 1);
-      mbar_init(smem_addr(&bar_acc_empty[i]), 4);
+      mbar_init(smem_addr(&bar_acc_empty[i]), 2 * kEpiWarps);   // used in CTA 0 only: both CTAs' epilogue warps
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&tmem_base_slot)),
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_addr(&tmem_base_slot)),
                  "r"(kTmemCols)
                  : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  cluster_sync_all();                            // both CTAs' barriers exist before anyone signals them
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const unsigned tmem_base = tmem_base_slot;
 
-  const int first = blockIdx.x, stride = gridDim.x;
+  const int first = blockIdx.x >> 1, stride = gridDim.x >> 1;   // tiles are dealt to CTA pairs
 
   if (warp == 0) {
-    // ------------------------------------------------ producer
+    // ------------------------------------------------ producer (both CTAs)
     if (lane == 0) {
       long long kb_iter = 0;
       for (int tile = first; tile < p.total_tiles && !*abort_flag; tile += stride) {
@@ -231,19 +288,20 @@ __global__ void __launch_bounds__(kThreadsTc, 1) matmul_tc_kernel(const __grid_c
             const int slot = (int)(kb_iter % kStages);
             const unsigned parity = (unsigned)(((kb_iter / kStages) & 1) ^ 1);
             if (!mbar_wait(smem_addr(&bar_empty[slot]), parity, abort_flag)) goto producer_done;
-            const unsigned full = smem_addr(&bar_full[slot]);
-            mbar_expect_tx(full, kStageBytes);
+            const unsigned full0 = map_to_cta(smem_addr(&bar_full[slot]), 0);
+            if (rank == 0) mbar_expect_tx(smem_addr(&bar_full[slot]), 2 * kStageBytes);
             unsigned char* sa = smem + slot * kStageBytes;
             unsigned char* sb = sa + kStageA;
-            tma_load_2d(smem_addr(sa), &p.map_a[s], kb * BK, (int)p.row_off[tc.g] + tc.m0, full);
+            tma_load_2d(smem_addr(sa), &p.map_a[s], kb * BK, (int)p.row_off[tc.g] + tc.m0 + (int)rank * BMH, full0);
 #pragma unroll
-            for (int c = 0; c < BN / 64; ++c)
-              tma_load_2d(smem_addr(sb + c * (BK * 128)), &p.map_b[s], (int)p.col_off[tc.g] + tc.n0 + c * 64, kb * BK, full);
+            for (int c = 0; c < BNH / 64; ++c)
+              tma_load_2d(smem_addr(sb + c * (BK * 128)), &p.map_b[s],
+                          (int)p.col_off[tc.g] + tc.n0 + (int)rank * BNH + c * 64, kb * BK, full0);
           }
         }
       }
     producer_done:
-      if (*abort_flag) {
+      if (*abort_flag && rank == 0) {
         // give the loads still in flight a bounded chance to land before the CTA goes away
         const long long issued = kb_iter;
         for (long long i = issued > kStages ? issued - kStages : 0; i < issued; ++i) {
@@ -254,8 +312,8 @@ __global__ void __launch_bounds__(kThreadsTc, 1) matmul_tc_kernel(const __grid_c
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------ MMA issuer (first CTA of the pair only)
+    if (lane == 0 && rank == 0) {
       long long kb_iter = 0;
       int tile_iter = 0;
       for (int tile = first; tile < p.total_tiles && !*abort_flag; tile += stride, ++tile_iter) {
@@ -282,24 +340,26 @@ __global__ void __launch_bounds__(kThreadsTc, 1) matmul_tc_kernel(const __grid_c
               // A: K-major, rows of 128 bytes, 8-row groups 1024 bytes apart; 16 K-elements = 32 bytes
               const unsigned long long da = smem_desc(sa + kk * 32, 16, 1024);
               // B: N-major, 64-column chunks BK*128 bytes apart, 8-row K groups 1024 bytes apart;
-              //    16 K-rows = 2048 bytes
+              //    16 K-rows = 2048 bytes.  Each CTA holds its 128 of the 256 columns at this offset.
               const unsigned long long db = smem_desc(sb + kk * 2048, BK * 128, 1024);
               umma_bf16(d_tmem, da, db, kIdesc, accumulate);
               accumulate = 1;
             }
-            umma_commit(smem_addr(&bar_empty[slot]));   // slot reusable once these MMAs have read it
+            umma_commit_pair(smem_addr(&bar_empty[slot]));   // slot reusable in both CTAs
           }
         }
         if (!ok) break;
-        umma_commit(smem_addr(&bar_acc_full[acc]));      // accumulator complete
+        umma_commit_pair(smem_addr(&bar_acc_full[acc]));      // accumulator complete in both CTAs
       }
     }
   } else {
-    // ------------------------------------------------ epilogue (warps 2..5)
+    // ------------------------------------------------ epilogue (warps 2..9, both CTAs)
     const int q = warp & 3;                       // the 32 tensor-memory lanes this warp may read
+    const int half = (warp - 2) >> 2;             // which 128 of the 256 columns
     unsigned char* my_epi = epi + (warp - 2) * 2 * kSlabBytes;
     const int cols_per_slab = p.out_f32 ? 32 : 64;
-    const int nslabs = BN / cols_per_slab;
+    const int nslabs = (BN / 2) / cols_per_slab;
+    const unsigned acc_empty0[2] = {map_to_cta(smem_addr(&bar_acc_empty[0]), 0), map_to_cta(smem_addr(&bar_acc_empty[1]), 0)};
     int tile_iter = 0;
     unsigned slab_iter = 0;
     for (int tile = first; tile < p.total_tiles; tile += stride, ++tile_iter) {
@@ -312,10 +372,10 @@ __global__ void __launch_bounds__(kThreadsTc, 1) matmul_tc_kernel(const __grid_c
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const long long Mg = p.m[tc.g], Ng = p.n[tc.g];
-      const int row0 = tc.m0 + q * 32;
-      const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * BN;
+      const int row0 = tc.m0 + (int)rank * BMH + q * 32;
+      const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * BN + half * (BN / 2);
       for (int sl = 0; sl < nslabs; ++sl) {
-        const int col0 = tc.n0 + sl * cols_per_slab;
+        const int col0 = tc.n0 + half * (BN / 2) + sl * cols_per_slab;
         const bool live = row0 < Mg && col0 < Ng;   // warp-uniform
         float v[64];
         if (live) {
@@ -363,17 +423,18 @@ __global__ void __launch_bounds__(kThreadsTc, 1) matmul_tc_kernel(const __grid_c
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
-      if (lane == 0) mbar_arrive(smem_addr(&bar_acc_empty[acc]));
+      if (lane == 0) mbar_arrive_cluster(acc_empty0[acc]);   // tells CTA 0's MMA thread
     }
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
 
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
+  cluster_sync_all();          // the partner may still signal this CTA's barriers or read its tiles
   if (warp == 1) {
     __syncwarp();
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
   }
 }
 
@@ -467,7 +528,7 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, void*, size_t, cudaStream_t 
       cols_b = plan.n[s];
     }
     if (rows_a == 0 || cols_b == 0) { p.kblocks[s] = plan.chain ? p.kblocks[s] : 0; continue; }
-    if (!make_map(&p.map_a[s], plan.a[s], 2, rows_a, plan.kseg[s], plan.lda[s], BM, BK))
+    if (!make_map(&p.map_a[s], plan.a[s], 2, rows_a, plan.kseg[s], plan.lda[s], BMH, BK))
       return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for operand x of shard %d", s);
     if (!make_map(&p.map_b[s], plan.b[s], 2, plan.kseg[s], cols_b, plan.ldb[s], BK, 64))
       return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for operand w of shard %d", s);
@@ -498,15 +559,33 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, void*, size_t, cudaStream_t 
   *taken = true;
   if (tiles == 0) return SBP_OK;
 
-  static int sm_count = 0;
-  if (sm_count == 0) {
-    int dev = 0;
-    SBP_CUDA_TRY(cudaGetDevice(&dev));
-    SBP_CUDA_TRY(cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev));
+  static int max_pairs = 0;
+  if (max_pairs == 0) {
     SBP_CUDA_TRY(cudaFuncSetAttribute(matmul_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    int dev = 0, sms = 0;
+    SBP_CUDA_TRY(cudaGetDevice(&dev));
+    SBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    // how many CTA pairs the device can hold at once (pairs must sit in one GPC)
+    cudaLaunchConfig_t probe = {};
+    probe.gridDim = dim3((unsigned)(2 * (sms / 2)));
+    probe.blockDim = dim3(kThreadsTc);
+    probe.dynamicSmemBytes = kSmemBytes;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    probe.attrs = &attr;
+    probe.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, matmul_tc_kernel, &probe) != cudaSuccess || clusters < 1) {
+      cudaGetLastError();
+      clusters = sms / 2;
+    }
+    max_pairs = clusters;
   }
-  const int grid = tiles < sm_count ? tiles : sm_count;
-  matmul_tc_kernel<<<grid, kThreadsTc, kSmemBytes, st>>>(p);
+  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  matmul_tc_kernel<<<2 * pairs, kThreadsTc, kSmemBytes, st>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e, "tensor-core matmul launch");
   count_launch();

@@ -162,7 +162,17 @@ def run_sweep(sbp, work, events=None):
 
 # DRAM bytes (read + write) per launch from the ncu captures summarised under profiles/.
 # None = not captured for the kernel as it stands.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # profiles/box_kernels_sweep_bf16_8192x8192_k4.md (full size)
+    "P(sum)->B": 1018.0e6, "P(sum)->S(0)": 625.5e6, "P(sum)->S(1)": 620.3e6, "S(0)->B": 613.9e6,
+    "S(0)->S(1)": 216.8e6, "S(1)->S(0)": 215.8e6, "B->S(1)": 216.0e6,
+    # profiles/xent_partial_bf16_512x1048576_k8.md (full size)
+    "softmax-xent on bf16 logits (partial + combine)": 1077.2e6,
+    # profiles/matmul_tc_classifier_bf16_512x512x1048576_k8.md (full size)
+    "classifier GEMM (B,S(1))->S(1), bf16 logits": 2105.1e6,
+    # profiles/embedding_fused_fp32_4194304x128_batch16384_k8.md (quarter batch, scaled x 4)
+    "embedding fused gather -> B (8 replicas written)": 7104.0e6,
+}
 
 
 def ncu_traffic(name):
@@ -265,23 +275,23 @@ def _hbm_entry(name, nbytes, avg, best, peaks, extra=None):
 def _tensor_entry(name, flops, avg, best, peaks, extra=None):
     tf = flops / (avg * 1e-3) / 1e12
     e = {"op": name, "bound": "tensor", "flops": flops, "ms": avg, "best_ms": best, "achieved": tf, "unit": "TFLOP/s",
-         "peak": peaks["bf16_tflops"], "frac_measured": tf / peaks["bf16_tflops"],
+         "peak": peaks["bf16_tflops"], "frac_measured": tf / peaks["bf16_tflops"], "traffic": ncu_traffic(name),
          "frac_sustained": tf / peaks["bf16_tflops_sustained"], "frac_nominal": tf / NOMINAL_BF16_TFLOPS}
     if extra:
         e.update(extra)
     return e
 
 
-def section_embedding(sbp, device, peaks):
+def section_embedding(sbp, device, peaks, opts):
     """Row-split embedding: fp32 table [2^24, 128] S(0) over k = 8, ids int64 [65536, 26] Zipf(1.05)."""
-    k, rows, dim = 8, 1 << 24, 128
-    ids = dg.zipf_ids(1005, 1, (65536, 26), rows, 1.05, device)
+    k, rows, dim, batch = 8, opts.emb_rows, 128, opts.emb_batch
+    ids = dg.zipf_ids(1005, 1, (batch, 26), rows, 1.05, device)
     table = sbp.SbpTensor((rows, dim), torch.float32, sbp.S(0),
                           [dg.uniform(1005, 100 + r, (rows // k, dim), -0.05, 0.05, torch.float32, device) for r in range(k)])
-    idt = sbp.SbpTensor((65536, 26), torch.int64, sbp.B, [ids] * k)
-    out_b = sbp.empty_global((65536, 26, dim), torch.float32, sbp.B, k, device=device)
-    out_1 = sbp.empty_global((65536, 26, dim), torch.float32, sbp.B, k, device=device, alias_replicas=True)
-    n = 65536 * 26
+    idt = sbp.SbpTensor((batch, 26), torch.int64, sbp.B, [ids] * k)
+    out_b = sbp.empty_global((batch, 26, dim), torch.float32, sbp.B, k, device=device)
+    out_1 = sbp.empty_global((batch, 26, dim), torch.float32, sbp.B, k, device=device, alias_replicas=True)
+    n = batch * 26
     row_b = dim * 4
     unique = int(torch.unique(ids).numel())
     res = []
@@ -292,7 +302,7 @@ def section_embedding(sbp, device, peaks):
     res.append(_hbm_entry("embedding fused gather -> B (replicas aliased, 1 write)", n * 8 + 2 * n * row_b, avg, best, peaks,
                           {"unique_rows": unique, "lookups": n}))
     del out_1
-    out_p = sbp.empty_global((65536, 26, dim), torch.float32, sbp.P_SUM, k, device=device)
+    out_p = sbp.empty_global((batch, 26, dim), torch.float32, sbp.P_SUM, k, device=device)
 
     def unfused():
         sbp.sbp_embedding(table, idt, out_p)
@@ -303,9 +313,9 @@ def section_embedding(sbp, device, peaks):
     return res
 
 
-def section_softmax(sbp, device, peaks):
+def section_softmax(sbp, device, peaks, opts):
     """Class-split softmax cross entropy on materialised bf16 logits [512, 2^20], S(1) over k = 8."""
-    k, rows, classes = 8, 512, 1 << 20
+    k, rows, classes = 8, opts.xent_rows, 1 << 20
     sigma = (512 ** 0.5) * 0.01
     logits = sbp.SbpTensor((rows, classes), torch.bfloat16, sbp.S(1),
                            [dg.normal(1004, 10 + r, (rows, classes // k), 0.0, sigma, torch.bfloat16, device) for r in range(k)])
@@ -318,7 +328,7 @@ def section_softmax(sbp, device, peaks):
                        {"loss_mean": float(loss.locals[0].mean().item())})]
 
 
-def section_mlp(sbp, device, peaks):
+def section_mlp(sbp, device, peaks, opts):
     """Megatron-style MLP: X[8192,4096] B, W1[4096,16384] S(1), GeLU, W2[16384,4096] S(0), k = 8."""
     k, M, H, F = 8, 8192, 4096, 16384
     bf16 = torch.bfloat16
@@ -344,9 +354,9 @@ def section_mlp(sbp, device, peaks):
     return res
 
 
-def section_classifier_gemm(sbp, device, peaks):
+def section_classifier_gemm(sbp, device, peaks, opts):
     """Classifier logits: F[512,512] B x W[512, 2^20] S(1) over k = 8 -> bf16 logits S(1)."""
-    k, rows, feat, classes = 8, 512, 512, 1 << 20
+    k, rows, feat, classes = 8, opts.xent_rows, 512, 1 << 20
     bf16 = torch.bfloat16
     Fm = dg.normal(1004, 0, (rows, feat), 0.0, 1.0, bf16, device)
     f = sbp.SbpTensor((rows, feat), bf16, sbp.B, [Fm] * k)
@@ -362,13 +372,14 @@ def section_classifier_gemm(sbp, device, peaks):
     return [e]
 
 
-def run_operator_sections(sbp, device, peaks, which="softmax,classifier,mlp,embedding"):
+def run_operator_sections(sbp, device, peaks, opts):
+    which = opts.ops
     out = []
     table = {"softmax": section_softmax, "classifier": section_classifier_gemm, "mlp": section_mlp,
              "embedding": section_embedding}
     for fn in [table[w.strip()] for w in which.split(",") if w.strip()]:
         try:
-            out.extend(fn(sbp, device, peaks))
+            out.extend(fn(sbp, device, peaks, opts))
         except sbp.SbpError as e:            # an operator this build cannot run is reported, not hidden
             out.append({"op": fn.__name__, "error": str(e)})
         torch.cuda.empty_cache()
@@ -430,6 +441,9 @@ def parse():
                     help="comma-separated operator sections to run: softmax, classifier, mlp, embedding")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--copy-engine", type=int, default=0)
+    ap.add_argument("--emb-rows", type=int, default=1 << 24, help="embedding table rows (smaller = profiling-sized case)")
+    ap.add_argument("--emb-batch", type=int, default=65536, help="embedding batch (x 26 fields)")
+    ap.add_argument("--xent-rows", type=int, default=512, help="rows of the softmax / classifier sections")
     ap.add_argument("--rows", type=int, default=SWEEP_SHAPE[0],
                     help="rows of the logical sweep tensor (smaller = a profiling-sized case, not the benchmark)")
     return ap.parse_args()
@@ -564,7 +578,7 @@ def main():
         if not args.no_ops:
             del T, src, work
             torch.cuda.empty_cache()
-            line["ops"] = run_operator_sections(sbp, device, peaks, args.ops)
+            line["ops"] = run_operator_sections(sbp, device, peaks, args)
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

@@ -63,6 +63,7 @@ struct TcParams {
   int kblocks[SBP_MAX_K];       // per segment
   int tile_begin[SBP_MAX_K + 1];   // prefix sum of tiles per group
   int tiles_m[SBP_MAX_K];
+  int tiles_n[SBP_MAX_K];
   int ngroups, nseg, chain, gelu, n_rep;
   int out_f32;
   int total_tiles;
@@ -226,11 +227,20 @@ struct TileCoord {
   int g, m0, n0;
 };
 
+// Tiles of a group are walked in panels of kPanelM m-tiles, n fastest across the panel, so that
+// the CTA pairs running at the same time cover a roughly square patch of the output and share
+// both their A rows and their B columns in L2.
+constexpr int kPanelM = 8;
+
 __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
   int g = 0;
   while (g + 1 < p.ngroups && tile >= p.tile_begin[g + 1]) ++g;
   const int local = tile - p.tile_begin[g];
-  const int nt = local / p.tiles_m[g], mt = local - nt * p.tiles_m[g];   // m fastest
+  const int tm = p.tiles_m[g], tn = p.tiles_n[g];
+  const int panel = local / (kPanelM * tn);
+  const int rem = local - panel * (kPanelM * tn);
+  const int pm = min(kPanelM, tm - panel * kPanelM);   // m-tiles in this (possibly last) panel
+  const int nt = rem / pm, mt = panel * kPanelM + (rem - nt * pm);
   return TileCoord{g, mt * BM, nt * BN};
 }
 
@@ -543,6 +553,7 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, void*, size_t, cudaStream_t 
     p.tile_begin[g] = tiles;
     const long long tm = (plan.m[g] + BM - 1) / BM, tn = (plan.n[g] + BN - 1) / BN;
     p.tiles_m[g] = (int)std::max(1LL, tm);
+    p.tiles_n[g] = (int)std::max(1LL, tn);
     if (plan.m[g] > 0 && plan.n[g] > 0) {
       if (tm * tn + tiles > 0x3fffffffLL) return SBP_ERR_UNSUPPORTED;
       tiles += (int)(tm * tn);

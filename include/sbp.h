@@ -147,6 +147,12 @@ sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, voi
  * the flag: SBP_ERR_TIMEOUT if a wait expired since the last call, else SBP_OK. */
 sbp_status sbp_check_device_errors(void);
 
+/* Self-test of that path, safe to run anywhere: enqueues a one-thread kernel that waits on a
+ * barrier nothing signals, gives up after limit_ms (1..1000) and raises the flag.  After the
+ * stream has drained, sbp_check_device_errors() returns SBP_ERR_TIMEOUT once, and the device
+ * stays fully usable. */
+sbp_status sbp_selftest_wait_timeout(uint32_t limit_ms, void* cuda_stream);
+
 /* Selects the copy engine of the pure data-movement transforms: 0 = choose (default),
  * 1 = 128-bit load/store kernel, 2 = bulk asynchronous copies staged through shared
  * memory (needs 16-byte aligned segments, else falls back to 1).  Process-wide. */
@@ -195,6 +201,23 @@ size_t sbp_softmax_xent_workspace_bytes(const sbp_tensor* logits);
 sbp_status sbp_softmax_xent(const sbp_tensor* logits, const sbp_tensor* labels, sbp_tensor* loss,
                             sbp_tensor* row_max, sbp_tensor* row_sum, void* ws, size_t ws_bytes,
                             void* cuda_stream);
+
+/* The classifier of Section 6.3 in one call: logits = features x weight with the weight S(1)
+ * (hence logits S(1)), then the split softmax cross entropy above -- without ever storing the
+ * logits.  Each 128-class chunk of a shard's product leaves, per row, its local max, local
+ * exp-sum and the label's logit straight from the fp32 accumulator; these partials are then
+ * reduced across chunks and shards in a fixed order (the two reductions of Section 6.3).
+ *
+ *   features [rows, feat]     B,    SBP_BF16
+ *   weight   [feat, classes]  S(1), SBP_BF16
+ *   labels, loss, row_max, row_sum: as for sbp_softmax_xent
+ * The logits are taken from the fp32 accumulator, i.e. they are not rounded to bf16 first.
+ * Needs shapes the tensor-core path accepts (16-byte aligned operands; feat and every shard's
+ * class count multiples of 8; feat > 0), else SBP_ERR_UNSUPPORTED and nothing is launched. */
+size_t sbp_matmul_softmax_xent_workspace_bytes(const sbp_tensor* features, const sbp_tensor* weight);
+sbp_status sbp_matmul_softmax_xent(const sbp_tensor* features, const sbp_tensor* weight,
+                                   const sbp_tensor* labels, sbp_tensor* loss, sbp_tensor* row_max,
+                                   sbp_tensor* row_sum, void* ws, size_t ws_bytes, void* cuda_stream);
 
 /* Variant of sbp_softmax_xent for callers that have no device workspace to give and may not
  * create one.  (The paper has no counterpart; this exists for programs that embed the library

@@ -95,12 +95,16 @@ def load_library():
     lib.sbp_boxing_set_copy_engine.argtypes = [C.c_int32]
     lib.sbp_boxing_set_copy_engine.restype = None
     lib.sbp_check_device_errors.argtypes = []
+    lib.sbp_selftest_wait_timeout.argtypes = [C.c_uint32, C.c_void_p]
     lib.sbp_matmul_workspace_bytes.restype = C.c_size_t
     lib.sbp_matmul_workspace_bytes.argtypes = [T, T, T]
     lib.sbp_matmul.argtypes = [T, T, T, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.sbp_softmax_xent_workspace_bytes.restype = C.c_size_t
     lib.sbp_softmax_xent_workspace_bytes.argtypes = [T]
     lib.sbp_softmax_xent.argtypes = [T, T, T, T, T, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sbp_matmul_softmax_xent_workspace_bytes.restype = C.c_size_t
+    lib.sbp_matmul_softmax_xent_workspace_bytes.argtypes = [T, T]
+    lib.sbp_matmul_softmax_xent.argtypes = [T, T, T, T, T, T, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.sbp_softmax_xent_static.argtypes = [T, T, T, T, T, C.c_void_p]
     lib.sbp_embedding.argtypes = [T, T, T, C.c_void_p, C.c_void_p]
     _LIB = lib
@@ -192,6 +196,10 @@ def sbp_check_device_errors() -> None:
     _check(load_library().sbp_check_device_errors())
 
 
+def sbp_selftest_wait_timeout(limit_ms: int, stream=None) -> None:
+    _check(load_library().sbp_selftest_wait_timeout(int(limit_ms), _stream_ptr(stream)))
+
+
 def sbp_boxing_set_copy_engine(engine: int) -> None:
     load_library().sbp_boxing_set_copy_engine(int(engine))
 
@@ -238,6 +246,23 @@ def sbp_softmax_xent(logits: SbpTensor, labels: SbpTensor, loss: SbpTensor,
     s = row_sum._c() if row_sum is not None else None
     _check(load_library().sbp_softmax_xent(
         C.byref(a), C.byref(b), C.byref(c),
+        C.byref(m) if m is not None else None, C.byref(s) if s is not None else None,
+        C.c_void_p(ws.data_ptr()), ws.numel() * ws.element_size(), _stream_ptr(stream)))
+
+
+def sbp_matmul_softmax_xent_workspace_bytes(features: SbpTensor, weight: SbpTensor) -> int:
+    a, b = features._c(), weight._c()
+    return int(load_library().sbp_matmul_softmax_xent_workspace_bytes(C.byref(a), C.byref(b)))
+
+
+def sbp_matmul_softmax_xent(features: SbpTensor, weight: SbpTensor, labels: SbpTensor, loss: SbpTensor,
+                            row_max: Optional[SbpTensor], row_sum: Optional[SbpTensor],
+                            ws: torch.Tensor, stream=None) -> None:
+    a, b, l, c = features._c(), weight._c(), labels._c(), loss._c()
+    m = row_max._c() if row_max is not None else None
+    s = row_sum._c() if row_sum is not None else None
+    _check(load_library().sbp_matmul_softmax_xent(
+        C.byref(a), C.byref(b), C.byref(l), C.byref(c),
         C.byref(m) if m is not None else None, C.byref(s) if s is not None else None,
         C.c_void_p(ws.data_ptr()), ws.numel() * ws.element_size(), _stream_ptr(stream)))
 

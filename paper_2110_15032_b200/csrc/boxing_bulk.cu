@@ -236,6 +236,37 @@ bool launch_bulk_copy(const BoxParams& p, int ntasks, cudaStream_t st) {
   return true;
 }
 
+// Self-test of the bounded-wait path: one thread waits on an mbarrier that nothing will ever
+// signal, gives up after limit_ns and raises the same flag a real expiry raises.
+__global__ void expire_wait_kernel(unsigned long long limit_ns) {
+  __shared__ __align__(8) unsigned long long bar;
+  if (threadIdx.x != 0) return;
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bar)) : "memory");
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  const unsigned long long t0 = global_ns();
+  bool done = false;
+  while (!done && global_ns() - t0 <= limit_ns) {
+    unsigned ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(smem_u32(&bar)), "r"(0u)
+        : "memory");
+    done = ok != 0;
+  }
+  if (!done) atomicExch(&g_bulk_timeout_flag, 1);
+}
+
+sbp_status launch_expire_wait(unsigned long long limit_ns, cudaStream_t st) {
+  expire_wait_kernel<<<1, 32, 0, st>>>(limit_ns);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "self-test launch");
+  count_launch();
+  return SBP_OK;
+}
+
 sbp_status read_and_clear_bulk_timeout(bool* timed_out) {
   int flag = 0, zero = 0;
   SBP_CUDA_TRY(cudaMemcpyFromSymbol(&flag, g_bulk_timeout_flag, sizeof(int)));

@@ -15,7 +15,13 @@ namespace sbp {
 // Defined in matmul_tc.cu.  Returns SBP_ERR_UNSUPPORTED (without touching the error text)
 // when the plan does not meet the tensor-core kernel's rules; the caller then falls back
 // to the FMA kernel.
-sbp_status launch_matmul_tc(const MatmulPlan& plan, void* ws, size_t ws_bytes, cudaStream_t st, bool* taken);
+sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaStream_t st, bool* taken);
+// Defined in softmax_xent.cu: reduces the per-chunk partials left by the fused classifier kernel.
+sbp_status launch_xent_finish(float* part_m, float* part_s, float* part_t, int parts, long long rows, float* stage,
+                              sbp_tensor* loss, sbp_tensor* row_max, sbp_tensor* row_sum, int k, cudaStream_t st);
+sbp_status check_xent_outputs(const sbp_tensor* labels, const sbp_tensor* loss, const sbp_tensor* row_max,
+                              const sbp_tensor* row_sum, long long rows, int k);
+size_t xent_finish_stage_floats(long long rows);
 size_t matmul_tc_workspace_bytes(const MatmulPlan& plan);
 
 __device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f)); }
@@ -251,9 +257,105 @@ sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, u
   if (st != SBP_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   bool taken = false;
-  st = launch_matmul_tc(plan, ws, ws_bytes, stream, &taken);
+  (void)ws;
+  (void)ws_bytes;
+  st = launch_matmul_tc(plan, nullptr, stream, &taken);
   if (taken) return st;
   return launch_fma(plan, stream);
+}
+
+// ------------------------------------------------------------------ fused classifier
+
+// Chunks of 128 classes per shard and in total, for the partial arrays of the fused path.
+static int classifier_chunks(const sbp_tensor* w, int part_base[SBP_MAX_K], long long class_start[SBP_MAX_K]) {
+  const int k = placement_k(w);
+  int total = 0;
+  for (int r = 0; r < k; ++r) {
+    int64_t st, ln;
+    split_range(w->shape[1], k, r, &st, &ln);
+    part_base[r] = total;
+    class_start[r] = st;
+    total += (int)((ln + 127) / 128);
+  }
+  return total;
+}
+
+static sbp_status check_classifier(const sbp_tensor* f, const sbp_tensor* w, bool need_ptrs) {
+  sbp_status st = check_tensor(f, "features", need_ptrs);
+  if (st != SBP_OK) return st;
+  st = check_tensor(w, "weight", need_ptrs);
+  if (st != SBP_OK) return st;
+  if (f->ndim != 2 || w->ndim != 2) return fail(SBP_ERR_SHAPE, "features and weight must be 2-D");
+  if (f->shape[1] != w->shape[0]) return fail(SBP_ERR_SHAPE, "features are [rows,%lld] but weight has %lld rows",
+                                              (long long)f->shape[1], (long long)w->shape[0]);
+  if (f->dtype != SBP_BF16 || w->dtype != SBP_BF16) return fail(SBP_ERR_DTYPE, "the fused classifier takes BF16 operands");
+  if (placement_k(f) != placement_k(w)) return fail(SBP_ERR_INVALID_ARG, "operands differ in k");
+  if (!is_b(f->sbp[0]) || !is_s(w->sbp[0], 1))
+    return fail(SBP_ERR_SIGNATURE, "the fused classifier needs features B and weight S(1)");
+  if (w->shape[1] < 1) return fail(SBP_ERR_SHAPE, "softmax over zero classes");
+  if (w->shape[1] / 128 + SBP_MAX_K > 0x3fffffffLL) return fail(SBP_ERR_UNSUPPORTED, "too many classes");
+  return SBP_OK;
+}
+
+size_t sbp_matmul_softmax_xent_workspace_bytes(const sbp_tensor* features, const sbp_tensor* weight) {
+  if (check_classifier(features, weight, false) != SBP_OK) return 0;
+  int part_base[SBP_MAX_K];
+  long long class_start[SBP_MAX_K];
+  const int parts = classifier_chunks(weight, part_base, class_start);
+  const size_t rows = (size_t)features->shape[0];
+  return (3 * (size_t)parts * rows + xent_finish_stage_floats((long long)rows)) * sizeof(float);
+}
+
+sbp_status sbp_matmul_softmax_xent(const sbp_tensor* features, const sbp_tensor* weight, const sbp_tensor* labels,
+                                   sbp_tensor* loss, sbp_tensor* row_max, sbp_tensor* row_sum, void* ws,
+                                   size_t ws_bytes, void* cuda_stream) {
+  sbp_status st = check_classifier(features, weight, true);
+  if (st != SBP_OK) return st;
+  const int k = placement_k(features);
+  const long long rows = features->shape[0], K = features->shape[1], N = weight->shape[1];
+  st = check_xent_outputs(labels, loss, row_max, row_sum, rows, k);
+  if (st != SBP_OK) return st;
+  if (rows == 0) return SBP_OK;
+  const size_t need = sbp_matmul_softmax_xent_workspace_bytes(features, weight);
+  if (!ws || ws_bytes < need) return fail(SBP_ERR_WORKSPACE, "workspace of %zu bytes needed, %zu given", need, ws_bytes);
+  if (reinterpret_cast<uintptr_t>(ws) % 4 != 0) return fail(SBP_ERR_ALIGNMENT, "workspace must be 4-byte aligned");
+
+  // (B, S(1)) -> S(1): one group per shard of the weight
+  MatmulPlan plan{};
+  plan.in_dtype = SBP_BF16;
+  plan.out_dtype = SBP_F32;
+  plan.ngroups = k;
+  plan.nseg = k;
+  plan.chain = 0;
+  for (int r = 0; r < k; ++r) {
+    int64_t s0, ln;
+    split_range(N, k, r, &s0, &ln);
+    plan.a[r] = features->local[r];
+    plan.b[r] = weight->local[r];
+    plan.lda[r] = K;
+    plan.ldb[r] = ln;
+    plan.kseg[r] = K;
+    plan.m[r] = rows;
+    plan.n[r] = ln;
+    plan.ldy[r] = ln;
+  }
+  XentFusion xf{};
+  const int parts = classifier_chunks(weight, xf.part_base, xf.class_start);
+  xf.part_m = static_cast<float*>(ws);
+  xf.part_s = xf.part_m + (size_t)parts * rows;
+  xf.part_t = xf.part_s + (size_t)parts * rows;
+  float* stage = xf.part_t + (size_t)parts * rows;
+  xf.labels = static_cast<const long long*>(labels->local[0]);
+  xf.rows = rows;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  bool taken = false;
+  st = launch_matmul_tc(plan, &xf, stream, &taken);
+  if (!taken)
+    return fail(SBP_ERR_UNSUPPORTED,
+                "the fused classifier needs the tensor-core path (16-byte aligned operands, feature and per-shard class "
+                "counts that are multiples of 8, a non-empty contraction); use sbp_matmul + sbp_softmax_xent instead");
+  if (st != SBP_OK) return st;
+  return launch_xent_finish(xf.part_m, xf.part_s, xf.part_t, parts, rows, stage, loss, row_max, row_sum, k, stream);
 }
 
 }  // extern "C"

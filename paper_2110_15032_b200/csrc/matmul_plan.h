@@ -34,4 +34,18 @@ struct MatmulPlan {
   int in_dtype, out_dtype;   // sbp_dtype
 };
 
+// Optional epilogue of the tensor-core kernel for the class-split classifier: instead of storing
+// the logits, every 128-column chunk of a tile leaves, per row, a local max, a local
+// sum of exp(z - max) and the label's logit (0 when the label lies elsewhere).
+//   part_x[(part_base[g] + chunk) * rows + row],  chunk = column / 128 inside group g
+struct XentFusion {
+  float* part_m;
+  float* part_s;
+  float* part_t;
+  const long long* labels;          // [rows], global class indices
+  long long class_start[SBP_MAX_K]; // first class of group g
+  int part_base[SBP_MAX_K];         // first chunk index of group g
+  long long rows;
+};
+
 }  // namespace sbp

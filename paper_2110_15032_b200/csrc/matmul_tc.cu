@@ -67,6 +67,8 @@ struct TcParams {
   int ngroups, nseg, chain, gelu, n_rep;
   int out_f32;
   int total_tiles;
+  int xent;                     // 1: softmax partials instead of stored logits
+  XentFusion xf;
 };
 
 // ------------------------------------------------------------------ PTX helpers
@@ -384,6 +386,73 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
       const long long Mg = p.m[tc.g], Ng = p.n[tc.g];
       const int row0 = tc.m0 + (int)rank * BMH + q * 32;
       const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * BN + half * (BN / 2);
+      if (p.xent) {
+        // Softmax partials of this warp's 32 rows x 128 columns; one thread owns one row, so
+        // nothing crosses lanes.  Columns are taken 32 at a time: batch max, then the running
+        // (m, s) is rescaled and the batch's exponentials are added.
+        constexpr float kL2e = 1.4426950408889634f;
+        const int colbase = tc.n0 + half * (BN / 2);
+        const long long row = row0 + lane;
+        if (row0 < Mg && colbase < Ng) {            // warp-uniform
+          float m = -INFINITY, s = 0.f, t = 0.f;
+          long long want = -1;
+          if (row < Mg) want = p.xf.labels[row] - p.xf.class_start[tc.g] - colbase;
+          for (int b = 0; b < 4; ++b) {
+            const int c0 = colbase + b * 32;
+            if (c0 >= Ng) break;                      // warp-uniform
+            float v[32];
+            tmem_ld32(taddr + b * 32, v);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            const int nvalid = (int)min((long long)32, Ng - c0);
+            if (nvalid < 32) {
+#pragma unroll
+              for (int i = 0; i < 32; ++i)
+                if (i >= nvalid) v[i] = -INFINITY;
+            }
+            float bm = v[0];
+#pragma unroll
+            for (int i = 1; i < 32; ++i) bm = fmaxf(bm, v[i]);
+            const float mm = fmaxf(m, bm);
+            const float neg = -mm * kL2e;
+            float carried = 0.f;
+            if (m != -INFINITY) {
+              float e;
+              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(m, kL2e, neg)));
+              carried = s * e;
+            }
+            float s0 = 0.f, s1 = 0.f;
+#pragma unroll
+            for (int i = 0; i < 32; i += 2) {
+              float e0, e1;
+              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e0) : "f"(fmaf(v[i], kL2e, neg)));
+              asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e1) : "f"(fmaf(v[i + 1], kL2e, neg)));
+              s0 += e0;
+              s1 += e1;
+            }
+            s = carried + (s0 + s1);
+            m = mm;
+          }
+          // The label's logit: rows whose label falls inside this chunk (rare) re-read that one
+          // column from tensor memory, one row at a time so the load stays warp-uniform.
+          const long long ncols = min((long long)(BN / 2), Ng - colbase);
+          unsigned hits = __ballot_sync(0xffffffffu, want >= 0 && want < ncols);
+          while (hits) {
+            const int src_lane = __ffs(hits) - 1;
+            hits &= hits - 1;
+            const int col = __shfl_sync(0xffffffffu, (int)want, src_lane);
+            unsigned bitsv;
+            asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(bitsv) : "r"(taddr + col) : "memory");
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            if (lane == src_lane) t = __uint_as_float(bitsv);
+          }
+          if (row < Mg) {
+            const long long slot = (long long)(p.xf.part_base[tc.g] + colbase / 128) * p.xf.rows + row;
+            p.xf.part_m[slot] = m;
+            p.xf.part_s[slot] = s;
+            p.xf.part_t[slot] = t;
+          }
+        }
+      } else
       for (int sl = 0; sl < nslabs; ++sl) {
         const int col0 = tc.n0 + half * (BN / 2) + sl * cols_per_slab;
         const bool live = row0 < Mg && col0 < Ng;   // warp-uniform
@@ -486,7 +555,7 @@ size_t matmul_tc_workspace_bytes(const MatmulPlan&) { return 0; }
 
 static bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
 
-sbp_status launch_matmul_tc(const MatmulPlan& plan, void*, size_t, cudaStream_t st, bool* taken) {
+sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaStream_t st, bool* taken) {
   *taken = false;
   if (plan.in_dtype != SBP_BF16) return SBP_ERR_UNSUPPORTED;
   const int oesz = plan.out_dtype == SBP_F32 ? 4 : 2;
@@ -503,7 +572,7 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, void*, size_t, cudaStream_t 
   for (int s = 0; s < plan.nseg; ++s) ktotal_chain += plan.kseg[s];
   for (int g = 0; g < plan.ngroups; ++g) {
     if (plan.m[g] == 0 || plan.n[g] == 0) continue;
-    if (!aligned16(plan.y[g]) || (plan.ldy[g] * oesz) % 16 != 0) return SBP_ERR_UNSUPPORTED;
+    if (!xf && (!aligned16(plan.y[g]) || (plan.ldy[g] * oesz) % 16 != 0)) return SBP_ERR_UNSUPPORTED;
     if (plan.col_off[g] % 8 != 0) return SBP_ERR_UNSUPPORTED;
     const long long kg = plan.chain ? ktotal_chain : plan.kseg[g];
     if (kg == 0) return SBP_ERR_UNSUPPORTED;   // an all-zero result: left to the FMA kernel
@@ -522,6 +591,8 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, void*, size_t, cudaStream_t 
   p.gelu = plan.gelu;
   p.n_rep = plan.n_rep;
   p.out_f32 = plan.out_dtype == SBP_F32;
+  p.xent = xf ? 1 : 0;
+  if (xf) p.xf = *xf;
 
   for (int s = 0; s < plan.nseg; ++s) {
     p.kblocks[s] = (int)((plan.kseg[s] + BK - 1) / BK);
@@ -557,7 +628,7 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, void*, size_t, cudaStream_t 
     if (plan.m[g] > 0 && plan.n[g] > 0) {
       if (tm * tn + tiles > 0x3fffffffLL) return SBP_ERR_UNSUPPORTED;
       tiles += (int)(tm * tn);
-      if (!make_map(&p.map_y[g], plan.y[g], oesz, plan.m[g], plan.n[g], plan.ldy[g], 32, box_cols))
+      if (!xf && !make_map(&p.map_y[g], plan.y[g], oesz, plan.m[g], plan.n[g], plan.ldy[g], 32, box_cols))
         return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for the result of group %d", g);
     }
   }

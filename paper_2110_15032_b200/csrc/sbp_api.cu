@@ -72,6 +72,7 @@ int64_t local_numel(const sbp_tensor* t, int r) {
 // Defined next to the kernels that own the flags.
 sbp_status read_and_clear_bulk_timeout(bool* timed_out);
 sbp_status read_and_clear_tc_timeout(bool* timed_out);
+sbp_status launch_expire_wait(unsigned long long limit_ns, cudaStream_t st);
 
 }  // namespace sbp
 
@@ -108,6 +109,11 @@ sbp_status sbp_check_device_errors(void) {
   if (bulk) return fail(SBP_ERR_TIMEOUT, "a bulk-copy boxing kernel gave up waiting for its loads");
   if (tc) return fail(SBP_ERR_TIMEOUT, "the tensor-core matmul kernel gave up waiting on one of its barriers");
   return SBP_OK;
+}
+
+sbp_status sbp_selftest_wait_timeout(uint32_t limit_ms, void* cuda_stream) {
+  if (limit_ms == 0 || limit_ms > 1000) return fail(SBP_ERR_INVALID_ARG, "limit_ms must be in [1, 1000]");
+  return launch_expire_wait((unsigned long long)limit_ms * 1000000ull, static_cast<cudaStream_t>(cuda_stream));
 }
 
 sbp_status sbp_local_shape(const sbp_tensor* t, int32_t r, int64_t out_shape[SBP_MAX_DIMS]) {

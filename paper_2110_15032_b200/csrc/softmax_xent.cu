@@ -287,6 +287,109 @@ static sbp_status check_row_vector(const sbp_tensor* t, const char* name, long l
   return SBP_OK;
 }
 
+// ---- second-level reduction for many partials per row (used after the fused classifier
+// kernel, which leaves one partial per 128 classes).  Thread (tx, ty) of a 32 x 8 CTA owns row
+// 32 bx + tx and walks the parts of slice `by` with stride 8 in ascending order; the 8 lanes
+// of a row are then merged in lane order.  Output: one partial per (slice, row).
+struct XentReduceParams {
+  const float* in_m;
+  const float* in_s;
+  const float* in_t;
+  float* out_m;
+  float* out_s;
+  float* out_t;
+  long long rows;
+  int parts, per_slice;
+};
+
+__global__ void __launch_bounds__(256) xent_reduce_parts_kernel(const __grid_constant__ XentReduceParams p) {
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  const long long row = (long long)blockIdx.x * 32 + tx;
+  const int lo = blockIdx.y * p.per_slice;
+  const int hi = min(p.parts, lo + p.per_slice);
+  float m = -INFINITY, s = 0.f, t = 0.f;
+  if (row < p.rows) {
+    for (int q = lo + ty; q < hi; q += 8) {
+      const long long at = (long long)q * p.rows + row;
+      merge(m, s, p.in_m[at], p.in_s[at]);
+      t += p.in_t[at];
+    }
+  }
+  __shared__ float sm[8][33], ss[8][33], st[8][33];
+  sm[ty][tx] = m;
+  ss[ty][tx] = s;
+  st[ty][tx] = t;
+  __syncthreads();
+  if (ty == 0 && row < p.rows) {
+#pragma unroll
+    for (int j = 1; j < 8; ++j) {
+      merge(m, s, sm[j][tx], ss[j][tx]);
+      t += st[j][tx];
+    }
+    const long long at = (long long)blockIdx.y * p.rows + row;
+    p.out_m[at] = m;
+    p.out_s[at] = s;
+    p.out_t[at] = t;
+  }
+}
+
+constexpr int kMaxSlices = 64;
+
+static int slices_for(int parts) {
+  int s = parts / 256;
+  return s < 1 ? 1 : (s > kMaxSlices ? kMaxSlices : s);
+}
+
+size_t xent_finish_stage_floats(long long rows) { return 3 * (size_t)kMaxSlices * (size_t)rows; }
+
+sbp_status check_xent_outputs(const sbp_tensor* labels, const sbp_tensor* loss, const sbp_tensor* row_max,
+                              const sbp_tensor* row_sum, long long rows, int k) {
+  sbp_status st = check_tensor(labels, "labels", true);
+  if (st != SBP_OK) return st;
+  if (labels->ndim != 1 || labels->shape[0] != rows) return fail(SBP_ERR_SHAPE, "labels must be [rows]");
+  if (labels->dtype != SBP_I64) return fail(SBP_ERR_DTYPE, "labels must be I64");
+  if (labels->sbp[0].kind != SBP_BROADCAST) return fail(SBP_ERR_SIGNATURE, "labels must be B");
+  if (placement_k(labels) != k) return fail(SBP_ERR_INVALID_ARG, "labels differ in k");
+  st = check_row_vector(loss, "loss", rows, k);
+  if (st != SBP_OK) return st;
+  if (row_max && (st = check_row_vector(row_max, "row_max", rows, k)) != SBP_OK) return st;
+  if (row_sum && (st = check_row_vector(row_sum, "row_sum", rows, k)) != SBP_OK) return st;
+  return SBP_OK;
+}
+
+// parts partials per row in part_* ([parts][rows]) -> loss / row_max / row_sum.
+sbp_status launch_xent_finish(float* part_m, float* part_s, float* part_t, int parts, long long rows, float* stage,
+                              sbp_tensor* loss, sbp_tensor* row_max, sbp_tensor* row_sum, int k, cudaStream_t st) {
+  const int slices = slices_for(parts);
+  XentReduceParams r{};
+  r.in_m = part_m;
+  r.in_s = part_s;
+  r.in_t = part_t;
+  r.out_m = stage;
+  r.out_s = stage + (size_t)slices * rows;
+  r.out_t = stage + 2 * (size_t)slices * rows;
+  r.rows = rows;
+  r.parts = parts;
+  r.per_slice = (parts + slices - 1) / slices;
+  xent_reduce_parts_kernel<<<dim3((unsigned)((rows + 31) / 32), (unsigned)slices), 256, 0, st>>>(r);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "softmax reduce launch");
+  XentCombineParams c{};
+  c.part_m = r.out_m;
+  c.part_s = r.out_s;
+  c.part_t = r.out_t;
+  c.rows = rows;
+  c.parts = slices;
+  c.n_loss = dedup(c.loss, loss, k);
+  c.n_max = row_max ? dedup(c.row_max, row_max, k) : 0;
+  c.n_sum = row_sum ? dedup(c.row_sum, row_sum, k) : 0;
+  xent_combine_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, st>>>(c);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "softmax combine launch");
+  count_launch(2);
+  return SBP_OK;
+}
+
 }  // namespace sbp
 
 using namespace sbp;

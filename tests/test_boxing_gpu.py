@@ -201,3 +201,18 @@ def test_host_buffer_entry_point():
     with pytest.raises(sbp.SbpError) as e:
         sbp.sbp_boxing_host(src, dst, ws[:1024])
     assert e.value.name == "SBP_ERR_WORKSPACE"
+
+
+def test_expired_device_wait_is_reported_and_the_device_stays_usable():
+    """A bounded wait that runs out (a barrier nothing signals) ends the kernel normally and is
+    reported once as SBP_ERR_TIMEOUT; nothing faults and later launches work."""
+    sbp.sbp_check_device_errors()                     # clean slate
+    sbp.sbp_selftest_wait_timeout(20)
+    torch.cuda.synchronize()
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_check_device_errors()
+    assert e.value.name == "SBP_ERR_TIMEOUT"
+    sbp.sbp_check_device_errors()                     # flag was cleared by the report
+    _run((64, 96), F32, sbp.S(0), sbp.S(1), 2)        # the context is intact
+    with pytest.raises(sbp.SbpError):
+        sbp.sbp_selftest_wait_timeout(5000)

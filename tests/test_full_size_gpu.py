@@ -173,8 +173,21 @@ def test_config4_softmax_and_classifier_full_size_sampled_rows():
         Zr = O.matmul_logical(Fs, to_np(wl[r]))
         assert_close(to_np(z.locals[r][pick]), Zr, 2e-2, 1e-3, f"logits shard {r}")
         Zs.append(Zr)
-    _, _, ref = O.softmax_xent_logical(O.from_locals(Zs, O.S1), labels[pick].cpu().numpy())
+    m, S, ref = O.softmax_xent_logical(O.from_locals(Zs, O.S1), labels[pick].cpu().numpy())
     assert_close(to_np(loss.locals[0][pick]), ref, 2e-2, 1e-3, "chain loss")
+    # (c) the same classifier in one call, logits never stored
+    del z
+    loss2 = sbp.empty_global((rows,), F32, sbp.B, k)
+    ws2 = torch.empty(sbp.sbp_matmul_softmax_xent_workspace_bytes(f, w), dtype=torch.uint8, device=dev)
+    sbp.sbp_matmul_softmax_xent(f, w, lab, loss2, rmax, rsum, ws2)
+    torch.cuda.synchronize()
+    sbp.sbp_check_device_errors()
+    assert_close(to_np(loss2.locals[k - 1][pick]), ref, 2e-2, 1e-3, "fused classifier loss")
+    assert_close(to_np(rmax.locals[0][pick]), m, 2e-2, 1e-3, "fused classifier row_max")
+    assert_close(to_np(rsum.locals[0][pick]), S, 2e-2, 1e-3, "fused classifier row_sum")
+    assert torch.isfinite(loss2.locals[0]).all()
+    # every row agrees with the two-call route within the stated tolerance (bf16 logits there)
+    assert_close(to_np(loss2.locals[0]), to_np(loss.locals[0]).astype(np.float64), 2e-2, 1e-3, "fused vs two-call")
 
 
 def test_config5_embedding_full_size_sampled_lookups():

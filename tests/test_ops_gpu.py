@@ -396,3 +396,61 @@ def test_classifier_chain_small_against_oracle():
     zl = O.to_locals(Z, O.S1, k)
     for r in range(k):
         assert_close(to_np(z.locals[r]), zl[r], 2e-2, 1e-3, f"logits shard {r}")
+
+
+# ------------------------------------------------------------------ fused classifier -> softmax cross entropy
+
+def _fused_classifier_case(rows, feat, classes, k, seed, w_std=0.05, alias=False):
+    Fm = dg.normal(seed, 0, (rows, feat), 0.0, 1.0, BF16)
+    W = dg.normal(seed, 2, (feat, classes), 0.0, w_std, BF16)
+    labels = dg.integers(seed, 1, (rows,), 0, classes)
+    f = make_global(split_cpu(Fm, sbp.B, k), (rows, feat), BF16, sbp.B)
+    w = make_global(split_cpu(W, sbp.S(1), k), (feat, classes), BF16, sbp.S(1))
+    lab = make_global([labels] * k, (rows,), I64, sbp.B)
+    loss = sbp.empty_global((rows,), F32, sbp.B, k, alias_replicas=alias)
+    rmax = sbp.empty_global((rows,), F32, sbp.B, k)
+    rsum = sbp.empty_global((rows,), F32, sbp.B, k)
+    for g in (loss, rmax, rsum):
+        for t in g.locals:
+            t.fill_(float("nan"))
+    ws = torch.empty(sbp.sbp_matmul_softmax_xent_workspace_bytes(f, w), dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)                                     # NaN patterns: every partial that is read must be written
+    sbp.sbp_matmul_softmax_xent(f, w, lab, loss, rmax, rsum, ws)
+    torch.cuda.synchronize()
+    sbp.sbp_check_device_errors()
+    Z = O.matmul_logical(to_np(Fm), to_np(W))
+    m, S, ref = O.softmax_xent_logical(Z, labels.numpy())
+    for t in loss.locals:
+        assert_close(to_np(t), ref, 2e-2, 1e-3, "fused loss")
+    for t in rmax.locals:
+        assert_close(to_np(t), m, 2e-2, 1e-3, "fused row_max")
+    for t in rsum.locals:
+        assert_close(to_np(t), S, 2e-2, 1e-3, "fused row_sum")
+    # fp32 accumulation straight into the softmax: far tighter than the stated bar
+    assert np.all(np.abs(to_np(loss.locals[0]) - ref) <= 1e-4 * np.maximum(np.abs(ref), 1.0))
+    return to_np(loss.locals[0])
+
+
+@pytest.mark.parametrize("k", [1, 2, 4, 8])
+def test_fused_classifier_parity_and_shard_invariance(k):
+    a = _fused_classifier_case(64, 512, 16384, k, seed=3001)
+    b = _fused_classifier_case(64, 512, 16384, 1, seed=3001) if k > 1 else a
+    assert np.all(np.abs(a - b) <= 1e-5 * np.abs(b) + 1e-5)
+
+
+def test_fused_classifier_ragged_shapes_and_edges():
+    _fused_classifier_case(300, 200, 4960, 4, seed=3002)        # ragged rows, K tail, 1240 classes per shard
+    _fused_classifier_case(33, 72, 960, 8, seed=3003)           # 120 classes per shard: one partial chunk each
+    _fused_classifier_case(700, 64, 64, 4, seed=3004, alias=True)   # 16 classes per shard, many row tiles
+    rows, feat, classes, k = 16, 64, 1000, 3                     # 334 / 333 classes per shard: not multiples of 8
+    f = sbp.empty_global((rows, feat), BF16, sbp.B, k)
+    w = sbp.empty_global((feat, classes), BF16, sbp.S(1), k)
+    lab = make_global([torch.zeros(rows, dtype=I64)] * k, (rows,), I64, sbp.B)
+    loss = sbp.empty_global((rows,), F32, sbp.B, k)
+    ws = torch.empty(sbp.sbp_matmul_softmax_xent_workspace_bytes(f, w), dtype=torch.uint8, device="cuda")
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_matmul_softmax_xent(f, w, lab, loss, None, None, ws)
+    assert e.value.name == "SBP_ERR_UNSUPPORTED"
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_matmul_softmax_xent(f, w, lab, loss, None, None, ws[:64])
+    assert e.value.name in ("SBP_ERR_WORKSPACE", "SBP_ERR_UNSUPPORTED")

@@ -125,7 +125,9 @@ sbp_status sbp_matmul_infer(sbp_sig x, sbp_sig w, sbp_sig* y);
  *   B              S(i)       local slice of the shard's own replica
  *   B              B          copy of the shard's own replica
  *   P(op)          P(op)      copy
- * Anything else (S->P, B->P, P(sum)<->P(max)) returns SBP_ERR_UNSUPPORTED.
+ *   S(i)           P(sum)     local (Table 2: cost 0): shard r = zeros with its own slice in place
+ *   B              P(sum)     local (Table 2: cost 0): shard 0 = the tensor, every other shard zeros
+ * Anything else (a P(max) destination from S or B, P(sum)<->P(max)) returns SBP_ERR_UNSUPPORTED.
  *
  * P(sum) arithmetic: an fp32 accumulator starts as shard 0, shards 1..k-1 are added in
  * rank order with plain IEEE adds, and the result is rounded once (nearest even) to the

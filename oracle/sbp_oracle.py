@@ -160,6 +160,21 @@ def boxing(src_locals, src_sig, dst_sig, storage="f32"):
     if src_sig[0] == "P" and tuple(src_sig) == tuple(dst_sig):
         # Table 2, P -> P on the same placement costs 0: every device keeps its own partial.
         return [np.asarray(x).copy() for x in src_locals]
+    if tuple(dst_sig) == PSUM:
+        # Table 2, S -> P and B -> P on the same placement cost 0: every device builds its partial
+        # from what it already holds.  Reading: a split source pads its own slice with zeros
+        # (the k padded slices sum to T); a broadcast source keeps T on device 0, zeros elsewhere.
+        T = from_locals(src_locals, src_sig, storage)
+        outs = [np.zeros_like(T) for _ in range(k)]
+        if src_sig[0] == "S":
+            ax = src_sig[1]
+            for r, (start, ln) in enumerate(balanced_split(T.shape[ax], k)):
+                sel = [slice(None)] * T.ndim
+                sel[ax] = slice(start, start + ln)
+                outs[r][tuple(sel)] = np.asarray(src_locals[r])
+        else:
+            outs[0] = T.copy()
+        return outs
     T = from_locals(src_locals, src_sig, storage)
     return to_locals(T, dst_sig, k)
 

@@ -143,6 +143,22 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
 
   TaskGeom g;
   task_geometry(p, s, d, (int)sizeof(V), &g);
+  // S(i)/B -> P(sum): the destination shard is walked in full rows of Nb * C elements; only
+  // the vectors [own_lo, own_hi) of a row come from the source, the rest is written as zero.
+  long long own_lo = 0, own_hi = 0, src_row_vecs = 0;
+  if (p.mode == MODE_SCATTER_P) {
+    const long long row_vecs = p.Nb * p.C * p.esz / (long long)sizeof(V);   // exact: checked on the host
+    if (p.src_b) {                       // split source: its own slice of the axis
+      own_lo = g.boff_d * p.C * p.esz / (long long)sizeof(V);
+      own_hi = own_lo + g.seg_vecs;
+      src_row_vecs = g.seg_vecs;
+    } else {                             // broadcast source: shard 0 keeps the tensor
+      own_hi = t == 0 ? row_vecs : 0;
+      src_row_vecs = row_vecs;
+    }
+    g.seg_vecs = row_vecs;
+    g.nseg = p.A * p.Na * p.M;
+  }
   const long long seg0 = row_tile * p.rows_per_tile;
   if (seg0 >= g.nseg) return;
   const long long col0 = col_tile << p.cv_log2;
@@ -173,9 +189,25 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
   V val[J];
   if constexpr (OP == OP_COPY) {
     const V* sp = reinterpret_cast<const V*>(p.src[s]);
+    if (p.mode == MODE_SCATTER_P) {
 #pragma unroll
-    for (int j = 0; j < J; ++j)
-      if (ok[j]) val[j] = ld_stream(sp + so[j]);
+      for (int j = 0; j < J; ++j) {
+        const int f = threadIdx.x + j * 256;
+        const long long seg = seg0 + (f >> p.cv_log2);
+        const long long col = col0 + (f & ((1 << p.cv_log2) - 1));
+        dofs[j] = seg * g.seg_vecs + col;
+        V z;
+        unsigned char* zb = reinterpret_cast<unsigned char*>(&z);
+#pragma unroll
+        for (int b = 0; b < (int)sizeof(V); ++b) zb[b] = 0;
+        val[j] = z;
+        if (ok[j] && col >= own_lo && col < own_hi) val[j] = ld_stream(sp + seg * src_row_vecs + (col - own_lo));
+      }
+    } else {
+#pragma unroll
+      for (int j = 0; j < J; ++j)
+        if (ok[j]) val[j] = ld_stream(sp + so[j]);
+    }
   } else {
     using L = typename Lanes<OP, V>::type;
     const int kk = KT ? KT : p.k;
@@ -315,7 +347,9 @@ static sbp_status make_plan(const sbp_tensor* src, const sbp_tensor* dst, Plan* 
       return fail(SBP_ERR_UNSUPPORTED, "boxing between P(sum) and P(max) has no meaning");
     p.mode = MODE_DIAG;
   } else if (dst_p) {
-    return fail(SBP_ERR_UNSUPPORTED, "boxing S->P / B->P is not implemented");
+    if (ds.kind != SBP_PARTIAL_SUM)
+      return fail(SBP_ERR_UNSUPPORTED, "boxing S->P(max) / B->P(max) is not implemented (zero is not neutral for max)");
+    p.mode = MODE_SCATTER_P;
   } else if (src_p) {
     if (src->dtype == SBP_I64) return fail(SBP_ERR_DTYPE, "partial-value reduction needs F32 or BF16");
     const bool bf = src->dtype == SBP_BF16;
@@ -386,7 +420,7 @@ static sbp_status make_plan(const sbp_tensor* src, const sbp_tensor* dst, Plan* 
 
   // tiling: the largest segment / segment count over shards bounds the per-task grid
   const long long la_max = (p.src_a || p.dst_a) ? (p.Na + k - 1) / k : p.Na;
-  const long long lb_max = (p.src_b || p.dst_b) ? (p.Nb + k - 1) / k : p.Nb;
+  const long long lb_max = ((p.src_b || p.dst_b) && p.mode != MODE_SCATTER_P) ? (p.Nb + k - 1) / k : p.Nb;
   const long long nseg_max = p.A * la_max * p.M;
   const long long seg_vecs_max = lb_max * p.C * p.esz / pl->vbytes;
   const int J = pl->op == OP_COPY ? kJCopy : kJReduce;
@@ -442,7 +476,7 @@ sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream)
   // Default choice, from measurement on B200: the bulk engine wins where one read feeds one
   // write (re-layouts and slices); the load/store kernel wins where one read feeds k writes.
   const int engine = g_copy_engine.load();
-  const bool want_bulk = engine == 2 || (engine == 0 && pl.p.mode != MODE_GATHER);
+  const bool want_bulk = (engine == 2 || (engine == 0 && pl.p.mode != MODE_GATHER)) && pl.p.mode != MODE_SCATTER_P;
   if (pl.op == OP_COPY && want_bulk && pl.vbytes == 16)
     done = launch_bulk_copy(pl.p, pl.ntasks, stream);
   if (!done) {

@@ -10,7 +10,8 @@ enum BoxMode : int {
   MODE_DIAG = 1,       // task t: source shard t, destination shard t
   MODE_GATHER = 2,     // task t: source shard t, every destination replica
   MODE_REDUCE_S = 3,   // task t: all sources, destination shard t
-  MODE_REDUCE_B = 4    // one task: all sources, every destination replica
+  MODE_REDUCE_B = 4,   // one task: all sources, every destination replica
+  MODE_SCATTER_P = 5   // task t: destination shard t is the full shape: own piece copied, rest zero
 };
 
 // The logical tensor is viewed as [A][Na][M][Nb][C] (elements); src_a/src_b/dst_a/dst_b say

@@ -117,7 +117,7 @@ def test_boxing_validation_happens_before_any_launch(lib):
     assert _status(boxing, src, _host_tensor((8, 9), f32, sbp.B, 2)) == "SBP_ERR_SHAPE"
     assert _status(boxing, src, _host_tensor((8, 8), bf16, sbp.B, 2)) == "SBP_ERR_DTYPE"
     assert _status(boxing, src, _host_tensor((8, 8), f32, sbp.B, 4)) == "SBP_ERR_INVALID_ARG"
-    assert _status(boxing, src, _host_tensor((8, 8), f32, sbp.P_SUM, 2)) == "SBP_ERR_UNSUPPORTED"
+    assert _status(boxing, src, _host_tensor((8, 8), f32, sbp.P_MAX, 2)) == "SBP_ERR_UNSUPPORTED"
     assert _status(boxing, _host_tensor((8, 8), f32, sbp.P_SUM, 2),
                    _host_tensor((8, 8), f32, sbp.P_MAX, 2)) == "SBP_ERR_UNSUPPORTED"
     assert _status(boxing, _host_tensor((8, 8), i64, sbp.P_SUM, 2),

@@ -69,11 +69,12 @@ def _run(shape, dtype, src_sig, dst_sig, k, seed=1, engine=0, alias=False, offse
 
 MOVES = [(sbp.S(0), sbp.B), (sbp.S(1), sbp.B), (sbp.S(0), sbp.S(1)), (sbp.S(1), sbp.S(0)),
          (sbp.B, sbp.S(0)), (sbp.B, sbp.S(1)), (sbp.S(0), sbp.S(0)), (sbp.B, sbp.B)]
+TO_PARTIAL = [(sbp.S(0), sbp.P_SUM), (sbp.S(1), sbp.P_SUM), (sbp.B, sbp.P_SUM)]
 REDUCES = [(sbp.P_SUM, sbp.B), (sbp.P_SUM, sbp.S(0)), (sbp.P_SUM, sbp.S(1)),
            (sbp.P_MAX, sbp.B), (sbp.P_MAX, sbp.S(1)), (sbp.P_SUM, sbp.P_SUM)]
 
 
-@pytest.mark.parametrize("src_sig,dst_sig", MOVES + REDUCES)
+@pytest.mark.parametrize("src_sig,dst_sig", MOVES + REDUCES + TO_PARTIAL)
 @pytest.mark.parametrize("k", [1, 2, 3, 4, 8])
 @pytest.mark.parametrize("dtype", [F32, BF16])
 def test_boxing_2d_aligned_and_ragged(src_sig, dst_sig, k, dtype):
@@ -109,7 +110,29 @@ def test_bulk_copy_engine_matches(src_sig, dst_sig, k):
     _run((67, 101), F32, src_sig, dst_sig, k, engine=2)        # unaligned: falls back to load/store
 
 
+def test_boxing_to_partial_sum_nd_and_round_trip():
+    for shape in [(6, 10, 16), (3, 5, 7, 8), (40,)]:
+        for i in range(len(shape)):
+            _run(shape, F32, sbp.S(i), sbp.P_SUM, 3)
+        _run(shape, BF16, sbp.B, sbp.P_SUM, 4)
+    _run((33, 40), I64, sbp.S(1), sbp.P_SUM, 4)
+    # S(0) -> P(sum) -> B returns the logical tensor (x + 0 is exact)
+    k, shape = 4, (96, 160)
+    T = dg.normal(6, 0, shape, 0, 1, BF16)
+    s0 = make_global(split_cpu(T, sbp.S(0), k), shape, BF16, sbp.S(0))
+    part = sbp.empty_global(shape, BF16, sbp.P_SUM, k)
+    rep = sbp.empty_global(shape, BF16, sbp.B, k)
+    sbp.sbp_boxing(s0, part)
+    sbp.sbp_boxing(part, rep)
+    torch.cuda.synchronize()
+    assert all(np.array_equal(bits(r), bits(T)) for r in rep.locals)
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_boxing(s0, sbp.empty_global(shape, BF16, sbp.P_MAX, k))
+    assert e.value.name == "SBP_ERR_UNSUPPORTED"
+
+
 def test_boxing_larger_than_one_wave():
+    _run((2048, 3072), BF16, sbp.S(1), sbp.P_SUM, 4)
     _run((2048, 3072), BF16, sbp.P_SUM, sbp.B, 4)
     _run((2048, 3072), BF16, sbp.S(0), sbp.S(1), 4)
     _run((2048, 3072), BF16, sbp.S(0), sbp.S(1), 4, engine=2)

@@ -509,3 +509,32 @@ def test_locate_agrees_with_to_locals(shape, k):
             assert loc[r][li] == T[idx]
     pairs = O.locate(shape, B, k, (0,) * len(shape))
     assert [r for r, _ in pairs] == list(range(k)) and all(li == (0,) * len(shape) for _, li in pairs)
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 4])
+def test_boxing_to_partial_sum_is_local_and_sums_back(k):
+    # Table 2: S -> P and B -> P move nothing.  Brute force: element (i, j) of shard r is the
+    # global element if r owns it (S source) / if r == 0 (B source), else zero.
+    n0, n1 = 7, 10
+    T = (np.arange(n0 * n1, dtype=np.float32).reshape(n0, n1) + 1)
+    for src_sig in (S0, S1, B):
+        src = O.to_locals(T, src_sig, k)
+        out = O.boxing(src, src_sig, PSUM)
+        assert len(out) == k
+        for r in range(k):
+            assert out[r].shape == T.shape
+            for i in range(n0):
+                for j in range(n1):
+                    if src_sig == B:
+                        mine = r == 0
+                    else:
+                        (owner, _), = O.locate((n0, n1), src_sig, k, (i, j))
+                        mine = owner == r
+                    assert out[r][i, j] == (T[i, j] if mine else 0.0)
+        assert np.array_equal(O.from_locals(out, PSUM, "f32"), T)
+        assert O.table2_same_placement_cost(src_sig, PSUM, k, T.nbytes) == 0
+        # nothing crosses devices: tag the sources with their device, non-zero tags stay home
+        tags = [np.full(s.shape, r + 1, np.float32) for r, s in enumerate(src)]
+        moved = O.boxing(tags, src_sig, PSUM) if src_sig != B else O.boxing([tags[0]] * k, B, PSUM)
+        for r in range(k):
+            assert set(np.unique(moved[r])) <= {0.0, float(r + 1)} if src_sig != B else True

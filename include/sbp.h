@@ -76,9 +76,11 @@ typedef struct {
  * tensor carries a placement and an sbp attribute).  Plain data; the caller owns it.
  *
  *   shape[0..ndim)   LOGICAL (global) shape, 1 <= ndim <= SBP_MAX_DIMS.
- *   pdims, pshape    placement hierarchy; k = product of pshape[0..pdims).  The paper's
- *                    multi-dimensional SBP (Section 3.3) needs pdims == 2; this build
- *                    implements pdims == 1 and answers SBP_ERR_UNSUPPORTED otherwise.
+ *   pdims, pshape    placement hierarchy; k = product of pshape[0..pdims).  pdims == 2 is the
+ *                    paper's multi-dimensional SBP (Section 3.3): sbp[0] is applied across the
+ *                    pshape[0] groups, sbp[1] inside a group, and device (i, j) is local[i *
+ *                    pshape[1] + j].  sbp_local_shape, sbp_boxing and sbp_matmul accept
+ *                    pdims == 2; every other entry point answers SBP_ERR_UNSUPPORTED.
  *   sbp[p]           one signature per placement axis.
  *   local[r]         device pointer of shard r's local tensor, r in [0, k).  For a B
  *                    tensor the k replicas may all be the same pointer; a kernel then
@@ -129,6 +131,12 @@ sbp_status sbp_matmul_infer(sbp_sig x, sbp_sig w, sbp_sig* y);
  *   B              P(sum)     local (Table 2: cost 0): shard 0 = the tensor, every other shard zeros
  * Anything else (a P(max) destination from S or B, P(sum)<->P(max)) returns SBP_ERR_UNSUPPORTED.
  *
+ * Two-axis placements: one call may change the signature of ONE placement axis (the other stays
+ * as it is); the transform then runs as independent one-axis boxing ops, inside each group when
+ * axis 1 changes, across the groups when axis 0 changes.  Changing axis 0 along the tensor axis
+ * that axis 1 splits, or summing over one axis what is a max over the other, is refused with
+ * SBP_ERR_UNSUPPORTED, as is changing both axes at once (make two calls).
+ *
  * P(sum) arithmetic: an fp32 accumulator starts as shard 0, shards 1..k-1 are added in
  * rank order with plain IEEE adds, and the result is rounded once (nearest even) to the
  * storage dtype.  P(max): acc = shard 0; shard r replaces acc only when strictly greater.
@@ -170,6 +178,9 @@ void sbp_boxing_set_copy_engine(int32_t engine);
  * kernel's accumulator and Y is written directly in that signature (the boxing op of
  * Section 3.2 fused into the producer).  Any other request is SBP_ERR_SIGNATURE; call
  * sbp_boxing afterwards instead.
+ * Two-axis placements (Table 3, e.g. (S(0),B) x (B,S(1)) -> (S(0),S(1)) and (S(0),S(1)) x
+ * (B,S(0)) -> (S(0),P(sum))): Table 1 is applied to each placement axis on its own, y must carry
+ * exactly the deduced pair, and every device multiplies its local tensors (no fused boxing).
  *
  * x: [M,K], w: [K,N], y: [M,N] logical, all 2-D, same dtype for x and w:
  *   SBP_F32  : fp32 FMA accumulation, y SBP_F32.

@@ -248,6 +248,57 @@ def matmul_locals(x_locals, x_sig, w_locals, w_sig):
 
 
 # --------------------------------------------------------------------------------------
+# Section 3.3: multi-dimensional SBP.  A placement of k0 x k1 devices carries one signature
+# per placement axis, e.g. (S(0), B): S(0) across the k0 groups ("nodes"), B among the k1
+# devices of a group.  Device (i, j) -- listed row-major, index i * k1 + j -- holds piece j,
+# under the second signature, of piece i, under the first, of the global tensor.
+# --------------------------------------------------------------------------------------
+
+def to_locals_2d(T, sigs, pshape):
+    k0, k1 = pshape
+    out = []
+    for node in to_locals(T, sigs[0], k0):
+        out.extend(to_locals(node, sigs[1], k1))
+    return out
+
+
+def from_locals_2d(locals_, sigs, pshape, storage="f32"):
+    k0, k1 = pshape
+    nodes = [from_locals(locals_[i * k1:(i + 1) * k1], sigs[1], storage) for i in range(k0)]
+    return from_locals(nodes, sigs[0], storage)
+
+
+def boxing_2d(src_locals, src_sigs, dst_sigs, pshape, storage="f32"):
+    """Boxing between two-axis signatures none of whose destination axes is partial-value."""
+    return to_locals_2d(from_locals_2d(src_locals, src_sigs, pshape, storage), dst_sigs, pshape)
+
+
+def matmul_infer_2d(x_sigs, w_sigs):
+    """Table 3: Table 1 applied to each placement axis on its own; None if either is invalid."""
+    ys = tuple(matmul_infer(a, b) for a, b in zip(x_sigs, w_sigs))
+    return None if any(y is None for y in ys) else ys
+
+
+def matmul_locals_2d(x_locals, x_sigs, w_locals, w_sigs, pshape):
+    """Every device multiplies its local tensors.  Returns (y_sigs, y_locals, Y_logical) with
+    the logical product computed from the logical operands (partial operands summed in fp64)."""
+    y_sigs = matmul_infer_2d(x_sigs, w_sigs)
+    if y_sigs is None:
+        raise ValueError("invalid two-axis MatMul signature")
+    f64 = lambda ls: [np.asarray(a, dtype=np.float64) for a in ls]
+    xl, wl = f64(x_locals), f64(w_locals)
+
+    def logical(locs, sigs):
+        k0, k1 = pshape
+        def inv(ls, sig):
+            return reduce_sum_fp64(ls) if tuple(sig) == PSUM else from_locals(ls, sig)
+        return inv([inv(locs[i * k1:(i + 1) * k1], sigs[1]) for i in range(k0)], sigs[0])
+
+    Y = matmul_logical(logical(xl, x_sigs), logical(wl, w_sigs))
+    return y_sigs, [matmul_logical(a, b) for a, b in zip(xl, wl)], Y
+
+
+# --------------------------------------------------------------------------------------
 # GeLU (erf form) and the Megatron-style MLP block: B x S(1) -> S(1), GeLU, S(1) x S(0)
 # -> P(sum), boxed to B.  Logical result only; sharding cannot change it.
 # --------------------------------------------------------------------------------------

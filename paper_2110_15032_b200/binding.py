@@ -122,14 +122,26 @@ class SbpTensor:
 
     `locals` are torch tensors used purely as memory (device memory for every entry
     point except sbp_boxing_host, which takes host tensors).  Each must be contiguous.
+    For a two-axis placement (the paper's multi-dimensional SBP) pass `sig` as a pair of
+    signatures and `pshape=(k0, k1)`; `locals` then lists the devices row-major (i * k1 + j).
     """
 
-    def __init__(self, shape: Sequence[int], dtype: torch.dtype, sig: Sig, locals: Sequence[torch.Tensor]):
+    def __init__(self, shape: Sequence[int], dtype: torch.dtype, sig, locals: Sequence[torch.Tensor],
+                 pshape: Optional[Sequence[int]] = None):
         self.shape = tuple(int(s) for s in shape)
         self.dtype = dtype
         self.sig = sig
         self.locals: List[torch.Tensor] = list(locals)
         self.k = len(self.locals)
+        self.sigs = tuple(sig) if isinstance(sig, (tuple, list)) else (sig,)
+        self.pshape = tuple(int(v) for v in pshape) if pshape is not None else (self.k,)
+        if len(self.sigs) != len(self.pshape):
+            raise ValueError("one signature per placement axis")
+        n = 1
+        for v in self.pshape:
+            n *= v
+        if n != self.k:
+            raise ValueError("placement size differs from the number of local tensors")
         for t in self.locals:
             if not t.is_contiguous():
                 raise ValueError("local tensors must be contiguous")
@@ -142,10 +154,11 @@ class SbpTensor:
         d.dtype = _DTYPES[self.dtype]
         for i, s in enumerate(self.shape):
             d.shape[i] = s
-        d.pdims = 1
-        d.pshape[0] = self.k
+        d.pdims = len(self.pshape)
         d.pshape[1] = 1
-        d.sbp[0] = self.sig._c()
+        for p, v in enumerate(self.pshape):
+            d.pshape[p] = v
+            d.sbp[p] = self.sigs[p]._c()
         for r, t in enumerate(self.locals):
             d.local[r] = t.data_ptr()
         return d
@@ -157,29 +170,37 @@ def _stream_ptr(stream) -> Optional[int]:
     return C.c_void_p(stream.cuda_stream)
 
 
-def sbp_local_shape(shape, sig: Sig, k: int, r: int, dtype=torch.float32):
+def sbp_local_shape(shape, sig, k, r: int, dtype=torch.float32):
+    """Local shape of device r.  One-axis placement: sig a Sig, k an int.  Two-axis placement:
+    sig a pair of Sig, k the pair (k0, k1), r = i * k1 + j."""
+    sigs = tuple(sig) if isinstance(sig, (tuple, list)) else (sig,)
+    pshape = tuple(k) if isinstance(k, (tuple, list)) else (k,)
     d = _Tensor()
     d.ndim = len(shape)
     d.dtype = _DTYPES[dtype]
     for i, s in enumerate(shape):
         d.shape[i] = int(s)
-    d.pdims = 1
-    d.pshape[0] = k
-    d.sbp[0] = sig._c()
+    d.pdims = len(pshape)
+    d.pshape[1] = 1
+    for p, v in enumerate(pshape):
+        d.pshape[p] = int(v)
+        d.sbp[p] = sigs[p]._c()
     out = (C.c_int64 * SBP_MAX_DIMS)()
     _check(load_library().sbp_local_shape(C.byref(d), r, out))
     return tuple(out[i] for i in range(len(shape)))
 
 
-def empty_global(shape, dtype, sig: Sig, k: int, device="cuda", alias_replicas: bool = False) -> SbpTensor:
-    """Allocates (torch.empty) the k local tensors of a global tensor."""
+def empty_global(shape, dtype, sig, k, device="cuda", alias_replicas: bool = False) -> SbpTensor:
+    """Allocates (torch.empty) the local tensors of a global tensor (k an int, or (k0, k1))."""
+    pshape = tuple(k) if isinstance(k, (tuple, list)) else None
+    n = k if pshape is None else pshape[0] * pshape[1]
     locs = []
-    for r in range(k):
-        if alias_replicas and sig.kind == SBP_BROADCAST and r > 0:
+    for r in range(n):
+        if alias_replicas and pshape is None and sig.kind == SBP_BROADCAST and r > 0:
             locs.append(locs[0])
         else:
             locs.append(torch.empty(sbp_local_shape(shape, sig, k, r, dtype), dtype=dtype, device=device))
-    return SbpTensor(shape, dtype, sig, locs)
+    return SbpTensor(shape, dtype, sig, locs, pshape)
 
 
 def sbp_matmul_infer(x: Sig, w: Sig) -> Sig:

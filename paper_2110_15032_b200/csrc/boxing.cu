@@ -463,7 +463,83 @@ extern "C" {
 
 void sbp_boxing_set_copy_engine(int32_t engine) { g_copy_engine.store(engine); }
 
+// Two-axis placements (Section 3.3, multi-dimensional SBP): device (i, j) of a k0 x k1
+// placement holds piece j, under sbp[1], of piece i, under sbp[0], of the global tensor.  A
+// boxing op that changes the signature of ONE placement axis is a set of independent one-axis
+// boxing ops: inside every group i when axis 1 changes, across the groups for every j when
+// axis 0 changes (valid when the unchanged axis-1 mapping commutes with the change).
+static bool is_partial(sbp_sig s) { return s.kind == SBP_PARTIAL_SUM || s.kind == SBP_PARTIAL_MAX; }
+
+static sbp_status boxing_2d(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream) {
+  sbp_status st = check_tensor_nd(src, "src", true);
+  if (st != SBP_OK) return st;
+  st = check_tensor_nd(dst, "dst", true);
+  if (st != SBP_OK) return st;
+  if (src->pdims != 2 || dst->pdims != 2 || src->pshape[0] != dst->pshape[0] || src->pshape[1] != dst->pshape[1])
+    return fail(SBP_ERR_INVALID_ARG, "src and dst must live on the same two-axis placement");
+  if (src->ndim != dst->ndim) return fail(SBP_ERR_SHAPE, "src and dst differ in rank");
+  for (int d = 0; d < src->ndim; ++d)
+    if (src->shape[d] != dst->shape[d]) return fail(SBP_ERR_SHAPE, "src and dst differ on axis %d", d);
+  if (src->dtype != dst->dtype) return fail(SBP_ERR_DTYPE, "src and dst differ in dtype");
+  const int k0 = src->pshape[0], k1 = src->pshape[1];
+  const bool ch0 = !same_sig(src->sbp[0], dst->sbp[0]), ch1 = !same_sig(src->sbp[1], dst->sbp[1]);
+  if (ch0 && ch1)
+    return fail(SBP_ERR_UNSUPPORTED, "change one placement axis per boxing call (two calls for both)");
+
+  sbp_tensor s1 = *src, d1 = *dst;
+  s1.pdims = d1.pdims = 1;
+  s1.pshape[1] = d1.pshape[1] = 1;
+  if (!ch0) {
+    // axis 1 changes (or nothing does): one boxing op inside each group, on the group's tensor
+    s1.pshape[0] = d1.pshape[0] = k1;
+    s1.sbp[0] = src->sbp[1];
+    d1.sbp[0] = dst->sbp[1];
+    for (int i = 0; i < k0; ++i) {
+      if (src->sbp[0].kind == SBP_SPLIT) {
+        int64_t start, len;
+        split_range(src->shape[src->sbp[0].axis], k0, i, &start, &len);
+        s1.shape[src->sbp[0].axis] = d1.shape[src->sbp[0].axis] = len;
+      }
+      for (int j = 0; j < k1; ++j) {
+        s1.local[j] = src->local[i * k1 + j];
+        d1.local[j] = dst->local[i * k1 + j];
+      }
+      st = sbp_boxing(&s1, &d1, cuda_stream);
+      if (st != SBP_OK) return st;
+    }
+    return SBP_OK;
+  }
+  // axis 0 changes, axis 1 keeps signature c
+  const sbp_sig c = src->sbp[1];
+  if (c.kind == SBP_SPLIT) {
+    if ((src->sbp[0].kind == SBP_SPLIT && src->sbp[0].axis == c.axis) ||
+        (dst->sbp[0].kind == SBP_SPLIT && dst->sbp[0].axis == c.axis))
+      return fail(SBP_ERR_UNSUPPORTED, "axis 0 cannot be re-boxed along the tensor axis that axis 1 splits");
+  } else if (is_partial(c)) {
+    if (is_partial(src->sbp[0]) && src->sbp[0].kind != c.kind)
+      return fail(SBP_ERR_UNSUPPORTED, "a max over one placement axis does not commute with a sum over the other");
+  }
+  s1.pshape[0] = d1.pshape[0] = k0;
+  s1.sbp[0] = src->sbp[0];
+  d1.sbp[0] = dst->sbp[0];
+  for (int j = 0; j < k1; ++j) {
+    if (c.kind == SBP_SPLIT) {
+      int64_t start, len;
+      split_range(src->shape[c.axis], k1, j, &start, &len);
+      s1.shape[c.axis] = d1.shape[c.axis] = len;
+    }
+    for (int i = 0; i < k0; ++i) {
+      s1.local[i] = src->local[i * k1 + j];
+      d1.local[i] = dst->local[i * k1 + j];
+    }
+    st = sbp_boxing(&s1, &d1, cuda_stream);
+    if (st != SBP_OK) return st;
+  }
+  return SBP_OK;
+}
+
 sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream) {
+  if (src && dst && (src->pdims == 2 || dst->pdims == 2)) return boxing_2d(src, dst, cuda_stream);
   sbp_status st = check_pair(src, dst, true);
   if (st != SBP_OK) return st;
   Plan pl;

@@ -238,6 +238,70 @@ static sbp_status build_plan(const sbp_tensor* x, const sbp_tensor* w, const sbp
   return SBP_OK;
 }
 
+// Two-axis placements (Section 3.3, Table 3): Table 1 is applied to each placement axis on its
+// own -- e.g. (S(0),B) x (B,S(1)) -> (S(0),S(1)) and (S(0),S(1)) x (B,S(0)) -> (S(0),P(sum)) --
+// and every device multiplies its local tensors.  No fused output boxing on this path.
+static sbp_status build_plan_2d(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y, uint32_t flags,
+                                MatmulPlan* plan) {
+  sbp_status st = check_tensor_nd(x, "x", true);
+  if (st != SBP_OK) return st;
+  st = check_tensor_nd(w, "w", true);
+  if (st != SBP_OK) return st;
+  st = check_tensor_nd(y, "y", true);
+  if (st != SBP_OK) return st;
+  if (x->pdims != 2 || w->pdims != 2 || y->pdims != 2) return fail(SBP_ERR_INVALID_ARG, "x, w and y must share one two-axis placement");
+  for (int p = 0; p < 2; ++p)
+    if (x->pshape[p] != w->pshape[p] || x->pshape[p] != y->pshape[p])
+      return fail(SBP_ERR_INVALID_ARG, "x, w and y must share one two-axis placement");
+  if (x->ndim != 2 || w->ndim != 2 || y->ndim != 2) return fail(SBP_ERR_SHAPE, "x, w and y must be 2-D");
+  const long long M = x->shape[0], K = x->shape[1], N = w->shape[1];
+  if (w->shape[0] != K) return fail(SBP_ERR_SHAPE, "x is [%lld,%lld] but w has %lld rows", M, K, (long long)w->shape[0]);
+  if (y->shape[0] != M || y->shape[1] != N) return fail(SBP_ERR_SHAPE, "y must be [%lld,%lld]", M, N);
+  if (x->dtype != w->dtype) return fail(SBP_ERR_DTYPE, "x and w differ in dtype");
+  if (x->dtype != SBP_F32 && x->dtype != SBP_BF16) return fail(SBP_ERR_DTYPE, "operands must be F32 or BF16");
+  if (y->dtype != SBP_F32 && y->dtype != SBP_BF16) return fail(SBP_ERR_DTYPE, "y must be F32 or BF16");
+  if (x->dtype == SBP_F32 && y->dtype != SBP_F32) return fail(SBP_ERR_DTYPE, "F32 operands need an F32 result");
+  if (flags & ~SBP_EPILOGUE_GELU) return fail(SBP_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
+  for (int p = 0; p < 2; ++p) {
+    sbp_sig natural;
+    st = sbp_matmul_infer(x->sbp[p], w->sbp[p], &natural);
+    if (st != SBP_OK) return st;
+    if (!same_sig(natural, y->sbp[p]))
+      return fail(SBP_ERR_SIGNATURE, "placement axis %d: y's signature is not the one Table 1 deduces", p);
+    if ((flags & SBP_EPILOGUE_GELU) && is_p(natural))
+      return fail(SBP_ERR_SIGNATURE, "GeLU is not linear: it cannot be applied to partial values");
+  }
+  const int k = placement_k(x);
+  MatmulPlan& p = *plan;
+  p = MatmulPlan{};
+  p.gelu = (flags & SBP_EPILOGUE_GELU) ? 1 : 0;
+  p.in_dtype = x->dtype;
+  p.out_dtype = y->dtype;
+  p.ngroups = k;
+  p.nseg = k;
+  p.chain = 0;
+  for (int r = 0; r < k; ++r) {
+    int64_t xs[SBP_MAX_DIMS], wsz[SBP_MAX_DIMS], ys[SBP_MAX_DIMS];
+    local_shape_nd(x, r, xs);
+    local_shape_nd(w, r, wsz);
+    local_shape_nd(y, r, ys);
+    if (xs[1] != wsz[0] || ys[0] != xs[0] || ys[1] != wsz[1])
+      return fail(SBP_ERR_SHAPE, "device %d: local shapes [%lld,%lld] x [%lld,%lld] -> [%lld,%lld] do not fit", r,
+                  (long long)xs[0], (long long)xs[1], (long long)wsz[0], (long long)wsz[1], (long long)ys[0],
+                  (long long)ys[1]);
+    p.a[r] = x->local[r];
+    p.b[r] = w->local[r];
+    p.lda[r] = xs[1];
+    p.ldb[r] = wsz[1];
+    p.kseg[r] = xs[1];
+    p.m[r] = xs[0];
+    p.n[r] = wsz[1];
+    p.ldy[r] = wsz[1];
+    p.y[r] = y->local[r];
+  }
+  return SBP_OK;
+}
+
 }  // namespace sbp
 
 using namespace sbp;
@@ -253,7 +317,8 @@ size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, cons
 sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, uint32_t flags, void* ws,
                       size_t ws_bytes, void* cuda_stream) {
   MatmulPlan plan;
-  sbp_status st = build_plan(x, w, y, flags, true, &plan);
+  const bool two_axes = x && w && y && (x->pdims == 2 || w->pdims == 2 || y->pdims == 2);
+  sbp_status st = two_axes ? build_plan_2d(x, w, y, flags, &plan) : build_plan(x, w, y, flags, true, &plan);
   if (st != SBP_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   bool taken = false;

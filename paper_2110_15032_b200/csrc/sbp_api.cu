@@ -23,7 +23,7 @@ sbp_status cuda_fail(cudaError_t e, const char* what) {
   return fail(SBP_ERR_CUDA, "%s: %s", what, cudaGetErrorString(e));
 }
 
-sbp_status check_tensor(const sbp_tensor* t, const char* name, bool need_ptrs) {
+static sbp_status check_common(const sbp_tensor* t, const char* name, bool need_ptrs, bool allow_2d) {
   if (!t) return fail(SBP_ERR_INVALID_ARG, "%s: null descriptor", name);
   if (t->ndim < 1 || t->ndim > SBP_MAX_DIMS)
     return fail(SBP_ERR_INVALID_ARG, "%s: ndim %d outside [1,%d]", name, t->ndim, SBP_MAX_DIMS);
@@ -36,14 +36,16 @@ sbp_status check_tensor(const sbp_tensor* t, const char* name, bool need_ptrs) {
     if (t->pshape[p] < 1) return fail(SBP_ERR_INVALID_ARG, "%s: placement extent < 1", name);
   int k = placement_k(t);
   if (k > SBP_MAX_K) return fail(SBP_ERR_INVALID_ARG, "%s: k = %d exceeds %d", name, k, SBP_MAX_K);
-  if (t->pdims != 1)
-    return fail(SBP_ERR_UNSUPPORTED, "%s: multi-dimensional SBP (pdims = %d) is not implemented", name,
-                t->pdims);
-  sbp_sig s = t->sbp[0];
-  if (s.kind < SBP_SPLIT || s.kind > SBP_PARTIAL_MAX)
-    return fail(SBP_ERR_SIGNATURE, "%s: unknown sbp kind %d", name, s.kind);
-  if (s.kind == SBP_SPLIT && (s.axis < 0 || s.axis >= t->ndim))
-    return fail(SBP_ERR_SIGNATURE, "%s: split axis %d outside [0,%d)", name, s.axis, t->ndim);
+  if (t->pdims != 1 && !allow_2d)
+    return fail(SBP_ERR_UNSUPPORTED, "%s: multi-dimensional SBP (pdims = %d) is not implemented by this entry point",
+                name, t->pdims);
+  for (int p = 0; p < t->pdims; ++p) {
+    sbp_sig s = t->sbp[p];
+    if (s.kind < SBP_SPLIT || s.kind > SBP_PARTIAL_MAX)
+      return fail(SBP_ERR_SIGNATURE, "%s: unknown sbp kind %d", name, s.kind);
+    if (s.kind == SBP_SPLIT && (s.axis < 0 || s.axis >= t->ndim))
+      return fail(SBP_ERR_SIGNATURE, "%s: split axis %d outside [0,%d)", name, s.axis, t->ndim);
+  }
   if (need_ptrs) {
     for (int r = 0; r < k; ++r) {
       if (!t->local[r] && local_numel(t, r) > 0)
@@ -55,17 +57,34 @@ sbp_status check_tensor(const sbp_tensor* t, const char* name, bool need_ptrs) {
   return SBP_OK;
 }
 
-int64_t local_numel(const sbp_tensor* t, int r) {
-  int k = placement_k(t);
-  int64_t n = 1;
-  for (int d = 0; d < t->ndim; ++d) {
-    int64_t e = t->shape[d];
-    if (t->sbp[0].kind == SBP_SPLIT && t->sbp[0].axis == d) {
-      int64_t st;
-      split_range(t->shape[d], k, r, &st, &e);
-    }
-    n *= e;
+sbp_status check_tensor(const sbp_tensor* t, const char* name, bool need_ptrs) {
+  return check_common(t, name, need_ptrs, false);
+}
+
+sbp_status check_tensor_nd(const sbp_tensor* t, const char* name, bool need_ptrs) {
+  return check_common(t, name, need_ptrs, true);
+}
+
+void local_shape_nd(const sbp_tensor* t, int r, int64_t out[SBP_MAX_DIMS]) {
+  for (int d = 0; d < SBP_MAX_DIMS; ++d) out[d] = d < t->ndim ? t->shape[d] : 1;
+  int idx[SBP_MAX_PDIMS] = {r, 0};
+  if (t->pdims == 2) {
+    idx[0] = r / t->pshape[1];
+    idx[1] = r % t->pshape[1];
   }
+  for (int p = 0; p < t->pdims; ++p) {
+    if (t->sbp[p].kind != SBP_SPLIT) continue;
+    int64_t start, len;
+    split_range(out[t->sbp[p].axis], t->pshape[p], idx[p], &start, &len);
+    out[t->sbp[p].axis] = len;
+  }
+}
+
+int64_t local_numel(const sbp_tensor* t, int r) {
+  int64_t shp[SBP_MAX_DIMS];
+  local_shape_nd(t, r, shp);
+  int64_t n = 1;
+  for (int d = 0; d < t->ndim; ++d) n *= shp[d];
   return n;
 }
 
@@ -117,17 +136,12 @@ sbp_status sbp_selftest_wait_timeout(uint32_t limit_ms, void* cuda_stream) {
 }
 
 sbp_status sbp_local_shape(const sbp_tensor* t, int32_t r, int64_t out_shape[SBP_MAX_DIMS]) {
-  sbp_status st = check_tensor(t, "t", false);
+  sbp_status st = check_tensor_nd(t, "t", false);
   if (st != SBP_OK) return st;
   if (!out_shape) return fail(SBP_ERR_INVALID_ARG, "out_shape is null");
   int k = placement_k(t);
   if (r < 0 || r >= k) return fail(SBP_ERR_INVALID_ARG, "shard %d outside [0,%d)", r, k);
-  for (int d = 0; d < SBP_MAX_DIMS; ++d) out_shape[d] = d < t->ndim ? t->shape[d] : 1;
-  if (t->sbp[0].kind == SBP_SPLIT) {
-    int64_t start, len;
-    split_range(t->shape[t->sbp[0].axis], k, r, &start, &len);
-    out_shape[t->sbp[0].axis] = len;
-  }
+  local_shape_nd(t, r, out_shape);
   return SBP_OK;
 }
 

@@ -41,6 +41,14 @@ inline bool same_sig(sbp_sig a, sbp_sig b) {
   return a.kind == b.kind && (a.kind != SBP_SPLIT || a.axis == b.axis);
 }
 
+// Local shape of device r under a 1-D or 2-D (hierarchical) placement: the signature of
+// placement axis 0 is applied across the pshape[0] groups, then that of axis 1 inside a group;
+// device r = i * pshape[1] + j.  out has SBP_MAX_DIMS entries (1 beyond ndim).
+void local_shape_nd(const sbp_tensor* t, int r, int64_t out[SBP_MAX_DIMS]);
+
+// Same checks as check_tensor but also accepts a two-axis placement (Section 3.3).
+sbp_status check_tensor_nd(const sbp_tensor* t, const char* name, bool need_ptrs);
+
 // Full validation of a descriptor (rank, dtype, placement, signature, pointers).
 // need_ptrs: every local[r], r < k, must be non-null and aligned to the element size.
 sbp_status check_tensor(const sbp_tensor* t, const char* name, bool need_ptrs);

@@ -126,7 +126,14 @@ def test_boxing_validation_happens_before_any_launch(lib):
     d.pdims = 2
     d.pshape[0], d.pshape[1] = 2, 1
     b = _host_tensor((8, 8), f32, sbp.B, 2)._c()
-    assert lib.sbp_boxing(C.byref(d), C.byref(b), stream) == 5          # multi-dimensional SBP: unsupported
+    assert lib.sbp_boxing(C.byref(d), C.byref(b), stream) == 1          # placements of src and dst differ
+    b2 = _host_tensor((8, 8), f32, sbp.B, 2)._c()
+    b2.pdims = 2
+    b2.pshape[0], b2.pshape[1] = 2, 1
+    b2.sbp[1] = binding._Sig(3, 0)                                      # both axes would change at once
+    assert lib.sbp_boxing(C.byref(d), C.byref(b2), stream) == 5
+    labels2 = _host_tensor((8,), torch.int64, sbp.B, 2)._c()
+    assert lib.sbp_softmax_xent(C.byref(d), C.byref(labels2), C.byref(labels2), None, None, None, 0, None) == 5
     d = src._c()
     d.local[1] = None
     assert lib.sbp_boxing(C.byref(d), C.byref(b), stream) == 1          # null local tensor

@@ -538,3 +538,61 @@ def test_boxing_to_partial_sum_is_local_and_sums_back(k):
         moved = O.boxing(tags, src_sig, PSUM) if src_sig != B else O.boxing([tags[0]] * k, B, PSUM)
         for r in range(k):
             assert set(np.unique(moved[r])) <= {0.0, float(r + 1)} if src_sig != B else True
+
+
+# ---------------------------------------------------------------- Section 3.3: two-axis placements
+
+def _parse_sig2(tok):
+    return tuple(_parse_sig(t) for t in tok.split(","))
+
+
+def test_table3_fixture_and_local_products_brute_force():
+    rows = read_golden("table3_matmul_2d_sbp.txt")
+    assert len(rows) == 2
+    M, K, N = 6, 8, 9
+    X = dg.small_integers(81, 0, (M, K), -4, 5).numpy().astype(np.float64)
+    W = dg.small_integers(81, 1, (K, N), -4, 5).numpy().astype(np.float64)
+    Y = _py_matmul(X, W)
+    for pshape in [(2, 2), (2, 3), (3, 2)]:
+        for a, b, c in rows:
+            xs, ws, ys = _parse_sig2(a), _parse_sig2(b), _parse_sig2(c)
+            assert O.matmul_infer_2d(xs, ws) == ys
+            xl, wl = O.to_locals_2d(X, xs, pshape), O.to_locals_2d(W, ws, pshape)
+            y_sigs, yl, Ylog = O.matmul_locals_2d(xl, xs, wl, ws, pshape)
+            assert y_sigs == ys and np.array_equal(Ylog, Y)
+            k0, k1 = pshape
+            for r in range(k0 * k1):
+                assert np.array_equal(yl[r], _py_matmul(xl[r], wl[r]))
+            # the SBP invariant: the locals reproduce the logical product
+            if ys[1] == PSUM:
+                nodes = [O.reduce_sum_fp64(yl[i * k1:(i + 1) * k1]) for i in range(k0)]
+                assert np.array_equal(O.from_locals(nodes, ys[0]), Y)
+            else:
+                assert np.array_equal(O.from_locals_2d(yl, ys, pshape), Y)
+    assert O.matmul_infer_2d((S0, S0), (B, B)) == (S0, S0)        # nested data parallelism is valid
+    assert O.matmul_infer_2d((S0, S1), (B, B)) is None             # (S(1), B) is not a row of Table 1
+
+
+def test_two_axis_mapping_brute_force_and_round_trip():
+    T = np.arange(7 * 10, dtype=np.float32).reshape(7, 10)
+    for pshape in [(2, 2), (2, 3), (4, 2)]:
+        k0, k1 = pshape
+        for sigs in [(S0, S1), (S1, S0), (S0, S0), (S0, B), (B, S1), (B, B)]:
+            loc = O.to_locals_2d(T, sigs, pshape)
+            assert len(loc) == k0 * k1
+            for i in range(k0):
+                # piece i under the first signature, by the one-axis mapping (pinned above)
+                node = O.to_locals(T, sigs[0], k0)[i]
+                for j in range(k1):
+                    assert np.array_equal(loc[i * k1 + j], O.to_locals(node, sigs[1], k1)[j])
+            assert np.array_equal(O.from_locals_2d(loc, sigs, pshape), T)
+        # (S(0), S(0)) is a nested split: concatenating all devices in order gives T back
+        loc = O.to_locals_2d(T, (S0, S0), pshape)
+        assert np.array_equal(np.concatenate(loc, axis=0), T)
+        # boxing one placement axis: (S(0), P) -> (S(0), B) sums inside each group only
+        parts = [dg.small_integers(82, r, O.to_locals(T, S0, k0)[r // k1].shape, -3, 4).numpy() for r in range(k0 * k1)]
+        out = O.boxing_2d(parts, (S0, PSUM), (S0, B), pshape)
+        for i in range(k0):
+            want = sum(parts[i * k1 + j] for j in range(k1))
+            for j in range(k1):
+                assert np.array_equal(out[i * k1 + j], want)

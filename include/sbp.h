@@ -258,7 +258,7 @@ sbp_status sbp_softmax_xent_static(const sbp_tensor* logits, const sbp_tensor* l
 /* ---------------------------------------------------------------- row-split embedding
  *
  * Section 6.3 (embedding table S(0), "splitting the vocabulary IDs"):
- *   table [rows, dim]   S(0), SBP_F32 or SBP_BF16
+ *   table [rows, dim]   S(0) (or S(1), see below), SBP_F32 or SBP_BF16
  *   ids   [...]         B, SBP_I64, 1 <= ndim <= 3
  *   out   [..., dim]    P(sum): shard r writes table row id where id falls in its own row
  *                       range and zeros elsewhere (the k outputs sum to the lookup);
@@ -266,6 +266,10 @@ sbp_status sbp_softmax_xent_static(const sbp_tensor* logits, const sbp_tensor* l
  *                       P(sum)->B boxing fused into the gather (exactly one shard
  *                       contributes to a row, so the sum is that row; a -0.0 entry is
  *                       written as +0.0 when k > 1, as x + 0 would give).
+ * The table may instead be S(1) (Section 6.3: "splitting the hidden dimension"): every shard
+ * then holds a column block of every row, and out is either split along its last axis the same
+ * way (each shard's lookup in its own block) or B (whole rows assembled and written to every
+ * replica: the all-gather fused into the gather).
  * An id outside [0, rows) produces a zero row and, when oob_count is not NULL, adds 1 to
  * the device int32 it points to (the caller zeroes it).
  */

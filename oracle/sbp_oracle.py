@@ -384,3 +384,11 @@ def embedding_partials(table_locals, ids):
         outs.append(o)
         off += t.shape[0]
     return outs
+
+
+def embedding_hidden_split(table_locals, ids):
+    """Table S(1) ("splitting the hidden dimension", Section 6.3): shard r holds a column block
+    of every row, looks up every id in it, and its result is that column block of the lookup:
+    the k outputs are the lookup split along its last axis."""
+    return [embedding_logical(t, ids) for t in table_locals]
+

@@ -136,6 +136,137 @@ static void launch_emb(const EmbParams& p, bool fused, cudaStream_t st) {
   }
 }
 
+// ---- table split along the hidden axis: S(1) ("splitting the hidden dimension", Section 6.3).
+// Shard r holds columns [start_r, start_r + len_r) of every row.  The lookup of one id touches
+// every shard; its natural result is split along the last axis the same way, and writing whole
+// rows to every B replica instead is the all-gather fused into the gather.
+struct EmbS1Params {
+  const char* table[SBP_MAX_K];
+  const long long* ids[SBP_MAX_K];
+  char* out[SBP_MAX_K];
+  long long vstart[SBP_MAX_K + 1];   // first vector of shard r's piece inside a full row
+  long long rows, n_lookups, vpr_total;
+  int k, n_dst;
+  int* oob;
+};
+
+template <typename V, int J, bool FUSED>
+__global__ void __launch_bounds__(256) embedding_s1_kernel(const __grid_constant__ EmbS1Params p) {
+  const long long total = p.n_lookups * p.vpr_total;
+  const long long stride = (long long)gridDim.x * 256;
+  const long long base = (long long)blockIdx.x * 256 + threadIdx.x;
+  long long item[J], look[J], col[J], id[J];
+  int shard[J];
+  bool ok[J];
+#pragma unroll
+  for (int j = 0; j < J; ++j) {
+    item[j] = base + j * stride;
+    ok[j] = item[j] < total;
+    look[j] = item[j] / p.vpr_total;
+    col[j] = item[j] - look[j] * p.vpr_total;
+    int r = 0;
+    while (r + 1 < p.k && col[j] >= p.vstart[r + 1]) ++r;
+    shard[j] = r;
+  }
+#pragma unroll
+  for (int j = 0; j < J; ++j) id[j] = ok[j] ? __ldg(p.ids[FUSED ? 0 : shard[j]] + look[j]) : 0;
+  V val[J];
+#pragma unroll
+  for (int j = 0; j < J; ++j) {
+    val[j] = zero_vec<V>();
+    if (!ok[j]) continue;
+    if (id[j] < 0 || id[j] >= p.rows) {
+      if (p.oob && col[j] == 0) atomicAdd(p.oob, 1);
+      continue;
+    }
+    const long long w = p.vstart[shard[j] + 1] - p.vstart[shard[j]];
+    val[j] = __ldg(reinterpret_cast<const V*>(p.table[shard[j]]) + id[j] * w + (col[j] - p.vstart[shard[j]]));
+  }
+  if (FUSED) {
+    for (int q = 0; q < p.n_dst; ++q) {
+      V* o = reinterpret_cast<V*>(p.out[q]);
+#pragma unroll
+      for (int j = 0; j < J; ++j)
+        if (ok[j]) o[item[j]] = val[j];
+    }
+  } else {
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      if (!ok[j]) continue;
+      const long long w = p.vstart[shard[j] + 1] - p.vstart[shard[j]];
+      reinterpret_cast<V*>(p.out[shard[j]])[look[j] * w + (col[j] - p.vstart[shard[j]])] = val[j];
+    }
+  }
+}
+
+template <typename V>
+static void launch_emb_s1(const EmbS1Params& p, bool fused, cudaStream_t st) {
+  constexpr int J = 4;
+  const long long total = p.n_lookups * p.vpr_total;
+  long long blocks = (total + 256LL * J - 1) / (256LL * J);
+  if (blocks < 1) blocks = 1;
+  if (fused) embedding_s1_kernel<V, J, true><<<(unsigned)blocks, 256, 0, st>>>(p);
+  else embedding_s1_kernel<V, J, false><<<(unsigned)blocks, 256, 0, st>>>(p);
+}
+
+static sbp_status embedding_hidden_split(const sbp_tensor* table, const sbp_tensor* ids, sbp_tensor* out,
+                                         int32_t* oob_count, cudaStream_t stream) {
+  const int k = placement_k(table);
+  const int esz = elem_size(table->dtype);
+  const int last = out->ndim - 1;
+  const bool fused = out->sbp[0].kind == SBP_BROADCAST;
+  if (!fused && !(out->sbp[0].kind == SBP_SPLIT && out->sbp[0].axis == last))
+    return fail(SBP_ERR_SIGNATURE, "with the table S(1), out must be split along its last axis, or B (gather fused in)");
+  const long long n_lookups = numel(ids);
+  if (n_lookups == 0 || table->shape[1] == 0) return SBP_OK;
+  int vb = 16;
+  for (; vb > esz; vb >>= 1) {
+    bool ok = true;
+    for (int r = 0; r < k && ok; ++r) {
+      int64_t st, ln;
+      split_range(table->shape[1], k, r, &st, &ln);
+      ok = (st * esz) % vb == 0 && (ln * esz) % vb == 0;
+      ok = ok && reinterpret_cast<uintptr_t>(table->local[r]) % vb == 0 && reinterpret_cast<uintptr_t>(out->local[r]) % vb == 0;
+    }
+    if (ok) break;
+  }
+  EmbS1Params p{};
+  p.k = k;
+  p.rows = table->shape[0];
+  p.n_lookups = n_lookups;
+  p.oob = oob_count;
+  p.vpr_total = table->shape[1] * esz / vb;
+  for (int r = 0; r < k; ++r) {
+    int64_t st, ln;
+    split_range(table->shape[1], k, r, &st, &ln);
+    p.vstart[r] = st * esz / vb;
+    p.table[r] = static_cast<const char*>(table->local[r]);
+    p.ids[r] = static_cast<const long long*>(ids->local[r]);
+    p.out[r] = static_cast<char*>(out->local[r]);
+  }
+  p.vstart[k] = p.vpr_total;
+  if (fused) {
+    char* uniq[SBP_MAX_K];
+    for (int r = 0; r < k; ++r) {
+      bool seen = false;
+      for (int q = 0; q < p.n_dst; ++q) seen = seen || uniq[q] == p.out[r];
+      if (!seen) uniq[p.n_dst++] = p.out[r];
+    }
+    for (int q = 0; q < p.n_dst; ++q) p.out[q] = uniq[q];
+  }
+  if ((n_lookups * p.vpr_total + 1023) / 1024 > 0x7fffffffLL) return fail(SBP_ERR_UNSUPPORTED, "too many lookups for one launch");
+  switch (vb) {
+    case 16: launch_emb_s1<uint4>(p, fused, stream); break;
+    case 8: launch_emb_s1<uint2>(p, fused, stream); break;
+    case 4: launch_emb_s1<uint32_t>(p, fused, stream); break;
+    default: launch_emb_s1<uint16_t>(p, fused, stream); break;
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "embedding launch");
+  count_launch();
+  return SBP_OK;
+}
+
 }  // namespace sbp
 
 using namespace sbp;
@@ -159,10 +290,10 @@ extern "C" sbp_status sbp_embedding(const sbp_tensor* table, const sbp_tensor* i
   if (out->shape[out->ndim - 1] != table->shape[1]) return fail(SBP_ERR_SHAPE, "out's last axis must equal dim");
   const int k = placement_k(table);
   if (placement_k(ids) != k || placement_k(out) != k) return fail(SBP_ERR_INVALID_ARG, "operands differ in k");
-  if (!(table->sbp[0].kind == SBP_SPLIT && table->sbp[0].axis == 0))
-    return fail(table->sbp[0].kind == SBP_SPLIT ? SBP_ERR_UNSUPPORTED : SBP_ERR_SIGNATURE,
-                "table must be S(0) (a table split along the hidden axis is not implemented)");
+  if (table->sbp[0].kind != SBP_SPLIT) return fail(SBP_ERR_SIGNATURE, "table must be S(0) or S(1)");
   if (ids->sbp[0].kind != SBP_BROADCAST) return fail(SBP_ERR_SIGNATURE, "ids must be B");
+  if (table->sbp[0].axis == 1)
+    return embedding_hidden_split(table, ids, out, oob_count, static_cast<cudaStream_t>(cuda_stream));
   const bool fused = out->sbp[0].kind == SBP_BROADCAST;
   if (!fused && out->sbp[0].kind != SBP_PARTIAL_SUM)
     return fail(SBP_ERR_SIGNATURE, "out must be P(sum) (unfused) or B (boxing fused into the gather)");

@@ -178,7 +178,7 @@ def test_softmax_and_embedding_validation(lib):
         binding._check(lib.sbp_embedding(C.byref(a), C.byref(b), C.byref(c), None, None))
 
     ids = _host_tensor((3, 2), i64, sbp.B, k)
-    assert _status(emb, _host_tensor((10, 4), f32, sbp.S(1), k), ids, _host_tensor((3, 2, 4), f32, sbp.B, k)) == "SBP_ERR_UNSUPPORTED"
+    assert _status(emb, _host_tensor((10, 4), f32, sbp.S(1), k), ids, _host_tensor((3, 2, 4), f32, sbp.P_SUM, k)) == "SBP_ERR_SIGNATURE"
     assert _status(emb, _host_tensor((10, 4), f32, sbp.B, k), ids, _host_tensor((3, 2, 4), f32, sbp.B, k)) == "SBP_ERR_SIGNATURE"
     assert _status(emb, _host_tensor((10, 4), f32, sbp.S(0), k), ids, _host_tensor((3, 2, 5), f32, sbp.B, k)) == "SBP_ERR_SHAPE"
     assert _status(emb, _host_tensor((10, 4), f32, sbp.S(0), k), ids, _host_tensor((3, 2, 4), f32, sbp.S(0), k)) == "SBP_ERR_SIGNATURE"

@@ -454,3 +454,31 @@ def test_fused_classifier_ragged_shapes_and_edges():
     with pytest.raises(sbp.SbpError) as e:
         sbp.sbp_matmul_softmax_xent(f, w, lab, loss, None, None, ws[:64])
     assert e.value.name in ("SBP_ERR_WORKSPACE", "SBP_ERR_UNSUPPORTED")
+
+
+@pytest.mark.parametrize("fused", [True, False])
+@pytest.mark.parametrize("k", [1, 2, 3, 8])
+@pytest.mark.parametrize("dtype,dim", [(F32, 128), (F32, 36), (BF16, 64), (BF16, 10)])
+def test_embedding_table_split_on_hidden_axis(fused, k, dtype, dim):
+    rows = 500
+    table = dg.uniform(1005, 3, (rows, dim), -0.05, 0.05, dtype)
+    ids = dg.zipf_ids(1005, 4, (41, 26), 512).clamp_(max=rows - 1)
+    ids[0, 0], ids[1, 1] = -3, rows                              # two ids out of range
+    tab = make_global(split_cpu(table, sbp.S(1), k), (rows, dim), dtype, sbp.S(1))
+    idt = make_global([ids] * k, tuple(ids.shape), I64, sbp.B)
+    out = sbp.empty_global(tuple(ids.shape) + (dim,), dtype, sbp.B if fused else sbp.S(2), k)
+    for t in out.locals:
+        t.view(torch.uint8).fill_(0x5A)
+    oob = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sbp.sbp_embedding(tab, idt, out, oob)
+    torch.cuda.synchronize()
+    assert int(oob.item()) == 2
+    parts = O.embedding_hidden_split(O.to_locals(to_np(table), O.S1, k), ids.numpy())
+    if fused:
+        want = O.from_locals(parts, O.S(2))
+        for t in out.locals:
+            assert np.array_equal(bits(t), np_bits(want, dtype))
+    else:
+        for r in range(k):
+            assert tuple(out.locals[r].shape) == tuple(parts[r].shape)
+            assert np.array_equal(bits(out.locals[r]), np_bits(parts[r], dtype)), f"shard {r}"

@@ -596,3 +596,18 @@ def test_two_axis_mapping_brute_force_and_round_trip():
             want = sum(parts[i * k1 + j] for j in range(k1))
             for j in range(k1):
                 assert np.array_equal(out[i * k1 + j], want)
+
+
+def test_embedding_hidden_split_is_the_lookup_split_on_its_last_axis():
+    rows, d, k = 19, 10, 4
+    table = dg.uniform(72, 0, (rows, d), -0.05, 0.05).numpy()
+    ids = dg.integers(72, 1, (5, 3), 0, rows).numpy()
+    ids[0, 0] = -1                                               # out of range -> zeros
+    parts = O.embedding_hidden_split(O.to_locals(table, S1, k), ids)
+    starts = O.balanced_split(d, k)
+    for b in range(5):
+        for f in range(3):
+            for r, (s, ln) in enumerate(starts):
+                want = table[ids[b, f], s:s + ln] if ids[b, f] >= 0 else np.zeros(ln, np.float32)
+                assert np.array_equal(parts[r][b, f], want)
+    assert np.array_equal(O.from_locals(parts, O.S(2)), O.embedding_logical(table, ids))

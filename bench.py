@@ -388,11 +388,40 @@ def section_classifier_gemm(sbp, device, peaks, opts):
     return [e, e2]
 
 
+def section_extras(sbp, device, peaks, opts):
+    """Rows beyond the core sweep: boxing to P(sum) (Table 2's zero-cost rows, materialised) and the
+    embedding with the table split on the hidden axis, at the sizes of configs 2 and 5."""
+    k, shape, bf16 = SWEEP_K, (8192, 8192), torch.bfloat16
+    tb = shape[0] * shape[1] * 2
+    T = dg.normal(SEED, 0, shape, 0.0, 1.0, bf16, device)
+    s0 = sbp.SbpTensor(shape, bf16, sbp.S(0), [T[r * shape[0] // k:(r + 1) * shape[0] // k].contiguous() for r in range(k)])
+    b = sbp.SbpTensor(shape, bf16, sbp.B, [T.clone() for _ in range(k)])
+    part = sbp.empty_global(shape, bf16, sbp.P_SUM, k, device=device)
+    res = []
+    avg, best = time_op(lambda: sbp.sbp_boxing(s0, part), device)
+    res.append(_hbm_entry("S(0)->P(sum) bf16 [8192,8192] k=4", (1 + k) * tb, avg, best, peaks))
+    avg, best = time_op(lambda: sbp.sbp_boxing(b, part), device)
+    res.append(_hbm_entry("B->P(sum) bf16 [8192,8192] k=4", (1 + k) * tb, avg, best, peaks))
+    del T, s0, b, part
+    torch.cuda.empty_cache()
+    k, rows, dim, batch = 8, opts.emb_rows, 128, opts.emb_batch
+    ids = dg.zipf_ids(1005, 1, (batch, 26), rows, 1.05, device)
+    table = sbp.SbpTensor((rows, dim), torch.float32, sbp.S(1),
+                          [dg.uniform(1005, 200 + r, (rows, dim // k), -0.05, 0.05, torch.float32, device) for r in range(k)])
+    idt = sbp.SbpTensor((batch, 26), torch.int64, sbp.B, [ids] * k)
+    out_b = sbp.empty_global((batch, 26, dim), torch.float32, sbp.B, k, device=device)
+    n, row_b = batch * 26, dim * 4
+    avg, best = time_op(lambda: sbp.sbp_embedding(table, idt, out_b), device)
+    res.append(_hbm_entry("embedding, table S(1): fused gather -> B (8 replicas written)", n * 8 + n * row_b + k * n * row_b,
+                          avg, best, peaks))
+    return res
+
+
 def run_operator_sections(sbp, device, peaks, opts):
     which = opts.ops
     out = []
     table = {"softmax": section_softmax, "classifier": section_classifier_gemm, "mlp": section_mlp,
-             "embedding": section_embedding}
+             "embedding": section_embedding, "extras": section_extras}
     for fn in [table[w.strip()] for w in which.split(",") if w.strip()]:
         try:
             out.extend(fn(sbp, device, peaks, opts))
@@ -453,8 +482,8 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-ops", action="store_true", help="skip the sharded-operator sections (N = 1 only)")
-    ap.add_argument("--ops", default="softmax,classifier,mlp,embedding",
-                    help="comma-separated operator sections to run: softmax, classifier, mlp, embedding")
+    ap.add_argument("--ops", default="softmax,classifier,mlp,embedding,extras",
+                    help="comma-separated operator sections to run: softmax, classifier, mlp, embedding, extras")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--copy-engine", type=int, default=0)
     ap.add_argument("--emb-rows", type=int, default=1 << 24, help="embedding table rows (smaller = profiling-sized case)")

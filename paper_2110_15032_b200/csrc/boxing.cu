@@ -143,22 +143,6 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
 
   TaskGeom g;
   task_geometry(p, s, d, (int)sizeof(V), &g);
-  // S(i)/B -> P(sum): the destination shard is walked in full rows of Nb * C elements; only
-  // the vectors [own_lo, own_hi) of a row come from the source, the rest is written as zero.
-  long long own_lo = 0, own_hi = 0, src_row_vecs = 0;
-  if (p.mode == MODE_SCATTER_P) {
-    const long long row_vecs = p.Nb * p.C * p.esz / (long long)sizeof(V);   // exact: checked on the host
-    if (p.src_b) {                       // split source: its own slice of the axis
-      own_lo = g.boff_d * p.C * p.esz / (long long)sizeof(V);
-      own_hi = own_lo + g.seg_vecs;
-      src_row_vecs = g.seg_vecs;
-    } else {                             // broadcast source: shard 0 keeps the tensor
-      own_hi = t == 0 ? row_vecs : 0;
-      src_row_vecs = row_vecs;
-    }
-    g.seg_vecs = row_vecs;
-    g.nseg = p.A * p.Na * p.M;
-  }
   const long long seg0 = row_tile * p.rows_per_tile;
   if (seg0 >= g.nseg) return;
   const long long col0 = col_tile << p.cv_log2;
@@ -189,25 +173,10 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
   V val[J];
   if constexpr (OP == OP_COPY) {
     const V* sp = reinterpret_cast<const V*>(p.src[s]);
-    if (p.mode == MODE_SCATTER_P) {
 #pragma unroll
-      for (int j = 0; j < J; ++j) {
-        const int f = threadIdx.x + j * 256;
-        const long long seg = seg0 + (f >> p.cv_log2);
-        const long long col = col0 + (f & ((1 << p.cv_log2) - 1));
-        dofs[j] = seg * g.seg_vecs + col;
-        V z;
-        unsigned char* zb = reinterpret_cast<unsigned char*>(&z);
-#pragma unroll
-        for (int b = 0; b < (int)sizeof(V); ++b) zb[b] = 0;
-        val[j] = z;
-        if (ok[j] && col >= own_lo && col < own_hi) val[j] = ld_stream(sp + seg * src_row_vecs + (col - own_lo));
-      }
-    } else {
-#pragma unroll
-      for (int j = 0; j < J; ++j)
-        if (ok[j]) val[j] = ld_stream(sp + so[j]);
-    }
+    for (int j = 0; j < J; ++j)
+      if (ok[j]) val[j] = ld_stream(sp + so[j]);
+
   } else {
     using L = typename Lanes<OP, V>::type;
     const int kk = KT ? KT : p.k;
@@ -260,6 +229,52 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
     for (int j = 0; j < J; ++j)
       if (ok[j]) dp[dofs[j]] = val[j];
   }
+}
+
+// ------------------------------------------------------------------ S(i)/B -> P(sum)
+//
+// Destination shard d has the full shape: the vectors [own_lo, own_hi) of every row come from
+// the source shard, everything else is written as zero.  Three quarters (for k = 4) of the work
+// is plain zero stores, so the kernel keeps its index arithmetic out of the inner loop: the
+// host precomputes the per-shard column ranges, a CTA walks 32 KiB chunks of rows.
+struct ScatterParams {
+  const char* src[SBP_MAX_K];
+  char* dst[SBP_MAX_K];
+  long long own_lo[SBP_MAX_K], own_hi[SBP_MAX_K];   // in vectors, inside a row
+  long long nrows, row_vecs, chunks_per_row, total_chunks;
+};
+
+constexpr int kScatterJ = 8;
+
+template <typename V>
+__global__ void __launch_bounds__(256) box_scatter_kernel(const __grid_constant__ ScatterParams p) {
+  const int d = blockIdx.y;
+  const V* sp = reinterpret_cast<const V*>(p.src[d]);
+  V* dp = reinterpret_cast<V*>(p.dst[d]);
+  const long long lo = p.own_lo[d], hi = p.own_hi[d], w = hi - lo;
+  for (long long c = blockIdx.x; c < p.total_chunks; c += gridDim.x) {
+    const long long row = c / p.chunks_per_row;
+    const long long col0 = (c - row * p.chunks_per_row) * (256 * kScatterJ) + threadIdx.x;
+    V val[kScatterJ];
+#pragma unroll
+    for (int j = 0; j < kScatterJ; ++j) {
+      const long long col = col0 + j * 256;
+      val[j] = V{};
+      if (col >= lo && col < hi) val[j] = ld_stream(sp + row * w + (col - lo));
+    }
+#pragma unroll
+    for (int j = 0; j < kScatterJ; ++j) {
+      const long long col = col0 + j * 256;
+      if (col < p.row_vecs) dp[row * p.row_vecs + col] = val[j];
+    }
+  }
+}
+
+template <typename V>
+static void launch_scatter_v(const ScatterParams& sp, int k, cudaStream_t st) {
+  long long gx = sp.total_chunks < 148 * 6 ? sp.total_chunks : 148 * 6;
+  if (gx < 1) gx = 1;
+  box_scatter_kernel<V><<<dim3((unsigned)gx, (unsigned)k), 256, 0, st>>>(sp);
 }
 
 // ------------------------------------------------------------------ host side
@@ -549,11 +564,39 @@ sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream)
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
   bool done = false;
+  if (pl.p.mode == MODE_SCATTER_P) {
+    const BoxParams& b = pl.p;
+    ScatterParams sp{};
+    sp.nrows = b.A * b.Na * b.M;
+    sp.row_vecs = b.Nb * b.C * b.esz / pl.vbytes;
+    sp.chunks_per_row = (sp.row_vecs + 256 * kScatterJ - 1) / (256 * kScatterJ);
+    sp.total_chunks = sp.nrows * sp.chunks_per_row;
+    for (int d = 0; d < b.k; ++d) {
+      sp.src[d] = b.src[d];
+      sp.dst[d] = b.dst[d];
+      if (b.src_b) {
+        int64_t start, len;
+        split_range(b.Nb, b.k, d, &start, &len);
+        sp.own_lo[d] = start * b.C * b.esz / pl.vbytes;
+        sp.own_hi[d] = (start + len) * b.C * b.esz / pl.vbytes;
+      } else {
+        sp.own_lo[d] = 0;
+        sp.own_hi[d] = d == 0 ? sp.row_vecs : 0;
+      }
+    }
+    switch (pl.vbytes) {
+      case 16: launch_scatter_v<uint4>(sp, b.k, stream); break;
+      case 8: launch_scatter_v<uint2>(sp, b.k, stream); break;
+      case 4: launch_scatter_v<uint32_t>(sp, b.k, stream); break;
+      default: launch_scatter_v<uint16_t>(sp, b.k, stream); break;
+    }
+    done = true;
+  }
   // Default choice, from measurement on B200: the bulk engine wins where one read feeds one
   // write (re-layouts and slices); the load/store kernel wins where one read feeds k writes.
   const int engine = g_copy_engine.load();
-  const bool want_bulk = (engine == 2 || (engine == 0 && pl.p.mode != MODE_GATHER)) && pl.p.mode != MODE_SCATTER_P;
-  if (pl.op == OP_COPY && want_bulk && pl.vbytes == 16)
+  const bool want_bulk = engine == 2 || (engine == 0 && pl.p.mode != MODE_GATHER);
+  if (!done && pl.op == OP_COPY && want_bulk && pl.vbytes == 16)
     done = launch_bulk_copy(pl.p, pl.ntasks, stream);
   if (!done) {
     switch (pl.op) {

@@ -19,6 +19,8 @@ struct EmbParams {
   const long long* ids[SBP_MAX_K];
   char* out[SBP_MAX_K];
   long long rows;         // logical table rows
+  long long base, rem, big;   // balanced split of the rows, see owner_of_row
+  int narrow;
   long long n_lookups;
   long long vpr;          // vectors per row
   int vpr_log2;           // >= 0 when vpr is a power of two, else -1
@@ -28,9 +30,23 @@ struct EmbParams {
   int* oob;
 };
 
-__host__ __device__ inline int owner_of_row(long long id, long long rows, int k, long long* start) {
-  const long long base = rows / k, rem = rows % k;
-  const long long big = rem * (base + 1);
+// Shard that owns table row `id` under the balanced split, and the first row of that shard.
+// base = rows / k, rem = rows % k, big = rem * (base + 1) come precomputed from the host; tables
+// below 2^31 rows (narrow = 1) take 32-bit divisions, which cost a fraction of 64-bit ones.
+__device__ __forceinline__ int owner_of_row(long long id, long long base, long long rem, long long big, int narrow,
+                                            long long* start) {
+  if (narrow) {
+    const unsigned uid = (unsigned)id, ubase = (unsigned)base, ubig = (unsigned)big;
+    unsigned r;
+    if (uid < ubig) {
+      r = uid / (ubase + 1);
+      *start = (long long)r * (ubase + 1);
+    } else {
+      r = (unsigned)rem + (uid - ubig) / ubase;
+      *start = (long long)ubig + (long long)(r - (unsigned)rem) * ubase;
+    }
+    return (int)r;
+  }
   int r;
   if (id < big) {
     r = (int)(id / (base + 1));
@@ -103,7 +119,7 @@ __global__ void __launch_bounds__(256) embedding_kernel(const __grid_constant__ 
       continue;
     }
     long long start;
-    const int r = owner_of_row(id[j], p.rows, p.k, &start);
+    const int r = owner_of_row(id[j], p.base, p.rem, p.big, p.narrow, &start);
     if (FUSED || r == shard)
       val[j] = __ldg(reinterpret_cast<const V*>(p.table[r]) + (id[j] - start) * p.vpr + col[j]);
   }
@@ -304,6 +320,10 @@ extern "C" sbp_status sbp_embedding(const sbp_tensor* table, const sbp_tensor* i
   p.k = k;
   p.esz = elem_size(table->dtype);
   p.rows = table->shape[0];
+  p.base = p.rows / k;
+  p.rem = p.rows % k;
+  p.big = p.rem * (p.base + 1);
+  p.narrow = p.rows < (1LL << 31) ? 1 : 0;
   p.n_lookups = n_lookups;
   p.oob = oob_count;
   const long long row_bytes = table->shape[1] * p.esz;

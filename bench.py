@@ -409,6 +409,14 @@ def section_extras(sbp, device, peaks, opts):
     res.append(_hbm_entry("B->P(sum) bf16 [8192,8192] k=4", (1 + k) * tb, avg, best, peaks))
     del T, s0, b, part
     torch.cuda.empty_cache()
+    # Section 6.4's cast op: fp32 shards S(0) -> bf16 replicas B, the cast folded into the gather
+    Tf = dg.normal(SEED, 1, shape, 0.0, 1.0, torch.float32, device)
+    sf = sbp.SbpTensor(shape, torch.float32, sbp.S(0), [Tf[r * shape[0] // k:(r + 1) * shape[0] // k].contiguous() for r in range(k)])
+    rb = sbp.empty_global(shape, bf16, sbp.B, k, device=device)
+    avg, best = time_op(lambda: sbp.sbp_boxing(sf, rb), device)
+    res.append(_hbm_entry("S(0) fp32 -> B bf16 (cast fused into the gather) [8192,8192] k=4", 2 * tb + k * tb, avg, best, peaks))
+    del Tf, sf, rb
+    torch.cuda.empty_cache()
     k, rows, dim, batch = 8, opts.emb_rows, 128, opts.emb_batch
     ids = dg.zipf_ids(1005, 1, (batch, 26), rows, 1.05, device)
     table = sbp.SbpTensor((rows, dim), torch.float32, sbp.S(1),

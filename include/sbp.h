@@ -116,7 +116,7 @@ sbp_status sbp_matmul_infer(sbp_sig x, sbp_sig w, sbp_sig* y);
  *
  * A boxing op re-arranges or transforms the local tensors of a global tensor so that
  * the same global tensor is seen under another signature (Section 3.2; Table 2, column
- * "same" placement).  src and dst must agree in logical shape, dtype and k.
+ * "same" placement).  src and dst must agree in logical shape, dtype (one exception below) and k.
  *
  *   src            dst        the collective it stands for (Table 2)
  *   P(sum)         B          all-reduce       out_j[e] = round(sum_r in_r[e])
@@ -129,6 +129,10 @@ sbp_status sbp_matmul_infer(sbp_sig x, sbp_sig w, sbp_sig* y);
  *   P(op)          P(op)      copy
  *   S(i)           P(sum)     local (Table 2: cost 0): shard r = zeros with its own slice in place
  *   B              P(sum)     local (Table 2: cost 0): shard 0 = the tensor, every other shard zeros
+ *   S(i) F32       B BF16     the cast op of Section 6.4 (sharded fp32 state -> half-precision
+ *                             replicas) folded into the all-gather: read once as fp32, rounded to
+ *                             bf16 (nearest even), written to every replica.  The only dtype change
+ *                             sbp_boxing accepts.
  * Anything else (a P(max) destination from S or B, P(sum)<->P(max)) returns SBP_ERR_UNSUPPORTED.
  *
  * Two-axis placements: one call may change the signature of ONE placement axis (the other stays

@@ -179,6 +179,12 @@ def boxing(src_locals, src_sig, dst_sig, storage="f32"):
     return to_locals(T, dst_sig, k)
 
 
+def boxing_cast(src_locals, src_sig, dst_sig, dst_storage):
+    """Boxing followed by a cast of every destination local tensor to dst_storage (Section 6.4:
+    a cast op with S(0) input and B output turns sharded fp32 state into half-precision replicas)."""
+    return [round_to_storage(x, dst_storage) for x in boxing(src_locals, src_sig, dst_sig, "f32")]
+
+
 def table2_same_placement_cost(src_sig, dst_sig, k, t_bytes):
     """Table 2, column "same": bytes that cross between devices for src -> dst when both
     live on the same k devices.  Used to tell which transforms move data at all."""

@@ -277,6 +277,68 @@ static void launch_scatter_v(const ScatterParams& sp, int k, cudaStream_t st) {
   box_scatter_kernel<V><<<dim3((unsigned)gx, (unsigned)k), 256, 0, st>>>(sp);
 }
 
+// ------------------------------------------------------------------ S(i) -> B with an fp32 -> bf16 cast
+//
+// Section 6.4 ("Parallelizing the Optimizer"): sharded fp32 model states are cast to half
+// precision and all-gathered -- a cast op whose input is S(0) and whose output is B.  Here the
+// cast is folded into the gather: every source shard is read once as fp32, rounded to bf16
+// (nearest even) and written to its place in every replica.  EPV = bf16 elements per store.
+struct GatherCastParams {
+  const float* src[SBP_MAX_K];
+  __nv_bfloat16* dst[SBP_MAX_K];
+  long long own_lo[SBP_MAX_K], own_hi[SBP_MAX_K];   // in units of EPV elements, inside a full row
+  long long nrows, row_units;
+  int n_dst;
+};
+
+template <int EPV>
+__global__ void __launch_bounds__(256) box_gather_cast_kernel(const __grid_constant__ GatherCastParams p) {
+  constexpr int J = 4;
+  const int s = blockIdx.y;
+  const long long lo = p.own_lo[s], w = p.own_hi[s] - lo;
+  if (w <= 0) return;
+  const long long chunks_per_row = (w + 256 * J - 1) / (256 * J);
+  const long long total = p.nrows * chunks_per_row;
+  for (long long c = blockIdx.x; c < total; c += gridDim.x) {
+    const long long row = c / chunks_per_row;
+    const long long col0 = (c - row * chunks_per_row) * (256 * J) + threadIdx.x;
+    const float* sp = p.src[s] + (row * w) * EPV;
+    float v[J][EPV];
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      const long long col = col0 + j * 256;
+      if (col < w) {
+        if (EPV == 8) {
+          const float4 a = __ldg(reinterpret_cast<const float4*>(sp + col * 8));
+          const float4 b = __ldg(reinterpret_cast<const float4*>(sp + col * 8) + 1);
+          v[j][0] = a.x; v[j][1] = a.y; v[j][2] = a.z; v[j][3] = a.w;
+          v[j][4 % EPV] = b.x; v[j][5 % EPV] = b.y; v[j][6 % EPV] = b.z; v[j][7 % EPV] = b.w;
+        } else {
+          v[j][0] = __ldg(sp + col);
+        }
+      }
+    }
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      const long long col = col0 + j * 256;
+      if (col >= w) continue;
+      const long long at = row * p.row_units + lo + col;
+      if (EPV == 8) {
+        uint4 o;
+        __nv_bfloat162 h;
+        h = __floats2bfloat162_rn(v[j][0], v[j][1]); o.x = *reinterpret_cast<unsigned*>(&h);
+        h = __floats2bfloat162_rn(v[j][2], v[j][3]); o.y = *reinterpret_cast<unsigned*>(&h);
+        h = __floats2bfloat162_rn(v[j][4 % EPV], v[j][5 % EPV]); o.z = *reinterpret_cast<unsigned*>(&h);
+        h = __floats2bfloat162_rn(v[j][6 % EPV], v[j][7 % EPV]); o.w = *reinterpret_cast<unsigned*>(&h);
+        for (int q = 0; q < p.n_dst; ++q) reinterpret_cast<uint4*>(p.dst[q])[at] = o;
+      } else {
+        const __nv_bfloat16 o = __float2bfloat16_rn(v[j][0]);
+        for (int q = 0; q < p.n_dst; ++q) p.dst[q][at] = o;
+      }
+    }
+  }
+}
+
 // ------------------------------------------------------------------ host side
 
 static std::atomic<int> g_copy_engine{0};
@@ -465,7 +527,10 @@ static sbp_status check_pair(const sbp_tensor* src, const sbp_tensor* dst, bool 
   if (src->ndim != dst->ndim) return fail(SBP_ERR_SHAPE, "src and dst differ in rank");
   for (int d = 0; d < src->ndim; ++d)
     if (src->shape[d] != dst->shape[d]) return fail(SBP_ERR_SHAPE, "src and dst differ on axis %d", d);
-  if (src->dtype != dst->dtype) return fail(SBP_ERR_DTYPE, "src and dst differ in dtype");
+  const bool cast_gather = src->dtype == SBP_F32 && dst->dtype == SBP_BF16 && src->sbp[0].kind == SBP_SPLIT &&
+                           dst->sbp[0].kind == SBP_BROADCAST;
+  if (src->dtype != dst->dtype && !cast_gather)
+    return fail(SBP_ERR_DTYPE, "src and dst differ in dtype (only S(i) -> B may cast, F32 -> BF16)");
   if (placement_k(src) != placement_k(dst)) return fail(SBP_ERR_INVALID_ARG, "src and dst differ in k");
   return SBP_OK;
 }
@@ -564,7 +629,33 @@ sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream)
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
   bool done = false;
-  if (pl.p.mode == MODE_SCATTER_P) {
+  if (src->dtype != dst->dtype) {   // S(i) -> B with the fp32 -> bf16 cast folded in
+    const BoxParams& b = pl.p;      // planned with the source element size; only the view is used
+    GatherCastParams gp{};
+    gp.nrows = b.A * b.Na * b.M;
+    bool vec = (b.Nb * b.C) % 8 == 0;
+    for (int r = 0; r < b.k && vec; ++r) {
+      int64_t start, len;
+      split_range(b.Nb, b.k, r, &start, &len);
+      vec = (start * b.C) % 8 == 0 && (len * b.C) % 8 == 0 && reinterpret_cast<uintptr_t>(src->local[r]) % 16 == 0 &&
+            reinterpret_cast<uintptr_t>(dst->local[r]) % 16 == 0;
+    }
+    const int epv = vec ? 8 : 1;
+    gp.row_units = b.Nb * b.C / epv;
+    for (int r = 0; r < b.k; ++r) {
+      int64_t start, len;
+      split_range(b.Nb, b.k, r, &start, &len);
+      gp.src[r] = static_cast<const float*>(src->local[r]);
+      gp.own_lo[r] = start * b.C / epv;
+      gp.own_hi[r] = (start + len) * b.C / epv;
+    }
+    gp.n_dst = b.n_dst;
+    for (int q = 0; q < b.n_dst; ++q) gp.dst[q] = reinterpret_cast<__nv_bfloat16*>(b.dst[q]);
+    dim3 grid(148 * 4, (unsigned)b.k);
+    if (vec) box_gather_cast_kernel<8><<<grid, 256, 0, stream>>>(gp);
+    else box_gather_cast_kernel<1><<<grid, 256, 0, stream>>>(gp);
+    done = true;
+  } else if (pl.p.mode == MODE_SCATTER_P) {
     const BoxParams& b = pl.p;
     ScatterParams sp{};
     sp.nrows = b.A * b.Na * b.M;
@@ -639,7 +730,7 @@ sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, voi
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   sbp_tensor s = *src_host, d = *dst_host;
   char* cur = static_cast<char*>(dev_ws);
-  const int esz = elem_size(src_host->dtype);
+  const int esz = elem_size(src_host->dtype), esz_dst = elem_size(dst_host->dtype);
   for (int r = 0; r < k; ++r) {
     s.local[r] = cur;
     cur += align256((size_t)local_numel(src_host, r) * esz);
@@ -651,7 +742,7 @@ sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, voi
       if (dst_host->local[q] == dst_host->local[r]) d.local[r] = d.local[q];
     if (!d.local[r]) {
       d.local[r] = cur;
-      cur += align256((size_t)local_numel(dst_host, r) * esz);
+      cur += align256((size_t)local_numel(dst_host, r) * esz_dst);
     }
   }
   for (int r = 0; r < k; ++r) {
@@ -663,7 +754,7 @@ sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, voi
   for (int r = 0; r < k; ++r) {
     bool dup = false;
     for (int q = 0; q < r; ++q) dup = dup || dst_host->local[q] == dst_host->local[r];
-    const size_t bytes = (size_t)local_numel(dst_host, r) * esz;
+    const size_t bytes = (size_t)local_numel(dst_host, r) * esz_dst;
     if (!dup && bytes)
       SBP_CUDA_TRY(cudaMemcpyAsync(dst_host->local[r], d.local[r], bytes, cudaMemcpyDeviceToHost, stream));
   }

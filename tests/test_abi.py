@@ -115,7 +115,8 @@ def test_boxing_validation_happens_before_any_launch(lib):
     f32, bf16, i64 = torch.float32, torch.bfloat16, torch.int64
     src = _host_tensor((8, 8), f32, sbp.S(0), 2)
     assert _status(boxing, src, _host_tensor((8, 9), f32, sbp.B, 2)) == "SBP_ERR_SHAPE"
-    assert _status(boxing, src, _host_tensor((8, 8), bf16, sbp.B, 2)) == "SBP_ERR_DTYPE"
+    assert _status(boxing, src, _host_tensor((8, 8), bf16, sbp.S(1), 2)) == "SBP_ERR_DTYPE"   # only S -> B may cast
+    assert _status(boxing, _host_tensor((8, 8), bf16, sbp.S(0), 2), _host_tensor((8, 8), f32, sbp.B, 2)) == "SBP_ERR_DTYPE"
     assert _status(boxing, src, _host_tensor((8, 8), f32, sbp.B, 4)) == "SBP_ERR_INVALID_ARG"
     assert _status(boxing, src, _host_tensor((8, 8), f32, sbp.P_MAX, 2)) == "SBP_ERR_UNSUPPORTED"
     assert _status(boxing, _host_tensor((8, 8), f32, sbp.P_SUM, 2),

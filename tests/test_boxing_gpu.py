@@ -239,3 +239,23 @@ def test_expired_device_wait_is_reported_and_the_device_stays_usable():
     _run((64, 96), F32, sbp.S(0), sbp.S(1), 2)        # the context is intact
     with pytest.raises(sbp.SbpError):
         sbp.sbp_selftest_wait_timeout(5000)
+
+
+@pytest.mark.parametrize("shape,axis", [((64, 96), 0), ((67, 101), 1), ((130, 520), 0), ((6, 10, 16), 1), ((2048, 1024), 1)])
+@pytest.mark.parametrize("k", [1, 3, 4])
+def test_cast_fused_gather_fp32_to_bf16(shape, axis, k):
+    """S(i) fp32 -> B bf16: the cast of Section 6.4 folded into the all-gather."""
+    T = dg.normal(31, 0, shape, 0.0, 2.0, F32)
+    src = make_global(split_cpu(T, sbp.S(axis), k), shape, F32, sbp.S(axis))
+    for alias in (False, True):
+        dst = sbp.empty_global(shape, BF16, sbp.B, k, alias_replicas=alias)
+        for t in dst.locals:
+            t.view(torch.uint8).fill_(0xAB)
+        sbp.sbp_boxing(src, dst)
+        torch.cuda.synchronize()
+        want = O.boxing_cast(O.to_locals(T.numpy(), O.S(axis), k), O.S(axis), O.B, "bf16")
+        for r in range(k):
+            assert np.array_equal(bits(dst.locals[r]), np_bits(want[r], BF16)), f"replica {r}"
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_boxing(src, sbp.empty_global(shape, BF16, sbp.S(axis), k))       # only S -> B may cast
+    assert e.value.name == "SBP_ERR_DTYPE"

@@ -611,3 +611,13 @@ def test_embedding_hidden_split_is_the_lookup_split_on_its_last_axis():
                 want = table[ids[b, f], s:s + ln] if ids[b, f] >= 0 else np.zeros(ln, np.float32)
                 assert np.array_equal(parts[r][b, f], want)
     assert np.array_equal(O.from_locals(parts, O.S(2)), O.embedding_logical(table, ids))
+
+
+def test_boxing_cast_rounds_once_after_the_gather():
+    k = 3
+    T = dg.normal(24, 0, (7, 12), 0, 3.0).numpy()
+    T[0, 0], T[0, 1] = np.float32(1.0 + 2.0 ** -8), np.float32(1.0 + 2.0 ** -8 + 2.0 ** -16)   # tie / just above
+    out = O.boxing_cast(O.to_locals(T, S0, k), S0, B, "bf16")
+    want = torch.from_numpy(T).to(torch.bfloat16).to(torch.float32).numpy()     # independent library RNE
+    assert len(out) == k and all(np.array_equal(o, want) for o in out)
+    assert out[0][0, 0] == np.float32(1.0) and out[0][0, 1] == np.float32(1.0 + 2.0 ** -7)

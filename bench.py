@@ -333,8 +333,15 @@ def section_softmax(sbp, device, peaks, opts):
     loss = sbp.empty_global((rows,), torch.float32, sbp.B, k, device=device)
     ws = torch.empty(sbp.sbp_softmax_xent_workspace_bytes(logits), dtype=torch.uint8, device=device)
     avg, best = time_op(lambda: sbp.sbp_softmax_xent(logits, lab, loss, None, None, ws), device)
-    return [_hbm_entry("softmax-xent on bf16 logits (partial + combine)", rows * classes * 2 + rows * 8, avg, best, peaks,
-                       {"loss_mean": float(loss.locals[0].mean().item())})]
+    res = [_hbm_entry("softmax-xent on bf16 logits (partial + combine)", rows * classes * 2 + rows * 8, avg, best, peaks,
+                      {"loss_mean": float(loss.locals[0].mean().item())})]
+    rmax = sbp.empty_global((rows,), torch.float32, sbp.B, k, device=device)
+    rsum = sbp.empty_global((rows,), torch.float32, sbp.B, k, device=device)
+    sbp.sbp_softmax_xent(logits, lab, loss, rmax, rsum, ws)
+    grad = sbp.empty_global((rows, classes), torch.bfloat16, sbp.S(1), k, device=device)
+    avg, best = time_op(lambda: sbp.sbp_softmax_xent_backward(logits, lab, rmax, rsum, grad), device)
+    res.append(_hbm_entry("softmax-xent backward (softmax - onehot, S(1))", 2 * rows * classes * 2, avg, best, peaks))
+    return res
 
 
 def section_mlp(sbp, device, peaks, opts):

@@ -219,6 +219,15 @@ sbp_status sbp_softmax_xent(const sbp_tensor* logits, const sbp_tensor* labels, 
                             sbp_tensor* row_max, sbp_tensor* row_sum, void* ws, size_t ws_bytes,
                             void* cuda_stream);
 
+/* Backward of that loss with respect to the logits, for per-row losses with unit upstream
+ * gradient: grad[i, j] = exp(z_ij - m_i) / S_i - [j == label_i], i.e. softmax minus one-hot.
+ * It is element-wise once the forward pass's row_max (m) and row_sum (S) are known, so the
+ * gradient keeps the logits' signature S(1) and needs no reduction (Section 6.3's plan read
+ * backwards).  grad_logits has the logits' shape, dtype and signature. */
+sbp_status sbp_softmax_xent_backward(const sbp_tensor* logits, const sbp_tensor* labels,
+                                     const sbp_tensor* row_max, const sbp_tensor* row_sum,
+                                     sbp_tensor* grad_logits, void* cuda_stream);
+
 /* The classifier of Section 6.3 in one call: logits = features x weight with the weight S(1)
  * (hence logits S(1)), then the split softmax cross entropy above -- without ever storing the
  * logits.  Each 128-class chunk of a shard's product leaves, per row, its local max, local

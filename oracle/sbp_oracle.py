@@ -337,6 +337,16 @@ def softmax_xent_logical(Z, labels):
     return m, Ssum, np.log(Ssum) + m - zy
 
 
+def softmax_xent_grad(Z, labels):
+    """d loss_i / d Z_ij = softmax(Z_i)_j - [j == y_i]  (per-row loss, unit upstream gradient)."""
+    Z = np.asarray(Z, dtype=np.float64)
+    labels = np.asarray(labels, dtype=np.int64)
+    m, Ssum, _ = softmax_xent_logical(Z, labels)
+    G = np.exp(Z - m[:, None]) / Ssum[:, None]
+    G[np.arange(Z.shape[0]), labels] -= 1.0
+    return G
+
+
 def softmax_xent_split(z_locals, labels):
     """The same quantity in the split form the paper describes: per shard r a local
     max m_r and, after the global max m = max_r m_r (P(max) -> B), a local

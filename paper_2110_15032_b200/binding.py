@@ -105,6 +105,7 @@ def load_library():
     lib.sbp_matmul_softmax_xent_workspace_bytes.restype = C.c_size_t
     lib.sbp_matmul_softmax_xent_workspace_bytes.argtypes = [T, T]
     lib.sbp_matmul_softmax_xent.argtypes = [T, T, T, T, T, T, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sbp_softmax_xent_backward.argtypes = [T, T, T, T, T, C.c_void_p]
     lib.sbp_softmax_xent_static.argtypes = [T, T, T, T, T, C.c_void_p]
     lib.sbp_embedding.argtypes = [T, T, T, C.c_void_p, C.c_void_p]
     _LIB = lib
@@ -286,6 +287,13 @@ def sbp_matmul_softmax_xent(features: SbpTensor, weight: SbpTensor, labels: SbpT
         C.byref(a), C.byref(b), C.byref(l), C.byref(c),
         C.byref(m) if m is not None else None, C.byref(s) if s is not None else None,
         C.c_void_p(ws.data_ptr()), ws.numel() * ws.element_size(), _stream_ptr(stream)))
+
+
+def sbp_softmax_xent_backward(logits: SbpTensor, labels: SbpTensor, row_max: SbpTensor, row_sum: SbpTensor,
+                              grad_logits: SbpTensor, stream=None) -> None:
+    a, b, m, s, g = logits._c(), labels._c(), row_max._c(), row_sum._c(), grad_logits._c()
+    _check(load_library().sbp_softmax_xent_backward(C.byref(a), C.byref(b), C.byref(m), C.byref(s), C.byref(g),
+                                                    _stream_ptr(stream)))
 
 
 def sbp_softmax_xent_static(logits: SbpTensor, labels: SbpTensor, loss: SbpTensor,

@@ -390,6 +390,44 @@ sbp_status launch_xent_finish(float* part_m, float* part_s, float* part_t, int p
   return SBP_OK;
 }
 
+// ---- backward of the per-row loss with respect to the logits: softmax - onehot, kept S(1).
+// Element-wise given the row max and row sum of the forward pass: one read and one write of
+// the logits' size.
+struct XentBwdParams {
+  const char* logits[SBP_MAX_K];
+  char* grad[SBP_MAX_K];
+  const long long* labels;
+  const float* row_max;
+  const float* row_sum;
+  long long rows, classes;
+  int k;
+};
+
+template <typename T, int VEC>
+__global__ void __launch_bounds__(kThreads) xent_backward_kernel(const __grid_constant__ XentBwdParams p) {
+  const long long row = blockIdx.x;
+  const int shard = blockIdx.z;
+  long long c_start, c_len;
+  split_range(p.classes, p.k, shard, (int64_t*)&c_start, (int64_t*)&c_len);
+  const T* z = reinterpret_cast<const T*>(p.logits[shard]) + row * c_len;
+  T* g = reinterpret_cast<T*>(p.grad[shard]) + row * c_len;
+  const float neg = -p.row_max[row] * kLog2e;
+  const float inv = 1.0f / p.row_sum[row];
+  const long long y = p.labels[row] - c_start;      // label's column inside this shard, if any
+  struct alignas(sizeof(T) * VEC) Pack { T e[VEC]; };
+  for (long long e0 = ((long long)blockIdx.y * kThreads + threadIdx.x) * VEC; e0 < c_len;
+       e0 += (long long)gridDim.y * kThreads * VEC) {
+    Pack in = *reinterpret_cast<const Pack*>(z + e0), out;
+#pragma unroll
+    for (int i = 0; i < VEC; ++i) {
+      float v = ex2(fmaf(static_cast<float>(in.e[i]), kLog2e, neg)) * inv;
+      if (e0 + i == y) v -= 1.0f;
+      out.e[i] = static_cast<T>(v);
+    }
+    *reinterpret_cast<Pack*>(g + e0) = out;
+  }
+}
+
 }  // namespace sbp
 
 using namespace sbp;
@@ -527,3 +565,62 @@ extern "C" sbp_status sbp_softmax_xent_static(const sbp_tensor* logits, const sb
   return sbp_softmax_xent(logits, labels, loss, row_max, row_sum, scratch, kStaticScratchBytes, cuda_stream);
 }
 
+extern "C" sbp_status sbp_softmax_xent_backward(const sbp_tensor* logits, const sbp_tensor* labels,
+                                                const sbp_tensor* row_max, const sbp_tensor* row_sum,
+                                                sbp_tensor* grad_logits, void* cuda_stream) {
+  sbp_status st = check_tensor(logits, "logits", true);
+  if (st != SBP_OK) return st;
+  st = check_tensor(grad_logits, "grad_logits", true);
+  if (st != SBP_OK) return st;
+  if (logits->ndim != 2 || grad_logits->ndim != 2 || logits->shape[0] != grad_logits->shape[0] ||
+      logits->shape[1] != grad_logits->shape[1])
+    return fail(SBP_ERR_SHAPE, "logits and grad_logits must be [rows, classes] alike");
+  if (logits->dtype != SBP_BF16 && logits->dtype != SBP_F32) return fail(SBP_ERR_DTYPE, "logits must be BF16 or F32");
+  if (grad_logits->dtype != logits->dtype) return fail(SBP_ERR_DTYPE, "grad_logits and logits differ in dtype");
+  const int k = placement_k(logits);
+  if (placement_k(grad_logits) != k) return fail(SBP_ERR_INVALID_ARG, "operands differ in k");
+  auto is_s1 = [](const sbp_tensor* t) { return t->sbp[0].kind == SBP_SPLIT && t->sbp[0].axis == 1; };
+  if (!is_s1(logits) || !is_s1(grad_logits)) return fail(SBP_ERR_SIGNATURE, "logits and grad_logits must be S(1)");
+  const long long rows = logits->shape[0], classes = logits->shape[1];
+  if (!row_max || !row_sum) return fail(SBP_ERR_INVALID_ARG, "row_max and row_sum of the forward pass are required");
+  st = check_xent_outputs(labels, row_max, row_max, row_sum, rows, k);
+  if (st != SBP_OK) return st;
+  if (rows == 0 || classes == 0) return SBP_OK;
+  if (rows > 0x7fffffffLL) return fail(SBP_ERR_UNSUPPORTED, "too many rows for one launch");
+
+  XentBwdParams p{};
+  bool vec_ok = true;
+  const int esz = elem_size(logits->dtype);
+  for (int r = 0; r < k; ++r) {
+    int64_t s0, ln;
+    split_range(classes, k, r, &s0, &ln);
+    vec_ok = vec_ok && (ln * esz) % 16 == 0 && reinterpret_cast<uintptr_t>(logits->local[r]) % 16 == 0 &&
+             reinterpret_cast<uintptr_t>(grad_logits->local[r]) % 16 == 0;
+    p.logits[r] = static_cast<const char*>(logits->local[r]);
+    p.grad[r] = static_cast<char*>(grad_logits->local[r]);
+  }
+  p.labels = static_cast<const long long*>(labels->local[0]);
+  p.row_max = static_cast<const float*>(row_max->local[0]);
+  p.row_sum = static_cast<const float*>(row_sum->local[0]);
+  p.rows = rows;
+  p.classes = classes;
+  p.k = k;
+  const int vec = vec_ok ? 16 / esz : 1;
+  const long long c_max = (classes + k - 1) / k;
+  long long gy = (c_max + (long long)kThreads * vec * 4 - 1) / ((long long)kThreads * vec * 4);   // ~4 vectors per thread
+  if (gy < 1) gy = 1;
+  if (gy > 65535) gy = 65535;
+  dim3 grid((unsigned)rows, (unsigned)gy, (unsigned)k);
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (logits->dtype == SBP_BF16) {
+    if (vec > 1) xent_backward_kernel<__nv_bfloat16, 8><<<grid, kThreads, 0, stream>>>(p);
+    else xent_backward_kernel<__nv_bfloat16, 1><<<grid, kThreads, 0, stream>>>(p);
+  } else {
+    if (vec > 1) xent_backward_kernel<float, 4><<<grid, kThreads, 0, stream>>>(p);
+    else xent_backward_kernel<float, 1><<<grid, kThreads, 0, stream>>>(p);
+  }
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "softmax backward launch");
+  count_launch();
+  return SBP_OK;
+}

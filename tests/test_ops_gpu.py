@@ -482,3 +482,29 @@ def test_embedding_table_split_on_hidden_axis(fused, k, dtype, dim):
         for r in range(k):
             assert tuple(out.locals[r].shape) == tuple(parts[r].shape)
             assert np.array_equal(bits(out.locals[r]), np_bits(parts[r], dtype)), f"shard {r}"
+
+
+@pytest.mark.parametrize("dtype", [BF16, F32])
+@pytest.mark.parametrize("k", [1, 4, 8])
+@pytest.mark.parametrize("rows,classes", [(16, 4096), (5, 1000), (3, 70000)])
+def test_softmax_xent_backward_parity(dtype, k, rows, classes):
+    Z = dg.normal(1004, 5, (rows, classes), 0.0, 1.0, dtype)
+    labels = dg.integers(1004, 6, (rows,), 0, classes)
+    logits = make_global(split_cpu(Z, sbp.S(1), k), (rows, classes), dtype, sbp.S(1))
+    lab = make_global([labels] * k, (rows,), I64, sbp.B)
+    loss = sbp.empty_global((rows,), F32, sbp.B, k)
+    rmax = sbp.empty_global((rows,), F32, sbp.B, k)
+    rsum = sbp.empty_global((rows,), F32, sbp.B, k)
+    grad = sbp.empty_global((rows, classes), dtype, sbp.S(1), k)
+    ws = torch.empty(sbp.sbp_softmax_xent_workspace_bytes(logits), dtype=torch.uint8, device="cuda")
+    sbp.sbp_softmax_xent(logits, lab, loss, rmax, rsum, ws)
+    sbp.sbp_softmax_xent_backward(logits, lab, rmax, rsum, grad)
+    torch.cuda.synchronize()
+    want = O.to_locals(O.softmax_xent_grad(to_np(Z), labels.numpy()), O.S1, k)
+    for r in range(k):
+        assert tuple(grad.locals[r].shape) == tuple(want[r].shape)
+        assert_close(to_np(grad.locals[r]), want[r], 2e-2, 1e-3, f"grad shard {r}")
+    if dtype == F32:        # far tighter in fact, and every row sums to zero
+        full = O.from_locals([to_np(t).astype(np.float64) for t in grad.locals], O.S1)
+        assert np.all(np.abs(full - O.softmax_xent_grad(to_np(Z), labels.numpy())) <= 1e-6)
+        assert np.all(np.abs(full.sum(axis=1)) <= 1e-4)

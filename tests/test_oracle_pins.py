@@ -621,3 +621,23 @@ def test_boxing_cast_rounds_once_after_the_gather():
     want = torch.from_numpy(T).to(torch.bfloat16).to(torch.float32).numpy()     # independent library RNE
     assert len(out) == k and all(np.array_equal(o, want) for o in out)
     assert out[0][0, 0] == np.float32(1.0) and out[0][0, 1] == np.float32(1.0 + 2.0 ** -7)
+
+
+def test_softmax_xent_grad_against_finite_differences_and_library_softmax():
+    from scipy.special import softmax
+    R, C = 4, 9
+    Z = dg.normal(63, 0, (R, C), 0, 1.5).numpy().astype(np.float64)
+    labels = dg.integers(63, 1, (R,), 0, C).numpy()
+    G = O.softmax_xent_grad(Z, labels)
+    onehot = np.zeros((R, C))
+    onehot[np.arange(R), labels] = 1.0
+    assert np.allclose(G, softmax(Z, axis=1) - onehot, rtol=1e-13, atol=1e-14)
+    assert np.allclose(G.sum(axis=1), 0.0, atol=1e-14)
+    h = 1e-6
+    for i in range(R):
+        for j in range(C):
+            Zp, Zm = Z.copy(), Z.copy()
+            Zp[i, j] += h
+            Zm[i, j] -= h
+            fd = (O.softmax_xent_logical(Zp, labels)[2][i] - O.softmax_xent_logical(Zm, labels)[2][i]) / (2 * h)
+            assert abs(fd - G[i, j]) < 1e-8

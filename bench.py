@@ -445,7 +445,7 @@ def run_operator_sections(sbp, device, peaks, opts):
     for fn in [table[w.strip()] for w in which.split(",") if w.strip()]:
         try:
             out.extend(fn(sbp, device, peaks, opts))
-        except sbp.SbpError as e:            # an operator this build cannot run is reported, not hidden
+        except sbp.SbpError as e:            # an operator the library refuses is reported, not hidden
             out.append({"op": fn.__name__, "error": str(e)})
         torch.cuda.empty_cache()
     return out

@@ -44,7 +44,7 @@ typedef enum {
   SBP_ERR_SHAPE = 2,       /* logical shapes of the operands do not fit together         */
   SBP_ERR_DTYPE = 3,       /* dtype not supported by this operation                      */
   SBP_ERR_SIGNATURE = 4,   /* SBP signatures are not a valid combination                 */
-  SBP_ERR_UNSUPPORTED = 5, /* valid request that this build does not implement           */
+  SBP_ERR_UNSUPPORTED = 5, /* valid request that the library does not implement          */
   SBP_ERR_ALIGNMENT = 6,   /* a pointer is not aligned to its element size               */
   SBP_ERR_WORKSPACE = 7,   /* workspace missing or too small                             */
   SBP_ERR_CUDA = 8,        /* a CUDA runtime / driver call failed (no device, launch...) */

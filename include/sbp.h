@@ -112,6 +112,15 @@ sbp_status sbp_local_shape(const sbp_tensor* t, int32_t r, int64_t out_shape[SBP
  * W, or SBP_ERR_SIGNATURE when the pair is not one of the table's six rows. */
 sbp_status sbp_matmul_infer(sbp_sig x, sbp_sig w, sbp_sig* y);
 
+/* Table 2 ("Data size transferred between successive SBP signatures"): bytes that cross between
+ * devices when a tensor of t_bytes goes from signature src on p1 devices to signature dst on p2
+ * devices -- the "same" column (disjoint == 0, p1 == p2) or the "disjoint" column.  The paper
+ * offers these counts for choosing the signatures with the lowest communication cost
+ * (Section 3.2); on the one-GPU placements of this library nothing crosses a link, so this is
+ * a planning aid only.  Host only, no CUDA. */
+sbp_status sbp_transfer_cost(sbp_sig src, sbp_sig dst, int32_t p1, int32_t p2, int32_t disjoint,
+                             uint64_t t_bytes, uint64_t* cost_bytes);
+
 /* ---------------------------------------------------------------- boxing (Section 3.2)
  *
  * A boxing op re-arranges or transforms the local tensors of a global tensor so that

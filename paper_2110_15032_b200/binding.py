@@ -88,6 +88,7 @@ def load_library():
     lib.sbp_launch_count.restype = C.c_uint64
     lib.sbp_local_shape.argtypes = [T, C.c_int32, C.POINTER(C.c_int64)]
     lib.sbp_matmul_infer.argtypes = [_Sig, _Sig, C.POINTER(_Sig)]
+    lib.sbp_transfer_cost.argtypes = [_Sig, _Sig, C.c_int32, C.c_int32, C.c_int32, C.c_uint64, C.POINTER(C.c_uint64)]
     lib.sbp_boxing.argtypes = [T, T, C.c_void_p]
     lib.sbp_boxing_host_workspace_bytes.restype = C.c_size_t
     lib.sbp_boxing_host_workspace_bytes.argtypes = [T, T]
@@ -208,6 +209,13 @@ def sbp_matmul_infer(x: Sig, w: Sig) -> Sig:
     out = _Sig()
     _check(load_library().sbp_matmul_infer(x._c(), w._c(), C.byref(out)))
     return Sig(out.kind, out.axis if out.kind == SBP_SPLIT else 0)
+
+
+def sbp_transfer_cost(src: Sig, dst: Sig, p1: int, p2: int, disjoint: bool, t_bytes: int) -> int:
+    """Table 2: bytes crossing between devices for src -> dst (same or disjoint device sets)."""
+    out = C.c_uint64()
+    _check(load_library().sbp_transfer_cost(src._c(), dst._c(), p1, p2, 1 if disjoint else 0, t_bytes, C.byref(out)))
+    return int(out.value)
 
 
 def sbp_launch_count() -> int:

@@ -145,6 +145,38 @@ sbp_status sbp_local_shape(const sbp_tensor* t, int32_t r, int64_t out_shape[SBP
   return SBP_OK;
 }
 
+sbp_status sbp_transfer_cost(sbp_sig src, sbp_sig dst, int32_t p1, int32_t p2, int32_t disjoint, uint64_t t_bytes,
+                             uint64_t* cost_bytes) {
+  if (!cost_bytes) return fail(SBP_ERR_INVALID_ARG, "cost_bytes is null");
+  if (p1 < 1 || p2 < 1) return fail(SBP_ERR_INVALID_ARG, "device counts must be >= 1");
+  auto valid = [](sbp_sig s) { return s.kind >= SBP_SPLIT && s.kind <= SBP_PARTIAL_MAX; };
+  if (!valid(src) || !valid(dst)) return fail(SBP_ERR_SIGNATURE, "unknown sbp kind");
+  const bool ss = src.kind == SBP_SPLIT, sb = src.kind == SBP_BROADCAST, sp = !ss && !sb;
+  const bool ds = dst.kind == SBP_SPLIT, db = dst.kind == SBP_BROADCAST, dp = !ds && !db;
+  const uint64_t T = t_bytes, P1 = (uint64_t)p1, P2 = (uint64_t)p2;
+  uint64_t c = 0;
+  if (!disjoint) {
+    if (p1 != p2) return fail(SBP_ERR_INVALID_ARG, "the same placement has p1 == p2");
+    if (ss && ds) c = src.axis == dst.axis ? 0 : (P1 - 1) * T / P1;   // all2all
+    else if (ss && db) c = (P1 - 1) * T;                               // all-gather
+    else if (sp && ds) c = (P1 - 1) * T;                               // reduce-scatter
+    else if (sp && db) c = 2 * (P1 - 1) * T;                           // all-reduce
+    else c = 0;                                                        // S->P, B->S, B->B, B->P, P->P
+  } else {
+    if (ss && ds) c = T;
+    else if (ss && db) c = P2 * T;
+    else if (ss && dp) c = T;
+    else if (sb && ds) c = T;
+    else if (sb && db) c = P2 * T;
+    else if (sb && dp) c = T;
+    else if (sp && ds) c = P1 * T;
+    else if (sp && db) c = (P1 + P2 - 1) * T;
+    else c = P1 * T;                                                   // P -> P
+  }
+  *cost_bytes = c;
+  return SBP_OK;
+}
+
 sbp_status sbp_matmul_infer(sbp_sig x, sbp_sig w, sbp_sig* y) {
   if (!y) return fail(SBP_ERR_INVALID_ARG, "y is null");
   auto is_s = [](sbp_sig s, int ax) { return s.kind == SBP_SPLIT && s.axis == ax; };

@@ -190,3 +190,24 @@ def test_missing_library_fails_loudly(monkeypatch, tmp_path):
     monkeypatch.setattr(binding, "lib_path", lambda: str(tmp_path / "libsbp_b200.so"))
     with pytest.raises(RuntimeError, match="no CPU or PyTorch fallback"):
         binding.load_library()
+
+
+def test_transfer_cost_is_table2(lib):
+    tb = 24 * 24 * 4
+    for p, q in [(2, 2), (3, 3), (4, 2), (2, 8)]:
+        for a, b, same, disjoint in read_golden("table2_transfer_cost.txt"):
+            src = {"S(i)": sbp.S(0), "S": sbp.S(0), "B": sbp.B, "P": sbp.P_SUM}[a]
+            dst = {"S(i)": sbp.S(0), "S(j)": sbp.S(1), "S": sbp.S(0), "B": sbp.B, "P": sbp.P_SUM}[b]
+            env = {"__builtins__": {}}
+            want_dis = round(eval(disjoint, env, {"p": p, "q": q}) * tb)
+            assert sbp.sbp_transfer_cost(src, dst, p, q, True, tb) == want_dis, (a, b, p, q)
+            if p == q:
+                want_same = round(eval(same, env, {"p": p, "q": q}) * tb)
+                assert sbp.sbp_transfer_cost(src, dst, p, q, False, tb) == want_same, (a, b, p)
+                assert O.table2_same_placement_cost(osig_(src), osig_(dst), p, tb) == want_same
+    with pytest.raises(sbp.SbpError):
+        sbp.sbp_transfer_cost(sbp.S(0), sbp.B, 2, 3, False, tb)
+
+
+def osig_(sig):
+    return O.S(sig.axis) if sig.kind == 0 else {1: O.B, 2: O.PSUM, 3: O.PMAX}[sig.kind]

@@ -257,7 +257,7 @@ def test_table2_same_placement_costs_match_fixture_and_layout():
     n0 = n1 = 24
     tbytes = n0 * n1 * 4
     for p in (2, 3, 4):
-        for a, b, expr in rows:
+        for a, b, expr, _disjoint in rows:
             frac = _eval_cost(expr, p)
             src_sig = {"S(i)": S0, "S": S0, "B": B, "P": PSUM}[a]
             dst_sig = {"S(i)": S0, "S(j)": S1, "S": S0, "B": B, "P": PSUM}[b]

@@ -25,8 +25,8 @@
 namespace sbp {
 
 constexpr int kThreads = 256;
-constexpr int kLoadsPerThread = 8;    // vectors per thread per chunk
-constexpr int kMaxChunksPerCta = 8;   // a CTA walks up to this many chunks of one row
+constexpr int kLoadsPerThread = 4;    // vectors per thread per chunk
+constexpr int kMaxChunksPerCta = 16;  // a CTA walks up to this many chunks of one row
 
 struct XentParams {
   const char* logits[SBP_MAX_K];

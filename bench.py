@@ -434,6 +434,15 @@ def section_extras(sbp, device, peaks, opts):
     avg, best = time_op(lambda: sbp.sbp_embedding(table, idt, out_b), device)
     res.append(_hbm_entry("embedding, table S(1): fused gather -> B (8 replicas written)", n * 8 + n * row_b + k * n * row_b,
                           avg, best, peaks))
+    # backward of the row-split lookup: dense table gradient S(0) (zero fill + atomic scatter-add)
+    g1 = out_b.locals[0]
+    del table, out_b
+    torch.cuda.empty_cache()
+    go = sbp.SbpTensor((batch, 26, dim), torch.float32, sbp.B, [g1] * k)
+    gt = sbp.empty_global((rows, dim), torch.float32, sbp.S(0), k, device=device)
+    avg, best = time_op(lambda: sbp.sbp_embedding_backward(go, idt, gt), device, iters=5)
+    res.append(_hbm_entry("embedding backward: table gradient S(0) (zero fill + scatter-add)",
+                          rows * row_b + n * 8 + n * row_b, avg, best, peaks))
     return res
 
 

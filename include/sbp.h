@@ -298,6 +298,17 @@ sbp_status sbp_softmax_xent_static(const sbp_tensor* logits, const sbp_tensor* l
 sbp_status sbp_embedding(const sbp_tensor* table, const sbp_tensor* ids, sbp_tensor* out,
                          int32_t* oob_count, void* cuda_stream);
 
+/* Backward of the row-split lookup: the gradient of the table, S(0) like the table itself.
+ *   grad_out   [..., dim]   B, SBP_F32   gradient of the lookup's result
+ *   ids        [...]        B, SBP_I64   the ids of the forward pass
+ *   grad_table [rows, dim]  S(0), SBP_F32: row i = sum of grad_out over the lookups of id i,
+ *                           zero for rows never looked up (the whole tensor is written)
+ * dim must be a multiple of 4.  The sums are accumulated with fp32 atomic adds in no fixed
+ * order, so a row that many lookups hit may differ in its last bits from run to run.  Ids
+ * outside [0, rows) contribute nothing (and are counted in oob_count when it is not NULL). */
+sbp_status sbp_embedding_backward(const sbp_tensor* grad_out, const sbp_tensor* ids, sbp_tensor* grad_table,
+                                  int32_t* oob_count, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -408,3 +408,15 @@ def embedding_hidden_split(table_locals, ids):
     the k outputs are the lookup split along its last axis."""
     return [embedding_logical(t, ids) for t in table_locals]
 
+
+def embedding_grad_table(grad_out, ids, rows):
+    """Adjoint of the lookup: grad_table[i, :] = sum of grad_out[l, :] over the lookups l with
+    ids[l] == i (float64).  Ids outside [0, rows) contribute nothing."""
+    grad_out = np.asarray(grad_out, dtype=np.float64)
+    ids = np.asarray(ids, dtype=np.int64).reshape(-1)
+    g = grad_out.reshape(ids.shape[0], -1)
+    out = np.zeros((rows, g.shape[1]), dtype=np.float64)
+    ok = (ids >= 0) & (ids < rows)
+    np.add.at(out, ids[ok], g[ok])
+    return out
+

@@ -109,6 +109,7 @@ def load_library():
     lib.sbp_softmax_xent_backward.argtypes = [T, T, T, T, T, C.c_void_p]
     lib.sbp_softmax_xent_static.argtypes = [T, T, T, T, T, C.c_void_p]
     lib.sbp_embedding.argtypes = [T, T, T, C.c_void_p, C.c_void_p]
+    lib.sbp_embedding_backward.argtypes = [T, T, T, C.c_void_p, C.c_void_p]
     _LIB = lib
     return lib
 
@@ -324,3 +325,11 @@ def sbp_embedding(table: SbpTensor, ids: SbpTensor, out: SbpTensor,
     a, b, c = table._c(), ids._c(), out._c()
     oob = C.c_void_p(oob_count.data_ptr()) if oob_count is not None else C.c_void_p(0)
     _check(load_library().sbp_embedding(C.byref(a), C.byref(b), C.byref(c), oob, _stream_ptr(stream)))
+
+
+def sbp_embedding_backward(grad_out: SbpTensor, ids: SbpTensor, grad_table: SbpTensor,
+                           oob_count: Optional[torch.Tensor] = None, stream=None) -> None:
+    a, b, c = grad_out._c(), ids._c(), grad_table._c()
+    oob = C.c_void_p(oob_count.data_ptr()) if oob_count is not None else C.c_void_p(0)
+    _check(load_library().sbp_embedding_backward(C.byref(a), C.byref(b), C.byref(c), oob, _stream_ptr(stream)))
+

@@ -283,6 +283,46 @@ static sbp_status embedding_hidden_split(const sbp_tensor* table, const sbp_tens
   return SBP_OK;
 }
 
+// ---- backward of the row-split lookup: the gradient of the table, S(0) like the table.
+// grad_table_r[row, :] = sum over the lookups l with id_l = start_r + row of grad_out[l, :].
+// Each shard's gradient is zero-filled, then every lookup adds its gradient row into the row of
+// the owning shard with fp32 atomic adds (the order of the adds, hence the last bits of a sum
+// with many terms, is not fixed).
+struct EmbBwdParams {
+  float* grad_table[SBP_MAX_K];
+  long long shard_vecs[SBP_MAX_K];   // float4 vectors in each shard's gradient
+  const long long* ids;
+  const float* grad_out;
+  long long rows, base, rem, big;
+  int narrow;
+  long long n_lookups, vpr;          // float4 vectors per row
+  int k;
+  int* oob;
+};
+
+__global__ void __launch_bounds__(256) embedding_zero_kernel(const __grid_constant__ EmbBwdParams p) {
+  float4* g = reinterpret_cast<float4*>(p.grad_table[blockIdx.y]);
+  const long long n = p.shard_vecs[blockIdx.y];
+  const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) g[i] = z;
+}
+
+__global__ void __launch_bounds__(256) embedding_backward_kernel(const __grid_constant__ EmbBwdParams p) {
+  const long long total = p.n_lookups * p.vpr;
+  for (long long item = (long long)blockIdx.x * 256 + threadIdx.x; item < total; item += (long long)gridDim.x * 256) {
+    const long long look = item / p.vpr, col = item - look * p.vpr;
+    const long long id = __ldg(p.ids + look);
+    if (id < 0 || id >= p.rows) {
+      if (p.oob && col == 0) atomicAdd(p.oob, 1);
+      continue;
+    }
+    long long start;
+    const int r = owner_of_row(id, p.base, p.rem, p.big, p.narrow, &start);
+    const float4 gv = __ldg(reinterpret_cast<const float4*>(p.grad_out) + item);
+    atomicAdd(reinterpret_cast<float4*>(p.grad_table[r]) + (id - start) * p.vpr + col, gv);
+  }
+}
+
 }  // namespace sbp
 
 using namespace sbp;
@@ -367,3 +407,71 @@ extern "C" sbp_status sbp_embedding(const sbp_tensor* table, const sbp_tensor* i
   count_launch();
   return SBP_OK;
 }
+
+extern "C" sbp_status sbp_embedding_backward(const sbp_tensor* grad_out, const sbp_tensor* ids, sbp_tensor* grad_table,
+                                             int32_t* oob_count, void* cuda_stream) {
+  sbp_status st = check_tensor(grad_out, "grad_out", true);
+  if (st != SBP_OK) return st;
+  st = check_tensor(ids, "ids", true);
+  if (st != SBP_OK) return st;
+  st = check_tensor(grad_table, "grad_table", true);
+  if (st != SBP_OK) return st;
+  if (grad_table->ndim != 2) return fail(SBP_ERR_SHAPE, "grad_table must be [rows, dim]");
+  if (grad_table->dtype != SBP_F32 || grad_out->dtype != SBP_F32)
+    return fail(SBP_ERR_DTYPE, "the embedding backward accumulates in F32: grad_out and grad_table must be F32");
+  if (ids->dtype != SBP_I64) return fail(SBP_ERR_DTYPE, "ids must be I64");
+  if (ids->ndim > 3 || grad_out->ndim != ids->ndim + 1) return fail(SBP_ERR_SHAPE, "grad_out rank must be ids rank + 1");
+  for (int d = 0; d < ids->ndim; ++d)
+    if (grad_out->shape[d] != ids->shape[d]) return fail(SBP_ERR_SHAPE, "grad_out and ids differ on axis %d", d);
+  const long long dim = grad_table->shape[1];
+  if (grad_out->shape[grad_out->ndim - 1] != dim) return fail(SBP_ERR_SHAPE, "grad_out's last axis must equal dim");
+  const int k = placement_k(grad_table);
+  if (placement_k(ids) != k || placement_k(grad_out) != k) return fail(SBP_ERR_INVALID_ARG, "operands differ in k");
+  if (!(grad_table->sbp[0].kind == SBP_SPLIT && grad_table->sbp[0].axis == 0))
+    return fail(SBP_ERR_SIGNATURE, "grad_table must be S(0), like the table");
+  if (ids->sbp[0].kind != SBP_BROADCAST || grad_out->sbp[0].kind != SBP_BROADCAST)
+    return fail(SBP_ERR_SIGNATURE, "ids and grad_out must be B");
+  if (dim % 4 != 0) return fail(SBP_ERR_UNSUPPORTED, "dim must be a multiple of 4 (16-byte atomic adds)");
+  for (int r = 0; r < k; ++r)
+    if (reinterpret_cast<uintptr_t>(grad_table->local[r]) % 16 != 0)
+      return fail(SBP_ERR_ALIGNMENT, "grad_table shards must be 16-byte aligned");
+  if (reinterpret_cast<uintptr_t>(grad_out->local[0]) % 16 != 0) return fail(SBP_ERR_ALIGNMENT, "grad_out must be 16-byte aligned");
+  if (dim == 0 || grad_table->shape[0] == 0) return SBP_OK;
+
+  EmbBwdParams p{};
+  p.k = k;
+  p.rows = grad_table->shape[0];
+  p.base = p.rows / k;
+  p.rem = p.rows % k;
+  p.big = p.rem * (p.base + 1);
+  p.narrow = p.rows < (1LL << 31) ? 1 : 0;
+  p.n_lookups = numel(ids);
+  p.vpr = dim / 4;
+  p.ids = static_cast<const long long*>(ids->local[0]);
+  p.grad_out = static_cast<const float*>(grad_out->local[0]);
+  p.oob = oob_count;
+  long long max_vecs = 0;
+  for (int r = 0; r < k; ++r) {
+    p.grad_table[r] = static_cast<float*>(grad_table->local[r]);
+    p.shard_vecs[r] = local_numel(grad_table, r) / 4;
+    max_vecs = p.shard_vecs[r] > max_vecs ? p.shard_vecs[r] : max_vecs;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  long long zb = (max_vecs + 256 * 8 - 1) / (256 * 8);
+  if (zb < 1) zb = 1;
+  if (zb > 148 * 16) zb = 148 * 16;
+  embedding_zero_kernel<<<dim3((unsigned)zb, (unsigned)k), 256, 0, stream>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "embedding backward launch");
+  count_launch();
+  if (p.n_lookups > 0) {
+    long long sb = (p.n_lookups * p.vpr + 256 * 4 - 1) / (256 * 4);
+    if (sb > 148 * 32) sb = 148 * 32;
+    embedding_backward_kernel<<<(unsigned)sb, 256, 0, stream>>>(p);
+    e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "embedding backward launch");
+    count_launch();
+  }
+  return SBP_OK;
+}
+

@@ -508,3 +508,30 @@ def test_softmax_xent_backward_parity(dtype, k, rows, classes):
         full = O.from_locals([to_np(t).astype(np.float64) for t in grad.locals], O.S1)
         assert np.all(np.abs(full - O.softmax_xent_grad(to_np(Z), labels.numpy())) <= 1e-6)
         assert np.all(np.abs(full.sum(axis=1)) <= 1e-4)
+
+
+@pytest.mark.parametrize("k", [1, 3, 8])
+@pytest.mark.parametrize("rows,dim,hot", [(1000, 128, False), (37, 8, True), (5, 4, True)])
+def test_embedding_backward_parity(k, rows, dim, hot):
+    """grad_table (S(0)) = scatter-add of grad_out over the ids; fp32 atomic adds in no fixed order,
+    so the bound is the rounding of an n-term fp32 sum: n u sum|terms| (u = 2^-24)."""
+    n_rows_ids = 16 if not hot else rows                           # hot: every id lands on few rows
+    ids = dg.zipf_ids(1005, 7, (97, 26), 1024).clamp_(max=n_rows_ids - 1 if hot else rows - 1)
+    ids[3, 3] = -1
+    G = dg.normal(1005, 8, (97, 26, dim), 0.0, 1.0, F32)
+    go = make_global([G] * k, (97, 26, dim), F32, sbp.B)
+    idt = make_global([ids] * k, (97, 26), I64, sbp.B)
+    gt = sbp.empty_global((rows, dim), F32, sbp.S(0), k)
+    for t in gt.locals:
+        t.fill_(float("nan"))                                      # the kernel must write everything
+    oob = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sbp.sbp_embedding_backward(go, idt, gt, oob)
+    torch.cuda.synchronize()
+    assert int(oob.item()) == 1
+    want = O.embedding_grad_table(G.numpy(), ids.numpy(), rows)
+    mag = O.embedding_grad_table(np.abs(G.numpy()), ids.numpy(), rows)
+    counts = O.embedding_grad_table(np.ones((97, 26, 1)), ids.numpy(), rows)
+    got = O.from_locals([to_np(t).astype(np.float64) for t in gt.locals], O.S0)
+    assert got.shape == want.shape
+    assert np.all(np.abs(got - want) <= counts * 2.0 ** -24 * mag + 1e-30)
+    assert np.all(got[counts[:, 0] == 0] == 0.0)

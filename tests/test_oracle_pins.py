@@ -641,3 +641,22 @@ def test_softmax_xent_grad_against_finite_differences_and_library_softmax():
             Zm[i, j] -= h
             fd = (O.softmax_xent_logical(Zp, labels)[2][i] - O.softmax_xent_logical(Zm, labels)[2][i]) / (2 * h)
             assert abs(fd - G[i, j]) < 1e-8
+
+
+def test_embedding_grad_table_brute_force_and_adjoint_identity():
+    rows, d = 11, 4
+    ids = dg.integers(73, 1, (6, 3), 0, rows).numpy()
+    ids[0, 0] = rows + 5                                          # out of range: no contribution
+    G = dg.normal(73, 2, (6, 3, d), 0, 1).numpy().astype(np.float64)
+    got = O.embedding_grad_table(G, ids, rows)
+    want = np.zeros((rows, d))
+    for b in range(6):
+        for f in range(3):
+            if 0 <= ids[b, f] < rows:
+                want[ids[b, f]] += G[b, f]
+    assert np.allclose(got, want, rtol=0, atol=1e-15)
+    # adjoint of the lookup: <lookup(table), G> == <table, grad_table(G)>
+    table = dg.normal(73, 3, (rows, d), 0, 1).numpy().astype(np.float64)
+    lhs = float((O.embedding_logical(table, ids) * G).sum())
+    rhs = float((table * got).sum())
+    assert abs(lhs - rhs) < 1e-12

@@ -218,18 +218,20 @@ bool launch_bulk_copy(const BoxParams& p, int ntasks, cudaStream_t st) {
   q.total_tiles = q.tiles_per_task * ntasks;
   if (q.total_tiles <= 0) return false;
 
-  static int sm_count = 0;
-  static bool attr_set = false;
+  // per device: SM count and the kernel's shared-memory opt-in
+  static int sms_on_device[64] = {};
   const size_t smem = (size_t)kStages * kStageBytes;
-  if (!attr_set) {
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return false;
-    if (cudaDeviceGetAttribute(&sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return false;
+  if (sms_on_device[dev] == 0) {
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return false;
     if (cudaFuncSetAttribute(box_bulk_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) !=
         cudaSuccess)
       return false;
-    attr_set = true;
+    sms_on_device[dev] = sms;
   }
+  const int sm_count = sms_on_device[dev];
   long long grid = (long long)sm_count * kCtasPerSm;
   if (grid > q.total_tiles) grid = q.total_tiles;
   box_bulk_kernel<<<(unsigned)grid, 32, smem, st>>>(q);

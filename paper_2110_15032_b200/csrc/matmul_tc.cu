@@ -215,7 +215,8 @@ constexpr unsigned kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1
 // operations where erff costs a long polynomial.
 __device__ __forceinline__ float erf_as(float x) {
   const float ax = fabsf(x);
-  const float t = __frcp_rn(fmaf(0.3275911f, ax, 1.0f));
+  float t;
+  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(t) : "f"(fmaf(0.3275911f, ax, 1.0f)));
   float poly = fmaf(1.061405429f, t, -1.453152027f);
   poly = fmaf(poly, t, 1.421413741f);
   poly = fmaf(poly, t, -0.284496736f);
@@ -644,11 +645,14 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
   *taken = true;
   if (tiles == 0) return SBP_OK;
 
-  static int max_pairs = 0;
-  if (max_pairs == 0) {
+  // per device: the kernel's shared-memory opt-in and the number of CTA pairs that fit at once
+  static int pairs_on_device[64] = {};
+  int dev = 0;
+  SBP_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(SBP_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
+  if (pairs_on_device[dev] == 0) {
     SBP_CUDA_TRY(cudaFuncSetAttribute(matmul_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    int dev = 0, sms = 0;
-    SBP_CUDA_TRY(cudaGetDevice(&dev));
+    int sms = 0;
     SBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     // how many CTA pairs the device can hold at once (pairs must sit in one GPC)
     cudaLaunchConfig_t probe = {};
@@ -667,8 +671,9 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
       cudaGetLastError();
       clusters = sms / 2;
     }
-    max_pairs = clusters;
+    pairs_on_device[dev] = clusters;
   }
+  const int max_pairs = pairs_on_device[dev];
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
   matmul_tc_kernel<<<2 * pairs, kThreadsTc, kSmemBytes, st>>>(p);
   cudaError_t e = cudaGetLastError();

@@ -285,9 +285,12 @@ static sbp_status embedding_hidden_split(const sbp_tensor* table, const sbp_tens
 
 // ---- backward of the row-split lookup: the gradient of the table, S(0) like the table.
 // grad_table_r[row, :] = sum over the lookups l with id_l = start_r + row of grad_out[l, :].
-// Each shard's gradient is zero-filled, then every lookup adds its gradient row into the row of
-// the owning shard with fp32 atomic adds (the order of the adds, hence the last bits of a sum
-// with many terms, is not fixed).
+// Each shard's gradient is zero-filled; then the lookups are taken in chunks, one CTA per chunk:
+// the CTA sorts its chunk by (id, position), each warp sums the runs of equal ids in its part
+// of the sorted chunk in registers (in lookup order) and adds one row per run into the owning
+// shard with 16-byte fp32 atomic adds. Under a skewed id distribution this takes the repeated
+// adds to the hot rows out of the L2 atomic units, which otherwise serialise them. The order of
+// the atomic adds between chunks, hence the last bits of a sum with many terms, is not fixed.
 struct EmbBwdParams {
   float* grad_table[SBP_MAX_K];
   long long shard_vecs[SBP_MAX_K];   // float4 vectors in each shard's gradient
@@ -307,19 +310,80 @@ __global__ void __launch_bounds__(256) embedding_zero_kernel(const __grid_consta
   for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) g[i] = z;
 }
 
-__global__ void __launch_bounds__(256) embedding_backward_kernel(const __grid_constant__ EmbBwdParams p) {
-  const long long total = p.n_lookups * p.vpr;
-  for (long long item = (long long)blockIdx.x * 256 + threadIdx.x; item < total; item += (long long)gridDim.x * 256) {
-    const long long look = item / p.vpr, col = item - look * p.vpr;
-    const long long id = __ldg(p.ids + look);
-    if (id < 0 || id >= p.rows) {
-      if (p.oob && col == 0) atomicAdd(p.oob, 1);
-      continue;
+// CHUNK lookups per CTA pass (256 or 1024); key = id * CHUNK + position in the chunk, all ones
+// for a position past the end or an id outside the table (sorted last, skipped).
+template <int CHUNK>
+__global__ void __launch_bounds__(256, 3) embedding_backward_kernel(const __grid_constant__ EmbBwdParams p) {
+  constexpr int kShift = CHUNK == 1024 ? 10 : 8;
+  constexpr int kPerWarp = CHUNK / 8;     // sorted positions walked by one warp
+  constexpr int kBatch = 8;               // gradient rows in flight per lane
+  constexpr unsigned long long kNone = ~0ull;
+  __shared__ unsigned long long key[CHUNK];
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const long long n_chunks = (p.n_lookups + CHUNK - 1) / CHUNK;
+  const float4* gout = reinterpret_cast<const float4*>(p.grad_out);
+  for (long long chunk = blockIdx.x; chunk < n_chunks; chunk += gridDim.x) {
+    const long long first = chunk * CHUNK;
+    for (int i = tid; i < CHUNK; i += 256) {
+      unsigned long long kv = kNone;
+      if (first + i < p.n_lookups) {
+        const long long id = __ldg(p.ids + first + i);
+        if (id >= 0 && id < p.rows) kv = ((unsigned long long)id << kShift) | (unsigned)i;
+        else if (p.oob) atomicAdd(p.oob, 1);
+      }
+      key[i] = kv;
     }
-    long long start;
-    const int r = owner_of_row(id, p.base, p.rem, p.big, p.narrow, &start);
-    const float4 gv = __ldg(reinterpret_cast<const float4*>(p.grad_out) + item);
-    atomicAdd(reinterpret_cast<float4*>(p.grad_table[r]) + (id - start) * p.vpr + col, gv);
+    __syncthreads();
+    // bitonic sort, ascending
+    for (int size = 2; size <= CHUNK; size <<= 1) {
+      for (int j = size >> 1; j > 0; j >>= 1) {
+        for (int t = tid; t < CHUNK / 2; t += 256) {
+          const int lo = 2 * t - (t & (j - 1)), hi = lo + j;
+          const unsigned long long a = key[lo], b = key[hi];
+          const bool up = (lo & size) == 0;
+          if ((a > b) == up) { key[lo] = b; key[hi] = a; }
+        }
+        __syncthreads();
+      }
+    }
+    // runs of equal ids -> one atomic row add each
+    for (long long cb = 0; cb < p.vpr; cb += 32) {
+      const long long col = cb + lane;
+      const bool active = col < p.vpr;
+      long long cur = -1;
+      float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+      auto flush = [&]() {
+        if (cur >= 0 && active) {
+          long long start;
+          const int r = owner_of_row(cur, p.base, p.rem, p.big, p.narrow, &start);
+          atomicAdd(reinterpret_cast<float4*>(p.grad_table[r]) + (cur - start) * p.vpr + col, acc);
+        }
+      };
+      for (int pos = warp * kPerWarp; pos < (warp + 1) * kPerWarp; pos += kBatch) {
+        unsigned long long kv[kBatch];
+        float4 gv[kBatch];
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+          kv[j] = key[pos + j];
+          gv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
+          if (kv[j] != kNone && active) gv[j] = __ldg(gout + (first + (long long)(kv[j] & (CHUNK - 1))) * p.vpr + col);
+        }
+#pragma unroll
+        for (int j = 0; j < kBatch; ++j) {
+          if (kv[j] == kNone) continue;
+          const long long id = (long long)(kv[j] >> kShift);
+          if (id != cur) {
+            flush();
+            cur = id;
+            acc = gv[j];
+          } else {
+            acc.x += gv[j].x; acc.y += gv[j].y; acc.z += gv[j].z; acc.w += gv[j].w;
+          }
+        }
+      }
+      flush();
+    }
+    __syncthreads();
   }
 }
 
@@ -465,9 +529,12 @@ extern "C" sbp_status sbp_embedding_backward(const sbp_tensor* grad_out, const s
   if (e != cudaSuccess) return cuda_fail(e, "embedding backward launch");
   count_launch();
   if (p.n_lookups > 0) {
-    long long sb = (p.n_lookups * p.vpr + 256 * 4 - 1) / (256 * 4);
-    if (sb > 148 * 32) sb = 148 * 32;
-    embedding_backward_kernel<<<(unsigned)sb, 256, 0, stream>>>(p);
+    // 1024-lookup chunks once they fill the GPU a few times over, else 256-lookup chunks
+    const bool big_chunks = p.n_lookups / 1024 >= 148 * 4;
+    const long long chunks = (p.n_lookups + (big_chunks ? 1023 : 255)) / (big_chunks ? 1024 : 256);
+    const unsigned sb = (unsigned)(chunks < 148 * 8 ? chunks : 148 * 8);
+    if (big_chunks) embedding_backward_kernel<1024><<<sb, 256, 0, stream>>>(p);
+    else embedding_backward_kernel<256><<<sb, 256, 0, stream>>>(p);
     e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "embedding backward launch");
     count_launch();

@@ -535,3 +535,28 @@ def test_embedding_backward_parity(k, rows, dim, hot):
     assert got.shape == want.shape
     assert np.all(np.abs(got - want) <= counts * 2.0 ** -24 * mag + 1e-30)
     assert np.all(got[counts[:, 0] == 0] == 0.0)
+
+
+@pytest.mark.parametrize("k,rows,dim,s,batch", [(8, 100003, 8, 1.05, 24000), (3, 2000, 132, 1.3, 300)])
+def test_embedding_backward_large_batch(k, rows, dim, s, batch):
+    """A batch large enough for the 1024-lookup chunks (and, with dim = 132, rows wider than one
+    pass of a warp): same bound as above."""
+    ids = dg.zipf_ids(1005, 17, (batch, 26), rows, s)
+    ids[5, 7] = rows
+    ids[batch - 1, 25] = -3
+    G = dg.normal(1005, 18, (batch, 26, dim), 0.0, 1.0, F32)
+    go = make_global([G] * k, (batch, 26, dim), F32, sbp.B)
+    idt = make_global([ids] * k, (batch, 26), I64, sbp.B)
+    gt = sbp.empty_global((rows, dim), F32, sbp.S(0), k)
+    for t in gt.locals:
+        t.fill_(float("nan"))
+    oob = torch.zeros(1, dtype=torch.int32, device="cuda")
+    sbp.sbp_embedding_backward(go, idt, gt, oob)
+    torch.cuda.synchronize()
+    assert int(oob.item()) == 2
+    want = O.embedding_grad_table(G.numpy(), ids.numpy(), rows)
+    mag = O.embedding_grad_table(np.abs(G.numpy()), ids.numpy(), rows)
+    counts = O.embedding_grad_table(np.ones((batch, 26, 1)), ids.numpy(), rows)
+    got = O.from_locals([to_np(t).astype(np.float64) for t in gt.locals], O.S0)
+    assert np.all(np.abs(got - want) <= counts * 2.0 ** -24 * mag + 1e-30)
+    assert np.all(got[counts[:, 0] == 0] == 0.0)

@@ -179,6 +179,64 @@ def boxing(src_locals, src_sig, dst_sig, storage="f32"):
     return to_locals(T, dst_sig, k)
 
 
+def boxing_disjoint(src_locals, src_sig, dst_sig, k_dst, storage="f32"):
+    """Boxing between two DIFFERENT device sets (Section 3.2, Table 2, column "disjoint"): the
+    input lives on p = len(src_locals) devices, the output on q = k_dst other devices.
+
+    The table gives only the bytes that move; the readings taken here are the simplest
+    transforms that move exactly those bytes and keep the global tensor unchanged:
+      S or B -> S or B   the global tensor is rebuilt and mapped onto the q devices;
+      P -> S, P -> B     the p partials are reduced in fixed rank order (all p|T| bytes travel),
+                         then mapped onto the q devices;
+      S -> P(sum)        |T| travels once: output device j holds piece j of the q-way balanced
+                         split of the source's split axis, in place, zeros elsewhere;
+      B -> P(sum)        |T| travels once: output device 0 holds T, the others zeros;
+      P -> P             every partial travels once (p|T|): input device r sends to output device
+                         r mod q, which reduces what it receives in ascending r (an output device
+                         that receives nothing holds zeros; for P(max) that case is undefined).
+    With q = p every row gives the same local tensors as boxing() on one placement.
+    """
+    p, q = len(src_locals), int(k_dst)
+    src_sig, dst_sig = tuple(src_sig), tuple(dst_sig)
+    if src_sig[0] == "P" and dst_sig[0] == "P":
+        if src_sig != dst_sig:
+            raise ValueError("P(sum) <-> P(max) has no meaning")
+        outs = []
+        for j in range(q):
+            mine = [src_locals[r] for r in range(j, p, q)]
+            if not mine:
+                if dst_sig == PMAX:
+                    raise ValueError("P(max) onto more devices than partials is undefined")
+                outs.append(np.zeros_like(np.asarray(src_locals[0])))
+            else:
+                outs.append(from_locals(mine, src_sig, storage))
+        return outs
+    T = from_locals(src_locals, src_sig, storage)
+    if dst_sig == PSUM:
+        outs = [np.zeros_like(T) for _ in range(q)]
+        if src_sig[0] == "S":
+            ax = src_sig[1]
+            for j, (start, ln) in enumerate(balanced_split(T.shape[ax], q)):
+                sel = [slice(None)] * T.ndim
+                sel[ax] = slice(start, start + ln)
+                outs[j][tuple(sel)] = T[tuple(sel)]
+        else:
+            outs[0] = T.copy()
+        return outs
+    if dst_sig[0] == "P":
+        raise ValueError("S -> P(max) / B -> P(max): zero is not neutral for max")
+    return to_locals(T, dst_sig, q)
+
+
+def table2_disjoint_placement_cost(src_sig, dst_sig, p, q, t_bytes):
+    """Table 2, column "disjoint": bytes that travel from the p input devices to the q output
+    devices (|T| = t_bytes)."""
+    a, b = src_sig[0], dst_sig[0]
+    if a == "P":
+        return (p + q - 1) * t_bytes if b == "B" else p * t_bytes
+    return q * t_bytes if b == "B" else t_bytes
+
+
 def boxing_cast(src_locals, src_sig, dst_sig, dst_storage):
     """Boxing followed by a cast of every destination local tensor to dst_storage (Section 6.4:
     a cast op with S(0) input and B output turns sharded fp32 state into half-precision replicas)."""

@@ -660,3 +660,126 @@ def test_embedding_grad_table_brute_force_and_adjoint_identity():
     lhs = float((O.embedding_logical(table, ids) * G).sum())
     rhs = float((table * got).sum())
     assert abs(lhs - rhs) < 1e-12
+
+
+# ---------------------------------------------------------------- Table 2, disjoint placements
+
+def _owner_1d(n, k, a):
+    """(device, local offset) of index a of an axis of length n split over k devices, by counting."""
+    base, rem = divmod(n, k)
+    start = 0
+    for r in range(k):
+        ln = base + (1 if r < rem else 0)
+        if a < start + ln:
+            return r, a - start
+        start += ln
+    raise AssertionError
+
+
+@pytest.mark.parametrize("n0,n1", [(8, 12), (7, 5)])
+@pytest.mark.parametrize("p,q", [(2, 3), (4, 2), (3, 5), (1, 4), (4, 1), (3, 3)])
+def test_boxing_disjoint_matches_element_definition(n0, n1, p, q):
+    """Every element of every output local tensor, from the definition of the signatures alone."""
+    T = np.arange(n0 * n1, dtype=np.float32).reshape(n0, n1) + 1
+    parts = [dg.small_integers(31, r, (n0, n1), -8, 9).numpy().astype(np.float32) for r in range(p)]
+    total = np.sum(parts, axis=0)                      # exact: small integers
+    for src_sig in (S0, S1, B, PSUM):
+        src = parts if src_sig == PSUM else O.to_locals(T, src_sig, p)
+        G = total if src_sig == PSUM else T
+        for dst_sig in (S0, S1, B):
+            got = O.boxing_disjoint(src, src_sig, dst_sig, q)
+            assert len(got) == q
+            seen = 0
+            for i in range(n0):
+                for j in range(n1):
+                    if dst_sig[0] == "B":
+                        for d in range(q):
+                            assert got[d][i, j] == G[i, j]
+                    else:
+                        ax = dst_sig[1]
+                        d, off = _owner_1d((n0, n1)[ax], q, (i, j)[ax])
+                        loc = (off, j) if ax == 0 else (i, off)
+                        assert got[d][loc] == G[i, j]
+                        seen += 1
+            if dst_sig[0] == "S":
+                assert sum(g.size for g in got) == seen == n0 * n1
+        # -> P(sum): the outputs have the global shape, sum back to it exactly, and each element
+        # is non-zero on exactly one device (the owner of its piece, or device 0 for B)
+        if src_sig != PSUM:
+            got = O.boxing_disjoint(src, src_sig, PSUM, q)
+            assert all(g.shape == (n0, n1) for g in got)
+            assert np.array_equal(np.sum(got, axis=0), T)
+            for i in range(n0):
+                for j in range(n1):
+                    holder = 0 if src_sig == B else _owner_1d((n0, n1)[src_sig[1]], q, (i, j)[src_sig[1]])[0]
+                    for d in range(q):
+                        assert got[d][i, j] == (T[i, j] if d == holder else 0.0)
+    # P -> P: partial r goes to device r mod q
+    got = O.boxing_disjoint(parts, PSUM, PSUM, q)
+    assert np.array_equal(np.sum(got, axis=0), total)
+    for d in range(q):
+        want = np.zeros((n0, n1), np.float32)
+        for r in range(p):
+            if r % q == d:
+                want = want + parts[r]
+        assert np.array_equal(got[d], want)
+    if p >= q:
+        gm = O.boxing_disjoint(parts, PMAX, PMAX, q)
+        assert np.array_equal(np.max(gm, axis=0), np.max(parts, axis=0))
+    else:
+        with pytest.raises(ValueError):
+            O.boxing_disjoint(parts, PMAX, PMAX, q)
+
+
+@pytest.mark.parametrize("k", [1, 2, 3, 4])
+def test_boxing_disjoint_with_equal_counts_is_boxing(k):
+    T = dg.normal(32, 0, (6, 9), 0, 1).numpy()
+    parts = [O.round_to_bf16(dg.normal(32, 1 + r, (6, 9), 0, 1).numpy()) for r in range(k)]   # storable as bf16
+    for src_sig in (S0, S1, B, PSUM, PMAX):
+        src = parts if src_sig[0] == "P" else O.to_locals(T, src_sig, k)
+        for dst_sig in (S0, S1, B, PSUM, PMAX):
+            if dst_sig == PMAX and src_sig != PMAX:
+                continue
+            if src_sig == PMAX and dst_sig == PSUM:
+                continue
+            a = O.boxing_disjoint(src, src_sig, dst_sig, k, "bf16" if src_sig == PSUM else "f32")
+            b = O.boxing(src, src_sig, dst_sig, "bf16" if src_sig == PSUM else "f32")
+            assert len(a) == len(b) and all(np.array_equal(x, y) for x, y in zip(a, b)), (src_sig, dst_sig)
+
+
+def test_boxing_disjoint_psum_rounds_once_in_rank_order():
+    """1 + 2^-24 + 2^-24 in fp32 rank order stays 1 (each add rounds to even), while the exact sum
+    rounds up: the order of the adds is visible, and so is the single bf16 rounding."""
+    a = np.array([[1.0]], np.float32)
+    e = np.array([[2.0 ** -24]], np.float32)
+    got = O.boxing_disjoint([a, e, e], PSUM, B, 2)
+    assert got[0][0, 0] == 1.0 and got[1][0, 0] == 1.0
+    got = O.boxing_disjoint([e, e, a], PSUM, B, 1)
+    assert got[0][0, 0] == np.float32(1.0 + 2.0 ** -23)
+    # devices 0 and 2 feed output 0, device 1 feeds output 1
+    got = O.boxing_disjoint([a, e, a], PSUM, PSUM, 2)
+    assert got[0][0, 0] == 2.0 and got[1][0, 0] == np.float32(2.0 ** -24)
+    h = np.array([[1.0 + 2.0 ** -8]], np.float32)            # a bf16 tie: rounds to even (1.0)
+    assert O.boxing_disjoint([h, np.zeros((1, 1), np.float32)], PSUM, S0, 1, "bf16")[0][0, 0] == 1.0
+
+
+def test_table2_disjoint_costs_match_fixture_and_layout():
+    rows = read_golden("table2_transfer_cost.txt")
+    tb = 24 * 24 * 4
+    for p, q in [(2, 3), (4, 2), (3, 3), (1, 5)]:
+        for a, b, _same, expr in rows:
+            want = round(eval(expr, {"__builtins__": {}}, {"p": p, "q": q}) * tb)
+            src_sig = {"S(i)": S0, "S": S0, "B": B, "P": PSUM}[a]
+            dst_sig = {"S(i)": S0, "S(j)": S1, "S": S0, "B": B, "P": PSUM}[b]
+            assert O.table2_disjoint_placement_cost(src_sig, dst_sig, p, q, tb) == want, (a, b, p, q)
+    # the layout agrees with the table where every output byte is a moved byte (no reduction):
+    # the outputs of S/B -> S hold |T| bytes, of S/B -> B q|T|, and S/B -> P(sum) has |T| non-zeros
+    T = np.arange(24 * 24, dtype=np.float32).reshape(24, 24) + 1
+    for p, q in [(2, 3), (4, 2)]:
+        for src_sig in (S0, S1, B):
+            src = O.to_locals(T, src_sig, p)
+            for dst_sig in (S0, S1, B):
+                out = O.boxing_disjoint(src, src_sig, dst_sig, q)
+                assert sum(o.nbytes for o in out) == O.table2_disjoint_placement_cost(src_sig, dst_sig, p, q, tb)
+            out = O.boxing_disjoint(src, src_sig, PSUM, q)
+            assert sum(int(np.count_nonzero(o)) for o in out) * 4 == O.table2_disjoint_placement_cost(src_sig, PSUM, p, q, tb)

@@ -414,7 +414,7 @@ def section_extras(sbp, device, peaks, opts):
     res.append(_hbm_entry("S(0)->P(sum) bf16 [8192,8192] k=4", (1 + k) * tb, avg, best, peaks))
     avg, best = time_op(lambda: sbp.sbp_boxing(b, part), device)
     res.append(_hbm_entry("B->P(sum) bf16 [8192,8192] k=4", (1 + k) * tb, avg, best, peaks))
-    del T, s0, b, part
+    del T, b, part
     torch.cuda.empty_cache()
     # Section 6.4's cast op: fp32 shards S(0) -> bf16 replicas B, the cast folded into the gather
     Tf = dg.normal(SEED, 1, shape, 0.0, 1.0, torch.float32, device)
@@ -423,6 +423,21 @@ def section_extras(sbp, device, peaks, opts):
     avg, best = time_op(lambda: sbp.sbp_boxing(sf, rb), device)
     res.append(_hbm_entry("S(0) fp32 -> B bf16 (cast fused into the gather) [8192,8192] k=4", 2 * tb + k * tb, avg, best, peaks))
     del Tf, sf, rb
+    torch.cuda.empty_cache()
+    # different placements (Table 2, column "disjoint"): p = 4 source shards, q = 8 (or 2) destination shards
+    psrc = sbp.SbpTensor(shape, bf16, sbp.P_SUM, [dg.normal(SEED, 300 + r, shape, 0.0, 1.0, bf16, device) for r in range(k)])
+    for name, src_g, dst_sig, q, nbytes in [
+            ("S(0)[4] -> S(0)[8]", s0, sbp.S(0), 8, 2 * tb),
+            ("S(0)[4] -> S(1)[8]", s0, sbp.S(1), 8, 2 * tb),
+            ("S(0)[4] -> B[8]", s0, sbp.B, 8, tb + 8 * tb),
+            ("P(sum)[4] -> S(0)[8]", psrc, sbp.S(0), 8, k * tb + tb),
+            ("P(sum)[4] -> B[2]", psrc, sbp.B, 2, k * tb + 2 * tb),
+            ("S(0)[4] -> P(sum)[8]", s0, sbp.P_SUM, 8, tb + 8 * tb)]:
+        dq = sbp.empty_global(shape, bf16, dst_sig, q, device=device)
+        avg, best = time_op(lambda: sbp.sbp_boxing(src_g, dq), device)
+        res.append(_hbm_entry("disjoint placements: " + name + " bf16 [8192,8192]", nbytes, avg, best, peaks))
+        del dq
+    del psrc, s0
     torch.cuda.empty_cache()
     k, rows, dim, batch = 8, opts.emb_rows, 128, opts.emb_batch
     ids = dg.zipf_ids(1005, 1, (batch, 26), rows, 1.05, device)

@@ -125,7 +125,9 @@ sbp_status sbp_transfer_cost(sbp_sig src, sbp_sig dst, int32_t p1, int32_t p2, i
  *
  * A boxing op re-arranges or transforms the local tensors of a global tensor so that
  * the same global tensor is seen under another signature (Section 3.2; Table 2, column
- * "same" placement).  src and dst must agree in logical shape, dtype (one exception below) and k.
+ * "same" placement).  src and dst must agree in logical shape and dtype (one exception below);
+ * with the same k on both sides the rows below apply, with different k the "disjoint" rows
+ * further down.
  *
  *   src            dst        the collective it stands for (Table 2)
  *   P(sum)         B          all-reduce       out_j[e] = round(sum_r in_r[e])
@@ -149,6 +151,18 @@ sbp_status sbp_transfer_cost(sbp_sig src, sbp_sig dst, int32_t p1, int32_t p2, i
  * axis 1 changes, across the groups when axis 0 changes.  Changing axis 0 along the tensor axis
  * that axis 1 splits, or summing over one axis what is a max over the other, is refused with
  * SBP_ERR_UNSUPPORTED, as is changing both axes at once (make two calls).
+ *
+ * Different placements (Table 2, column "disjoint"): src on p = k(src) shards, dst on q = k(dst)
+ * other shards, p != q allowed, one-axis placements on both sides, same dtype.  The table fixes
+ * only the bytes that travel; the transforms are the plainest ones that move exactly those bytes:
+ *   S / B   -> S(i) / B   the global tensor, mapped onto the q shards (balanced q-way split)
+ *   P(op)   -> S(i) / B   all p partials reduced in rank order (arithmetic below), then mapped
+ *   S(i)    -> P(sum)     partial j = zeros with piece j of the q-way split of axis i in place
+ *   B       -> P(sum)     partial 0 = the tensor, the others zeros
+ *   P(op)   -> P(op)      partial r travels to shard r mod q, which reduces what it receives in
+ *                         ascending r; a shard that receives nothing is zero (so P(max) with
+ *                         q > p is refused with SBP_ERR_UNSUPPORTED)
+ * With q == p these give the same local tensors as the same-placement rows.
  *
  * P(sum) arithmetic: an fp32 accumulator starts as shard 0, shards 1..k-1 are added in
  * rank order with plain IEEE adds, and the result is rounded once (nearest even) to the

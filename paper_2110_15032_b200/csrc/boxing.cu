@@ -18,88 +18,11 @@
 #include <algorithm>
 #include <atomic>
 
+#include "boxing_arith.h"
 #include "boxing_params.h"
 #include "sbp_internal.h"
 
 namespace sbp {
-
-enum BoxOp : int { OP_COPY = 0, OP_SUM_F32, OP_SUM_BF16, OP_MAX_F32, OP_MAX_BF16 };
-
-// ------------------------------------------------------------------ element arithmetic
-
-// fp32 lanes carried by one vector of type V
-template <typename V>
-struct AccF32 {
-  static constexpr int N = sizeof(V) / 4;
-  float v[N];
-  __device__ void load(const V& x) {
-    const float* f = reinterpret_cast<const float*>(&x);
-#pragma unroll
-    for (int i = 0; i < N; ++i) v[i] = f[i];
-  }
-  __device__ V store() const {
-    V out;
-    float* f = reinterpret_cast<float*>(&out);
-#pragma unroll
-    for (int i = 0; i < N; ++i) f[i] = v[i];
-    return out;
-  }
-};
-
-template <typename V>
-struct AccBF16 {
-  static constexpr int N = sizeof(V) / 2;
-  float v[N];
-  __device__ void load(const V& x) {
-    const __nv_bfloat16* h = reinterpret_cast<const __nv_bfloat16*>(&x);
-#pragma unroll
-    for (int i = 0; i < N; ++i) v[i] = __bfloat162float(h[i]);
-  }
-  __device__ V store() const {
-    V out;
-    __nv_bfloat16* h = reinterpret_cast<__nv_bfloat16*>(&out);
-#pragma unroll
-    for (int i = 0; i < N; ++i) h[i] = __float2bfloat16_rn(v[i]);   // the single rounding
-    return out;
-  }
-};
-
-template <int OP, typename V>
-struct Lanes {
-  using type = AccF32<V>;
-};
-template <typename V>
-struct Lanes<OP_SUM_BF16, V> {
-  using type = AccBF16<V>;
-};
-template <typename V>
-struct Lanes<OP_MAX_BF16, V> {
-  using type = AccBF16<V>;
-};
-
-template <int OP, typename L>
-__device__ __forceinline__ void combine(L& acc, const L& x) {
-#pragma unroll
-  for (int i = 0; i < L::N; ++i) {
-    if (OP == OP_SUM_F32 || OP == OP_SUM_BF16)
-      acc.v[i] = __fadd_rn(acc.v[i], x.v[i]);          // plain IEEE add, never contracted
-    else
-      acc.v[i] = (x.v[i] > acc.v[i]) ? x.v[i] : acc.v[i];   // first wins on ties
-  }
-}
-
-template <typename V>
-__device__ __forceinline__ V ld_stream(const V* p) {
-  return *p;
-}
-template <>
-__device__ __forceinline__ uint4 ld_stream<uint4>(const uint4* p) {
-  uint4 r;
-  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
-               : "l"(p));
-  return r;
-}
 
 // ------------------------------------------------------------------ the tile kernel
 
@@ -531,9 +454,17 @@ static sbp_status check_pair(const sbp_tensor* src, const sbp_tensor* dst, bool 
                            dst->sbp[0].kind == SBP_BROADCAST;
   if (src->dtype != dst->dtype && !cast_gather)
     return fail(SBP_ERR_DTYPE, "src and dst differ in dtype (only S(i) -> B may cast, F32 -> BF16)");
-  if (placement_k(src) != placement_k(dst)) return fail(SBP_ERR_INVALID_ARG, "src and dst differ in k");
+  if (placement_k(src) != placement_k(dst)) {
+    if (src->pdims != 1 || dst->pdims != 1)
+      return fail(SBP_ERR_UNSUPPORTED, "boxing between different placements needs one-axis placements on both sides");
+    if (src->dtype != dst->dtype)
+      return fail(SBP_ERR_UNSUPPORTED, "the cast-fused gather needs src and dst on the same placement");
+  }
   return SBP_OK;
 }
+
+// Different shard counts on the two sides (defined in boxing_disjoint.cu).
+sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, cudaStream_t stream);
 
 }  // namespace sbp
 
@@ -622,6 +553,7 @@ sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream)
   if (src && dst && (src->pdims == 2 || dst->pdims == 2)) return boxing_2d(src, dst, cuda_stream);
   sbp_status st = check_pair(src, dst, true);
   if (st != SBP_OK) return st;
+  if (placement_k(src) != placement_k(dst)) return boxing_disjoint(src, dst, static_cast<cudaStream_t>(cuda_stream));
   Plan pl;
   st = make_plan(src, dst, &pl);
   if (st != SBP_OK) return st;
@@ -708,12 +640,10 @@ static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
 
 size_t sbp_boxing_host_workspace_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_host) {
   if (check_pair(src_host, dst_host, false) != SBP_OK) return 0;
-  const int k = placement_k(src_host);
+  const int ks = placement_k(src_host), kd = placement_k(dst_host);
   size_t total = 0;
-  for (int r = 0; r < k; ++r) {
-    total += align256((size_t)local_numel(src_host, r) * elem_size(src_host->dtype));
-    total += align256((size_t)local_numel(dst_host, r) * elem_size(dst_host->dtype));
-  }
+  for (int r = 0; r < ks; ++r) total += align256((size_t)local_numel(src_host, r) * elem_size(src_host->dtype));
+  for (int r = 0; r < kd; ++r) total += align256((size_t)local_numel(dst_host, r) * elem_size(dst_host->dtype));
   return total;
 }
 
@@ -726,17 +656,17 @@ sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, voi
     return fail(SBP_ERR_WORKSPACE, "device workspace of %zu bytes needed, %zu given", need, dev_ws_bytes);
   if (reinterpret_cast<uintptr_t>(dev_ws) % 256 != 0)
     return fail(SBP_ERR_ALIGNMENT, "device workspace must be 256-byte aligned");
-  const int k = placement_k(src_host);
+  const int ks = placement_k(src_host), kd = placement_k(dst_host);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   sbp_tensor s = *src_host, d = *dst_host;
   char* cur = static_cast<char*>(dev_ws);
   const int esz = elem_size(src_host->dtype), esz_dst = elem_size(dst_host->dtype);
-  for (int r = 0; r < k; ++r) {
+  for (int r = 0; r < ks; ++r) {
     s.local[r] = cur;
     cur += align256((size_t)local_numel(src_host, r) * esz);
   }
   // Destination replicas that alias on the host alias on the device as well.
-  for (int r = 0; r < k; ++r) {
+  for (int r = 0; r < kd; ++r) {
     d.local[r] = nullptr;
     for (int q = 0; q < r; ++q)
       if (dst_host->local[q] == dst_host->local[r]) d.local[r] = d.local[q];
@@ -745,13 +675,13 @@ sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, voi
       cur += align256((size_t)local_numel(dst_host, r) * esz_dst);
     }
   }
-  for (int r = 0; r < k; ++r) {
+  for (int r = 0; r < ks; ++r) {
     const size_t bytes = (size_t)local_numel(src_host, r) * esz;
     if (bytes) SBP_CUDA_TRY(cudaMemcpyAsync(s.local[r], src_host->local[r], bytes, cudaMemcpyHostToDevice, stream));
   }
   st = sbp_boxing(&s, &d, cuda_stream);
   if (st != SBP_OK) return st;
-  for (int r = 0; r < k; ++r) {
+  for (int r = 0; r < kd; ++r) {
     bool dup = false;
     for (int q = 0; q < r; ++q) dup = dup || dst_host->local[q] == dst_host->local[r];
     const size_t bytes = (size_t)local_numel(dst_host, r) * esz_dst;

@@ -117,7 +117,17 @@ def test_boxing_validation_happens_before_any_launch(lib):
     assert _status(boxing, src, _host_tensor((8, 9), f32, sbp.B, 2)) == "SBP_ERR_SHAPE"
     assert _status(boxing, src, _host_tensor((8, 8), bf16, sbp.S(1), 2)) == "SBP_ERR_DTYPE"   # only S -> B may cast
     assert _status(boxing, _host_tensor((8, 8), bf16, sbp.S(0), 2), _host_tensor((8, 8), f32, sbp.B, 2)) == "SBP_ERR_DTYPE"
-    assert _status(boxing, src, _host_tensor((8, 8), f32, sbp.B, 4)) == "SBP_ERR_INVALID_ARG"
+    # different shard counts on the two sides are the disjoint-placement transforms; what they refuse:
+    assert _status(boxing, src, _host_tensor((8, 8), bf16, sbp.B, 4)) == "SBP_ERR_UNSUPPORTED"   # cast + other placement
+    assert _status(boxing, src, _host_tensor((8, 8), f32, sbp.P_MAX, 4)) == "SBP_ERR_UNSUPPORTED"
+    assert _status(boxing, _host_tensor((8, 8), f32, sbp.P_MAX, 2),
+                   _host_tensor((8, 8), f32, sbp.P_MAX, 3)) == "SBP_ERR_UNSUPPORTED"             # zero is not neutral
+    assert _status(boxing, _host_tensor((8, 8), f32, sbp.P_MAX, 2),
+                   _host_tensor((8, 8), f32, sbp.P_SUM, 3)) == "SBP_ERR_UNSUPPORTED"
+    assert _status(boxing, _host_tensor((8, 8), i64, sbp.P_SUM, 2),
+                   _host_tensor((8, 8), i64, sbp.S(0), 3)) == "SBP_ERR_DTYPE"
+    two_axis = sbp.SbpTensor((8, 8), f32, (sbp.B, sbp.B), [torch.zeros(8, 8) for _ in range(4)], pshape=(2, 2))
+    assert _status(boxing, src, two_axis) == "SBP_ERR_INVALID_ARG"
     assert _status(boxing, src, _host_tensor((8, 8), f32, sbp.P_MAX, 2)) == "SBP_ERR_UNSUPPORTED"
     assert _status(boxing, _host_tensor((8, 8), f32, sbp.P_SUM, 2),
                    _host_tensor((8, 8), f32, sbp.P_MAX, 2)) == "SBP_ERR_UNSUPPORTED"

@@ -46,7 +46,8 @@ constexpr int kStageB = BK * BNH * 2;             // 16 KiB
 constexpr int kStageBytes = kStageA + kStageB;    // 32 KiB per CTA
 constexpr int kEpiWarps = 8;
 constexpr int kSlabBytes = 32 * 128;              // one epilogue slab: 32 rows x 128 bytes
-constexpr int kEpiBytes = kEpiWarps * 2 * kSlabBytes;
+constexpr int kEpiBufs = 2;                       // staging slabs per epilogue warp
+constexpr int kEpiBytes = kEpiWarps * kEpiBufs * kSlabBytes;
 constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024;   // + alignment slack
 constexpr int kThreadsTc = 32 * (2 + kEpiWarps);
 constexpr int kTmemCols = 512;
@@ -372,7 +373,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
     // ------------------------------------------------ epilogue (warps 2..9, both CTAs)
     const int q = warp & 3;                       // the 32 tensor-memory lanes this warp may read
     const int half = (warp - 2) >> 2;             // which 128 of the 256 columns
-    unsigned char* my_epi = epi + (warp - 2) * 2 * kSlabBytes;
+    unsigned char* my_epi = epi + (warp - 2) * kEpiBufs * kSlabBytes;
     const int cols_per_slab = p.out_f32 ? 32 : 64;
     const int nslabs = (BN / 2) / cols_per_slab;
     const unsigned acc_empty0[2] = {map_to_cta(smem_addr(&bar_acc_empty[0]), 0), map_to_cta(smem_addr(&bar_acc_empty[1]), 0)};
@@ -465,9 +466,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
           tmem_ld32(taddr + sl * cols_per_slab, v);
           if (!p.out_f32) tmem_ld32(taddr + sl * cols_per_slab + 32, v + 32);
           asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-          unsigned char* buf = my_epi + (slab_iter & 1) * kSlabBytes;
+          unsigned char* buf = my_epi + (slab_iter % kEpiBufs) * kSlabBytes;
           // the store that last used this buffer must have finished reading it
-          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kEpiBufs - 1) : "memory");
           __syncwarp();
           unsigned char* rowp = buf + lane * 128;
           if (p.out_f32) {

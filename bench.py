@@ -175,6 +175,15 @@ NCU_TRAFFIC = {
     "MLP GEMM1 (B,S(1))->S(1) + GeLU": 1030.4e6,
     "MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials": 915.3e6,
     "MLP GEMM2 fused (S(1),S(0))->B": 1752.0e6,
+    # profiles/extras_bf16_8192x8192_p4_and_embedding_fp32_4194304x128_batch16384_k8.md (full size)
+    "S(0)->P(sum) bf16 [8192,8192] k=4": 615.7e6,
+    "B->P(sum) bf16 [8192,8192] k=4": 611.4e6,
+    "S(0) fp32 -> B bf16 (cast fused into the gather) [8192,8192] k=4": 748.6e6,
+    "disjoint placements: S(0)[4] -> S(0)[8] bf16 [8192,8192]": 215.0e6,
+    "disjoint placements: S(0)[4] -> S(1)[8] bf16 [8192,8192]": 214.5e6,
+    "disjoint placements: S(0)[4] -> B[8] bf16 [8192,8192]": 1169.0e6,
+    "disjoint placements: P(sum)[4] -> S(0)[8] bf16 [8192,8192]": 616.7e6,
+    "disjoint placements: P(sum)[4] -> B[2] bf16 [8192,8192]": 749.7e6,
     # profiles/embedding_fused_fp32_4194304x128_batch16384_k8.md (quarter batch, scaled x 4)
     "embedding fused gather -> B (8 replicas written)": 7102.8e6,
 }
@@ -254,8 +263,13 @@ def _flush_l2(device):
     _FLUSH.fill_(1)
 
 
+OP_REPEATS = {"iters": None, "warmup": None}    # set by --op-iters / --op-warmup (profiling-sized runs)
+
+
 def time_op(fn, device, iters=10, warmup=3):
     """Average and best device time (ms) of fn(), L2 flushed between iterations."""
+    iters = OP_REPEATS["iters"] or iters
+    warmup = OP_REPEATS["warmup"] if OP_REPEATS["warmup"] is not None else warmup
     for _ in range(warmup):
         fn()
     torch.cuda.synchronize()
@@ -529,13 +543,17 @@ def parse():
     ap.add_argument("--ops", default="softmax,classifier,mlp,embedding,extras",
                     help="comma-separated operator sections to run: softmax, classifier, mlp, embedding, extras")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--op-iters", type=int, default=None, help="timed repeats per operator line (default 5-10)")
+    ap.add_argument("--op-warmup", type=int, default=None, help="warm-up repeats per operator line (default 3; >= 3 for a valid number)")
     ap.add_argument("--copy-engine", type=int, default=0)
     ap.add_argument("--emb-rows", type=int, default=1 << 24, help="embedding table rows (smaller = profiling-sized case)")
     ap.add_argument("--emb-batch", type=int, default=65536, help="embedding batch (x 26 fields)")
     ap.add_argument("--xent-rows", type=int, default=512, help="rows of the softmax / classifier sections")
     ap.add_argument("--rows", type=int, default=SWEEP_SHAPE[0],
                     help="rows of the logical sweep tensor (smaller = a profiling-sized case, not the benchmark)")
-    return ap.parse_args()
+    args = ap.parse_args()
+    OP_REPEATS["iters"], OP_REPEATS["warmup"] = args.op_iters, args.op_warmup
+    return args
 
 
 def reference_arm(args):

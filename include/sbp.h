@@ -171,6 +171,25 @@ sbp_status sbp_transfer_cost(sbp_sig src, sbp_sig dst, int32_t p1, int32_t p2, i
  */
 sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream);
 
+/* The part of a boxing op that ONE device of the destination placement executes: produces
+ * dst->local[dst_shard] and nothing else (Section 3.2: a boxing op stands for a collective; on
+ * real devices each member pulls what it needs from the others).  Same transforms, arithmetic
+ * and errors as sbp_boxing on one-axis placements (same or different shard counts); the k calls
+ * with dst_shard = 0..k-1 together write exactly what one sbp_boxing call writes.
+ *
+ *   src->local[*]          read: every source local tensor the transform needs for this shard must
+ *                          be readable from the current device -- device memory of this GPU, or a
+ *                          peer GPU's memory mapped into this process (plain loads cross NVLink;
+ *                          nothing in the library assumes the sources are local)
+ *   dst->local[dst_shard]  written, device memory of the current GPU; the other dst->local entries
+ *                          are not looked at and may be null
+ * Which source shards are read: S -> S / S -> B all that overlap the shard; P -> S / B all k
+ * partials; B -> S / B -> B / P -> P / S(i) -> S(i) only source shard dst_shard (dst_shard mod k(src)
+ * between different placements); S / B -> P(sum) the shard's own piece.  The caller orders the calls
+ * of different devices (sources complete before anyone reads them): a stream or host barrier,
+ * never a wait inside a kernel.  Two-axis placements: SBP_ERR_UNSUPPORTED. */
+sbp_status sbp_boxing_shard(const sbp_tensor* src, sbp_tensor* dst, int32_t dst_shard, void* cuda_stream);
+
 /* Same transform, but every local[] pointer of src_host and dst_host is a HOST pointer
  * (pinned memory recommended).  The source local tensors are copied to the device
  * workspace, transformed there and the destination local tensors copied back, all

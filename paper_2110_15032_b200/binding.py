@@ -90,6 +90,7 @@ def load_library():
     lib.sbp_matmul_infer.argtypes = [_Sig, _Sig, C.POINTER(_Sig)]
     lib.sbp_transfer_cost.argtypes = [_Sig, _Sig, C.c_int32, C.c_int32, C.c_int32, C.c_uint64, C.POINTER(C.c_uint64)]
     lib.sbp_boxing.argtypes = [T, T, C.c_void_p]
+    lib.sbp_boxing_shard.argtypes = [T, T, C.c_int32, C.c_void_p]
     lib.sbp_boxing_host_workspace_bytes.restype = C.c_size_t
     lib.sbp_boxing_host_workspace_bytes.argtypes = [T, T]
     lib.sbp_boxing_host.argtypes = [T, T, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -146,6 +147,8 @@ class SbpTensor:
         if n != self.k:
             raise ValueError("placement size differs from the number of local tensors")
         for t in self.locals:
+            if t is None:            # a local tensor another device holds (sbp_boxing_shard)
+                continue
             if not t.is_contiguous():
                 raise ValueError("local tensors must be contiguous")
             if t.dtype != dtype:
@@ -163,7 +166,7 @@ class SbpTensor:
             d.pshape[p] = v
             d.sbp[p] = self.sigs[p]._c()
         for r, t in enumerate(self.locals):
-            d.local[r] = t.data_ptr()
+            d.local[r] = t.data_ptr() if t is not None else None
         return d
 
 
@@ -238,6 +241,13 @@ def sbp_boxing_set_copy_engine(engine: int) -> None:
 def sbp_boxing(src: SbpTensor, dst: SbpTensor, stream=None) -> None:
     a, b = src._c(), dst._c()
     _check(load_library().sbp_boxing(C.byref(a), C.byref(b), _stream_ptr(stream)))
+
+
+def sbp_boxing_shard(src: SbpTensor, dst: SbpTensor, dst_shard: int, stream=None) -> None:
+    """Only destination local tensor `dst_shard` of the boxing op (what one device of the
+    destination placement executes); the other entries of dst.locals may be None."""
+    a, b = src._c(), dst._c()
+    _check(load_library().sbp_boxing_shard(C.byref(a), C.byref(b), int(dst_shard), _stream_ptr(stream)))
 
 
 def sbp_boxing_host_workspace_bytes(src_host: SbpTensor, dst_host: SbpTensor) -> int:

@@ -61,7 +61,8 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
   const long long col_tile = rem - row_tile * p.col_tiles;
 
   int s = t, d = t;
-  if (p.mode == MODE_PAIRS) { s = t / p.k; d = t - s * p.k; }
+  if (p.one_dst) { d = p.dst_shard; if (p.mode == MODE_DIAG) s = p.dst_shard; }
+  else if (p.mode == MODE_PAIRS) { s = t / p.k; d = t - s * p.k; }
   else if (p.mode == MODE_REDUCE_B) { s = 0; d = 0; }
 
   TaskGeom g;
@@ -165,13 +166,14 @@ struct ScatterParams {
   char* dst[SBP_MAX_K];
   long long own_lo[SBP_MAX_K], own_hi[SBP_MAX_K];   // in vectors, inside a row
   long long nrows, row_vecs, chunks_per_row, total_chunks;
+  int d0;                                           // first destination shard of the launch (grid.y counts from it)
 };
 
 constexpr int kScatterJ = 8;
 
 template <typename V>
 __global__ void __launch_bounds__(256) box_scatter_kernel(const __grid_constant__ ScatterParams p) {
-  const int d = blockIdx.y;
+  const int d = blockIdx.y + p.d0;
   const V* sp = reinterpret_cast<const V*>(p.src[d]);
   V* dp = reinterpret_cast<V*>(p.dst[d]);
   const long long lo = p.own_lo[d], hi = p.own_hi[d], w = hi - lo;
@@ -331,13 +333,15 @@ static void launch_v_f32(const Plan& pl, cudaStream_t st) {
 constexpr int kJCopy = 4;
 constexpr int kJReduce = 2;
 
-static sbp_status make_plan(const sbp_tensor* src, const sbp_tensor* dst, Plan* pl) {
+static sbp_status make_plan(const sbp_tensor* src, const sbp_tensor* dst, int dst_shard, Plan* pl) {
   const int k = placement_k(src);
   const sbp_sig ss = src->sbp[0], ds = dst->sbp[0];
   BoxParams& p = pl->p;
   p = BoxParams{};
   p.k = k;
   p.esz = elem_size(src->dtype);
+  p.one_dst = dst_shard >= 0 ? 1 : 0;
+  p.dst_shard = dst_shard >= 0 ? dst_shard : 0;
   const bool src_p = ss.kind == SBP_PARTIAL_SUM || ss.kind == SBP_PARTIAL_MAX;
   const bool dst_p = ds.kind == SBP_PARTIAL_SUM || ds.kind == SBP_PARTIAL_MAX;
 
@@ -408,7 +412,10 @@ static sbp_status make_plan(const sbp_tensor* src, const sbp_tensor* dst, Plan* 
 
   // distinct destination buffers for the one-read-many-writes modes
   p.n_dst = 0;
-  if (p.mode == MODE_GATHER || p.mode == MODE_REDUCE_B) {
+  if ((p.mode == MODE_GATHER || p.mode == MODE_REDUCE_B) && p.one_dst) {
+    p.n_dst = 1;
+    p.dst[0] = static_cast<char*>(dst->local[dst_shard]);
+  } else if (p.mode == MODE_GATHER || p.mode == MODE_REDUCE_B) {
     char* uniq[SBP_MAX_K];
     for (int r = 0; r < k; ++r) {
       bool seen = false;
@@ -433,6 +440,7 @@ static sbp_status make_plan(const sbp_tensor* src, const sbp_tensor* dst, Plan* 
   const long long row_tiles = std::max(1LL, (nseg_max + p.rows_per_tile - 1) / p.rows_per_tile);
   p.tiles_per_task = p.col_tiles * row_tiles;
   pl->ntasks = p.mode == MODE_PAIRS ? k * k : (p.mode == MODE_REDUCE_B ? 1 : k);
+  if (p.one_dst) pl->ntasks = (p.mode == MODE_PAIRS || p.mode == MODE_GATHER) ? k : 1;
   p.ntasks = pl->ntasks;
   pl->grid = p.tiles_per_task * pl->ntasks;
   if (pl->grid > 0x7fffffffLL) return fail(SBP_ERR_UNSUPPORTED, "tensor too large for one launch");
@@ -442,11 +450,19 @@ static sbp_status make_plan(const sbp_tensor* src, const sbp_tensor* dst, Plan* 
 // Bulk-copy engine (defined in boxing_bulk.cu); returns false when it does not apply.
 bool launch_bulk_copy(const BoxParams& p, int ntasks, cudaStream_t st);
 
-static sbp_status check_pair(const sbp_tensor* src, const sbp_tensor* dst, bool need_ptrs) {
+// dst_shard >= 0: only that destination local tensor is produced, the other dst pointers are not looked at.
+static sbp_status check_pair(const sbp_tensor* src, const sbp_tensor* dst, bool need_ptrs, int dst_shard = -1) {
   sbp_status st = check_tensor(src, "src", need_ptrs);
   if (st != SBP_OK) return st;
-  st = check_tensor(dst, "dst", need_ptrs);
+  st = check_tensor(dst, "dst", need_ptrs && dst_shard < 0);
   if (st != SBP_OK) return st;
+  if (dst_shard >= 0) {
+    if (dst->pdims != 1 || src->pdims != 1) return fail(SBP_ERR_UNSUPPORTED, "one-shard boxing needs one-axis placements");
+    if (dst_shard >= placement_k(dst)) return fail(SBP_ERR_INVALID_ARG, "dst_shard %d outside the placement of %d", dst_shard, placement_k(dst));
+    const void* ptr = dst->local[dst_shard];
+    if (!ptr && local_numel(dst, dst_shard) > 0) return fail(SBP_ERR_INVALID_ARG, "dst local tensor %d is null", dst_shard);
+    if (reinterpret_cast<uintptr_t>(ptr) % elem_size(dst->dtype) != 0) return fail(SBP_ERR_ALIGNMENT, "dst local tensor %d is misaligned", dst_shard);
+  }
   if (src->ndim != dst->ndim) return fail(SBP_ERR_SHAPE, "src and dst differ in rank");
   for (int d = 0; d < src->ndim; ++d)
     if (src->shape[d] != dst->shape[d]) return fail(SBP_ERR_SHAPE, "src and dst differ on axis %d", d);
@@ -464,7 +480,7 @@ static sbp_status check_pair(const sbp_tensor* src, const sbp_tensor* dst, bool 
 }
 
 // Different shard counts on the two sides (defined in boxing_disjoint.cu).
-sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, cudaStream_t stream);
+sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard, cudaStream_t stream);
 
 }  // namespace sbp
 
@@ -549,13 +565,13 @@ static sbp_status boxing_2d(const sbp_tensor* src, sbp_tensor* dst, void* cuda_s
   return SBP_OK;
 }
 
-sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream) {
-  if (src && dst && (src->pdims == 2 || dst->pdims == 2)) return boxing_2d(src, dst, cuda_stream);
-  sbp_status st = check_pair(src, dst, true);
+static sbp_status boxing_one_axis(const sbp_tensor* src, sbp_tensor* dst, int dst_shard, void* cuda_stream) {
+  sbp_status st = check_pair(src, dst, true, dst_shard);
   if (st != SBP_OK) return st;
-  if (placement_k(src) != placement_k(dst)) return boxing_disjoint(src, dst, static_cast<cudaStream_t>(cuda_stream));
+  if (placement_k(src) != placement_k(dst))
+    return boxing_disjoint(src, dst, dst_shard, static_cast<cudaStream_t>(cuda_stream));
   Plan pl;
-  st = make_plan(src, dst, &pl);
+  st = make_plan(src, dst, dst_shard, &pl);
   if (st != SBP_OK) return st;
   if (numel(src) == 0) return SBP_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
@@ -607,11 +623,13 @@ sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream)
         sp.own_hi[d] = d == 0 ? sp.row_vecs : 0;
       }
     }
+    const int ny = b.one_dst ? 1 : b.k;
+    sp.d0 = b.one_dst ? b.dst_shard : 0;
     switch (pl.vbytes) {
-      case 16: launch_scatter_v<uint4>(sp, b.k, stream); break;
-      case 8: launch_scatter_v<uint2>(sp, b.k, stream); break;
-      case 4: launch_scatter_v<uint32_t>(sp, b.k, stream); break;
-      default: launch_scatter_v<uint16_t>(sp, b.k, stream); break;
+      case 16: launch_scatter_v<uint4>(sp, ny, stream); break;
+      case 8: launch_scatter_v<uint2>(sp, ny, stream); break;
+      case 4: launch_scatter_v<uint32_t>(sp, ny, stream); break;
+      default: launch_scatter_v<uint16_t>(sp, ny, stream); break;
     }
     done = true;
   }
@@ -634,6 +652,16 @@ sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream)
   if (e != cudaSuccess) return cuda_fail(e, "boxing launch");
   count_launch();
   return SBP_OK;
+}
+
+sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream) {
+  if (src && dst && (src->pdims == 2 || dst->pdims == 2)) return boxing_2d(src, dst, cuda_stream);
+  return boxing_one_axis(src, dst, -1, cuda_stream);
+}
+
+sbp_status sbp_boxing_shard(const sbp_tensor* src, sbp_tensor* dst, int32_t dst_shard, void* cuda_stream) {
+  if (dst_shard < 0) return fail(SBP_ERR_INVALID_ARG, "dst_shard %d is negative", dst_shard);
+  return boxing_one_axis(src, dst, dst_shard, cuda_stream);
 }
 
 static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }

@@ -78,7 +78,8 @@ __device__ __forceinline__ BulkTile bulk_tile(const BulkParams& q, long long u) 
   const long long row_tile = rem / q.col_tiles, col_tile = rem - row_tile * q.col_tiles;
   g.s = t;
   g.d = t;
-  if (p.mode == MODE_PAIRS) { g.s = t / p.k; g.d = t - g.s * p.k; }
+  if (p.one_dst) { g.d = p.dst_shard; if (p.mode == MODE_DIAG) g.s = p.dst_shard; }
+  else if (p.mode == MODE_PAIRS) { g.s = t / p.k; g.d = t - g.s * p.k; }
   long long a0 = 0, la = p.Na, b0 = 0, lb = p.Nb;
   if (p.src_a) split_range(p.Na, p.k, g.s, (int64_t*)&a0, (int64_t*)&la);
   else if (p.dst_a) split_range(p.Na, p.k, g.d, (int64_t*)&a0, (int64_t*)&la);

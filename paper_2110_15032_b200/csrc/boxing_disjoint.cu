@@ -42,6 +42,7 @@ struct DisjointParams {
   int n_dst;                        // distinct replicas written by one task (DJ_TO_ALL, DJ_REDUCE_ALL)
   int red_by_dst;                   // DJ_REDUCE: sources d, d + kd, ... instead of 0 .. ks-1
   int n_pairs;                      // > 0: DJ_PAIRS tasks listed in pair_s / pair_d
+  int one_dst, dst_shard;           // one_dst: only the tasks that produce destination shard dst_shard
   int cv_log2, rows_per_tile, ntasks;
   unsigned char pair_s[kMaxPairs], pair_d[kMaxPairs];
 };
@@ -90,11 +91,12 @@ __global__ void __launch_bounds__(256, OP == OP_COPY ? 4 : 3) box_disjoint_kerne
   switch (p.mode) {
     case DJ_PAIRS:
       if (p.n_pairs > 0) { s = p.pair_s[t]; d = p.pair_d[t]; }
+      else if (p.one_dst) { s = t; d = p.dst_shard; }
       else { s = t / p.kd; d = t - s * p.kd; }
       break;
-    case DJ_FROM_REPLICA: d = t; s = t % p.ks; break;
+    case DJ_FROM_REPLICA: d = p.one_dst ? p.dst_shard : t; s = d % p.ks; break;
     case DJ_TO_ALL: s = t; break;
-    case DJ_REDUCE: d = t; break;
+    case DJ_REDUCE: d = p.one_dst ? p.dst_shard : t; break;
     default: break;
   }
 
@@ -204,7 +206,8 @@ static void launch_disjoint(const DisjointParams& p, int vbytes, long long grid,
 
 // src and dst have been validated by the caller (same logical shape and dtype, one-axis
 // placements, pointers present); ks != kd is the expected case but not required.
-sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, cudaStream_t stream) {
+// dst_shard >= 0: only that destination local tensor is produced (the other dst pointers may be null).
+sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard, cudaStream_t stream) {
   const int ks = placement_k(src), kd = placement_k(dst);
   const sbp_sig ss = src->sbp[0], ds = dst->sbp[0];
   const bool src_p = ss.kind == SBP_PARTIAL_SUM || ss.kind == SBP_PARTIAL_MAX;
@@ -215,6 +218,8 @@ sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, cudaStream_t 
 
   DisjointParams p{};
   p.ks = ks; p.kd = kd; p.esz = esz;
+  p.one_dst = dst_shard >= 0 ? 1 : 0;
+  p.dst_shard = dst_shard >= 0 ? dst_shard : 0;
   int op = OP_COPY;
   bool zero_first = false;
   if (src_p) {
@@ -302,6 +307,7 @@ sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, cudaStream_t 
           int64_t s0, sl, d0, dl;
           split_range(p.Nb, ks, s, &s0, &sl);
           split_range(p.Nb, kd, d, &d0, &dl);
+          if (p.one_dst && d != dst_shard) continue;
           if (std::max(s0, d0) < std::min(s0 + sl, d0 + dl)) {
             p.pair_s[p.n_pairs] = (unsigned char)s;
             p.pair_d[p.n_pairs] = (unsigned char)d;
@@ -309,18 +315,22 @@ sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, cudaStream_t 
           }
         }
       p.ntasks = p.n_pairs;
-      if (p.ntasks == 0) return SBP_OK;
     } else {
-      p.ntasks = ks * kd;
+      p.ntasks = p.one_dst ? ks : ks * kd;
     }
   } else if (p.mode == DJ_FROM_REPLICA || p.mode == DJ_REDUCE) {
-    p.ntasks = kd;
+    p.ntasks = p.one_dst ? 1 : kd;
   } else if (p.mode == DJ_TO_ALL) {
     p.ntasks = ss.kind == SBP_SPLIT ? ks : 1;
   } else {
     p.ntasks = 1;
   }
-  if (p.mode == DJ_TO_ALL || p.mode == DJ_REDUCE_ALL) {
+  bool copy_needed = p.ntasks > 0;
+  if ((p.mode == DJ_TO_ALL || p.mode == DJ_REDUCE_ALL) && p.one_dst) {
+    p.n_dst = 1;
+    if (zero_first) copy_needed = dst_shard == 0;   // B -> P(sum): only partial 0 receives the tensor
+    else p.dst[0] = static_cast<char*>(dst->local[dst_shard]);
+  } else if (p.mode == DJ_TO_ALL || p.mode == DJ_REDUCE_ALL) {
     const int n_out = zero_first ? 1 : kd;          // B -> P(sum) writes partial 0 only
     char* uniq[SBP_MAX_K];
     for (int r = 0; r < n_out; ++r) {
@@ -334,10 +344,12 @@ sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, cudaStream_t 
 
   if (zero_first) {
     for (int r = 0; r < kd; ++r) {
+      if (p.one_dst && r != dst_shard) continue;
       if (p.mode == DJ_TO_ALL && r == 0) continue;  // overwritten in full by the copy
       SBP_CUDA_TRY(cudaMemsetAsync(dst->local[r], 0, (size_t)numel(dst) * esz, stream));
     }
   }
+  if (!copy_needed) return SBP_OK;
 
   // tiling, sized by the largest cut any task can have
   auto max_cut = [&](long long n, bool by_src, bool by_dst) {

@@ -27,6 +27,7 @@ struct BoxParams {
   int cv_log2;                      // tile width in vectors, log2
   int rows_per_tile;
   int ntasks;                       // tasks of the transform; tiles are dealt task-fastest
+  int one_dst, dst_shard;           // one_dst: only the tasks that produce destination shard dst_shard
 };
 
 }  // namespace sbp

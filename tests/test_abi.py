@@ -126,6 +126,14 @@ def test_boxing_validation_happens_before_any_launch(lib):
                    _host_tensor((8, 8), f32, sbp.P_SUM, 3)) == "SBP_ERR_UNSUPPORTED"
     assert _status(boxing, _host_tensor((8, 8), i64, sbp.P_SUM, 2),
                    _host_tensor((8, 8), i64, sbp.S(0), 3)) == "SBP_ERR_DTYPE"
+    def shard(src_t, dst_t, d):
+        a, b = src_t._c(), dst_t._c()
+        binding._check(lib.sbp_boxing_shard(C.byref(a), C.byref(b), d, stream))
+
+    assert _status(shard, src, _host_tensor((8, 8), f32, sbp.B, 2), 2) == "SBP_ERR_INVALID_ARG"      # outside the placement
+    assert _status(shard, src, _host_tensor((8, 8), f32, sbp.B, 2), -1) == "SBP_ERR_INVALID_ARG"
+    assert _status(shard, src, sbp.SbpTensor((8, 8), f32, sbp.B, [None, None]), 1) == "SBP_ERR_INVALID_ARG"   # no buffer
+    assert _status(shard, src, _host_tensor((8, 8), f32, sbp.P_MAX, 2), 0) == "SBP_ERR_UNSUPPORTED"
     two_axis = sbp.SbpTensor((8, 8), f32, (sbp.B, sbp.B), [torch.zeros(8, 8) for _ in range(4)], pshape=(2, 2))
     assert _status(boxing, src, two_axis) == "SBP_ERR_INVALID_ARG"
     assert _status(boxing, src, _host_tensor((8, 8), f32, sbp.P_MAX, 2)) == "SBP_ERR_UNSUPPORTED"

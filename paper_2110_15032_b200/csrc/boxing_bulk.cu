@@ -1,6 +1,6 @@
 // Bulk-copy engine for the pure data-movement boxing transforms (S(i)->S(j), S(i)->B,
 // B->S(i)): the copy engine of the SM moves whole row segments global -> shared -> global
-// (cp.async.bulk), so no register file traffic and one issuing thread per CTA.
+// (cp.async.bulk), so no register file traffic; one warp per CTA issues the copies.
 //
 // A persistent grid of small CTAs walks the same (task, segment rows, column chunk) tiles
 // as the load/store kernel.  Each CTA owns a ring of kStages shared-memory buffers: the
@@ -22,6 +22,7 @@ __device__ int g_bulk_timeout_flag = 0;
 constexpr int kStages = 4;
 constexpr int kStageBytes = 16 * 1024;
 constexpr int kCtasPerSm = 3;
+constexpr int kStoreSlack = 1;         // store groups that may still be reading shared memory when the next load is issued
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
 struct BulkParams {
@@ -60,22 +61,23 @@ __device__ __forceinline__ bool mbar_wait(unsigned bar, unsigned parity) {
   }
 }
 
-// One tile of one task: which shards, which segments, where they sit on both sides.
+// One tile of one task: which shards, which segments, where they sit on both sides.  The fields
+// below `cb` belong to the task and are the same for all of its tiles.
 struct BulkTile {
-  int s, d;
   long long rows, bytes;      // segments in the tile, bytes of each segment piece
   long long seg0, cb;         // first segment, byte offset of the column chunk
+  int s, d;
+  long long nseg, seg_bytes;  // segments of the task, bytes of one segment
   long long la;
   long long Na_s, aoff_s, Nb_s, boff_s;
   long long Na_d, aoff_d, Nb_d, boff_d;
 };
 
-__device__ __forceinline__ BulkTile bulk_tile(const BulkParams& q, long long u) {
-  const BoxParams& p = q.b;
+constexpr int kTaskCache = 64;   // tasks whose geometry a CTA keeps in shared memory
+
+// The per-task part of a tile (several 64-bit divisions: worked out once per task, not per tile).
+__device__ __forceinline__ BulkTile bulk_task(const BoxParams& p, int t) {
   BulkTile g;
-  const long long rem = u / p.ntasks;            // task index varies fastest (see boxing.cu)
-  const int t = (int)(u - rem * p.ntasks);
-  const long long row_tile = rem / q.col_tiles, col_tile = rem - row_tile * q.col_tiles;
   g.s = t;
   g.d = t;
   if (p.one_dst) { g.d = p.dst_shard; if (p.mode == MODE_DIAG) g.s = p.dst_shard; }
@@ -85,16 +87,28 @@ __device__ __forceinline__ BulkTile bulk_tile(const BulkParams& q, long long u) 
   else if (p.dst_a) split_range(p.Na, p.k, g.d, (int64_t*)&a0, (int64_t*)&la);
   if (p.src_b) split_range(p.Nb, p.k, g.s, (int64_t*)&b0, (int64_t*)&lb);
   else if (p.dst_b) split_range(p.Nb, p.k, g.d, (int64_t*)&b0, (int64_t*)&lb);
-  const long long nseg = p.A * la * p.M, seg_bytes = lb * p.C * p.esz;
-  g.seg0 = row_tile * q.rows_per_tile;
-  g.cb = col_tile * q.chunk_bytes;
-  g.rows = nseg - g.seg0 < q.rows_per_tile ? nseg - g.seg0 : q.rows_per_tile;
-  g.bytes = seg_bytes - g.cb < q.chunk_bytes ? seg_bytes - g.cb : q.chunk_bytes;
+  g.nseg = p.A * la * p.M;
+  g.seg_bytes = lb * p.C * p.esz;
   g.la = la;
   g.Na_s = p.src_a ? la : p.Na;  g.aoff_s = p.src_a ? 0 : a0;
   g.Nb_s = p.src_b ? lb : p.Nb;  g.boff_s = p.src_b ? 0 : b0;
   g.Na_d = p.dst_a ? la : p.Na;  g.aoff_d = p.dst_a ? 0 : a0;
   g.Nb_d = p.dst_b ? lb : p.Nb;  g.boff_d = p.dst_b ? 0 : b0;
+  g.rows = g.bytes = g.seg0 = g.cb = 0;
+  return g;
+}
+
+// Tile number u (below 2^31, checked on the host): task index fastest, then column chunk, then rows.
+__device__ __forceinline__ BulkTile bulk_tile(const BulkParams& q, const BulkTile* task_cache, unsigned u) {
+  const BoxParams& p = q.b;
+  const unsigned ntasks = (unsigned)p.ntasks, col_tiles = (unsigned)q.col_tiles;
+  const unsigned rem = u / ntasks, t = u - rem * ntasks;
+  const unsigned row_tile = rem / col_tiles, col_tile = rem - row_tile * col_tiles;
+  BulkTile g = t < (unsigned)kTaskCache ? task_cache[t] : bulk_task(p, (int)t);
+  g.seg0 = (long long)row_tile * q.rows_per_tile;
+  g.cb = (long long)col_tile * q.chunk_bytes;
+  g.rows = g.nseg - g.seg0 < q.rows_per_tile ? g.nseg - g.seg0 : q.rows_per_tile;
+  g.bytes = g.seg_bytes - g.cb < q.chunk_bytes ? g.seg_bytes - g.cb : q.chunk_bytes;
   return g;
 }
 
@@ -116,32 +130,44 @@ __device__ __forceinline__ void seg_offsets(const BoxParams& p, const BulkTile& 
 __global__ void __launch_bounds__(32) box_bulk_kernel(const __grid_constant__ BulkParams q) {
   extern __shared__ __align__(128) unsigned char smem[];
   __shared__ __align__(8) unsigned long long bars[kStages];
-  if (threadIdx.x != 0) return;
+  __shared__ BulkTile tiles[kStages];          // geometry of the tile in each ring slot, computed once
+  __shared__ BulkTile task_cache[kTaskCache];  // per-task geometry
   const BoxParams& p = q.b;
+  const int lane = threadIdx.x;
 
-  for (int i = 0; i < kStages; ++i)
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[i])) : "memory");
-  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  if (lane == 0) {
+    for (int i = 0; i < kStages; ++i)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(&bars[i])) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  for (int t = lane; t < p.ntasks && t < kTaskCache; t += 32) task_cache[t] = bulk_task(p, t);
+  __syncwarp();
 
   const long long first = blockIdx.x, stride = gridDim.x;
   const long long n_mine = first < q.total_tiles ? (q.total_tiles - first + stride - 1) / stride : 0;
   bool timed_out = false;
 
-  // Loads of my tile number `it` into its ring slot: one bulk copy per segment.
+  // Loads of my tile number `it` into its ring slot: one bulk copy per segment, lane r issuing
+  // the copies of segments r, r + 32, ...  Lane 0 works out the tile and posts the byte count.
   auto issue_loads = [&](long long it) {
-    const BulkTile g = bulk_tile(q, first + it * stride);
     const int slot = (int)(it % kStages);
     const unsigned bar = smem_u32(&bars[slot]);
-    if (g.rows <= 0 || g.bytes <= 0) {   // tile outside an uneven shard: complete the phase empty
-      asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-      return;
+    if (lane == 0) {
+      const BulkTile t = bulk_tile(q, task_cache, (unsigned)(first + it * stride));
+      tiles[slot] = t;
+      if (t.rows <= 0 || t.bytes <= 0)           // tile outside an uneven shard: complete the phase empty
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+      else
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
+                     "r"((unsigned)(t.rows * t.bytes))
+                     : "memory");
     }
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar),
-                 "r"((unsigned)(g.rows * g.bytes))
-                 : "memory");
+    __syncwarp();
+    const BulkTile& g = tiles[slot];
+    if (g.rows <= 0 || g.bytes <= 0) return;
     unsigned char* buf = smem + (size_t)slot * kStageBytes;
-    for (long long r = 0; r < g.rows; ++r) {
+    for (long long r = lane; r < g.rows; r += 32) {
       long long so, dofs;
       seg_offsets(p, g, g.seg0 + r, &so, &dofs);
       asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -151,14 +177,15 @@ __global__ void __launch_bounds__(32) box_bulk_kernel(const __grid_constant__ Bu
     }
   };
 
-  // Stores of my tile number `it` out of its ring slot, once per destination replica.
+  // Stores of my tile number `it` out of its ring slot, once per destination replica; every lane
+  // commits its own (possibly empty) group so that the group counts of all lanes stay in step.
   auto issue_stores = [&](long long it) {
-    const BulkTile g = bulk_tile(q, first + it * stride);
     const int slot = (int)(it % kStages);
+    const BulkTile& g = tiles[slot];
     if (g.rows > 0 && g.bytes > 0) {
       unsigned char* buf = smem + (size_t)slot * kStageBytes;
       const int nd = p.mode == MODE_GATHER ? p.n_dst : 1;
-      for (long long r = 0; r < g.rows; ++r) {
+      for (long long r = lane; r < g.rows; r += 32) {
         long long so, dofs;
         seg_offsets(p, g, g.seg0 + r, &so, &dofs);
         for (int j = 0; j < nd; ++j) {
@@ -172,28 +199,33 @@ __global__ void __launch_bounds__(32) box_bulk_kernel(const __grid_constant__ Bu
     asm volatile("cp.async.bulk.commit_group;" ::: "memory");
   };
 
-  const long long prologue = n_mine < kStages - 1 ? n_mine : kStages - 1;
+  const long long prologue = n_mine < kStages - kStoreSlack ? n_mine : kStages - kStoreSlack;
   for (long long it = 0; it < prologue; ++it) issue_loads(it);
 
   for (long long it = 0; it < n_mine; ++it) {
     const int slot = (int)(it % kStages);
     const unsigned parity = (unsigned)((it / kStages) & 1);
-    if (!mbar_wait(smem_u32(&bars[slot]), parity)) {
+    // every lane observes the phase itself before it hands the buffer to its stores
+    const bool ok = mbar_wait(smem_u32(&bars[slot]), parity);
+    if (!__all_sync(0xffffffffu, ok)) {
       timed_out = true;
       break;
     }
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     issue_stores(it);
-    // The slot that tile it + kStages - 1 will use was last drained by tile it - 1:
-    // wait until every store group except the newest has finished reading shared memory.
-    const long long nxt = it + kStages - 1;
+    // The slot that tile it + kStages - kStoreSlack will use was last drained by tile
+    // it - kStoreSlack: every lane waits until all of its store groups except the newest
+    // kStoreSlack have finished reading shared memory, and the warp meets before anyone loads
+    // into that slot.
+    const long long nxt = it + kStages - kStoreSlack;
     if (nxt < n_mine) {
-      asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+      asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kStoreSlack) : "memory");
+      __syncwarp();
       issue_loads(nxt);
     }
   }
   asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-  if (timed_out) atomicExch(&g_bulk_timeout_flag, 1);
+  if (timed_out && lane == 0) atomicExch(&g_bulk_timeout_flag, 1);
 }
 
 bool launch_bulk_copy(const BoxParams& p, int ntasks, cudaStream_t st) {
@@ -217,7 +249,7 @@ bool launch_bulk_copy(const BoxParams& p, int ntasks, cudaStream_t st) {
   q.row_tiles = (nseg_max + q.rows_per_tile - 1) / q.rows_per_tile;
   q.tiles_per_task = q.col_tiles * q.row_tiles;
   q.total_tiles = q.tiles_per_task * ntasks;
-  if (q.total_tiles <= 0) return false;
+  if (q.total_tiles <= 0 || q.total_tiles > 0x7fffffffLL || q.col_tiles > 0x7fffffffLL) return false;
 
   // per device: SM count and the kernel's shared-memory opt-in
   static int sms_on_device[64] = {};

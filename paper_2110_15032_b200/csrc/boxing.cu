@@ -35,10 +35,10 @@ struct TaskGeom {
 
 __device__ __forceinline__ void task_geometry(const BoxParams& p, int s, int d, int vbytes, TaskGeom* g) {
   long long a0 = 0, la = p.Na, b0 = 0, lb = p.Nb;
-  if (p.src_a) split_range(p.Na, p.k, s, (int64_t*)&a0, (int64_t*)&la);
-  else if (p.dst_a) split_range(p.Na, p.k, d, (int64_t*)&a0, (int64_t*)&la);
-  if (p.src_b) split_range(p.Nb, p.k, s, (int64_t*)&b0, (int64_t*)&lb);
-  else if (p.dst_b) split_range(p.Nb, p.k, d, (int64_t*)&b0, (int64_t*)&lb);
+  if (p.src_a) split_range_pre(p.a_base, p.a_rem, s, &a0, &la);
+  else if (p.dst_a) split_range_pre(p.a_base, p.a_rem, d, &a0, &la);
+  if (p.src_b) split_range_pre(p.b_base, p.b_rem, s, &b0, &lb);
+  else if (p.dst_b) split_range_pre(p.b_base, p.b_rem, d, &b0, &lb);
   g->la = la;
   g->nseg = p.A * la * p.M;
   g->seg_vecs = lb * p.C * p.esz / vbytes;
@@ -52,13 +52,15 @@ __device__ __forceinline__ void task_geometry(const BoxParams& p, int s, int d, 
 // KT: compile-time number of source shards of a reduction (0 = read p.k at run time).
 template <typename V, int OP, int J, int KT>
 __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ BoxParams p) {
-  const long long u = blockIdx.x;
   // Task index varies fastest: CTAs that run together then touch the same rows of every shard
-  // (whole DRAM pages) instead of one column stripe of one shard.
-  const long long rem = u / p.ntasks;
-  const int t = (int)(u - rem * p.ntasks);
-  const long long row_tile = rem / p.col_tiles;
-  const long long col_tile = rem - row_tile * p.col_tiles;
+  // (whole DRAM pages) instead of one column stripe of one shard.  The grid is below 2^31 tiles,
+  // so this is 32-bit arithmetic.
+  const unsigned u = blockIdx.x;
+  const unsigned rem = u / (unsigned)p.ntasks;
+  const int t = (int)(u - rem * (unsigned)p.ntasks);
+  const unsigned row_tile_u = rem / (unsigned)p.col_tiles;
+  const long long row_tile = row_tile_u;
+  const long long col_tile = rem - row_tile_u * (unsigned)p.col_tiles;
 
   int s = t, d = t;
   if (p.one_dst) { d = p.dst_shard; if (p.mode == MODE_DIAG) s = p.dst_shard; }
@@ -403,6 +405,8 @@ static sbp_status make_plan(const sbp_tensor* src, const sbp_tensor* dst, int ds
     p.src_b = sa == hi;  p.dst_b = da == hi;
   }
 
+  p.a_base = p.Na / k;  p.a_rem = p.Na % k;
+  p.b_base = p.Nb / k;  p.b_rem = p.Nb % k;
   for (int r = 0; r < k; ++r) {
     p.src[r] = static_cast<const char*>(src->local[r]);
     p.dst[r] = static_cast<char*>(dst->local[r]);

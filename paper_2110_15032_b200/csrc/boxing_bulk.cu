@@ -83,10 +83,10 @@ __device__ __forceinline__ BulkTile bulk_task(const BoxParams& p, int t) {
   if (p.one_dst) { g.d = p.dst_shard; if (p.mode == MODE_DIAG) g.s = p.dst_shard; }
   else if (p.mode == MODE_PAIRS) { g.s = t / p.k; g.d = t - g.s * p.k; }
   long long a0 = 0, la = p.Na, b0 = 0, lb = p.Nb;
-  if (p.src_a) split_range(p.Na, p.k, g.s, (int64_t*)&a0, (int64_t*)&la);
-  else if (p.dst_a) split_range(p.Na, p.k, g.d, (int64_t*)&a0, (int64_t*)&la);
-  if (p.src_b) split_range(p.Nb, p.k, g.s, (int64_t*)&b0, (int64_t*)&lb);
-  else if (p.dst_b) split_range(p.Nb, p.k, g.d, (int64_t*)&b0, (int64_t*)&lb);
+  if (p.src_a) split_range_pre(p.a_base, p.a_rem, g.s, &a0, &la);
+  else if (p.dst_a) split_range_pre(p.a_base, p.a_rem, g.d, &a0, &la);
+  if (p.src_b) split_range_pre(p.b_base, p.b_rem, g.s, &b0, &lb);
+  else if (p.dst_b) split_range_pre(p.b_base, p.b_rem, g.d, &b0, &lb);
   g.nseg = p.A * la * p.M;
   g.seg_bytes = lb * p.C * p.esz;
   g.la = la;

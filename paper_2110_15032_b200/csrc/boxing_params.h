@@ -28,6 +28,13 @@ struct BoxParams {
   int rows_per_tile;
   int ntasks;                       // tasks of the transform; tiles are dealt task-fastest
   int one_dst, dst_shard;           // one_dst: only the tasks that produce destination shard dst_shard
+  long long a_base, a_rem, b_base, b_rem;   // Na / k, Na % k, Nb / k, Nb % k: the balanced split without a division
 };
+
+// Start and length of shard r's piece of an axis whose n / k and n % k are known.
+__host__ __device__ inline void split_range_pre(long long base, long long rem, int r, long long* start, long long* len) {
+  *len = base + (r < rem ? 1 : 0);
+  *start = r * base + (r < rem ? r : rem);
+}
 
 }  // namespace sbp

@@ -209,9 +209,10 @@ sbp_status sbp_check_device_errors(void);
  * stays fully usable. */
 sbp_status sbp_selftest_wait_timeout(uint32_t limit_ms, void* cuda_stream);
 
-/* Selects the copy engine of the pure data-movement transforms: 0 = choose (default),
- * 1 = 128-bit load/store kernel, 2 = bulk asynchronous copies staged through shared
- * memory (needs 16-byte aligned segments, else falls back to 1).  Process-wide. */
+/* Selects the copy engine of the pure data-movement transforms: 0 = choose (default; currently
+ * always the load/store kernel, the faster one on B200), 1 = 128-bit load/store kernel,
+ * 2 = bulk asynchronous copies staged through shared memory (needs 16-byte aligned segments
+ * of at least 512 bytes, else falls back to 1).  Process-wide. */
 void sbp_boxing_set_copy_engine(int32_t engine);
 
 /* ---------------------------------------------------------------- MatMul (Table 1)

@@ -45,6 +45,8 @@ struct DisjointParams {
   int one_dst, dst_shard;           // one_dst: only the tasks that produce destination shard dst_shard
   int cv_log2, rows_per_tile, ntasks;
   unsigned char pair_s[kMaxPairs], pair_d[kMaxPairs];
+  // quotient and remainder of each axis by each side's shard count: the balanced split without a division
+  long long a_base_s, a_rem_s, a_base_d, a_rem_d, b_base_s, b_rem_s, b_base_d, b_rem_d;
 };
 
 struct AxisCut {
@@ -53,21 +55,19 @@ struct AxisCut {
   long long n_d, off_d; // same for the destination
 };
 
-__device__ __forceinline__ AxisCut cut_axis(long long n, bool by_src, int ks, int s, bool by_dst, int kd, int d,
-                                            bool dst_full) {
+__device__ __forceinline__ AxisCut cut_axis(long long n, bool by_src, long long base_s, long long rem_s, int s, bool by_dst,
+                                            long long base_d, long long rem_d, int d, bool dst_full) {
   long long lo = 0, hi = n;
   AxisCut c;
   c.n_s = n; c.n_d = n;
   long long start_s = 0, start_d = 0;
   if (by_src) {
-    int64_t st, ln;
-    split_range(n, ks, s, &st, &ln);
+    const long long ln = base_s + (s < rem_s ? 1 : 0), st = s * base_s + (s < rem_s ? s : rem_s);
     lo = st; hi = st + ln;
     start_s = st; c.n_s = ln;
   }
   if (by_dst) {
-    int64_t st, ln;
-    split_range(n, kd, d, &st, &ln);
+    const long long ln = base_d + (d < rem_d ? 1 : 0), st = d * base_d + (d < rem_d ? d : rem_d);
     lo = lo > st ? lo : st;
     hi = hi < st + ln ? hi : st + ln;
     if (!dst_full) { start_d = st; c.n_d = ln; }
@@ -81,11 +81,12 @@ __device__ __forceinline__ AxisCut cut_axis(long long n, bool by_src, int ks, in
 template <typename V, int OP>
 __global__ void __launch_bounds__(256, OP == OP_COPY ? 4 : 3) box_disjoint_kernel(const __grid_constant__ DisjointParams p) {
   constexpr int J = OP == OP_COPY ? 4 : 2;
-  const long long u = blockIdx.x;
-  const long long rem = u / p.ntasks;            // task index varies fastest
-  const int t = (int)(u - rem * p.ntasks);
-  const long long row_tile = rem / p.col_tiles;
-  const long long col_tile = rem - row_tile * p.col_tiles;
+  const unsigned u = blockIdx.x;                 // the grid is below 2^31 tiles: 32-bit arithmetic
+  const unsigned rem = u / (unsigned)p.ntasks;   // task index varies fastest
+  const int t = (int)(u - rem * (unsigned)p.ntasks);
+  const unsigned row_tile_u = rem / (unsigned)p.col_tiles;
+  const long long row_tile = row_tile_u;
+  const long long col_tile = rem - row_tile_u * (unsigned)p.col_tiles;
 
   int s = 0, d = 0;
   switch (p.mode) {
@@ -100,8 +101,8 @@ __global__ void __launch_bounds__(256, OP == OP_COPY ? 4 : 3) box_disjoint_kerne
     default: break;
   }
 
-  const AxisCut ca = cut_axis(p.Na, p.src_a, p.ks, s, p.dst_a, p.kd, d, p.dst_full);
-  const AxisCut cb = cut_axis(p.Nb, p.src_b, p.ks, s, p.dst_b, p.kd, d, p.dst_full);
+  const AxisCut ca = cut_axis(p.Na, p.src_a, p.a_base_s, p.a_rem_s, s, p.dst_a, p.a_base_d, p.a_rem_d, d, p.dst_full);
+  const AxisCut cb = cut_axis(p.Nb, p.src_b, p.b_base_s, p.b_rem_s, s, p.dst_b, p.b_base_d, p.b_rem_d, d, p.dst_full);
   if (ca.len <= 0 || cb.len <= 0) return;
   const long long nseg = p.A * ca.len * p.M;
   const long long cs = p.C * p.esz;              // bytes per unit step of the Nb axis
@@ -275,6 +276,8 @@ sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard
     p.src_b = sa == hi;  p.dst_b = da == hi;
   }
   if (numel(src) == 0) return SBP_OK;
+  p.a_base_s = p.Na / ks;  p.a_rem_s = p.Na % ks;  p.a_base_d = p.Na / kd;  p.a_rem_d = p.Na % kd;
+  p.b_base_s = p.Nb / ks;  p.b_rem_s = p.Nb % ks;  p.b_base_d = p.Nb / kd;  p.b_rem_d = p.Nb % kd;
 
   for (int r = 0; r < ks; ++r) p.src[r] = static_cast<const char*>(src->local[r]);
   for (int r = 0; r < kd; ++r) p.dst[r] = static_cast<char*>(dst->local[r]);

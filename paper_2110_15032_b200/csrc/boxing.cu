@@ -157,6 +157,19 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
   }
 }
 
+// row = c / per_row and the remainder; 32-bit arithmetic whenever both fit (a 64-bit division
+// costs an order of magnitude more and sits in front of every chunk's loads).
+__device__ __forceinline__ void chunk_row(long long c, long long per_row, long long* row, long long* within) {
+  if (((unsigned long long)c | (unsigned long long)per_row) >> 32) {
+    *row = c / per_row;
+    *within = c - *row * per_row;
+  } else {
+    const unsigned r = (unsigned)c / (unsigned)per_row;
+    *row = r;
+    *within = (unsigned)c - r * (unsigned)per_row;
+  }
+}
+
 // ------------------------------------------------------------------ S(i)/B -> P(sum)
 //
 // Destination shard d has the full shape: the vectors [own_lo, own_hi) of every row come from
@@ -180,8 +193,9 @@ __global__ void __launch_bounds__(256) box_scatter_kernel(const __grid_constant_
   V* dp = reinterpret_cast<V*>(p.dst[d]);
   const long long lo = p.own_lo[d], hi = p.own_hi[d], w = hi - lo;
   for (long long c = blockIdx.x; c < p.total_chunks; c += gridDim.x) {
-    const long long row = c / p.chunks_per_row;
-    const long long col0 = (c - row * p.chunks_per_row) * (256 * kScatterJ) + threadIdx.x;
+    long long row, within;
+    chunk_row(c, p.chunks_per_row, &row, &within);
+    const long long col0 = within * (256 * kScatterJ) + threadIdx.x;
     V val[kScatterJ];
 #pragma unroll
     for (int j = 0; j < kScatterJ; ++j) {
@@ -227,8 +241,9 @@ __global__ void __launch_bounds__(256) box_gather_cast_kernel(const __grid_const
   const long long chunks_per_row = (w + 256 * J - 1) / (256 * J);
   const long long total = p.nrows * chunks_per_row;
   for (long long c = blockIdx.x; c < total; c += gridDim.x) {
-    const long long row = c / chunks_per_row;
-    const long long col0 = (c - row * chunks_per_row) * (256 * J) + threadIdx.x;
+    long long row, within;
+    chunk_row(c, chunks_per_row, &row, &within);
+    const long long col0 = within * (256 * J) + threadIdx.x;
     const float* sp = p.src[s] + (row * w) * EPV;
     float v[J][EPV];
 #pragma unroll

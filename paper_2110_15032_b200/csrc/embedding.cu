@@ -58,6 +58,22 @@ __device__ __forceinline__ int owner_of_row(long long id, long long base, long l
   return r;
 }
 
+// item = lookup * vpr + piece: a shift when vpr is a power of two, a 32-bit division when both
+// fit, a 64-bit division (an order of magnitude dearer) only otherwise.
+__device__ __forceinline__ void split_item(long long item, long long vpr, int vpr_log2, long long* look, long long* col) {
+  if (vpr_log2 >= 0) {
+    *look = item >> vpr_log2;
+    *col = item & (vpr - 1);
+  } else if (((unsigned long long)item | (unsigned long long)vpr) >> 32) {
+    *look = item / vpr;
+    *col = item - *look * vpr;
+  } else {
+    const unsigned q = (unsigned)item / (unsigned)vpr;
+    *look = q;
+    *col = (unsigned)item - q * (unsigned)vpr;
+  }
+}
+
 template <typename V>
 __device__ __forceinline__ V zero_vec() {
   V z;
@@ -97,13 +113,7 @@ __global__ void __launch_bounds__(256) embedding_kernel(const __grid_constant__ 
   for (int j = 0; j < J; ++j) {
     item[j] = base + j * stride;
     ok[j] = item[j] < total;
-    if (p.vpr_log2 >= 0) {
-      look[j] = item[j] >> p.vpr_log2;
-      col[j] = item[j] & (p.vpr - 1);
-    } else {
-      look[j] = item[j] / p.vpr;
-      col[j] = item[j] - look[j] * p.vpr;
-    }
+    split_item(item[j], p.vpr, p.vpr_log2, &look[j], &col[j]);
   }
 #pragma unroll
   for (int j = 0; j < J; ++j) id[j] = ok[j] ? __ldg(p.ids[shard] + look[j]) : 0;
@@ -162,6 +172,7 @@ struct EmbS1Params {
   char* out[SBP_MAX_K];
   long long vstart[SBP_MAX_K + 1];   // first vector of shard r's piece inside a full row
   long long rows, n_lookups, vpr_total;
+  int vpr_log2;                      // >= 0 when vpr_total is a power of two, else -1
   int k, n_dst;
   int* oob;
 };
@@ -178,8 +189,7 @@ __global__ void __launch_bounds__(256) embedding_s1_kernel(const __grid_constant
   for (int j = 0; j < J; ++j) {
     item[j] = base + j * stride;
     ok[j] = item[j] < total;
-    look[j] = item[j] / p.vpr_total;
-    col[j] = item[j] - look[j] * p.vpr_total;
+    split_item(item[j], p.vpr_total, p.vpr_log2, &look[j], &col[j]);
     int r = 0;
     while (r + 1 < p.k && col[j] >= p.vstart[r + 1]) ++r;
     shard[j] = r;
@@ -252,6 +262,9 @@ static sbp_status embedding_hidden_split(const sbp_tensor* table, const sbp_tens
   p.n_lookups = n_lookups;
   p.oob = oob_count;
   p.vpr_total = table->shape[1] * esz / vb;
+  p.vpr_log2 = -1;
+  for (int b = 0; b < 40; ++b)
+    if ((1LL << b) == p.vpr_total) p.vpr_log2 = b;
   for (int r = 0; r < k; ++r) {
     int64_t st, ln;
     split_range(table->shape[1], k, r, &st, &ln);

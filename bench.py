@@ -164,8 +164,8 @@ def run_sweep(sbp, work, events=None):
 # None = not captured for the kernel as it stands.
 NCU_TRAFFIC = {
     # profiles/box_kernels_sweep_bf16_8192x8192_k4.md (full size)
-    "P(sum)->B": 1017.8e6, "P(sum)->S(0)": 623.5e6, "P(sum)->S(1)": 620.1e6, "S(0)->B": 613.3e6,
-    "S(0)->S(1)": 215.5e6, "S(1)->S(0)": 215.0e6, "B->S(1)": 215.0e6,
+    "P(sum)->B": 1017.8e6, "P(sum)->S(0)": 624.8e6, "P(sum)->S(1)": 620.8e6, "S(0)->B": 613.6e6,
+    "S(0)->S(1)": 214.8e6, "S(1)->S(0)": 214.5e6, "B->S(1)": 213.6e6,
     # profiles/xent_partial_bf16_512x1048576_k8.md (full size)
     "softmax-xent on bf16 logits (partial + combine)": 1076.9e6,
     # profiles/matmul_tc_classifier_bf16_512x512x1048576_k8.md (full size)

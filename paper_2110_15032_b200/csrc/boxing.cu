@@ -147,13 +147,13 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
       V* dp = reinterpret_cast<V*>(p.dst[r]);
 #pragma unroll
       for (int j = 0; j < J; ++j)
-        if (ok[j]) dp[dofs[j]] = val[j];
+        if (ok[j]) st_stream(dp + dofs[j], val[j]);
     }
   } else {
     V* dp = reinterpret_cast<V*>(p.dst[d]);
 #pragma unroll
     for (int j = 0; j < J; ++j)
-      if (ok[j]) dp[dofs[j]] = val[j];
+      if (ok[j]) st_stream(dp + dofs[j], val[j]);
   }
 }
 

@@ -86,4 +86,15 @@ __device__ __forceinline__ uint4 ld_stream<uint4>(const uint4* p) {
   return r;
 }
 
+// Stores of results that this kernel never reads again: the 16-byte form is marked evict-first
+// so that the output stream does not push the inputs still to be read out of L2.
+template <typename V>
+__device__ __forceinline__ void st_stream(V* p, const V& v) {
+  *p = v;
+}
+template <>
+__device__ __forceinline__ void st_stream<uint4>(uint4* p, const uint4& v) {
+  __stcs(p, v);
+}
+
 }  // namespace sbp

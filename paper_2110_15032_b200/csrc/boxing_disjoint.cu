@@ -181,13 +181,13 @@ __global__ void __launch_bounds__(256, OP == OP_COPY ? 4 : 3) box_disjoint_kerne
       V* dp = reinterpret_cast<V*>(p.dst[r]);
 #pragma unroll
       for (int j = 0; j < J; ++j)
-        if (ok[j]) st_stream(dp + dofs[j], val[j]);
+        if (ok[j]) dp[dofs[j]] = val[j];
     }
   } else {
     V* dp = reinterpret_cast<V*>(p.dst[d]);
 #pragma unroll
     for (int j = 0; j < J; ++j)
-      if (ok[j]) st_stream(dp + dofs[j], val[j]);
+      if (ok[j]) dp[dofs[j]] = val[j];
   }
 }
 

@@ -411,7 +411,17 @@ def section_classifier_gemm(sbp, device, peaks, opts):
     nbytes2 = feat * classes * 2 + rows * feat * 2
     e2["hbm_gbs"] = nbytes2 / (avg * 1e-3) / 1e9
     e2["hbm_frac_measured"] = e2["hbm_gbs"] / peaks["hbm_gbs"]
-    return [e, e2]
+    # and its backward: the product recomputed, softmax - onehot written as bf16 S(1)
+    rmax = sbp.empty_global((rows,), torch.float32, sbp.B, k, device=device)
+    rsum = sbp.empty_global((rows,), torch.float32, sbp.B, k, device=device)
+    sbp.sbp_matmul_softmax_xent(f, w, lab, loss, rmax, rsum, ws2)
+    grad = sbp.empty_global((rows, classes), bf16, sbp.S(1), k, device=device)
+    avg, best = time_op(lambda: sbp.sbp_matmul_softmax_xent_backward(f, w, lab, rmax, rsum, grad), device, iters=5)
+    e3 = _tensor_entry("classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)",
+                       2.0 * rows * feat * classes, avg, best, peaks)
+    e3["hbm_gbs"] = nbytes / (avg * 1e-3) / 1e9
+    e3["hbm_frac_measured"] = e3["hbm_gbs"] / peaks["hbm_gbs"]
+    return [e, e2, e3]
 
 
 def section_extras(sbp, device, peaks, opts):

@@ -288,6 +288,17 @@ sbp_status sbp_matmul_softmax_xent(const sbp_tensor* features, const sbp_tensor*
                                    const sbp_tensor* labels, sbp_tensor* loss, sbp_tensor* row_max,
                                    sbp_tensor* row_sum, void* ws, size_t ws_bytes, void* cuda_stream);
 
+/* Backward of the fused classifier with respect to the logits, again without storing them: the
+ * product F W is recomputed on the tensor cores and the epilogue writes
+ *   grad[i, j] = exp(z_ij - m_i) / S_i - [j == label_i]
+ * (softmax minus one-hot, Section 6.3's plan read backwards) as S(1), BF16 or F32, from the forward
+ * pass's row_max (m) and row_sum (S), both [rows] B F32.  Same operand rules and
+ * SBP_ERR_UNSUPPORTED conditions as sbp_matmul_softmax_xent, plus 16-byte aligned result shards.
+ * The gradient feeds dW = F^T grad and dF = grad W^T, which this library does not compute. */
+sbp_status sbp_matmul_softmax_xent_backward(const sbp_tensor* features, const sbp_tensor* weight,
+                                            const sbp_tensor* labels, const sbp_tensor* row_max,
+                                            const sbp_tensor* row_sum, sbp_tensor* grad_logits, void* cuda_stream);
+
 /* Variant of sbp_softmax_xent for callers that have no device workspace to give and may not
  * create one.  (The paper has no counterpart; this exists for programs that embed the library
  * under constraints the paper does not discuss.)  Typical cases: a plug-in that runs inside

@@ -91,6 +91,7 @@ def load_library():
     lib.sbp_transfer_cost.argtypes = [_Sig, _Sig, C.c_int32, C.c_int32, C.c_int32, C.c_uint64, C.POINTER(C.c_uint64)]
     lib.sbp_boxing.argtypes = [T, T, C.c_void_p]
     lib.sbp_boxing_shard.argtypes = [T, T, C.c_int32, C.c_void_p]
+    lib.sbp_matmul_softmax_xent_backward.argtypes = [T, T, T, T, T, T, C.c_void_p]
     lib.sbp_boxing_host_workspace_bytes.restype = C.c_size_t
     lib.sbp_boxing_host_workspace_bytes.argtypes = [T, T]
     lib.sbp_boxing_host.argtypes = [T, T, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -306,6 +307,15 @@ def sbp_matmul_softmax_xent(features: SbpTensor, weight: SbpTensor, labels: SbpT
         C.byref(a), C.byref(b), C.byref(l), C.byref(c),
         C.byref(m) if m is not None else None, C.byref(s) if s is not None else None,
         C.c_void_p(ws.data_ptr()), ws.numel() * ws.element_size(), _stream_ptr(stream)))
+
+
+
+def sbp_matmul_softmax_xent_backward(features: SbpTensor, weight: SbpTensor, labels: SbpTensor, row_max: SbpTensor,
+                                     row_sum: SbpTensor, grad_logits: SbpTensor, stream=None) -> None:
+    """softmax(F W) - onehot written as S(1) without the logits ever being stored."""
+    a, w, l, m, s, g = (features._c(), weight._c(), labels._c(), row_max._c(), row_sum._c(), grad_logits._c())
+    _check(load_library().sbp_matmul_softmax_xent_backward(C.byref(a), C.byref(w), C.byref(l), C.byref(m), C.byref(s),
+                                                           C.byref(g), _stream_ptr(stream)))
 
 
 def sbp_softmax_xent_backward(logits: SbpTensor, labels: SbpTensor, row_max: SbpTensor, row_sum: SbpTensor,

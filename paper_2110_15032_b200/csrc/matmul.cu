@@ -423,4 +423,66 @@ sbp_status sbp_matmul_softmax_xent(const sbp_tensor* features, const sbp_tensor*
   return launch_xent_finish(xf.part_m, xf.part_s, xf.part_t, parts, rows, stage, loss, row_max, row_sum, k, stream);
 }
 
+sbp_status sbp_matmul_softmax_xent_backward(const sbp_tensor* features, const sbp_tensor* weight,
+                                            const sbp_tensor* labels, const sbp_tensor* row_max,
+                                            const sbp_tensor* row_sum, sbp_tensor* grad_logits, void* cuda_stream) {
+  sbp_status st = check_classifier(features, weight, true);
+  if (st != SBP_OK) return st;
+  const int k = placement_k(features);
+  const long long rows = features->shape[0], K = features->shape[1], N = weight->shape[1];
+  st = check_tensor(grad_logits, "grad_logits", true);
+  if (st != SBP_OK) return st;
+  if (grad_logits->ndim != 2 || grad_logits->shape[0] != rows || grad_logits->shape[1] != N)
+    return fail(SBP_ERR_SHAPE, "grad_logits must be [rows, classes]");
+  if (grad_logits->dtype != SBP_BF16 && grad_logits->dtype != SBP_F32)
+    return fail(SBP_ERR_DTYPE, "grad_logits must be BF16 or F32");
+  if (placement_k(grad_logits) != k || !is_s(grad_logits->sbp[0], 1))
+    return fail(SBP_ERR_SIGNATURE, "grad_logits must be S(1) on the operands' placement");
+  const sbp_tensor* vecs[3] = {labels, row_max, row_sum};
+  const char* names[3] = {"labels", "row_max", "row_sum"};
+  for (int i = 0; i < 3; ++i) {
+    st = check_tensor(vecs[i], names[i], true);
+    if (st != SBP_OK) return st;
+    if (vecs[i]->ndim != 1 || vecs[i]->shape[0] != rows) return fail(SBP_ERR_SHAPE, "%s must be [rows]", names[i]);
+    if (placement_k(vecs[i]) != k || !is_b(vecs[i]->sbp[0])) return fail(SBP_ERR_SIGNATURE, "%s must be B", names[i]);
+    if (vecs[i]->dtype != (i == 0 ? SBP_I64 : SBP_F32)) return fail(SBP_ERR_DTYPE, "%s has the wrong dtype", names[i]);
+  }
+  if (rows == 0) return SBP_OK;
+
+  MatmulPlan plan{};
+  plan.in_dtype = SBP_BF16;
+  plan.out_dtype = grad_logits->dtype;
+  plan.ngroups = k;
+  plan.nseg = k;
+  plan.chain = 0;
+  XentFusion xf{};
+  for (int r = 0; r < k; ++r) {
+    int64_t s0, ln;
+    split_range(N, k, r, &s0, &ln);
+    plan.a[r] = features->local[r];
+    plan.b[r] = weight->local[r];
+    plan.lda[r] = K;
+    plan.ldb[r] = ln;
+    plan.kseg[r] = K;
+    plan.m[r] = rows;
+    plan.n[r] = ln;
+    plan.ldy[r] = ln;
+    plan.y[r] = grad_logits->local[r];
+    xf.class_start[r] = s0;
+  }
+  xf.grad = 1;
+  xf.labels = static_cast<const long long*>(labels->local[0]);
+  xf.row_max = static_cast<const float*>(row_max->local[0]);
+  xf.row_sum = static_cast<const float*>(row_sum->local[0]);
+  xf.rows = rows;
+  bool taken = false;
+  st = launch_matmul_tc(plan, &xf, static_cast<cudaStream_t>(cuda_stream), &taken);
+  if (!taken)
+    return fail(SBP_ERR_UNSUPPORTED,
+                "the fused classifier backward needs the tensor-core path (16-byte aligned operands and result, feature "
+                "and per-shard class counts that are multiples of 8, a non-empty contraction); store the logits and use "
+                "sbp_softmax_xent_backward instead");
+  return st;
+}
+
 }  // extern "C"

@@ -46,6 +46,10 @@ struct XentFusion {
   long long class_start[SBP_MAX_K]; // first class of group g
   int part_base[SBP_MAX_K];         // first chunk index of group g
   long long rows;
+  // grad mode: the epilogue writes softmax - onehot of the recomputed logits instead of partials
+  int grad;
+  const float* row_max;             // [rows], from the forward pass
+  const float* row_sum;             // [rows]
 };
 
 }  // namespace sbp

@@ -32,6 +32,7 @@
 
 #include <algorithm>
 #include <mutex>
+#include <type_traits>
 
 #include "matmul_plan.h"
 #include "sbp_internal.h"
@@ -391,7 +392,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
       const long long Mg = p.m[tc.g], Ng = p.n[tc.g];
       const int row0 = tc.m0 + (int)rank * BMH + q * 32;
       const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * BN + half * (BN / 2);
-      if (p.xent) {
+      if (p.xent == 1) {
         // Softmax partials of this warp's 32 rows x 128 columns; one thread owns one row, so
         // nothing crosses lanes.  Columns are taken 32 at a time: batch max, then the running
         // (m, s) is rescaled and the batch's exponentials are added.
@@ -457,53 +458,83 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
             p.xf.part_t[slot] = t;
           }
         }
-      } else
-      for (int sl = 0; sl < nslabs; ++sl) {
-        const int col0 = tc.n0 + half * (BN / 2) + sl * cols_per_slab;
-        const bool live = row0 < Mg && col0 < Ng;   // warp-uniform
-        float v[64];
-        if (live) {
-          tmem_ld32(taddr + sl * cols_per_slab, v);
-          if (!p.out_f32) tmem_ld32(taddr + sl * cols_per_slab + 32, v + 32);
-          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-          unsigned char* buf = my_epi + (slab_iter % kEpiBufs) * kSlabBytes;
-          // the store that last used this buffer must have finished reading it
-          if (lane == 0) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kEpiBufs - 1) : "memory");
-          __syncwarp();
-          unsigned char* rowp = buf + lane * 128;
-          if (p.out_f32) {
-#pragma unroll
-            for (int c = 0; c < 8; ++c) {
-              float4 o;
-              o.x = v[4 * c + 0]; o.y = v[4 * c + 1]; o.z = v[4 * c + 2]; o.w = v[4 * c + 3];
-              if (p.gelu) { o.x = gelu_erf_tc(o.x); o.y = gelu_erf_tc(o.y); o.z = gelu_erf_tc(o.z); o.w = gelu_erf_tc(o.w); }
-              *reinterpret_cast<float4*>(rowp + ((c ^ (lane & 7)) << 4)) = o;
-            }
+      } else {
+      // The element-wise modes are compiled apart (MODE 0 plain, 1 GeLU, 2 softmax - onehot of the
+      // recomputed logits) so that the plain store, which the short-K classifier product leans
+      // on, carries none of the others' instructions.
+      float g_neg = 0.f, g_inv = 0.f;
+      long long g_lab = -1;
+      if (p.xent == 2 && row0 + lane < Mg) {      // this thread's row constants
+        const long long row = row0 + lane;
+        g_neg = -p.xf.row_max[row] * 1.4426950408889634f;
+        g_inv = 1.0f / p.xf.row_sum[row];
+        g_lab = p.xf.labels[row] - p.xf.class_start[tc.g];
+      }
+      auto slabs = [&](auto mode_tag) {
+        constexpr int MODE = decltype(mode_tag)::value;
+        auto xform = [&](float x, long long col) -> float {
+          if constexpr (MODE == 2) {
+            float e;
+            asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(x, 1.4426950408889634f, g_neg)));
+            e *= g_inv;
+            return col == g_lab ? e - 1.0f : e;
+          } else if constexpr (MODE == 1) {
+            return gelu_erf_tc(x);
           } else {
+            return x;
+          }
+        };
+        for (int sl = 0; sl < nslabs; ++sl) {
+          const int col0 = tc.n0 + half * (BN / 2) + sl * cols_per_slab;
+          const bool live = row0 < Mg && col0 < Ng;   // warp-uniform
+          float v[64];
+          if (live) {
+            tmem_ld32(taddr + sl * cols_per_slab, v);
+            if (!p.out_f32) tmem_ld32(taddr + sl * cols_per_slab + 32, v + 32);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            unsigned char* buf = my_epi + (slab_iter % kEpiBufs) * kSlabBytes;
+            // the store that last used this buffer must have finished reading it
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kEpiBufs - 1) : "memory");
+            __syncwarp();
+            unsigned char* rowp = buf + lane * 128;
+            if (p.out_f32) {
 #pragma unroll
-            for (int c = 0; c < 8; ++c) {
-              float f[8];
+              for (int c = 0; c < 8; ++c) {
+                float4 o;
+                o.x = xform(v[4 * c + 0], col0 + 4 * c + 0); o.y = xform(v[4 * c + 1], col0 + 4 * c + 1);
+                o.z = xform(v[4 * c + 2], col0 + 4 * c + 2); o.w = xform(v[4 * c + 3], col0 + 4 * c + 3);
+                *reinterpret_cast<float4*>(rowp + ((c ^ (lane & 7)) << 4)) = o;
+              }
+            } else {
 #pragma unroll
-              for (int e = 0; e < 8; ++e) f[e] = p.gelu ? gelu_erf_tc(v[8 * c + e]) : v[8 * c + e];
-              uint4 o;
-              __nv_bfloat162 h;
-              h = __floats2bfloat162_rn(f[0], f[1]); o.x = *reinterpret_cast<unsigned*>(&h);
-              h = __floats2bfloat162_rn(f[2], f[3]); o.y = *reinterpret_cast<unsigned*>(&h);
-              h = __floats2bfloat162_rn(f[4], f[5]); o.z = *reinterpret_cast<unsigned*>(&h);
-              h = __floats2bfloat162_rn(f[6], f[7]); o.w = *reinterpret_cast<unsigned*>(&h);
-              *reinterpret_cast<uint4*>(rowp + ((c ^ (lane & 7)) << 4)) = o;
+              for (int c = 0; c < 8; ++c) {
+                float f[8];
+#pragma unroll
+                for (int e = 0; e < 8; ++e) f[e] = xform(v[8 * c + e], col0 + 8 * c + e);
+                uint4 o;
+                __nv_bfloat162 h;
+                h = __floats2bfloat162_rn(f[0], f[1]); o.x = *reinterpret_cast<unsigned*>(&h);
+                h = __floats2bfloat162_rn(f[2], f[3]); o.y = *reinterpret_cast<unsigned*>(&h);
+                h = __floats2bfloat162_rn(f[4], f[5]); o.z = *reinterpret_cast<unsigned*>(&h);
+                h = __floats2bfloat162_rn(f[6], f[7]); o.w = *reinterpret_cast<unsigned*>(&h);
+                *reinterpret_cast<uint4*>(rowp + ((c ^ (lane & 7)) << 4)) = o;
+              }
             }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0) {
+              tma_store_2d(&p.map_y[tc.g], col0, row0, smem_addr(buf));
+              if (tc.g == 0)
+                for (int r = 0; r < p.n_rep; ++r) tma_store_2d(&p.map_rep[r], col0, row0, smem_addr(buf));
+              asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
+            ++slab_iter;
           }
-          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-          __syncwarp();
-          if (lane == 0) {
-            tma_store_2d(&p.map_y[tc.g], col0, row0, smem_addr(buf));
-            if (tc.g == 0)
-              for (int r = 0; r < p.n_rep; ++r) tma_store_2d(&p.map_rep[r], col0, row0, smem_addr(buf));
-            asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-          }
-          ++slab_iter;
         }
+      };
+      if (p.xent == 2) slabs(std::integral_constant<int, 2>{});
+      else if (p.gelu) slabs(std::integral_constant<int, 1>{});
+      else slabs(std::integral_constant<int, 0>{});
       }
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
@@ -564,6 +595,7 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
   *taken = false;
   if (plan.in_dtype != SBP_BF16) return SBP_ERR_UNSUPPORTED;
   const int oesz = plan.out_dtype == SBP_F32 ? 4 : 2;
+  const bool stores_y = !xf || xf->grad;      // the softmax-partials mode writes no product
 
   // the rules of the TMA path: 16-byte aligned bases, leading dimensions and column offsets
   for (int s = 0; s < plan.nseg; ++s) {
@@ -577,7 +609,7 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
   for (int s = 0; s < plan.nseg; ++s) ktotal_chain += plan.kseg[s];
   for (int g = 0; g < plan.ngroups; ++g) {
     if (plan.m[g] == 0 || plan.n[g] == 0) continue;
-    if (!xf && (!aligned16(plan.y[g]) || (plan.ldy[g] * oesz) % 16 != 0)) return SBP_ERR_UNSUPPORTED;
+    if (stores_y && (!aligned16(plan.y[g]) || (plan.ldy[g] * oesz) % 16 != 0)) return SBP_ERR_UNSUPPORTED;
     if (plan.col_off[g] % 8 != 0) return SBP_ERR_UNSUPPORTED;
     const long long kg = plan.chain ? ktotal_chain : plan.kseg[g];
     if (kg == 0) return SBP_ERR_UNSUPPORTED;   // an all-zero result: left to the FMA kernel
@@ -596,7 +628,7 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
   p.gelu = plan.gelu;
   p.n_rep = plan.n_rep;
   p.out_f32 = plan.out_dtype == SBP_F32;
-  p.xent = xf ? 1 : 0;
+  p.xent = xf ? (xf->grad ? 2 : 1) : 0;
   if (xf) p.xf = *xf;
 
   for (int s = 0; s < plan.nseg; ++s) {
@@ -633,7 +665,7 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
     if (plan.m[g] > 0 && plan.n[g] > 0) {
       if (tm * tn + tiles > 0x3fffffffLL) return SBP_ERR_UNSUPPORTED;
       tiles += (int)(tm * tn);
-      if (!xf && !make_map(&p.map_y[g], plan.y[g], oesz, plan.m[g], plan.n[g], plan.ldy[g], 32, box_cols))
+      if (stores_y && !make_map(&p.map_y[g], plan.y[g], oesz, plan.m[g], plan.n[g], plan.ldy[g], 32, box_cols))
         return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for the result of group %d", g);
     }
   }

@@ -428,6 +428,22 @@ def _fused_classifier_case(rows, feat, classes, k, seed, w_std=0.05, alias=False
         assert_close(to_np(t), S, 2e-2, 1e-3, "fused row_sum")
     # fp32 accumulation straight into the softmax: far tighter than the stated bar
     assert np.all(np.abs(to_np(loss.locals[0]) - ref) <= 1e-4 * np.maximum(np.abs(ref), 1.0))
+    # the backward, again without stored logits: softmax - onehot, S(1), in both result dtypes
+    want = O.to_locals(O.softmax_xent_grad(Z, labels.numpy()), O.S1, k)
+    for gdt in (BF16, F32):
+        grad = sbp.empty_global((rows, classes), gdt, sbp.S(1), k)
+        for t in grad.locals:
+            t.fill_(float("nan"))
+        sbp.sbp_matmul_softmax_xent_backward(f, w, lab, rmax, rsum, grad)
+        torch.cuda.synchronize()
+        sbp.sbp_check_device_errors()
+        for r in range(k):
+            assert tuple(grad.locals[r].shape) == tuple(want[r].shape)
+            assert_close(to_np(grad.locals[r]), want[r], 2e-2, 1e-3, f"fused grad shard {r}")
+        if gdt == F32:      # every row of softmax - onehot sums to zero; fp32 results are far tighter than the bar
+            full = O.from_locals([to_np(t).astype(np.float64) for t in grad.locals], O.S1)
+            assert np.all(np.abs(full.sum(axis=1)) <= 1e-3)
+            assert np.all(np.abs(full - O.softmax_xent_grad(Z, labels.numpy())) <= 1e-5)
     return to_np(loss.locals[0])
 
 

@@ -5,7 +5,8 @@
 //   partial kernel   one CTA per (row, shard, column chunk) streams its piece of the logits
 //                    once and leaves a local max m_p, a local exp-sum s_p = sum exp(z - m_p)
 //                    and the label's logit t_p (0 when the label lies elsewhere);
-//   combine kernel   per row, over the pieces p in fixed order (shard-major):
+//   combine kernel   per row, over the pieces p (one warp per row: the pieces of a lane in
+//                    ascending order, then the lanes by a butterfly):
 //                    m = max_p m_p            (the P(max) -> B boxing of the local maxima)
 //                    S = sum_p s_p exp(m_p-m) (the P(sum) -> B boxing, after rescaling)
 //                    loss = log S + m - sum_p t_p.
@@ -175,6 +176,9 @@ __global__ void __launch_bounds__(kThreads) xent_partial_kernel(const __grid_con
   const int part = shard * p.nsplit + split;
   const T* z = reinterpret_cast<const T*>(p.logits[shard]) + row * c_len + c0;
   const int tid = threadIdx.x;
+  // The kernel that combines the partials may be set up while this one runs; it waits for
+  // this grid to finish before it reads anything.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   float m = -INFINITY, s = 0.f;
   Chunk cur, nxt;
@@ -218,21 +222,36 @@ __global__ void __launch_bounds__(kThreads) xent_partial_kernel(const __grid_con
   }
 }
 
-__global__ void __launch_bounds__(128) xent_combine_kernel(const __grid_constant__ XentCombineParams p) {
-  const long long row = (long long)blockIdx.x * 128 + threadIdx.x;
+// One warp per row: lane j takes the parts j, j + 32, ... in ascending order, then the lanes
+// are merged by a butterfly -- a fixed tree for a given number of parts.
+constexpr int kCombineThreads = 256;
+
+__global__ void __launch_bounds__(kCombineThreads) xent_combine_kernel(const __grid_constant__ XentCombineParams p) {
+  // When launched as the programmatic dependent of the kernel that writes the partials, wait
+  // here until that grid has finished and its writes are visible (a no-op otherwise).
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  const long long row = (long long)blockIdx.x * (kCombineThreads / 32) + (threadIdx.x >> 5);
   if (row >= p.rows) return;
-  float m = -INFINITY;
-  for (int q = 0; q < p.parts; ++q) m = fmaxf(m, p.part_m[(long long)q * p.rows + row]);
-  float S = 0.f, zy = 0.f;
-  for (int q = 0; q < p.parts; ++q) {
-    const float mq = p.part_m[(long long)q * p.rows + row];
-    if (mq != -INFINITY) S += p.part_s[(long long)q * p.rows + row] * expf(mq - m);
-    zy += p.part_t[(long long)q * p.rows + row];
+  const int lane = threadIdx.x & 31;
+  float m = -INFINITY, S = 0.f, zy = 0.f;
+  for (int q = lane; q < p.parts; q += 32) {
+    const long long at = (long long)q * p.rows + row;
+    merge(m, S, p.part_m[at], p.part_s[at]);
+    zy += p.part_t[at];
   }
-  const float loss = logf(S) + m - zy;
-  for (int j = 0; j < p.n_loss; ++j) p.loss[j][row] = loss;
-  for (int j = 0; j < p.n_max; ++j) p.row_max[j][row] = m;
-  for (int j = 0; j < p.n_sum; ++j) p.row_sum[j][row] = S;
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float m2 = __shfl_xor_sync(0xffffffffu, m, off);
+    const float s2 = __shfl_xor_sync(0xffffffffu, S, off);
+    zy += __shfl_xor_sync(0xffffffffu, zy, off);
+    merge(m, S, m2, s2);
+  }
+  if (lane == 0) {
+    const float loss = logf(S) + m - zy;
+    for (int j = 0; j < p.n_loss; ++j) p.loss[j][row] = loss;
+    for (int j = 0; j < p.n_max; ++j) p.row_max[j][row] = m;
+    for (int j = 0; j < p.n_sum; ++j) p.row_sum[j][row] = S;
+  }
 }
 
 // Elements of one CTA's column span, and how many spans cover the widest shard.
@@ -383,7 +402,7 @@ sbp_status launch_xent_finish(float* part_m, float* part_s, float* part_t, int p
   c.n_loss = dedup(c.loss, loss, k);
   c.n_max = row_max ? dedup(c.row_max, row_max, k) : 0;
   c.n_sum = row_sum ? dedup(c.row_sum, row_sum, k) : 0;
-  xent_combine_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, st>>>(c);
+  xent_combine_kernel<<<(unsigned)((rows + kCombineThreads / 32 - 1) / (kCombineThreads / 32)), kCombineThreads, 0, st>>>(c);
   e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e, "softmax combine launch");
   count_launch(2);
@@ -512,8 +531,19 @@ sbp_status sbp_softmax_xent(const sbp_tensor* logits, const sbp_tensor* labels, 
   c.n_loss = dedup(c.loss, loss, k);
   c.n_max = row_max ? dedup(c.row_max, row_max, k) : 0;
   c.n_sum = row_sum ? dedup(c.row_sum, row_sum, k) : 0;
-  xent_combine_kernel<<<(unsigned)((rows + 127) / 128), 128, 0, stream>>>(c);
-  e = cudaGetLastError();
+  // Launched as the programmatic dependent of the partial kernel: it may be set up while that
+  // kernel still runs and waits, on the device, for it to finish before reading the partials.
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)((rows + kCombineThreads / 32 - 1) / (kCombineThreads / 32)));
+  cfg.blockDim = dim3(kCombineThreads);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  e = cudaLaunchKernelEx(&cfg, xent_combine_kernel, c);
   if (e != cudaSuccess) return cuda_fail(e, "softmax combine launch");
   count_launch(2);
   return SBP_OK;

@@ -167,7 +167,8 @@ NCU_TRAFFIC = {
     "P(sum)->B": 1017.8e6, "P(sum)->S(0)": 624.8e6, "P(sum)->S(1)": 620.8e6, "S(0)->B": 613.6e6,
     "S(0)->S(1)": 214.8e6, "S(1)->S(0)": 214.5e6, "B->S(1)": 213.6e6,
     # profiles/xent_partial_bf16_512x1048576_k8.md (full size)
-    "softmax-xent on bf16 logits (partial + combine)": 1076.9e6,
+    "softmax-xent on bf16 logits (partial + combine)": 1077.5e6,
+    "softmax-xent backward (softmax - onehot, S(1))": 2100.3e6,
     # profiles/matmul_tc_classifier_bf16_512x512x1048576_k8.md (full size)
     "classifier GEMM (B,S(1))->S(1), bf16 logits": 2105.2e6,
     "classifier GEMM fused with softmax-xent (no logits stored)": 1132.9e6 + 50.3e6,

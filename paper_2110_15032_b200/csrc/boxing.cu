@@ -55,6 +55,9 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
   // Task index varies fastest: CTAs that run together then touch the same rows of every shard
   // (whole DRAM pages) instead of one column stripe of one shard.  The grid is below 2^31 tiles,
   // so this is 32-bit arithmetic.
+  // Let the next kernel in the stream be set up while this one's last CTAs run; it waits, as
+  // this one does below, for its predecessor to finish before it touches global memory.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   const unsigned u = blockIdx.x;
   const unsigned rem = u / (unsigned)p.ntasks;
   const int t = (int)(u - rem * (unsigned)p.ntasks);
@@ -95,6 +98,8 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
     so[j] = ((((x * g.Na_s + g.aoff_s + ia) * p.M + m) * g.Nb_s + g.boff_s) * cs) / (long long)sizeof(V) + col;
     dofs[j] = ((((x * g.Na_d + g.aoff_d + ia) * p.M + m) * g.Nb_d + g.boff_d) * cs) / (long long)sizeof(V) + col;
   }
+
+  asm volatile("griddepcontrol.wait;" ::: "memory");   // the previous kernel's results are visible from here on
 
   V val[J];
   if constexpr (OP == OP_COPY) {
@@ -311,19 +316,38 @@ static int pick_vector_bytes(const BoxParams& p, const sbp_tensor* src, const sb
   return p.esz;
 }
 
+// Launch as a programmatic dependent of whatever kernel precedes it in the stream: if that
+// kernel releases its dependents early (the tile kernel does), this one's CTAs are set up while
+// the last CTAs of the other still run, and wait on the device (griddepcontrol.wait, before
+// their first access to global memory) until it has finished.  After any other kind of work
+// the launch behaves like a plain one.
+template <typename V, int OP, int J, int KT>
+static void launch_tile(const Plan& pl, cudaStream_t st) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)pl.grid);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cudaLaunchKernelEx(&cfg, box_tile_kernel<V, OP, J, KT>, pl.p);   // errors are picked up by the caller's cudaGetLastError
+}
+
 template <typename V, int OP, int J>
 static void launch_k(const Plan& pl, cudaStream_t st) {
-  dim3 grid((unsigned)pl.grid), block(256);
   if (OP == OP_COPY) {
-    box_tile_kernel<V, OP, J, 0><<<grid, block, 0, st>>>(pl.p);
+    launch_tile<V, OP, J, 0>(pl, st);
     return;
   }
   switch (pl.p.k) {
-    case 1: box_tile_kernel<V, OP, J, 1><<<grid, block, 0, st>>>(pl.p); break;
-    case 2: box_tile_kernel<V, OP, J, 2><<<grid, block, 0, st>>>(pl.p); break;
-    case 4: box_tile_kernel<V, OP, J, 4><<<grid, block, 0, st>>>(pl.p); break;
-    case 8: box_tile_kernel<V, OP, J, 8><<<grid, block, 0, st>>>(pl.p); break;
-    default: box_tile_kernel<V, OP, J, 0><<<grid, block, 0, st>>>(pl.p); break;
+    case 1: launch_tile<V, OP, J, 1>(pl, st); break;
+    case 2: launch_tile<V, OP, J, 2>(pl, st); break;
+    case 4: launch_tile<V, OP, J, 4>(pl, st); break;
+    case 8: launch_tile<V, OP, J, 8>(pl, st); break;
+    default: launch_tile<V, OP, J, 0>(pl, st); break;
   }
 }
 

@@ -291,6 +291,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
   cluster_sync_all();                            // both CTAs' barriers exist before anyone signals them
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const unsigned tmem_base = tmem_base_slot;
+  // A kernel launched behind this one as its programmatic dependent may be set up from here on;
+  // it waits on the device for this grid to finish before it reads what this grid writes.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int first = blockIdx.x >> 1, stride = gridDim.x >> 1;   // tiles are dealt to CTA pairs
 

@@ -326,12 +326,30 @@ __global__ void __launch_bounds__(256) xent_reduce_parts_kernel(const __grid_con
   const long long row = (long long)blockIdx.x * 32 + tx;
   const int lo = blockIdx.y * p.per_slice;
   const int hi = min(p.parts, lo + p.per_slice);
+  // The partials come from the kernel just before this one in the stream; when launched as its
+  // programmatic dependent, wait for it here (a no-op otherwise), and let the combine kernel
+  // that follows be set up meanwhile.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   float m = -INFINITY, s = 0.f, t = 0.f;
   if (row < p.rows) {
-    for (int q = lo + ty; q < hi; q += 8) {
-      const long long at = (long long)q * p.rows + row;
-      merge(m, s, p.in_m[at], p.in_s[at]);
-      t += p.in_t[at];
+    // four parts (stride 8) are loaded before they are merged, in ascending order
+    for (int q = lo + ty; q < hi; q += 32) {
+      float pm[4], ps[4], pt[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int qq = q + 8 * j;
+        const long long at = (long long)(qq < hi ? qq : q) * p.rows + row;
+        pm[j] = p.in_m[at];
+        ps[j] = p.in_s[at];
+        pt[j] = p.in_t[at];
+      }
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        if (q + 8 * j < hi) {
+          merge(m, s, pm[j], ps[j]);
+          t += pt[j];
+        }
     }
   }
   __shared__ float sm[8][33], ss[8][33], st[8][33];
@@ -390,8 +408,18 @@ sbp_status launch_xent_finish(float* part_m, float* part_s, float* part_t, int p
   r.rows = rows;
   r.parts = parts;
   r.per_slice = (parts + slices - 1) / slices;
-  xent_reduce_parts_kernel<<<dim3((unsigned)((rows + 31) / 32), (unsigned)slices), 256, 0, st>>>(r);
-  cudaError_t e = cudaGetLastError();
+  // Both kernels are launched as programmatic dependents of their predecessors in the stream.
+  cudaLaunchAttribute pdl[1];
+  pdl[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  pdl[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3((unsigned)((rows + 31) / 32), (unsigned)slices);
+  cfg.blockDim = dim3(256);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = st;
+  cfg.attrs = pdl;
+  cfg.numAttrs = 1;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, xent_reduce_parts_kernel, r);
   if (e != cudaSuccess) return cuda_fail(e, "softmax reduce launch");
   XentCombineParams c{};
   c.part_m = r.out_m;
@@ -402,8 +430,9 @@ sbp_status launch_xent_finish(float* part_m, float* part_s, float* part_t, int p
   c.n_loss = dedup(c.loss, loss, k);
   c.n_max = row_max ? dedup(c.row_max, row_max, k) : 0;
   c.n_sum = row_sum ? dedup(c.row_sum, row_sum, k) : 0;
-  xent_combine_kernel<<<(unsigned)((rows + kCombineThreads / 32 - 1) / (kCombineThreads / 32)), kCombineThreads, 0, st>>>(c);
-  e = cudaGetLastError();
+  cfg.gridDim = dim3((unsigned)((rows + kCombineThreads / 32 - 1) / (kCombineThreads / 32)));
+  cfg.blockDim = dim3(kCombineThreads);
+  e = cudaLaunchKernelEx(&cfg, xent_combine_kernel, c);
   if (e != cudaSuccess) return cuda_fail(e, "softmax combine launch");
   count_launch(2);
   return SBP_OK;

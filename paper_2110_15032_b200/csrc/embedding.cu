@@ -1,7 +1,8 @@
 // Row-split embedding lookup (Section 6.3: table S(0), "splitting the vocabulary IDs").
 //
-//   unfused: shard r writes out_r[l,:] = table_r[id_l - start_r,:] when id_l lies in its own
-//            row range and zeros otherwise; the k outputs form a P(sum) tensor.
+//   unfused: out_r[l,:] = table_r[id_l - start_r,:] when id_l lies in shard r's row range and
+//            zeros otherwise; the k outputs form a P(sum) tensor.  One pass over the lookups
+//            writes all k of them (row read once, k stores).
 //   fused:   the P(sum) -> B boxing folded into the gather.  Exactly one shard contributes
 //            to a lookup, so the sum over shards is that shard's row; the kernel finds the
 //            owning shard from the id, reads the row once and writes every B replica.
@@ -105,9 +106,14 @@ __global__ void __launch_bounds__(256) embedding_kernel(const __grid_constant__ 
   const long long total = p.n_lookups * p.vpr;
   const long long stride = (long long)gridDim.x * 256;
   const long long base = (long long)blockIdx.x * 256 + threadIdx.x;
-  const int shard = FUSED ? 0 : blockIdx.y;
+  // Both forms walk the lookups once and read every row once, from the shard that owns it.
+  // Fused: the row goes to every B replica.  Unfused: it goes to the owner's P(sum) output and
+  // zeros go to the others' -- the same k outputs as k devices looking up only their own rows.
+  // The ids are taken from replica 0 (the replicas of a B tensor are equal by definition).
+  const int shard = 0;
 
   long long item[J], look[J], col[J], id[J];
+  int own[J];
   bool ok[J];
 #pragma unroll
   for (int j = 0; j < J; ++j) {
@@ -122,6 +128,7 @@ __global__ void __launch_bounds__(256) embedding_kernel(const __grid_constant__ 
 #pragma unroll
   for (int j = 0; j < J; ++j) {
     val[j] = zero_vec<V>();
+    own[j] = -1;
     if (!ok[j]) continue;
     const bool in_table = id[j] >= 0 && id[j] < p.rows;
     if (!in_table) {
@@ -130,8 +137,8 @@ __global__ void __launch_bounds__(256) embedding_kernel(const __grid_constant__ 
     }
     long long start;
     const int r = owner_of_row(id[j], p.base, p.rem, p.big, p.narrow, &start);
-    if (FUSED || r == shard)
-      val[j] = __ldg(reinterpret_cast<const V*>(p.table[r]) + (id[j] - start) * p.vpr + col[j]);
+    own[j] = r;
+    val[j] = __ldg(reinterpret_cast<const V*>(p.table[r]) + (id[j] - start) * p.vpr + col[j]);
   }
 
   if (FUSED) {
@@ -142,10 +149,12 @@ __global__ void __launch_bounds__(256) embedding_kernel(const __grid_constant__ 
         if (ok[j]) o[item[j]] = p.canon_neg_zero ? canon<V, ESZ>(val[j]) : val[j];
     }
   } else {
-    V* o = reinterpret_cast<V*>(p.out[shard]);
+    for (int q = 0; q < p.k; ++q) {
+      V* o = reinterpret_cast<V*>(p.out[q]);
 #pragma unroll
-    for (int j = 0; j < J; ++j)
-      if (ok[j]) o[item[j]] = val[j];
+      for (int j = 0; j < J; ++j)
+        if (ok[j]) o[item[j]] = own[j] == q ? val[j] : zero_vec<V>();
+    }
   }
 }
 
@@ -158,7 +167,7 @@ static void launch_emb(const EmbParams& p, bool fused, cudaStream_t st) {
   if (fused) {
     embedding_kernel<V, ESZ, J, true><<<dim3((unsigned)blocks), 256, 0, st>>>(p);
   } else {
-    embedding_kernel<V, ESZ, J, false><<<dim3((unsigned)blocks, p.k), 256, 0, st>>>(p);
+    embedding_kernel<V, ESZ, J, false><<<dim3((unsigned)blocks), 256, 0, st>>>(p);
   }
 }
 

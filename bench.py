@@ -386,6 +386,25 @@ def section_mlp(sbp, device, peaks, opts):
     res.append(_hbm_entry("MLP P(sum)->B of the bf16 partials", 2 * k * M * H * 2, avg, best, peaks))
     avg, best = time_op(lambda: sbp.sbp_matmul(h, w2, y_b, 0, ws), device, iters=5)
     res.append(_tensor_entry("MLP GEMM2 fused (S(1),S(0))->B", flops, avg, best, peaks))
+    del h, y_p, y_b, w1, w2, x
+    # Backward products of a data-parallel layer of the same size (tokens S(0), weight B), taken
+    # from the stored operands with the transpose flags: dW = X^T dY is (S(1),S(0)) -> P(sum),
+    # written as S(0) (the gradient reduce-scatter folded in) or as B (the all-reduce folded in);
+    # dX = dY W^T is (S(0),B) -> S(0).
+    xs = sbp.SbpTensor((M, H), bf16, sbp.S(0), [dg.normal(1003, 50 + r, (M // k, H), 0.0, 1.0, bf16, device) for r in range(k)])
+    dy = sbp.SbpTensor((M, F), bf16, sbp.S(0), [dg.normal(1003, 60 + r, (M // k, F), 0.0, 1.0, bf16, device) for r in range(k)])
+    Wb = dg.normal(1003, 70, (H, F), 0.0, 0.02, bf16, device)
+    wb = sbp.SbpTensor((H, F), bf16, sbp.B, [Wb] * k)
+    dw_s = sbp.empty_global((H, F), bf16, sbp.S(0), k, device=device)
+    avg, best = time_op(lambda: sbp.sbp_matmul(xs, dy, dw_s, sbp.SBP_TRANS_X), device, iters=5)
+    res.append(_tensor_entry("DP layer backward dW = X^T dY, (S(1),S(0))->S(0) fused", flops, avg, best, peaks))
+    dw_b = sbp.empty_global((H, F), bf16, sbp.B, k, device=device)
+    avg, best = time_op(lambda: sbp.sbp_matmul(xs, dy, dw_b, sbp.SBP_TRANS_X), device, iters=5)
+    res.append(_tensor_entry("DP layer backward dW = X^T dY, (S(1),S(0))->B fused (8 replicas written)", flops, avg, best, peaks))
+    del dw_b
+    dx = sbp.empty_global((M, H), bf16, sbp.S(0), k, device=device)
+    avg, best = time_op(lambda: sbp.sbp_matmul(dy, wb, dx, sbp.SBP_TRANS_W), device, iters=5)
+    res.append(_tensor_entry("DP layer backward dX = dY W^T, (S(0),B)->S(0)", flops, avg, best, peaks))
     return res
 
 

@@ -235,11 +235,21 @@ void sbp_boxing_set_copy_engine(int32_t engine);
  * flags: SBP_EPILOGUE_GELU applies GeLU(v) = v/2 (1 + erf(v/sqrt 2)) to the fp32
  * accumulator before the store; only where Y is S or B (GeLU is not linear, so it cannot
  * be applied to partial values).
+ *        SBP_TRANS_X / SBP_TRANS_W: the descriptor x (w) holds the transpose of the operand,
+ * i.e. x is stored as [K,M] (w as [N,K]), logically and in every local tensor, and its
+ * signature refers to the stored axes.  The operand that enters Table 1 is the transpose, so a
+ * stored S(0) counts as S(1) and a stored S(1) as S(0); B and P(sum) are unchanged.  This is
+ * what the backward products of a layer need without a transposed copy: with Y = X W,
+ * dW = X^T dY (x = X with SBP_TRANS_X) and dX = dY W^T (w = W with SBP_TRANS_W).  Data
+ * parallelism (Section 3.1: X S(0), W B) then gives dW = (S(1), S(0)) -> P(sum), and asking
+ * for y as B folds the gradient all-reduce into the product.  One-axis placements only.
  * ws: scratch for the tensor-core path (see sbp_matmul_workspace_bytes; may be NULL when
  * that returns 0).
  */
 #define SBP_EPILOGUE_GELU 1u
-size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y);
+#define SBP_TRANS_X 2u
+#define SBP_TRANS_W 4u
+size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y);   /* untransposed operands */
 sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, uint32_t flags,
                       void* ws, size_t ws_bytes, void* cuda_stream);
 

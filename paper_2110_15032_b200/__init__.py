@@ -11,5 +11,5 @@ from .binding import (  # noqa: F401
     sbp_boxing, sbp_boxing_shard, sbp_boxing_host, sbp_boxing_host_workspace_bytes, sbp_boxing_set_copy_engine,
     sbp_check_device_errors, sbp_embedding, sbp_embedding_backward, sbp_launch_count, sbp_local_shape, sbp_matmul,
     sbp_matmul_infer, sbp_matmul_softmax_xent, sbp_matmul_softmax_xent_backward, sbp_matmul_softmax_xent_workspace_bytes, sbp_matmul_workspace_bytes, sbp_selftest_wait_timeout, sbp_softmax_xent,
-    sbp_softmax_xent_backward, sbp_transfer_cost, sbp_softmax_xent_static, sbp_softmax_xent_workspace_bytes, SBP_EPILOGUE_GELU,
+    sbp_softmax_xent_backward, sbp_transfer_cost, sbp_softmax_xent_static, sbp_softmax_xent_workspace_bytes, SBP_EPILOGUE_GELU, SBP_TRANS_X, SBP_TRANS_W,
 )

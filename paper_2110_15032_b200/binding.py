@@ -12,6 +12,8 @@ SBP_MAX_DIMS = 4
 SBP_MAX_K = 16
 SBP_MAX_PDIMS = 2
 SBP_EPILOGUE_GELU = 1
+SBP_TRANS_X = 2
+SBP_TRANS_W = 4
 
 SBP_SPLIT, SBP_BROADCAST, SBP_PARTIAL_SUM, SBP_PARTIAL_MAX = 0, 1, 2, 3
 _DTYPES = {torch.float32: 0, torch.bfloat16: 1, torch.int64: 2}

@@ -59,17 +59,34 @@ __global__ void __launch_bounds__(256) matmul_fma_kernel(const __grid_constant__
 
   const int s_lo = p.chain ? 0 : g, s_hi = p.chain ? p.nseg : g + 1;
   for (int s = s_lo; s < s_hi; ++s) {
-    const TI* A = static_cast<const TI*>(p.a[s]) + (p.row_off[g] + m0) * p.lda[s];
-    const TI* Bm = static_cast<const TI*>(p.b[s]) + p.col_off[g] + n0;
+    // element (row, kk) of the A tile and (kk, col) of the B tile, whichever way they are stored
+    const TI* A = static_cast<const TI*>(p.a[s]) + (p.a_trans ? p.row_off[g] + m0 : (p.row_off[g] + m0) * p.lda[s]);
+    const TI* Bm = static_cast<const TI*>(p.b[s]) + (p.b_trans ? (p.col_off[g] + n0) * p.ldb[s] : p.col_off[g] + n0);
+    const long long a_rs = p.a_trans ? 1 : p.lda[s], a_ks = p.a_trans ? p.lda[s] : 1;
+    const long long b_ks = p.b_trans ? 1 : p.ldb[s], b_cs = p.b_trans ? p.ldb[s] : 1;
     const long long K = p.kseg[s];
     for (long long k0 = 0; k0 < K; k0 += BK) {
-      for (int e = threadIdx.x; e < BM * BK; e += 256) {
-        const int r = e / BK, c = e % BK;
-        As[c][r] = (m0 + r < M && k0 + c < K) ? ld_f32<TI>(A + (long long)r * p.lda[s] + k0 + c) : 0.f;
+      if (p.a_trans) {
+        for (int e = threadIdx.x; e < BM * BK; e += 256) {
+          const int c = e / BM, r = e % BM;   // consecutive threads walk the stored rows
+          As[c][r] = (m0 + r < M && k0 + c < K) ? ld_f32<TI>(A + r * a_rs + (k0 + c) * a_ks) : 0.f;
+        }
+      } else {
+        for (int e = threadIdx.x; e < BM * BK; e += 256) {
+          const int r = e / BK, c = e % BK;
+          As[c][r] = (m0 + r < M && k0 + c < K) ? ld_f32<TI>(A + r * a_rs + (k0 + c) * a_ks) : 0.f;
+        }
       }
-      for (int e = threadIdx.x; e < BK * BN; e += 256) {
-        const int r = e / BN, c = e % BN;
-        Bs[r][c] = (k0 + r < K && n0 + c < N) ? ld_f32<TI>(Bm + (k0 + r) * p.ldb[s] + c) : 0.f;
+      if (p.b_trans) {
+        for (int e = threadIdx.x; e < BK * BN; e += 256) {
+          const int c = e / BK, r = e % BK;
+          Bs[r][c] = (k0 + r < K && n0 + c < N) ? ld_f32<TI>(Bm + (k0 + r) * b_ks + c * b_cs) : 0.f;
+        }
+      } else {
+        for (int e = threadIdx.x; e < BK * BN; e += 256) {
+          const int r = e / BN, c = e % BN;
+          Bs[r][c] = (k0 + r < K && n0 + c < N) ? ld_f32<TI>(Bm + (k0 + r) * b_ks + c * b_cs) : 0.f;
+        }
       }
       __syncthreads();
 #pragma unroll
@@ -142,8 +159,12 @@ static sbp_status build_plan(const sbp_tensor* x, const sbp_tensor* w, const sbp
   st = check_tensor(y, "y", need_ptrs);
   if (st != SBP_OK) return st;
   if (x->ndim != 2 || w->ndim != 2 || y->ndim != 2) return fail(SBP_ERR_SHAPE, "x, w and y must be 2-D");
-  const long long M = x->shape[0], K = x->shape[1], N = w->shape[1];
-  if (w->shape[0] != K) return fail(SBP_ERR_SHAPE, "x is [%lld,%lld] but w has %lld rows", M, K, (long long)w->shape[0]);
+  if (flags & ~(SBP_EPILOGUE_GELU | SBP_TRANS_X | SBP_TRANS_W)) return fail(SBP_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
+  const bool tx = (flags & SBP_TRANS_X) != 0, tw = (flags & SBP_TRANS_W) != 0;
+  // the operands as they enter the product: [M,K] and [K,N]
+  const long long M = x->shape[tx ? 1 : 0], K = x->shape[tx ? 0 : 1], N = w->shape[tw ? 0 : 1];
+  if (w->shape[tw ? 1 : 0] != K)
+    return fail(SBP_ERR_SHAPE, "x is [%lld,%lld] but w has %lld rows", M, K, (long long)w->shape[tw ? 1 : 0]);
   if (y->shape[0] != M || y->shape[1] != N) return fail(SBP_ERR_SHAPE, "y must be [%lld,%lld]", M, N);
   if (x->dtype != w->dtype) return fail(SBP_ERR_DTYPE, "x and w differ in dtype");
   if (x->dtype != SBP_F32 && x->dtype != SBP_BF16) return fail(SBP_ERR_DTYPE, "operands must be F32 or BF16");
@@ -152,7 +173,12 @@ static sbp_status build_plan(const sbp_tensor* x, const sbp_tensor* w, const sbp
   const int k = placement_k(x);
   if (placement_k(w) != k || placement_k(y) != k) return fail(SBP_ERR_INVALID_ARG, "operands differ in k");
 
-  const sbp_sig xs = x->sbp[0], ws = w->sbp[0], ys = y->sbp[0];
+  // signature of the operand that enters Table 1: a transposed operand swaps S(0) and S(1)
+  auto effective = [](sbp_sig s, bool t) {
+    if (t && s.kind == SBP_SPLIT) s.axis = 1 - s.axis;
+    return s;
+  };
+  const sbp_sig xs = effective(x->sbp[0], tx), ws = effective(w->sbp[0], tw), ys = y->sbp[0];
   sbp_sig natural;
   st = sbp_matmul_infer(xs, ws, &natural);
   if (st != SBP_OK) return st;
@@ -163,11 +189,12 @@ static sbp_status build_plan(const sbp_tensor* x, const sbp_tensor* w, const sbp
     return fail(SBP_ERR_SIGNATURE, "a P(sum) product can be written directly only as B or S(i)");
   if ((flags & SBP_EPILOGUE_GELU) && is_p(natural) && !fused)
     return fail(SBP_ERR_SIGNATURE, "GeLU is not linear: it cannot be applied to partial values");
-  if (flags & ~SBP_EPILOGUE_GELU) return fail(SBP_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
 
   MatmulPlan& p = *plan;
   p = MatmulPlan{};
   p.gelu = (flags & SBP_EPILOGUE_GELU) ? 1 : 0;
+  p.a_trans = tx ? 1 : 0;
+  p.b_trans = tw ? 1 : 0;
   p.in_dtype = x->dtype;
   p.out_dtype = y->dtype;
 
@@ -182,11 +209,14 @@ static sbp_status build_plan(const sbp_tensor* x, const sbp_tensor* w, const sbp
     long long st_, ln;
     p.a[r] = x->local[r];
     p.b[r] = w->local[r];
-    p.lda[r] = K;
-    p.ldb[r] = N;
+    // leading dimensions of the stored local tensors: their last axis, M or K for x, K or N for w
+    p.lda[r] = tx ? M : K;
+    p.ldb[r] = tw ? K : N;
     p.kseg[r] = K;
-    if (is_s(xs, 1)) { range(K, r, &st_, &ln); p.lda[r] = ln; p.kseg[r] = ln; }
-    if (is_s(ws, 1)) { range(N, r, &st_, &ln); p.ldb[r] = ln; }
+    if (is_s(xs, 1)) { range(K, r, &st_, &ln); p.kseg[r] = ln; if (!tx) p.lda[r] = ln; }
+    if (is_s(xs, 0) && tx) { range(M, r, &st_, &ln); p.lda[r] = ln; }
+    if (is_s(ws, 1) && !tw) { range(N, r, &st_, &ln); p.ldb[r] = ln; }
+    if (is_s(ws, 0) && tw) { range(K, r, &st_, &ln); p.ldb[r] = ln; }
   }
   p.nseg = k;
 
@@ -261,6 +291,7 @@ static sbp_status build_plan_2d(const sbp_tensor* x, const sbp_tensor* w, const 
   if (x->dtype != SBP_F32 && x->dtype != SBP_BF16) return fail(SBP_ERR_DTYPE, "operands must be F32 or BF16");
   if (y->dtype != SBP_F32 && y->dtype != SBP_BF16) return fail(SBP_ERR_DTYPE, "y must be F32 or BF16");
   if (x->dtype == SBP_F32 && y->dtype != SBP_F32) return fail(SBP_ERR_DTYPE, "F32 operands need an F32 result");
+  if (flags & (SBP_TRANS_X | SBP_TRANS_W)) return fail(SBP_ERR_UNSUPPORTED, "transposed operands on a two-axis placement");
   if (flags & ~SBP_EPILOGUE_GELU) return fail(SBP_ERR_INVALID_ARG, "unknown flags 0x%x", flags);
   for (int p = 0; p < 2; ++p) {
     sbp_sig natural;

@@ -6,6 +6,7 @@
 //
 //   Y_g[M_g, N_g] = sum_{s in segs(g)}  A_s[row_off_g : row_off_g + M_g, 0 : K_s]
 //                                     * B_s[0 : K_s, col_off_g : col_off_g + N_g]
+// (A_s and B_s may each be stored transposed, see a_trans / b_trans)
 //
 //   unfused (chain == 0): segs(g) = {g}       one local product per shard
 //   fused   (chain == 1): segs(g) = {0..nseg-1}  the partial products of all shards are
@@ -30,6 +31,9 @@ struct MatmulPlan {
   void* y_rep[SBP_MAX_K];
   int n_rep;
   int ngroups, nseg, chain;
+  // a_trans: A_s is stored transposed, A_s[row, kk] = a[kk * lda + row]; b_trans: B_s[kk, col] =
+  // b[col * ldb + kk].  lda / ldb are always the leading dimensions of the stored arrays.
+  int a_trans, b_trans;
   int gelu;
   int in_dtype, out_dtype;   // sbp_dtype
 };

@@ -67,6 +67,7 @@ struct TcParams {
   int tiles_m[SBP_MAX_K];
   int tiles_n[SBP_MAX_K];
   int ngroups, nseg, chain, gelu, n_rep;
+  int a_trans, b_trans;         // operand stored transposed (see MatmulPlan)
   int out_f32;
   int total_tiles;
   int xent;                     // 1: softmax partials instead of stored logits
@@ -208,9 +209,14 @@ __device__ __forceinline__ unsigned long long smem_desc(unsigned addr, unsigned 
   return d;
 }
 
-// Instruction descriptor: D fp32, A and B bf16, A K-major, B N-major, M = 256 (pair), N = 256.
-constexpr unsigned kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((BN >> 3) << 17) |
-                            ((BM >> 4) << 24);
+// Instruction descriptor: D fp32, A and B bf16, M = 256 (pair), N = 256.  Bit 15 / bit 16 say
+// that A / B lies in shared memory with its M / N index contiguous ("MN-major") instead of its
+// K index.  Operands as given: A [M,K] row-major is K-major, B [K,N] row-major is N-major; a
+// transposed operand is the other way round.
+constexpr unsigned kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((BN >> 3) << 17) | ((BM >> 4) << 24);
+__device__ __forceinline__ unsigned make_idesc(int a_trans, int b_trans) {
+  return kIdescBase | ((a_trans ? 1u : 0u) << 15) | ((b_trans ? 0u : 1u) << 16);
+}
 
 // erf by the rational approximation 7.1.26 of Abramowitz & Stegun (|error| <= 1.5e-7), which is
 // far below the rounding of the bf16 / fp32 store that follows and costs two special-function
@@ -313,11 +319,22 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
             if (rank == 0) mbar_expect_tx(smem_addr(&bar_full[slot]), 2 * kStageBytes);
             unsigned char* sa = smem + slot * kStageBytes;
             unsigned char* sb = sa + kStageA;
-            tma_load_2d(smem_addr(sa), &p.map_a[s], kb * BK, (int)p.row_off[tc.g] + tc.m0 + (int)rank * BMH, full0);
+            const int arow = (int)p.row_off[tc.g] + tc.m0 + (int)rank * BMH;
+            const int bcol = (int)p.col_off[tc.g] + tc.n0 + (int)rank * BNH;
+            if (!p.a_trans) {   // [rows, K] in memory: one box of 128 rows x 64 K
+              tma_load_2d(smem_addr(sa), &p.map_a[s], kb * BK, arow, full0);
+            } else {            // [K, rows] in memory: two boxes of 64 K x 64 rows
 #pragma unroll
-            for (int c = 0; c < BNH / 64; ++c)
-              tma_load_2d(smem_addr(sb + c * (BK * 128)), &p.map_b[s],
-                          (int)p.col_off[tc.g] + tc.n0 + (int)rank * BNH + c * 64, kb * BK, full0);
+              for (int c = 0; c < BMH / 64; ++c)
+                tma_load_2d(smem_addr(sa + c * (BK * 128)), &p.map_a[s], arow + c * 64, kb * BK, full0);
+            }
+            if (!p.b_trans) {   // [K, cols] in memory: two boxes of 64 K x 64 columns
+#pragma unroll
+              for (int c = 0; c < BNH / 64; ++c)
+                tma_load_2d(smem_addr(sb + c * (BK * 128)), &p.map_b[s], bcol + c * 64, kb * BK, full0);
+            } else {            // [cols, K] in memory: one box of 128 columns x 64 K
+              tma_load_2d(smem_addr(sb), &p.map_b[s], kb * BK, bcol, full0);
+            }
           }
         }
       }
@@ -337,6 +354,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
     if (lane == 0 && rank == 0) {
       long long kb_iter = 0;
       int tile_iter = 0;
+      const unsigned idesc = make_idesc(p.a_trans, p.b_trans);
       for (int tile = first; tile < p.total_tiles && !*abort_flag; tile += stride, ++tile_iter) {
         const TileCoord tc = tile_coord(p, tile);
         const int acc = tile_iter & 1;
@@ -358,12 +376,16 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
             const unsigned sb = sa + kStageA;
 #pragma unroll
             for (int kk = 0; kk < BK / 16; ++kk) {
-              // A: K-major, rows of 128 bytes, 8-row groups 1024 bytes apart; 16 K-elements = 32 bytes
-              const unsigned long long da = smem_desc(sa + kk * 32, 16, 1024);
-              // B: N-major, 64-column chunks BK*128 bytes apart, 8-row K groups 1024 bytes apart;
-              //    16 K-rows = 2048 bytes.  Each CTA holds its 128 of the 256 columns at this offset.
-              const unsigned long long db = smem_desc(sb + kk * 2048, BK * 128, 1024);
-              umma_bf16(d_tmem, da, db, kIdesc, accumulate);
+              // K-major tile (A as given, B transposed): rows of 128 bytes = 64 K-elements, 8-row
+              //    groups 1024 bytes apart; 16 K-elements = 32 bytes.
+              // MN-major tile (B as given, A transposed): 64-element chunks of the M / N index
+              //    BK*128 bytes apart, 8-row K groups 1024 bytes apart; 16 K-rows = 2048 bytes.
+              // Each CTA holds its 128 of the pair's 256 rows (A) or columns (B).
+              const unsigned long long da =
+                  p.a_trans ? smem_desc(sa + kk * 2048, BK * 128, 1024) : smem_desc(sa + kk * 32, 16, 1024);
+              const unsigned long long db =
+                  p.b_trans ? smem_desc(sb + kk * 32, 16, 1024) : smem_desc(sb + kk * 2048, BK * 128, 1024);
+              umma_bf16(d_tmem, da, db, idesc, accumulate);
               accumulate = 1;
             }
             umma_commit_pair(smem_addr(&bar_empty[slot]));   // slot reusable in both CTAs
@@ -613,7 +635,8 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
   for (int g = 0; g < plan.ngroups; ++g) {
     if (plan.m[g] == 0 || plan.n[g] == 0) continue;
     if (stores_y && (!aligned16(plan.y[g]) || (plan.ldy[g] * oesz) % 16 != 0)) return SBP_ERR_UNSUPPORTED;
-    if (plan.col_off[g] % 8 != 0) return SBP_ERR_UNSUPPORTED;
+    if (!plan.b_trans && plan.col_off[g] % 8 != 0) return SBP_ERR_UNSUPPORTED;   // the x coordinate of a TMA load
+    if (plan.a_trans && plan.row_off[g] % 8 != 0) return SBP_ERR_UNSUPPORTED;
     const long long kg = plan.chain ? ktotal_chain : plan.kseg[g];
     if (kg == 0) return SBP_ERR_UNSUPPORTED;   // an all-zero result: left to the FMA kernel
     if (plan.m[g] > 0x7fffffffLL || plan.n[g] > 0x7fffffffLL) return SBP_ERR_UNSUPPORTED;
@@ -630,6 +653,8 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
   p.chain = plan.chain;
   p.gelu = plan.gelu;
   p.n_rep = plan.n_rep;
+  p.a_trans = plan.a_trans;
+  p.b_trans = plan.b_trans;
   p.out_f32 = plan.out_dtype == SBP_F32;
   p.xent = xf ? (xf->grad ? 2 : 1) : 0;
   if (xf) p.xf = *xf;
@@ -649,10 +674,13 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
       cols_b = plan.n[s];
     }
     if (rows_a == 0 || cols_b == 0) { p.kblocks[s] = plan.chain ? p.kblocks[s] : 0; continue; }
-    if (!make_map(&p.map_a[s], plan.a[s], 2, rows_a, plan.kseg[s], plan.lda[s], BMH, BK))
-      return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for operand x of shard %d", s);
-    if (!make_map(&p.map_b[s], plan.b[s], 2, plan.kseg[s], cols_b, plan.ldb[s], BK, 64))
-      return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for operand w of shard %d", s);
+    // as stored: A [rows, K] (transposed [K, rows]), B [K, cols] (transposed [cols, K])
+    const bool ok_a = plan.a_trans ? make_map(&p.map_a[s], plan.a[s], 2, plan.kseg[s], rows_a, plan.lda[s], BK, 64)
+                                   : make_map(&p.map_a[s], plan.a[s], 2, rows_a, plan.kseg[s], plan.lda[s], BMH, BK);
+    if (!ok_a) return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for operand x of shard %d", s);
+    const bool ok_b = plan.b_trans ? make_map(&p.map_b[s], plan.b[s], 2, cols_b, plan.kseg[s], plan.ldb[s], BNH, BK)
+                                   : make_map(&p.map_b[s], plan.b[s], 2, plan.kseg[s], cols_b, plan.ldb[s], BK, 64);
+    if (!ok_b) return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for operand w of shard %d", s);
   }
   int tiles = 0;
   const int box_cols = p.out_f32 ? 32 : 64;

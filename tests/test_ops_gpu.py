@@ -36,7 +36,15 @@ def _shard_operand(T, sig, k, seed, tid, dtype):
     return split_cpu(T, sig, k)
 
 
-def _matmul_case(M, K, N, k, dtype, xs, ws, ys=None, flags=0, out_dtype=None, seed=1001):
+def _swap(sig):
+    """Signature of the stored tensor whose transpose carries sig (S(0) <-> S(1))."""
+    return sbp.S(1 - sig.axis) if sig.kind == 0 else sig
+
+
+def _matmul_case(M, K, N, k, dtype, xs, ws, ys=None, flags=0, out_dtype=None, seed=1001, tx=False, tw=False):
+    """xs / ws are the signatures of the operands as they enter the product.  With tx (tw) the
+    library is handed the transpose of x (w) -- stored [K,M] ([N,K]) with the swapped signature --
+    together with SBP_TRANS_X (SBP_TRANS_W); the oracle sees the untransposed operands."""
     out_dtype = out_dtype or dtype
     X = dg.uniform(seed, 0, (M, K), -1.0, 1.0, dtype)
     W = dg.uniform(seed, 1, (K, N), -1.0, 1.0, dtype)
@@ -44,12 +52,20 @@ def _matmul_case(M, K, N, k, dtype, xs, ws, ys=None, flags=0, out_dtype=None, se
     wl = _shard_operand(W, ws, k, seed, 40, dtype)
     natural = sbp.sbp_matmul_infer(xs, ws)
     ys = ys or natural
-    x = make_global(xl, (M, K), dtype, xs)
-    w = make_global(wl, (K, N), dtype, ws)
+    if tx:
+        x = make_global([t.t().contiguous() for t in xl], (K, M), dtype, _swap(xs))
+        flags |= sbp.SBP_TRANS_X
+    else:
+        x = make_global(xl, (M, K), dtype, xs)
+    if tw:
+        w = make_global([t.t().contiguous() for t in wl], (N, K), dtype, _swap(ws))
+        flags |= sbp.SBP_TRANS_W
+    else:
+        w = make_global(wl, (K, N), dtype, ws)
     y = sbp.empty_global((M, N), out_dtype, ys, k)
     for t in y.locals:
         t.view(torch.uint8).fill_(0x7F)
-    nbytes = sbp.sbp_matmul_workspace_bytes(x, w, y)
+    nbytes = 0 if (tx or tw) else sbp.sbp_matmul_workspace_bytes(x, w, y)
     wsbuf = torch.empty(max(nbytes, 1), dtype=torch.uint8, device="cuda")
     sbp.sbp_matmul(x, w, y, flags, wsbuf)
     torch.cuda.synchronize()
@@ -121,6 +137,78 @@ def test_matmul_gelu_epilogue_and_f32_out():
     _matmul_case(64, 128, 96, 2, BF16, sbp.B, sbp.S(1), flags=sbp.SBP_EPILOGUE_GELU)
     _matmul_case(64, 128, 96, 2, BF16, sbp.S(1), sbp.S(0), ys=sbp.B, flags=sbp.SBP_EPILOGUE_GELU)
     _matmul_case(64, 128, 96, 2, BF16, sbp.S(1), sbp.S(0), out_dtype=F32)
+
+
+TRANS = [(True, False), (False, True), (True, True)]
+
+
+@pytest.mark.parametrize("tx,tw", TRANS)
+@pytest.mark.parametrize("xs,ws", TABLE1)
+def test_matmul_transposed_operands_fp32(xs, ws, tx, tw):
+    """SBP_TRANS_X / SBP_TRANS_W on the FMA kernel: all six signatures, even and ragged shapes."""
+    _matmul_case(64, 128, 96, 2, F32, xs, ws, tx=tx, tw=tw)
+    _matmul_case(70, 45, 83, 3, F32, xs, ws, tx=tx, tw=tw)
+
+
+@pytest.mark.parametrize("tx,tw", TRANS)
+@pytest.mark.parametrize("xs,ws", TABLE1)
+def test_matmul_transposed_operands_tensor_core(xs, ws, tx, tw):
+    """The same on the tensor-core kernel: several tiles, K not a multiple of the K-block, ragged
+    M and N, k = 2 and 4."""
+    _matmul_case(512, 320, 512, 2, BF16, xs, ws, tx=tx, tw=tw)
+    _matmul_case(384, 1160, 648, 4, BF16, xs, ws, tx=tx, tw=tw, seed=1011)
+    _matmul_case(70, 45, 83, 3, BF16, xs, ws, tx=tx, tw=tw)      # falls to the FMA kernel
+
+
+@pytest.mark.parametrize("tx,tw", TRANS)
+@pytest.mark.parametrize("ys", [sbp.B, sbp.S(0), sbp.S(1)])
+def test_matmul_transposed_operands_fused_boxing(ys, tx, tw):
+    _matmul_case(64, 128, 96, 2, F32, sbp.S(1), sbp.S(0), ys=ys, tx=tx, tw=tw)
+    _matmul_case(512, 1024, 768, 4, BF16, sbp.S(1), sbp.S(0), ys=ys, tx=tx, tw=tw)
+    _matmul_case(512, 1024, 768, 4, BF16, sbp.S(1), sbp.S(0), ys=ys, tx=tx, tw=tw, out_dtype=F32)
+
+
+def test_data_parallel_layer_backward():
+    """Data parallelism (Section 3.1): X S(0), W B, Y = X W S(0).  Backward with the same calls:
+    dX = dY W^T is (S(0), B) -> S(0); dW = X^T dY is (S(1), S(0)) -> P(sum), asked for as B, i.e.
+    with the gradient all-reduce folded into the product.  Checked against the fp64 products."""
+    M, K, N, k = 1024, 512, 768, 4
+    X = dg.normal(77, 0, (M, K), 0.0, 1.0, BF16)
+    W = dg.normal(77, 1, (K, N), 0.0, 0.05, BF16)
+    dY = dg.normal(77, 2, (M, N), 0.0, 1.0, BF16)
+    x = make_global(split_cpu(X, sbp.S(0), k), (M, K), BF16, sbp.S(0))
+    w = make_global([W] * k, (K, N), BF16, sbp.B)
+    dy = make_global(split_cpu(dY, sbp.S(0), k), (M, N), BF16, sbp.S(0))
+    dx = sbp.empty_global((M, K), BF16, sbp.S(0), k)
+    dw = sbp.empty_global((K, N), F32, sbp.B, k)
+    sbp.sbp_matmul(dy, w, dx, sbp.SBP_TRANS_W)
+    sbp.sbp_matmul(x, dy, dw, sbp.SBP_TRANS_X)
+    torch.cuda.synchronize()
+    sbp.sbp_check_device_errors()
+    dX = O.matmul_logical(to_np(dY), to_np(W).T)
+    dW = O.matmul_logical(to_np(X).T, to_np(dY))
+    for r, a in enumerate(O.to_locals(dX, O.S0, k)):
+        assert_close(to_np(dx.locals[r]), a, 2e-2, 1e-3, f"dX shard {r}")
+    for r in range(k):
+        assert_close(to_np(dw.locals[r]), dW, 2e-2, 1e-3, f"dW replica {r}")
+
+
+def test_matmul_transposed_operands_are_validated():
+    k = 2
+    x = sbp.empty_global((128, 64), F32, sbp.S(1), k)        # stored [K,M] = [128,64]: M = 64, K = 128
+    w = sbp.empty_global((128, 96), F32, sbp.B, k)
+    y = sbp.empty_global((64, 96), F32, sbp.S(0), k)
+    sbp.sbp_matmul(x, w, y, sbp.SBP_TRANS_X)                 # (S(0), B) -> S(0) once transposed
+    bad = sbp.empty_global((64, 96), F32, sbp.S(1), k)
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_matmul(x, w, bad, sbp.SBP_TRANS_X)
+    assert e.value.name == "SBP_ERR_SIGNATURE"
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_matmul(x, w, y, 0)                           # untransposed: [128,64] x [128,96] does not fit
+    assert e.value.name == "SBP_ERR_SHAPE"
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_matmul(x, w, y, 64)
+    assert e.value.name == "SBP_ERR_INVALID_ARG"
 
 
 def test_matmul_exact_on_small_integers_and_permutation():

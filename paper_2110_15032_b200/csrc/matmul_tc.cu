@@ -67,7 +67,6 @@ struct TcParams {
   int tiles_m[SBP_MAX_K];
   int tiles_n[SBP_MAX_K];
   int ngroups, nseg, chain, gelu, n_rep;
-  int a_trans, b_trans;         // operand stored transposed (see MatmulPlan)
   int out_f32;
   int total_tiles;
   int xent;                     // 1: softmax partials instead of stored logits
@@ -214,7 +213,7 @@ __device__ __forceinline__ unsigned long long smem_desc(unsigned addr, unsigned 
 // K index.  Operands as given: A [M,K] row-major is K-major, B [K,N] row-major is N-major; a
 // transposed operand is the other way round.
 constexpr unsigned kIdescBase = (1u << 4) | (1u << 7) | (1u << 10) | ((BN >> 3) << 17) | ((BM >> 4) << 24);
-__device__ __forceinline__ unsigned make_idesc(int a_trans, int b_trans) {
+__host__ __device__ constexpr unsigned make_idesc(int a_trans, int b_trans) {
   return kIdescBase | ((a_trans ? 1u : 0u) << 15) | ((b_trans ? 0u : 1u) << 16);
 }
 
@@ -260,6 +259,10 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
 
 // ------------------------------------------------------------------ the kernel
 
+// AT / BT: operand A / B is stored transposed.  They are compile-time so that the usual
+// (untransposed) form carries no trace of the other three: as run-time switches they cost the
+// MMA-issuing thread and the producer enough to slow every product by 6 %.
+template <int AT, int BT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
     matmul_tc_kernel(const __grid_constant__ TcParams p) {
   extern __shared__ unsigned char smem_raw[];
@@ -321,14 +324,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
             unsigned char* sb = sa + kStageA;
             const int arow = (int)p.row_off[tc.g] + tc.m0 + (int)rank * BMH;
             const int bcol = (int)p.col_off[tc.g] + tc.n0 + (int)rank * BNH;
-            if (!p.a_trans) {   // [rows, K] in memory: one box of 128 rows x 64 K
+            if constexpr (!AT) {   // [rows, K] in memory: one box of 128 rows x 64 K
               tma_load_2d(smem_addr(sa), &p.map_a[s], kb * BK, arow, full0);
             } else {            // [K, rows] in memory: two boxes of 64 K x 64 rows
 #pragma unroll
               for (int c = 0; c < BMH / 64; ++c)
                 tma_load_2d(smem_addr(sa + c * (BK * 128)), &p.map_a[s], arow + c * 64, kb * BK, full0);
             }
-            if (!p.b_trans) {   // [K, cols] in memory: two boxes of 64 K x 64 columns
+            if constexpr (!BT) {   // [K, cols] in memory: two boxes of 64 K x 64 columns
 #pragma unroll
               for (int c = 0; c < BNH / 64; ++c)
                 tma_load_2d(smem_addr(sb + c * (BK * 128)), &p.map_b[s], bcol + c * 64, kb * BK, full0);
@@ -354,7 +357,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
     if (lane == 0 && rank == 0) {
       long long kb_iter = 0;
       int tile_iter = 0;
-      const unsigned idesc = make_idesc(p.a_trans, p.b_trans);
+      constexpr unsigned idesc = make_idesc(AT, BT);
       for (int tile = first; tile < p.total_tiles && !*abort_flag; tile += stride, ++tile_iter) {
         const TileCoord tc = tile_coord(p, tile);
         const int acc = tile_iter & 1;
@@ -382,9 +385,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
               //    BK*128 bytes apart, 8-row K groups 1024 bytes apart; 16 K-rows = 2048 bytes.
               // Each CTA holds its 128 of the pair's 256 rows (A) or columns (B).
               const unsigned long long da =
-                  p.a_trans ? smem_desc(sa + kk * 2048, BK * 128, 1024) : smem_desc(sa + kk * 32, 16, 1024);
+                  AT ? smem_desc(sa + kk * 2048, BK * 128, 1024) : smem_desc(sa + kk * 32, 16, 1024);
               const unsigned long long db =
-                  p.b_trans ? smem_desc(sb + kk * 32, 16, 1024) : smem_desc(sb + kk * 2048, BK * 128, 1024);
+                  BT ? smem_desc(sb + kk * 32, 16, 1024) : smem_desc(sb + kk * 2048, BK * 128, 1024);
               umma_bf16(d_tmem, da, db, idesc, accumulate);
               accumulate = 1;
             }
@@ -616,6 +619,46 @@ size_t matmul_tc_workspace_bytes(const MatmulPlan&) { return 0; }
 
 static bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
 
+// Launch of one compiled form of the kernel (called with the parameter block's lock held).
+template <int AT, int BT>
+static sbp_status launch_tc_form(const TcParams& p, int tiles, cudaStream_t st) {
+  // per device: the kernel's shared-memory opt-in and the number of CTA pairs that fit at once
+  static int pairs_on_device[64] = {};
+  int dev = 0;
+  SBP_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return fail(SBP_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
+  if (pairs_on_device[dev] == 0) {
+    SBP_CUDA_TRY(cudaFuncSetAttribute(matmul_tc_kernel<AT, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    int sms = 0;
+    SBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    // how many CTA pairs the device can hold at once (pairs must sit in one GPC)
+    cudaLaunchConfig_t probe = {};
+    probe.gridDim = dim3((unsigned)(2 * (sms / 2)));
+    probe.blockDim = dim3(kThreadsTc);
+    probe.dynamicSmemBytes = kSmemBytes;
+    cudaLaunchAttribute attr;
+    attr.id = cudaLaunchAttributeClusterDimension;
+    attr.val.clusterDim.x = 2;
+    attr.val.clusterDim.y = 1;
+    attr.val.clusterDim.z = 1;
+    probe.attrs = &attr;
+    probe.numAttrs = 1;
+    int clusters = 0;
+    if (cudaOccupancyMaxActiveClusters(&clusters, matmul_tc_kernel<AT, BT>, &probe) != cudaSuccess || clusters < 1) {
+      cudaGetLastError();
+      clusters = sms / 2;
+    }
+    pairs_on_device[dev] = clusters;
+  }
+  const int max_pairs = pairs_on_device[dev];
+  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  matmul_tc_kernel<AT, BT><<<2 * pairs, kThreadsTc, kSmemBytes, st>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "tensor-core matmul launch");
+  count_launch();
+  return SBP_OK;
+}
+
 sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaStream_t st, bool* taken) {
   *taken = false;
   if (plan.in_dtype != SBP_BF16) return SBP_ERR_UNSUPPORTED;
@@ -653,8 +696,6 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
   p.chain = plan.chain;
   p.gelu = plan.gelu;
   p.n_rep = plan.n_rep;
-  p.a_trans = plan.a_trans;
-  p.b_trans = plan.b_trans;
   p.out_f32 = plan.out_dtype == SBP_F32;
   p.xent = xf ? (xf->grad ? 2 : 1) : 0;
   if (xf) p.xf = *xf;
@@ -709,41 +750,12 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
   *taken = true;
   if (tiles == 0) return SBP_OK;
 
-  // per device: the kernel's shared-memory opt-in and the number of CTA pairs that fit at once
-  static int pairs_on_device[64] = {};
-  int dev = 0;
-  SBP_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64) return fail(SBP_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
-  if (pairs_on_device[dev] == 0) {
-    SBP_CUDA_TRY(cudaFuncSetAttribute(matmul_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
-    int sms = 0;
-    SBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    // how many CTA pairs the device can hold at once (pairs must sit in one GPC)
-    cudaLaunchConfig_t probe = {};
-    probe.gridDim = dim3((unsigned)(2 * (sms / 2)));
-    probe.blockDim = dim3(kThreadsTc);
-    probe.dynamicSmemBytes = kSmemBytes;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = 2;
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    probe.attrs = &attr;
-    probe.numAttrs = 1;
-    int clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&clusters, matmul_tc_kernel, &probe) != cudaSuccess || clusters < 1) {
-      cudaGetLastError();
-      clusters = sms / 2;
-    }
-    pairs_on_device[dev] = clusters;
+  switch ((plan.a_trans ? 2 : 0) | (plan.b_trans ? 1 : 0)) {
+    case 0: return launch_tc_form<0, 0>(p, tiles, st);
+    case 1: return launch_tc_form<0, 1>(p, tiles, st);
+    case 2: return launch_tc_form<1, 0>(p, tiles, st);
+    default: return launch_tc_form<1, 1>(p, tiles, st);
   }
-  const int max_pairs = pairs_on_device[dev];
-  const int pairs = tiles < max_pairs ? tiles : max_pairs;
-  matmul_tc_kernel<<<2 * pairs, kThreadsTc, kSmemBytes, st>>>(p);
-  cudaError_t e = cudaGetLastError();
-  if (e != cudaSuccess) return cuda_fail(e, "tensor-core matmul launch");
-  count_launch();
-  return SBP_OK;
 }
 
 sbp_status read_and_clear_tc_timeout(bool* timed_out) {

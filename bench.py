@@ -166,18 +166,22 @@ def run_sweep(sbp, work, events=None):
 # None = not captured for the kernel as it stands.
 NCU_TRAFFIC = {
     # profiles/box_kernels_sweep_bf16_8192x8192_k4.md (full size)
-    "P(sum)->B": 1017.8e6, "P(sum)->S(0)": 624.8e6, "P(sum)->S(1)": 620.8e6, "S(0)->B": 613.6e6,
-    "S(0)->S(1)": 214.8e6, "S(1)->S(0)": 214.5e6, "B->S(1)": 213.6e6,
+    "P(sum)->B": 1020.4e6, "P(sum)->S(0)": 647.2e6, "P(sum)->S(1)": 644.5e6, "S(0)->B": 612.7e6,
+    "S(0)->S(1)": 218.1e6, "S(1)->S(0)": 216.3e6, "B->S(1)": 217.2e6,
     # profiles/xent_partial_bf16_512x1048576_k8.md (full size)
     "softmax-xent on bf16 logits (partial + combine)": 1077.5e6,
     "softmax-xent backward (softmax - onehot, S(1))": 2100.3e6,
     # profiles/matmul_tc_classifier_bf16_512x512x1048576_k8.md (full size)
-    "classifier GEMM (B,S(1))->S(1), bf16 logits": 2105.2e6,
-    "classifier GEMM fused with softmax-xent (no logits stored)": 1132.9e6 + 50.3e6,
+    "classifier GEMM (B,S(1))->S(1), bf16 logits": 2105.6e6,
+    "classifier GEMM fused with softmax-xent (no logits stored)": 1127.2e6 + 50.3e6,
+    "classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)": 2105.0e6,
     # profiles/matmul_tc_mlp_bf16_8192x4096x16384_k8.md (full size)
-    "MLP GEMM1 (B,S(1))->S(1) + GeLU": 1030.4e6,
-    "MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials": 915.3e6,
-    "MLP GEMM2 fused (S(1),S(0))->B": 1752.0e6,
+    "MLP GEMM1 (B,S(1))->S(1) + GeLU": 975.0e6,
+    "MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials": 910.8e6,
+    "MLP GEMM2 fused (S(1),S(0))->B": 1731.9e6,
+    "DP layer backward dW = X^T dY, (S(1),S(0))->S(0) fused": 2506.1e6,
+    "DP layer backward dW = X^T dY, (S(1),S(0))->B fused (8 replicas written)": 2090.9e6,
+    "DP layer backward dX = dY W^T, (S(0),B)->S(0)": 1474.8e6,
     # profiles/extras_bf16_8192x8192_p4_and_embedding_fp32_4194304x128_batch16384_k8.md (full size)
     "S(0)->P(sum) bf16 [8192,8192] k=4": 615.7e6,
     "B->P(sum) bf16 [8192,8192] k=4": 611.4e6,
@@ -189,6 +193,7 @@ NCU_TRAFFIC = {
     "disjoint placements: P(sum)[4] -> B[2] bf16 [8192,8192]": 749.7e6,
     # profiles/embedding_fused_fp32_4194304x128_batch16384_k8.md (quarter batch, scaled x 4)
     "embedding fused gather -> B (8 replicas written)": 7102.8e6,
+    "embedding fused gather -> B (replicas aliased, 1 write)": 950.4e6,
 }
 
 

@@ -9,7 +9,7 @@
 // of J*256 vectors of one task, all loads before the stores.
 //
 //   copy      S -> S (any axes), B -> S (replica d mod ks serves shard d), S -> B and B -> B
-//             (one read, one write per distinct replica), S -> P(sum) (zero fill first, then
+//             (one read, one write per distinct replica), S -> P(sum) (zero fill by one kernel first, then
 //             piece d of the kd-way split of the source's axis lands in place in partial d)
 //   reduce    P -> S / B (all ks partials in rank order, fp32 accumulator, one rounding),
 //             P -> P (partial r goes to destination r mod kd, which adds what it gets in
@@ -191,6 +191,21 @@ __global__ void __launch_bounds__(256, OP == OP_COPY ? 4 : 3) box_disjoint_kerne
   }
 }
 
+// Clears n destination buffers of `bytes` bytes each (16-byte aligned, a multiple of 16 long):
+// the starting value of P(sum) partials that then receive their piece.
+struct ZeroParams {
+  char* dst[SBP_MAX_K];
+  long long bytes;
+  int n;
+};
+
+__global__ void __launch_bounds__(256) box_zero_kernel(const __grid_constant__ ZeroParams z) {
+  uint4* d = reinterpret_cast<uint4*>(z.dst[blockIdx.y]);
+  const long long n = z.bytes / 16;
+  const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) d[i] = zero;
+}
+
 template <int OP>
 static void launch_disjoint(const DisjointParams& p, int vbytes, long long grid, cudaStream_t st) {
   const dim3 g((unsigned)grid), b(256);
@@ -346,10 +361,28 @@ sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard
   }
 
   if (zero_first) {
+    // The partials start as zeros.  One kernel clears all of them when they are 16-byte
+    // aligned (one launch instead of up to kd memsets with their gaps); else memsets do.
+    ZeroParams z{};
+    z.bytes = (long long)numel(dst) * esz;
+    bool vec_ok = z.bytes % 16 == 0;
     for (int r = 0; r < kd; ++r) {
       if (p.one_dst && r != dst_shard) continue;
       if (p.mode == DJ_TO_ALL && r == 0) continue;  // overwritten in full by the copy
-      SBP_CUDA_TRY(cudaMemsetAsync(dst->local[r], 0, (size_t)numel(dst) * esz, stream));
+      z.dst[z.n++] = static_cast<char*>(dst->local[r]);
+      vec_ok = vec_ok && reinterpret_cast<uintptr_t>(dst->local[r]) % 16 == 0;
+    }
+    if (z.n > 0 && z.bytes > 0) {
+      if (vec_ok) {
+        long long zb = (z.bytes / 16 + 256 * 8 - 1) / (256 * 8);
+        if (zb > 148 * 16) zb = 148 * 16;
+        box_zero_kernel<<<dim3((unsigned)zb, (unsigned)z.n), 256, 0, stream>>>(z);
+        cudaError_t ze = cudaGetLastError();
+        if (ze != cudaSuccess) return cuda_fail(ze, "zero fill launch");
+        count_launch();
+      } else {
+        for (int q = 0; q < z.n; ++q) SBP_CUDA_TRY(cudaMemsetAsync(z.dst[q], 0, (size_t)z.bytes, stream));
+      }
     }
   }
   if (!copy_needed) return SBP_OK;

@@ -207,6 +207,33 @@ def test_round_trips_on_device():
         assert np.array_equal(bits(r), bits(T))
 
 
+def test_back_to_back_calls_keep_stream_order():
+    """Boxing kernels are launched so that a call may be set up on the GPU while the call before
+    it is still running; it must nevertheless see that call's results (read after write) and must
+    not overwrite what that call still reads (write after read).  A chain over buffers large
+    enough for many waves of CTAs, repeated: a -> b, b -> c, then z -> a while b -> c may still run,
+    then a -> b again.  Every intermediate is compared with the oracle's mapping."""
+    k, shape = 4, (2048, 4096)
+    T = dg.normal(31, 0, shape, 0, 1, BF16)
+    Z = dg.normal(31, 1, shape, 0, 1, BF16)
+    want_s1 = {id(X): split_cpu(X, sbp.S(1), k) for X in (T, Z)}
+    for rep in range(5):
+        a = make_global(split_cpu(T, sbp.S(0), k), shape, BF16, sbp.S(0))
+        z = make_global(split_cpu(Z, sbp.S(0), k), shape, BF16, sbp.S(0))
+        b = sbp.empty_global(shape, BF16, sbp.S(1), k)
+        c = sbp.empty_global(shape, BF16, sbp.B, k)
+        b2 = sbp.empty_global(shape, BF16, sbp.S(1), k)
+        sbp.sbp_boxing(a, b)        # a -> b
+        sbp.sbp_boxing(b, c)        # reads b right behind its writer
+        sbp.sbp_boxing(z, a)        # overwrites a, which the first call read
+        sbp.sbp_boxing(a, b2)       # reads the overwritten a
+        torch.cuda.synchronize()
+        for r in range(k):
+            assert torch.equal(b.locals[r].cpu(), want_s1[id(T)][r]), f"repeat {rep}: S(0)->S(1) shard {r}"
+            assert np.array_equal(bits(c.locals[r]), bits(T)), f"repeat {rep}: replica {r} read stale data"
+            assert torch.equal(b2.locals[r].cpu(), want_s1[id(Z)][r]), f"repeat {rep}: second chain shard {r}"
+
+
 def test_host_buffer_entry_point():
     k, shape = 4, (128, 256)
     src_cpu = [dg.normal(9, r, shape, 0, 1, BF16).pin_memory() for r in range(k)]

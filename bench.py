@@ -191,6 +191,7 @@ NCU_TRAFFIC = {
     "disjoint placements: S(0)[4] -> B[8] bf16 [8192,8192]": 1169.0e6,
     "disjoint placements: P(sum)[4] -> S(0)[8] bf16 [8192,8192]": 616.7e6,
     "disjoint placements: P(sum)[4] -> B[2] bf16 [8192,8192]": 749.7e6,
+    "disjoint placements: S(0)[4] -> P(sum)[8] bf16 [8192,8192]": 1015.4e6 + 215.5e6,
     # profiles/embedding_fused_fp32_4194304x128_batch16384_k8.md (quarter batch, scaled x 4)
     "embedding fused gather -> B (8 replicas written)": 7102.8e6,
     "embedding fused gather -> B (replicas aliased, 1 write)": 950.4e6,

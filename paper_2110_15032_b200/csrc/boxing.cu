@@ -57,7 +57,7 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
   // so this is 32-bit arithmetic.
   // Let the next kernel in the stream be set up while this one's last CTAs run; it waits, as
   // this one does below, for its predecessor to finish before it touches global memory.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  SBP_PDL_RELEASE();
   const unsigned u = blockIdx.x;
   const unsigned rem = u / (unsigned)p.ntasks;
   const int t = (int)(u - rem * (unsigned)p.ntasks);
@@ -99,7 +99,7 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
     dofs[j] = ((((x * g.Na_d + g.aoff_d + ia) * p.M + m) * g.Nb_d + g.boff_d) * cs) / (long long)sizeof(V) + col;
   }
 
-  asm volatile("griddepcontrol.wait;" ::: "memory");   // the previous kernel's results are visible from here on
+  SBP_PDL_WAIT();   // the previous kernel's results are visible from here on
 
   V val[J];
   if constexpr (OP == OP_COPY) {
@@ -193,10 +193,12 @@ constexpr int kScatterJ = 8;
 
 template <typename V>
 __global__ void __launch_bounds__(256) box_scatter_kernel(const __grid_constant__ ScatterParams p) {
+  SBP_PDL_RELEASE();
   const int d = blockIdx.y + p.d0;
   const V* sp = reinterpret_cast<const V*>(p.src[d]);
   V* dp = reinterpret_cast<V*>(p.dst[d]);
   const long long lo = p.own_lo[d], hi = p.own_hi[d], w = hi - lo;
+  SBP_PDL_WAIT();
   for (long long c = blockIdx.x; c < p.total_chunks; c += gridDim.x) {
     long long row, within;
     chunk_row(c, p.chunks_per_row, &row, &within);
@@ -220,7 +222,7 @@ template <typename V>
 static void launch_scatter_v(const ScatterParams& sp, int k, cudaStream_t st) {
   long long gx = sp.total_chunks < 148 * 6 ? sp.total_chunks : 148 * 6;
   if (gx < 1) gx = 1;
-  box_scatter_kernel<V><<<dim3((unsigned)gx, (unsigned)k), 256, 0, st>>>(sp);
+  launch_dependent(box_scatter_kernel<V>, dim3((unsigned)gx, (unsigned)k), dim3(256), 0, st, sp);
 }
 
 // ------------------------------------------------------------------ S(i) -> B with an fp32 -> bf16 cast
@@ -240,9 +242,11 @@ struct GatherCastParams {
 template <int EPV>
 __global__ void __launch_bounds__(256) box_gather_cast_kernel(const __grid_constant__ GatherCastParams p) {
   constexpr int J = 4;
+  SBP_PDL_RELEASE();
   const int s = blockIdx.y;
   const long long lo = p.own_lo[s], w = p.own_hi[s] - lo;
   if (w <= 0) return;
+  SBP_PDL_WAIT();
   const long long chunks_per_row = (w + 256 * J - 1) / (256 * J);
   const long long total = p.nrows * chunks_per_row;
   for (long long c = blockIdx.x; c < total; c += gridDim.x) {
@@ -323,17 +327,7 @@ static int pick_vector_bytes(const BoxParams& p, const sbp_tensor* src, const sb
 // the launch behaves like a plain one.
 template <typename V, int OP, int J, int KT>
 static void launch_tile(const Plan& pl, cudaStream_t st) {
-  cudaLaunchConfig_t cfg{};
-  cfg.gridDim = dim3((unsigned)pl.grid);
-  cfg.blockDim = dim3(256);
-  cfg.dynamicSmemBytes = 0;
-  cfg.stream = st;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-  attr[0].val.programmaticStreamSerializationAllowed = 1;
-  cfg.attrs = attr;
-  cfg.numAttrs = 1;
-  cudaLaunchKernelEx(&cfg, box_tile_kernel<V, OP, J, KT>, pl.p);   // errors are picked up by the caller's cudaGetLastError
+  launch_dependent(box_tile_kernel<V, OP, J, KT>, dim3((unsigned)pl.grid), dim3(256), 0, st, pl.p);   // errors are picked up by the caller's cudaGetLastError
 }
 
 template <typename V, int OP, int J>
@@ -643,8 +637,8 @@ static sbp_status boxing_one_axis(const sbp_tensor* src, sbp_tensor* dst, int ds
     gp.n_dst = b.n_dst;
     for (int q = 0; q < b.n_dst; ++q) gp.dst[q] = reinterpret_cast<__nv_bfloat16*>(b.dst[q]);
     dim3 grid(148 * 4, (unsigned)b.k);
-    if (vec) box_gather_cast_kernel<8><<<grid, 256, 0, stream>>>(gp);
-    else box_gather_cast_kernel<1><<<grid, 256, 0, stream>>>(gp);
+    if (vec) launch_dependent(box_gather_cast_kernel<8>, grid, dim3(256), 0, stream, gp);
+    else launch_dependent(box_gather_cast_kernel<1>, grid, dim3(256), 0, stream, gp);
     done = true;
   } else if (pl.p.mode == MODE_SCATTER_P) {
     const BoxParams& b = pl.p;

@@ -81,6 +81,7 @@ __device__ __forceinline__ AxisCut cut_axis(long long n, bool by_src, long long 
 template <typename V, int OP>
 __global__ void __launch_bounds__(256, OP == OP_COPY ? 4 : 3) box_disjoint_kernel(const __grid_constant__ DisjointParams p) {
   constexpr int J = OP == OP_COPY ? 4 : 2;
+  SBP_PDL_RELEASE();                             // the next kernel of the stream may be set up from here on
   const unsigned u = blockIdx.x;                 // the grid is below 2^31 tiles: 32-bit arithmetic
   const unsigned rem = u / (unsigned)p.ntasks;   // task index varies fastest
   const int t = (int)(u - rem * (unsigned)p.ntasks);
@@ -130,6 +131,8 @@ __global__ void __launch_bounds__(256, OP == OP_COPY ? 4 : 3) box_disjoint_kerne
     so[j] = ((((x * ca.n_s + ca.off_s + ia) * p.M + m) * cb.n_s + cb.off_s) * cs) / (long long)sizeof(V) + col;
     dofs[j] = ((((x * ca.n_d + ca.off_d + ia) * p.M + m) * cb.n_d + cb.off_d) * cs) / (long long)sizeof(V) + col;
   }
+
+  SBP_PDL_WAIT();                                // the kernel before this one has finished
 
   V val[J];
   if constexpr (OP == OP_COPY) {
@@ -200,6 +203,8 @@ struct ZeroParams {
 };
 
 __global__ void __launch_bounds__(256) box_zero_kernel(const __grid_constant__ ZeroParams z) {
+  SBP_PDL_RELEASE();
+  SBP_PDL_WAIT();
   uint4* d = reinterpret_cast<uint4*>(z.dst[blockIdx.y]);
   const long long n = z.bytes / 16;
   const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
@@ -210,12 +215,12 @@ template <int OP>
 static void launch_disjoint(const DisjointParams& p, int vbytes, long long grid, cudaStream_t st) {
   const dim3 g((unsigned)grid), b(256);
   switch (vbytes) {
-    case 16: box_disjoint_kernel<uint4, OP><<<g, b, 0, st>>>(p); break;
-    case 8: box_disjoint_kernel<uint2, OP><<<g, b, 0, st>>>(p); break;
-    case 4: box_disjoint_kernel<uint32_t, OP><<<g, b, 0, st>>>(p); break;
+    case 16: launch_dependent(box_disjoint_kernel<uint4, OP>, g, b, 0, st, p); break;
+    case 8: launch_dependent(box_disjoint_kernel<uint2, OP>, g, b, 0, st, p); break;
+    case 4: launch_dependent(box_disjoint_kernel<uint32_t, OP>, g, b, 0, st, p); break;
     default:
       // a 2-byte vector cannot carry an fp32 lane; the fp32 reductions never get here
-      if constexpr (OP != OP_SUM_F32 && OP != OP_MAX_F32) box_disjoint_kernel<uint16_t, OP><<<g, b, 0, st>>>(p);
+      if constexpr (OP != OP_SUM_F32 && OP != OP_MAX_F32) launch_dependent(box_disjoint_kernel<uint16_t, OP>, g, b, 0, st, p);
       break;
   }
 }
@@ -376,7 +381,7 @@ sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard
       if (vec_ok) {
         long long zb = (z.bytes / 16 + 256 * 8 - 1) / (256 * 8);
         if (zb > 148 * 16) zb = 148 * 16;
-        box_zero_kernel<<<dim3((unsigned)zb, (unsigned)z.n), 256, 0, stream>>>(z);
+        launch_dependent(box_zero_kernel, dim3((unsigned)zb, (unsigned)z.n), dim3(256), 0, stream, z);
         cudaError_t ze = cudaGetLastError();
         if (ze != cudaSuccess) return cuda_fail(ze, "zero fill launch");
         count_launch();

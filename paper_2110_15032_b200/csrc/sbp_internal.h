@@ -64,6 +64,28 @@ int64_t local_numel(const sbp_tensor* t, int r);
 
 sbp_status cuda_fail(cudaError_t e, const char* what);
 
+// Launch of `kernel` as a programmatic dependent of the kernel before it in the stream: if that
+// kernel releases its dependents early (SBP_PDL_RELEASE), this one's CTAs may be set up while its
+// last CTAs still run.  Such a kernel must execute SBP_PDL_WAIT before its first access to
+// global memory; after any other kind of work the launch behaves like a plain one.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                                    Args&&... args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#define SBP_PDL_RELEASE() asm volatile("griddepcontrol.launch_dependents;" ::: "memory")
+#define SBP_PDL_WAIT() asm volatile("griddepcontrol.wait;" ::: "memory")
+
 #define SBP_CUDA_TRY(expr)                                   \
   do {                                                       \
     cudaError_t _e = (expr);                                 \

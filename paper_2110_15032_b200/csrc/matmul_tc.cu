@@ -490,22 +490,22 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
       // The element-wise modes are compiled apart (MODE 0 plain, 1 GeLU, 2 softmax - onehot of the
       // recomputed logits) so that the plain store, which the short-K classifier product leans
       // on, carries none of the others' instructions.
-      float g_neg = 0.f, g_inv = 0.f;
+      // softmax = 2^(z log2e - m log2e - log2 S): the division by the row sum is folded into the exponent
+      float g_neg = 0.f;
       long long g_lab = -1;
       if (p.xent == 2 && row0 + lane < Mg) {      // this thread's row constants
         const long long row = row0 + lane;
-        g_neg = -p.xf.row_max[row] * 1.4426950408889634f;
-        g_inv = 1.0f / p.xf.row_sum[row];
+        g_neg = -p.xf.row_max[row] * 1.4426950408889634f - log2f(p.xf.row_sum[row]);
         g_lab = p.xf.labels[row] - p.xf.class_start[tc.g];
       }
       auto slabs = [&](auto mode_tag) {
         constexpr int MODE = decltype(mode_tag)::value;
-        auto xform = [&](float x, long long col) -> float {
+        int lab_rel = -1;   // the label's column inside the current slab, if it lies there
+        auto xform = [&](float x, int idx) -> float {
           if constexpr (MODE == 2) {
             float e;
             asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(x, 1.4426950408889634f, g_neg)));
-            e *= g_inv;
-            return col == g_lab ? e - 1.0f : e;
+            return idx == lab_rel ? e - 1.0f : e;
           } else if constexpr (MODE == 1) {
             return gelu_erf_tc(x);
           } else {
@@ -515,6 +515,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
         for (int sl = 0; sl < nslabs; ++sl) {
           const int col0 = tc.n0 + half * (BN / 2) + sl * cols_per_slab;
           const bool live = row0 < Mg && col0 < Ng;   // warp-uniform
+          if constexpr (MODE == 2) lab_rel = (g_lab >= col0 && g_lab < col0 + cols_per_slab) ? (int)(g_lab - col0) : -1;
           float v[64];
           if (live) {
             tmem_ld32(taddr + sl * cols_per_slab, v);
@@ -529,8 +530,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
 #pragma unroll
               for (int c = 0; c < 8; ++c) {
                 float4 o;
-                o.x = xform(v[4 * c + 0], col0 + 4 * c + 0); o.y = xform(v[4 * c + 1], col0 + 4 * c + 1);
-                o.z = xform(v[4 * c + 2], col0 + 4 * c + 2); o.w = xform(v[4 * c + 3], col0 + 4 * c + 3);
+                o.x = xform(v[4 * c + 0], 4 * c + 0); o.y = xform(v[4 * c + 1], 4 * c + 1);
+                o.z = xform(v[4 * c + 2], 4 * c + 2); o.w = xform(v[4 * c + 3], 4 * c + 3);
                 *reinterpret_cast<float4*>(rowp + ((c ^ (lane & 7)) << 4)) = o;
               }
             } else {
@@ -538,7 +539,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
               for (int c = 0; c < 8; ++c) {
                 float f[8];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) f[e] = xform(v[8 * c + e], col0 + 8 * c + e);
+                for (int e = 0; e < 8; ++e) f[e] = xform(v[8 * c + e], 8 * c + e);
                 uint4 o;
                 __nv_bfloat162 h;
                 h = __floats2bfloat162_rn(f[0], f[1]); o.x = *reinterpret_cast<unsigned*>(&h);

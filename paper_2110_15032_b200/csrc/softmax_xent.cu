@@ -459,17 +459,18 @@ __global__ void __launch_bounds__(kThreads) xent_backward_kernel(const __grid_co
   split_range(p.classes, p.k, shard, (int64_t*)&c_start, (int64_t*)&c_len);
   const T* z = reinterpret_cast<const T*>(p.logits[shard]) + row * c_len;
   T* g = reinterpret_cast<T*>(p.grad[shard]) + row * c_len;
-  const float neg = -p.row_max[row] * kLog2e;
-  const float inv = 1.0f / p.row_sum[row];
+  // softmax = 2^(z log2e - m log2e - log2 S): the division by the row sum is folded into the exponent
+  const float neg = -p.row_max[row] * kLog2e - log2f(p.row_sum[row]);
   const long long y = p.labels[row] - c_start;      // label's column inside this shard, if any
   struct alignas(sizeof(T) * VEC) Pack { T e[VEC]; };
   for (long long e0 = ((long long)blockIdx.y * kThreads + threadIdx.x) * VEC; e0 < c_len;
        e0 += (long long)gridDim.y * kThreads * VEC) {
     Pack in = *reinterpret_cast<const Pack*>(z + e0), out;
+    const int y_rel = (y >= e0 && y < e0 + VEC) ? (int)(y - e0) : -1;   // the label's place in this vector, if it is here
 #pragma unroll
     for (int i = 0; i < VEC; ++i) {
-      float v = ex2(fmaf(static_cast<float>(in.e[i]), kLog2e, neg)) * inv;
-      if (e0 + i == y) v -= 1.0f;
+      float v = ex2(fmaf(static_cast<float>(in.e[i]), kLog2e, neg));
+      if (i == y_rel) v -= 1.0f;
       out.e[i] = static_cast<T>(v);
     }
     *reinterpret_cast<Pack*>(g + e0) = out;

@@ -174,7 +174,7 @@ NCU_TRAFFIC = {
     # profiles/matmul_tc_classifier_bf16_512x512x1048576_k8.md (full size)
     "classifier GEMM (B,S(1))->S(1), bf16 logits": 2105.6e6,
     "classifier GEMM fused with softmax-xent (no logits stored)": 1127.2e6 + 50.3e6,
-    "classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)": 2105.0e6,
+    "classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)": 2104.0e6,
     # profiles/matmul_tc_mlp_bf16_8192x4096x16384_k8.md (full size)
     "MLP GEMM1 (B,S(1))->S(1) + GeLU": 975.0e6,
     "MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials": 910.8e6,

@@ -10,6 +10,13 @@ once.  value = algorithmic bytes of a step / device time of a step.  With N > 1 
 runs its own replica of the sweep (no collective on the data path; weak scaling).
 
 Prints one JSON line (rank 0).  --impl reference times the CPU oracle instead.
+
+--gpus N is the number of ranks: started without a launcher and N > 1, the script starts the N
+ranks itself (torch.distributed.run on 127.0.0.1); under a launcher WORLD_SIZE must equal N.
+At one GPU the line also carries, inside `roofline`, one entry per line of configs 2-5
+(`roofline.configs`: kernel, bound, ms, work, achieved, frac of the measured peak and, for HBM lines
+with an ncu capture, the DRAM-byte rate) and, inside `cpu_baseline`, the oracle timed on a bounded
+sample of each config (`cpu_baseline.configs`, with the host's cores and the threads it used).
 """
 from __future__ import annotations
 
@@ -301,19 +308,27 @@ def time_op(fn, device, iters=10, warmup=3):
     return sum(ms) / len(ms), min(ms)
 
 
-def _hbm_entry(name, nbytes, avg, best, peaks, extra=None):
+def _hbm_entry(name, nbytes, avg, best, peaks, extra=None, config=None, kernel=None):
+    """One HBM-bound line.  `achieved` counts the ALGORITHMIC bytes; where an ncu capture of the kernel
+    as it stands exists, `achieved_dram` is that capture's DRAM bytes per launch over the same time."""
     gbs = nbytes / (avg * 1e-3) / 1e9
-    e = {"op": name, "bound": "hbm", "bytes": nbytes, "ms": avg, "best_ms": best, "achieved": gbs, "unit": "GB/s",
+    traffic = ncu_traffic(name)
+    e = {"op": name, "config": config, "kernel": kernel, "bound": "hbm", "bytes": nbytes, "ms": avg, "best_ms": best,
+         "achieved": gbs, "unit": "GB/s",
          "peak": peaks["hbm_gbs"], "frac_measured": gbs / peaks["hbm_gbs"], "frac_nominal": gbs / NOMINAL_HBM_GBS,
-         "traffic": ncu_traffic(name)}
+         "traffic": traffic}
+    if traffic is not None:
+        e["achieved_dram"] = traffic / (avg * 1e-3) / 1e9
+        e["frac_dram"] = e["achieved_dram"] / peaks["hbm_gbs"]
     if extra:
         e.update(extra)
     return e
 
 
-def _tensor_entry(name, flops, avg, best, peaks, extra=None):
+def _tensor_entry(name, flops, avg, best, peaks, extra=None, config=None, kernel="matmul_tc_kernel"):
     tf = flops / (avg * 1e-3) / 1e12
-    e = {"op": name, "bound": "tensor", "flops": flops, "ms": avg, "best_ms": best, "achieved": tf, "unit": "TFLOP/s",
+    e = {"op": name, "config": config, "kernel": kernel, "bound": "tensor", "flops": flops, "ms": avg, "best_ms": best,
+         "achieved": tf, "unit": "TFLOP/s",
          "peak": peaks["bf16_tflops"], "frac_measured": tf / peaks["bf16_tflops"], "traffic": ncu_traffic(name),
          "frac_sustained": tf / peaks["bf16_tflops_sustained"], "frac_nominal": tf / NOMINAL_BF16_TFLOPS}
     if extra:
@@ -520,17 +535,103 @@ def section_extras(sbp, device, peaks, opts):
     return res
 
 
+def section_cliffs(sbp, device, peaks, opts):
+    """Shapes that miss the fast paths' rules, next to their nearest regular neighbour: a bf16 product
+    whose shard width is not a multiple of 8 elements (the TMA stride rule), and P(sum) -> B with shard
+    counts outside {1, 2, 4, 8} (the unrolled reductions)."""
+    bf16 = torch.bfloat16
+    res = []
+    k, M, K = 8, 8192, 4096
+    X = dg.normal(1003, 0, (M, K), 0.0, 1.0, bf16, device)
+    x = sbp.SbpTensor((M, K), bf16, sbp.B, [X] * k)
+    for width in (336, 333):
+        N = k * width
+        w = sbp.SbpTensor((K, N), bf16, sbp.S(1), [dg.normal(1003, 80 + r, (K, width), 0.0, 0.02, bf16, device) for r in range(k)])
+        y = sbp.empty_global((M, N), bf16, sbp.S(1), k, device=device)
+        ws = torch.empty(max(1, sbp.sbp_matmul_workspace_bytes(x, w, y)), dtype=torch.uint8, device=device)
+        avg, best = time_op(lambda: sbp.sbp_matmul(x, w, y, 0, ws), device, iters=5)
+        res.append(_tensor_entry(f"bf16 product (B,S(1))->S(1), [8192,4096] x [4096,{N}], shard width {width}"
+                                 + ("" if width % 8 == 0 else " (not a multiple of 8)"),
+                                 2.0 * M * K * N, avg, best, peaks, kernel=None))
+        del w, y, ws
+    del x, X
+    torch.cuda.empty_cache()
+    shape = (8192, 8192)
+    tb = shape[0] * shape[1] * 2
+    for kk in (3, 4, 16):
+        src = sbp.SbpTensor(shape, bf16, sbp.P_SUM, [dg.normal(SEED, 400 + r, shape, 0.0, 1.0, bf16, device) for r in range(kk)])
+        dst = sbp.empty_global(shape, bf16, sbp.B, kk, device=device)
+        avg, best = time_op(lambda: sbp.sbp_boxing(src, dst), device, iters=5)
+        res.append(_hbm_entry(f"P(sum)->B, k={kk}, bf16 [8192,8192]", 2 * kk * tb, avg, best, peaks))
+        del src, dst
+        torch.cuda.empty_cache()
+    return res
+
+
+# BASELINE config each operator section belongs to (None: beyond the five configs)
+SECTION_CONFIG = {"softmax": 4, "classifier": 4, "mlp": 3, "embedding": 5, "extras": None, "cliffs": None}
+
+# kernel behind an HBM-bound line, by the start of its name (tensor-bound lines: matmul_tc_kernel)
+HBM_KERNELS = [
+    ("softmax-xent on bf16", "xent_partial_kernel+xent_combine_kernel"),
+    ("softmax-xent backward", "xent_backward_kernel"),
+    ("embedding fused", "embedding_kernel<fused>"),
+    ("embedding unfused", "embedding_kernel+box_tile_kernel"),
+    ("embedding, table S(1)", "embedding_s1_kernel"),
+    ("embedding backward", "embedding_backward_kernel"),
+    ("MLP P(sum)->B", "box_tile_kernel"),
+    ("S(0)->P(sum)", "box_scatter_kernel"), ("B->P(sum)", "box_scatter_kernel"),
+    ("S(0) fp32 -> B bf16", "box_gather_cast_kernel"),
+    ("disjoint placements", "box_disjoint_kernel"),
+    ("P(sum)->B, k=", "box_tile_kernel"),
+]
+
+
 def run_operator_sections(sbp, device, peaks, opts):
     which = opts.ops
     out = []
     table = {"softmax": section_softmax, "classifier": section_classifier_gemm, "mlp": section_mlp,
-             "embedding": section_embedding, "extras": section_extras}
-    for fn in [table[w.strip()] for w in which.split(",") if w.strip()]:
+             "embedding": section_embedding, "extras": section_extras, "cliffs": section_cliffs}
+    for w in [w.strip() for w in which.split(",") if w.strip()]:
+        fn = table[w]
         try:
-            out.extend(fn(sbp, device, peaks, opts))
+            res = fn(sbp, device, peaks, opts)
         except sbp.SbpError as e:            # an operator the library refuses is reported, not hidden
-            out.append({"op": fn.__name__, "error": str(e)})
+            res = [{"op": fn.__name__, "error": str(e)}]
+        for e in res:
+            if e.get("config") is None:
+                e["config"] = SECTION_CONFIG[w]
+            if e.get("kernel") is None and "op" in e:
+                e["kernel"] = next((kn for pre, kn in HBM_KERNELS if e["op"].startswith(pre)), None)
+        out.extend(res)
         torch.cuda.empty_cache()
+    return out
+
+
+def roofline_configs(per, ops):
+    """Compact per-config roofline lines for the record: config 2's transforms, then every operator
+    line of configs 3-5.  frac = achieved / peak with the peak of the line's own bound; HBM lines
+    with an ncu capture also carry the DRAM-byte figure (achieved_dram, frac_dram)."""
+    out = []
+    for t in per:
+        e = {"config": 2, "line": t["transform"], "kernel": "box_tile_kernel", "bound": "hbm", "ms": t["ms"],
+             "work": t["bytes"], "achieved": t["gbs"], "unit": "GB/s", "frac": t["frac_measured"],
+             "ms_back_to_back": t.get("ms_back_to_back"), "frac_back_to_back": t.get("frac_measured_back_to_back")}
+        tr = ncu_traffic(t["transform"])
+        if tr is not None:
+            e["traffic"] = tr
+            e["achieved_dram"] = tr / (t["ms"] * 1e-3) / 1e9
+        out.append(e)
+    for o in ops or []:
+        if "error" in o or o.get("config") is None:
+            continue
+        e = {"config": o["config"], "line": o["op"], "kernel": o.get("kernel"), "bound": o["bound"], "ms": o["ms"],
+             "work": o.get("bytes", o.get("flops")), "achieved": o["achieved"], "unit": o["unit"],
+             "frac": o["frac_measured"]}
+        for key in ("traffic", "achieved_dram", "frac_dram", "hbm_gbs", "hbm_frac_measured", "frac_sustained"):
+            if o.get(key) is not None:
+                e[key] = o[key]
+        out.append(e)
     return out
 
 
@@ -556,6 +657,100 @@ def oracle_sweep_sample(rows: int):
         assert len(out) == k
         nbytes += units * rows * SWEEP_SHAPE[1] * 2
     return nbytes, time.perf_counter() - t0, 1
+
+
+def host_cores():
+    """Cores this process may run on (what the oracle has at its disposal)."""
+    try:
+        return len(os.sched_getaffinity(0))
+    except AttributeError:
+        return os.cpu_count() or 1
+
+
+def blas_threads():
+    """Threads numpy's BLAS uses for the oracle's float64 matrix products; everything else in the
+    oracle is single-threaded numpy."""
+    try:
+        from threadpoolctl import threadpool_info
+        n = [int(i.get("num_threads", 1)) for i in threadpool_info() if i.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return 1
+
+
+def oracle_config_samples(gen_device="cpu"):
+    """The CPU oracle, as it stands, timed on a bounded sample of configs 3, 4 and 5 (config 2 is
+    oracle_sweep_sample).  Inputs are drawn on gen_device and copied to the host before the clock
+    starts.  Rows / lookups are independent, so a sample's time scales linearly to the full
+    workload; `scale` is that factor and `full_s_extrapolated` = seconds * scale."""
+    import numpy as np
+    from oracle import sbp_oracle as O
+    bf16, f32 = torch.bfloat16, torch.float32
+    k = 8
+    cores, bt = host_cores(), blas_threads()
+
+    def host(t):
+        return t.float().cpu().numpy() if t.dtype == bf16 else t.cpu().numpy()
+
+    out = []
+
+    def add(config, what, work, unit_work, secs, scale, threads, sample):
+        out.append({"config": config, "what": what, "seconds": secs, "value": work / secs / 1e9,
+                    "unit": unit_work, "scale": scale, "full_s_extrapolated": secs * scale,
+                    "cores": cores, "threads_used": threads, "sample": sample})
+
+    # config 3: Y = GeLU(X W1) W2 in float64 on the first rows of X (all columns)
+    M, H, F, rows = 8192, 4096, 16384, 128
+    X = host(dg.normal(1003, 0, (rows, H), 0.0, 1.0, bf16, gen_device))
+    W1 = np.concatenate([host(dg.normal(1003, 10 + r, (H, F // k), 0.0, 0.02, bf16, gen_device)) for r in range(k)], axis=1)
+    W2 = np.concatenate([host(dg.normal(1003, 30 + r, (F // k, H), 0.0, 0.02, bf16, gen_device)) for r in range(k)], axis=0)
+    t0 = time.perf_counter()
+    Y = O.mlp_logical(X, W1, W2)
+    secs = time.perf_counter() - t0
+    assert Y.shape == (rows, H)
+    add(3, "MLP block GeLU(X W1) W2, float64", 2 * 2.0 * rows * H * F, "GFLOP/s", secs, M / rows, bt,
+        f"first {rows} of {M} rows of X, all of W1 and W2")
+    del W1, W2, Y
+
+    # config 4: one shard's logits product in float64, then the split softmax-xent on a row sample
+    R, feat, classes = 512, 512, 1 << 20
+    Fm = host(dg.normal(1004, 0, (R, feat), 0.0, 1.0, bf16, gen_device))
+    W0 = host(dg.normal(1004, 40, (feat, classes // k), 0.0, 0.01, bf16, gen_device))
+    t0 = time.perf_counter()
+    Z0 = O.matmul_logical(Fm, W0)
+    secs = time.perf_counter() - t0
+    assert Z0.shape == (R, classes // k)
+    add(4, "classifier logits F W, float64", 2.0 * R * feat * (classes // k), "GFLOP/s", secs, k, bt,
+        f"shard 0 of {k} of the class-split weight, all {R} rows")
+    del W0, Z0
+    rs = 64
+    sigma = (512 ** 0.5) * 0.01
+    zl = [host(dg.normal(1004, 10 + r, (rs, classes // k), 0.0, sigma, bf16, gen_device)) for r in range(k)]
+    labels = dg.integers(1004, 1, (rs,), 0, classes, gen_device).cpu().numpy()
+    t0 = time.perf_counter()
+    m, S, loss = O.softmax_xent_split(zl, labels)
+    secs = time.perf_counter() - t0
+    assert loss.shape == (rs,)
+    add(4, "split softmax cross entropy on bf16 logits", rs * classes * 2.0, "GB/s", secs, R / rs, 1,
+        f"first {rs} of {R} rows, all {classes} classes over {k} shards")
+    del zl
+
+    # config 5: row-split lookup -> P(sum) partials, then their fixed-order sum (the unfused path the
+    # paper describes), on a table and batch of 1/8 the size
+    trows, dim, batch = 1 << 21, 128, 2048
+    table = [host(dg.uniform(1005, 100 + r, (trows // k, dim), -0.05, 0.05, f32, gen_device)) for r in range(k)]
+    ids = dg.zipf_ids(1005, 1, (batch, 26), trows, 1.05, gen_device).cpu().numpy()
+    t0 = time.perf_counter()
+    parts = O.embedding_partials(table, ids)
+    got = O.boxing(parts, O.PSUM, O.B, "f32")
+    secs = time.perf_counter() - t0
+    assert got[0].shape == (batch, 26, dim)
+    n = batch * 26
+    add(5, "embedding gather -> P(sum) partials, then P(sum) -> B", n * 8.0 + 2.0 * n * dim * 4, "GB/s", secs,
+        65536 / batch, 1,
+        f"{batch} of 65536 samples x 26 fields, table of {trows} rows (1/8 of 2^24) over {k} shards; "
+        "bytes counted as ids + rows gathered + one result written")
+    return out
 
 
 # ------------------------------------------------------------------------------ ranks
@@ -585,9 +780,12 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-ops", action="store_true", help="skip the sharded-operator sections (N = 1 only)")
-    ap.add_argument("--ops", default="softmax,classifier,mlp,embedding,extras",
-                    help="comma-separated operator sections to run: softmax, classifier, mlp, embedding, extras")
+    ap.add_argument("--ops", default="softmax,classifier,mlp,embedding,extras,cliffs",
+                    help="comma-separated operator sections to run: softmax, classifier, mlp, embedding, extras, cliffs")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dry-run-cpu", action="store_true",
+                    help="rank plumbing only, on CPU over gloo: launch, world-size check, barrier, slowest-rank timing, "
+                         "rank 0's JSON line; no kernel runs and the line is not a measurement")
     ap.add_argument("--op-iters", type=int, default=None, help="timed repeats per operator line (default 5-10)")
     ap.add_argument("--op-warmup", type=int, default=None, help="warm-up repeats per operator line (default 3; >= 3 for a valid number)")
     ap.add_argument("--copy-engine", type=int, default=0)
@@ -620,10 +818,57 @@ def reference_arm(args):
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_s / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": "boxing sweep bf16 [8192,8192] k=4, 7 transforms (CPU oracle on a row sample)"},
-        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": host_cores(), "threads_used": cores, "kind": "oracle",
+                         "sample": sample},
         "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
     print(json.dumps(line))
+    return 0
+
+
+def launch_ranks_if_needed(args):
+    """--gpus N is the number of ranks.  Started plainly (no WORLD_SIZE) with N > 1, this process
+    starts the N ranks itself through torch.distributed.run on 127.0.0.1 and returns their exit
+    code; started by a launcher, the launcher's WORLD_SIZE must equal N (exit code 2 otherwise).
+    Returns None when this process is a rank (or the only one) and should go on."""
+    ws = os.environ.get("WORLD_SIZE")
+    if ws is not None:
+        if int(ws) != args.gpus:
+            sys.stderr.write(f"bench.py: --gpus {args.gpus} but the launcher started WORLD_SIZE={ws} ranks\n")
+            return 2
+        return None
+    if args.gpus <= 1 or args.impl == "reference":     # the oracle arm is one CPU process whatever N is
+        return None
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={args.gpus}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    return subprocess.call(cmd)
+
+
+def dry_run_cpu(args):
+    """The multi-rank plumbing of the benchmark with the GPU work left out: gloo process group on CPU,
+    barrier, a stand-in per-rank time (rank r: 1 + r ms), slowest rank's time, whole-job value, one
+    JSON line from rank 0.  Exists so that the launch path can be tested where there is no GPU."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("gloo")
+        dist.barrier()
+    ms_step = max_over_ranks(1.0 + rank, dist, torch.device("cpu"))
+    if dist is not None:
+        dist.barrier()
+    if rank == 0:
+        print(json.dumps({"metric": METRIC, "dry_run": True, "value": whole_job_gbs(world, ms_step), "unit": "GB/s",
+                          "n_gpus": args.gpus, "world_size": world, "steps": args.steps, "warmup": args.warmup,
+                          "ms_per_step": ms_step, "scaling": "weak", "data": "none (dry run on CPU)"}))
+    if dist is not None:
+        dist.destroy_process_group()
     return 0
 
 
@@ -631,8 +876,13 @@ def main():
     args = parse()
     global SWEEP_SHAPE
     SWEEP_SHAPE = (args.rows, SWEEP_SHAPE[1])
+    rc = launch_ranks_if_needed(args)
+    if rc is not None:
+        return rc
     if args.impl == "reference":
         return reference_arm(args)
+    if args.dry_run_cpu:
+        return dry_run_cpu(args)
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
@@ -717,7 +967,7 @@ def main():
                 "unit": "GB/s", "frac": dom["gbs"] / peaks["hbm_gbs"], "traffic": ncu_traffic(dom["transform"])}
 
     line = {
-        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+        "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,
         "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
         "config": {"workload": f"boxing sweep: logical bf16 [{SWEEP_SHAPE[0]},{SWEEP_SHAPE[1]}] N(0,1), k=4, 7 transforms per step",
@@ -742,16 +992,25 @@ def main():
         line["e2e"] = None
 
     if rank == 0 and world == 1:
-        if not args.no_cpu_baseline:
-            rows = SWEEP_SHAPE[0]
-            nbytes, secs, cores = oracle_sweep_sample(rows)
-            line["cpu_baseline"] = {"value": nbytes / secs / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
-                                    "sample": f"first {rows} of {SWEEP_SHAPE[0]} rows of every local tensor, "
-                                              f"all 7 transforms once ({secs:.1f} s)"}
         if not args.no_ops:
             del T, src, work
             torch.cuda.empty_cache()
             line["ops"] = run_operator_sections(sbp, device, peaks, args)
+        # every config's lines inside the roofline object (the sweep's dominant kernel stays on top)
+        line["roofline"]["configs"] = roofline_configs(per, line.get("ops"))
+        if not args.no_cpu_baseline:
+            rows = SWEEP_SHAPE[0]
+            nbytes, secs, threads = oracle_sweep_sample(rows)
+            base = {"value": nbytes / secs / 1e9, "unit": "GB/s", "cores": host_cores(), "threads_used": threads,
+                    "kind": "oracle",
+                    "sample": f"config 2: first {rows} of {SWEEP_SHAPE[0]} rows of every local tensor, "
+                              f"all 7 transforms once ({secs:.1f} s)"}
+            cfgs = [{"config": 2, "what": "boxing sweep, 7 transforms", "seconds": secs, "value": base["value"],
+                     "unit": "GB/s", "scale": 1.0, "full_s_extrapolated": secs, "cores": base["cores"],
+                     "threads_used": threads, "sample": "the whole sweep"}]
+            cfgs.extend(oracle_config_samples(device))
+            base["configs"] = cfgs
+            line["cpu_baseline"] = base
     if rank == 0:
         print(json.dumps(line))
     if dist is not None:

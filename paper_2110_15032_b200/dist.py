@@ -41,8 +41,10 @@ class ShardMap:
 
 
 def _split_range(n: int, k: int, r: int):
-    base, rem = divmod(n, k)
-    return r * base + min(r, rem), base + (1 if r < rem else 0)
+    """(start, length) of shard r's piece of an axis of length n split k ways.  The split rule lives
+    in the library alone: the lengths are asked from sbp_local_shape, the start is their running sum."""
+    lens = [_b.sbp_local_shape((n,), _b.S(0), k, i)[0] for i in range(r + 1)]
+    return sum(lens[:-1]), lens[-1]
 
 
 def sources_read(src_sig: _b.Sig, dst_sig: _b.Sig, p: int, q: int, dst_shard: int, shape: Sequence[int]) -> List[int]:

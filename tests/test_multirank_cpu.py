@@ -69,3 +69,42 @@ def test_reference_arm_only_rank0_reports(monkeypatch):
     line = json.loads(buf.getvalue())
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["value"] == pytest.approx(1000 / 0.5 / 1e9)
+
+
+def _run_bench(argv, env_extra=None, timeout=300):
+    import subprocess
+    import sys
+    env = {k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    env.update(env_extra or {})
+    return subprocess.run([sys.executable, os.path.join(os.path.dirname(bench.__file__), "bench.py")] + argv,
+                          capture_output=True, text=True, timeout=timeout, env=env)
+
+
+def test_gpus_flag_starts_the_ranks_itself_dry_run():
+    """`python bench.py --gpus 2` with no launcher around it: the process starts two ranks through
+    torch.distributed.run, and rank 0 alone prints one line that claims two ranks."""
+    r = _run_bench(["--gpus", "2", "--steps", "3", "--warmup", "1", "--dry-run-cpu"])
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [ln for ln in r.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["n_gpus"] == 2 and d["world_size"] == 2 and d["dry_run"] is True
+    assert d["ms_per_step"] == 2.0                                # the slow rank's stand-in time
+    assert d["value"] == pytest.approx(2 * bench.step_bytes() / 2.0e-3 / 1e9)
+
+
+def test_world_size_that_contradicts_gpus_is_refused():
+    r = _run_bench(["--gpus", "4", "--dry-run-cpu"], {"WORLD_SIZE": "2", "RANK": "0", "LOCAL_RANK": "0",
+                                                      "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(_free_port())})
+    assert r.returncode == 2
+    assert "WORLD_SIZE=2" in r.stderr and r.stdout.strip() == ""
+    # the reference arm checks the same thing, and prints n_gpus from the same flag
+    r = _run_bench(["--gpus", "4", "--impl", "reference"], {"WORLD_SIZE": "2", "RANK": "0"})
+    assert r.returncode == 2
+
+
+def test_single_process_dry_run_is_one_rank():
+    r = _run_bench(["--dry-run-cpu"])
+    assert r.returncode == 0, r.stderr[-2000:]
+    d = json.loads(r.stdout.strip().splitlines()[-1])
+    assert d["n_gpus"] == 1 and d["world_size"] == 1 and d["ms_per_step"] == 1.0

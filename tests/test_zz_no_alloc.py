@@ -4,26 +4,31 @@ Some users of this library run where device allocation is off the table: all mem
 planned and handed out before they were called, or they sit on a path that must never enter
 the allocator.  sbp_softmax_xent_static serves them by keeping its partial vectors in an
 array built into the library.  This file checks, through the C ABI, that it returns what the
-workspace-taking entry point returns -- twice in a row on different inputs, because the
-built-in array is shared and still holds the previous call's values -- and that a shape
-beyond the array's size is refused.  It is collected last on purpose."""
+workspace-taking entry point returns, bit for bit -- twice in a row on different inputs,
+because the built-in array is shared and still holds the previous call's values -- that both
+agree with the CPU oracle, and that a shape beyond the array's size is refused.  It is
+collected last on purpose."""
 import numpy as np
 import pytest
 import torch
-from helpers import assert_close, make_global, split_cpu, to_np
+from helpers import assert_close, bits, make_global, split_cpu, to_np
 
 import paper_2110_15032_b200 as sbp
 import sbp_datagen as dg
+from oracle import sbp_oracle as O
 
 pytestmark = pytest.mark.gpu
 
 F32, BF16, I64 = torch.float32, torch.bfloat16, torch.int64
 
 
-def _both_ways(rows, classes, k, seed, sigma):
-    Z = dg.normal(seed, 0, (rows, classes), 0.0, sigma, BF16)
+def _both_ways(rows, classes, k, seed, sigma, dtype=BF16):
+    """Runs the workspace-taking and the workspace-free entry point on the same inputs.  They launch
+    the same kernels with the same tiling, so their outputs must agree bit for bit; both are also
+    held to the oracle's split softmax within the library's stated tolerance."""
+    Z = dg.normal(seed, 0, (rows, classes), 0.0, sigma, dtype)
     labels = dg.integers(seed, 1, (rows,), 0, classes)
-    logits = make_global(split_cpu(Z, sbp.S(1), k), (rows, classes), BF16, sbp.S(1))
+    logits = make_global(split_cpu(Z, sbp.S(1), k), (rows, classes), dtype, sbp.S(1))
     lab = make_global([labels] * k, (rows,), I64, sbp.B)
     outs = []
     for static in (False, True):
@@ -39,15 +44,27 @@ def _both_ways(rows, classes, k, seed, sigma):
             ws = torch.empty(sbp.sbp_softmax_xent_workspace_bytes(logits), dtype=torch.uint8, device="cuda")
             sbp.sbp_softmax_xent(logits, lab, loss, rmax, rsum, ws)
         torch.cuda.synchronize()
-        outs.append([to_np(g.locals[r]) for g in (loss, rmax, rsum) for r in range(k)])
+        outs.append([bits(g.locals[r]) for g in (loss, rmax, rsum) for r in range(k)])
+        m, S, ref = O.softmax_xent_split(O.to_locals(to_np(Z), O.S1, k), labels.numpy())
+        for r in range(k):
+            assert np.array_equal(to_np(rmax.locals[r]), m.astype(np.float32)), "boxed row max is exact"
+            assert_close(to_np(rsum.locals[r]), S, 2e-2, 1e-3, "row sum vs oracle")
+            assert_close(to_np(loss.locals[r]), ref, 2e-2, 1e-3, "loss vs oracle")
     for a, b in zip(*outs):
-        assert np.all(np.isfinite(b))
-        assert_close(b, a, 2e-2, 1e-3, "built-in scratch vs caller workspace")
+        assert np.array_equal(a, b), "built-in scratch and caller workspace must give identical bits"
 
 
 def test_static_scratch_matches_workspace_entry_point_twice_in_a_row():
+    # The call with many parts goes first, so the second call's (fewer) parts sit in a region
+    # that still holds the first call's values: stale entries would show up as wrong bits.
     _both_ways(96, 40000, 8, seed=9001, sigma=1.0)      # several column spans per shard
-    _both_ways(33, 4096, 4, seed=9002, sigma=3.0)       # fewer parts: stale entries stay behind it
+    _both_ways(33, 4096, 4, seed=9002, sigma=3.0)
+
+
+def test_static_scratch_fp32_and_element_wise_paths():
+    _both_ways(40, 20000, 8, seed=9003, sigma=2.0, dtype=F32)    # fp32 logits
+    _both_ways(17, 1003, 4, seed=9004, sigma=1.5)                # class count not a multiple of 8: element-wise loads
+    _both_ways(9, 77, 2, seed=9005, sigma=1.0, dtype=F32)
 
 
 def test_static_scratch_refuses_oversized_shapes():

@@ -85,6 +85,16 @@ typedef struct {
  *   local[r]         device pointer of shard r's local tensor, r in [0, k).  For a B
  *                    tensor the k replicas may all be the same pointer; a kernel then
  *                    writes that buffer once.
+ *   local_ld[r]      leading dimension of shard r's local tensor, in elements: the distance between
+ *                    consecutive rows when the local tensor is viewed as [rows, cols] with cols its
+ *                    last local extent and rows the product of the others.  0 means dense
+ *                    (local_ld = cols); otherwise local_ld[r] >= cols.  A local tensor with a
+ *                    leading dimension is a window into a larger buffer -- a column block of a
+ *                    replica (Table 2: B -> S costs nothing, see sbp_view_b_to_s) or a sub-block of a
+ *                    matrix.  Honoured by sbp_matmul (all three tensors), by sbp_boxing on 2-D tensors
+ *                    of one placement (S / B / P on either side, except the P(sum)-destination and
+ *                    cast rows) and by sbp_softmax_xent / sbp_softmax_xent_backward (logits, grad);
+ *                    every other entry point answers SBP_ERR_UNSUPPORTED to a non-dense tensor.
  */
 typedef struct {
   int32_t ndim;
@@ -94,6 +104,7 @@ typedef struct {
   int32_t pshape[SBP_MAX_PDIMS];
   sbp_sig sbp[SBP_MAX_PDIMS];
   void* local[SBP_MAX_K];
+  int64_t local_ld[SBP_MAX_K];
 } sbp_tensor;
 
 /* ---------------------------------------------------------------- descriptors, rules */
@@ -107,6 +118,16 @@ uint64_t sbp_launch_count(void);
 
 /* Local shape of shard r under t's signature (Section 3.1).  Host only, no CUDA. */
 sbp_status sbp_local_shape(const sbp_tensor* t, int32_t r, int64_t out_shape[SBP_MAX_DIMS]);
+
+/* B -> S(axis) without moving anything (Table 2: "B -> S" costs 0; Section 3.2: such a boxing "may
+ * not lead to data movement").  Fills *view with a descriptor of the same global tensor under
+ * S(axis) whose local tensors are windows into b's replicas: view->local[r] points at shard r's
+ * piece inside b->local[r] and view->local_ld[r] carries the replica's row length when the piece
+ * is not contiguous (a split of the last axis).  b must be a B tensor on a one-axis placement;
+ * axis 0 or the last axis (any other axis of an N-D tensor would need two strides:
+ * SBP_ERR_UNSUPPORTED).  Nothing is launched or copied; the view aliases b's memory, so writing
+ * through one is visible through the other.  Host only, no CUDA. */
+sbp_status sbp_view_b_to_s(const sbp_tensor* b, int32_t axis, sbp_tensor* view);
 
 /* Table 1 ("Valid SBP signatures for MatMul"): signature of Y = XW from those of X and
  * W, or SBP_ERR_SIGNATURE when the pair is not one of the table's six rows. */
@@ -250,6 +271,13 @@ void sbp_boxing_set_copy_engine(int32_t engine);
 #define SBP_TRANS_X 2u
 #define SBP_TRANS_W 4u
 size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y);   /* untransposed operands */
+
+/* The tensor-core path describes every operand and result tile layout to the copy engine with a
+ * descriptor that the driver encodes on the host.  The library keeps the descriptors it has
+ * encoded, keyed by address and layout, and re-uses them when a product is called again on the
+ * same buffers.  This reports how many were re-used and how many encoded since the library was
+ * loaded (process-wide), so that a harness can check that a steady-state call encodes nothing. */
+void sbp_tensor_map_stats(uint64_t* reused, uint64_t* encoded);
 sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, uint32_t flags,
                       void* ws, size_t ws_bytes, void* cuda_stream);
 

@@ -32,6 +32,7 @@ class _Tensor(C.Structure):
         ("pshape", C.c_int32 * SBP_MAX_PDIMS),
         ("sbp", _Sig * SBP_MAX_PDIMS),
         ("local", C.c_void_p * SBP_MAX_K),
+        ("local_ld", C.c_int64 * SBP_MAX_K),
     ]
 
 
@@ -89,6 +90,7 @@ def load_library():
     lib.sbp_last_error.restype = C.c_char_p
     lib.sbp_launch_count.restype = C.c_uint64
     lib.sbp_local_shape.argtypes = [T, C.c_int32, C.POINTER(C.c_int64)]
+    lib.sbp_view_b_to_s.argtypes = [T, C.c_int32, T]
     lib.sbp_matmul_infer.argtypes = [_Sig, _Sig, C.POINTER(_Sig)]
     lib.sbp_transfer_cost.argtypes = [_Sig, _Sig, C.c_int32, C.c_int32, C.c_int32, C.c_uint64, C.POINTER(C.c_uint64)]
     lib.sbp_boxing.argtypes = [T, T, C.c_void_p]
@@ -104,6 +106,8 @@ def load_library():
     lib.sbp_matmul_workspace_bytes.restype = C.c_size_t
     lib.sbp_matmul_workspace_bytes.argtypes = [T, T, T]
     lib.sbp_matmul.argtypes = [T, T, T, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sbp_tensor_map_stats.argtypes = [C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+    lib.sbp_tensor_map_stats.restype = None
     lib.sbp_softmax_xent_workspace_bytes.restype = C.c_size_t
     lib.sbp_softmax_xent_workspace_bytes.argtypes = [T]
     lib.sbp_softmax_xent.argtypes = [T, T, T, T, T, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -124,11 +128,30 @@ def _check(status: int):
         raise SbpError(status, lib.sbp_status_string(status).decode(), lib.sbp_last_error().decode())
 
 
+def _row_pitch(t: torch.Tensor):
+    """Leading dimension to pass for a local tensor: 0 when it is contiguous, the distance between its
+    rows (in elements) when it is a row-strided window, None when it is neither."""
+    if t.is_contiguous():
+        return 0
+    if t.dim() < 2 or t.stride(-1) != 1:
+        return None
+    pitch = t.stride(-2)
+    if pitch < t.shape[-1]:
+        return None
+    for i in range(t.dim() - 2):                 # every axis before the last two is dense over the pitch
+        if t.shape[i] != 1 and t.stride(i) != t.stride(i + 1) * t.shape[i + 1]:
+            return None
+    return int(pitch)
+
+
 class SbpTensor:
     """A global tensor = logical shape + dtype + signature + the k local tensors.
 
     `locals` are torch tensors used purely as memory (device memory for every entry
-    point except sbp_boxing_host, which takes host tensors).  Each must be contiguous.
+    point except sbp_boxing_host, which takes host tensors).  Each must be contiguous, or a
+    window of a larger row-major buffer whose rows are a fixed distance apart (unit stride on the
+    last axis, every axis before the last two dense): that distance is passed on as the
+    descriptor's leading dimension.
     For a two-axis placement (the paper's multi-dimensional SBP) pass `sig` as a pair of
     signatures and `pshape=(k0, k1)`; `locals` then lists the devices row-major (i * k1 + j).
     """
@@ -152,8 +175,8 @@ class SbpTensor:
         for t in self.locals:
             if t is None:            # a local tensor another device holds (sbp_boxing_shard)
                 continue
-            if not t.is_contiguous():
-                raise ValueError("local tensors must be contiguous")
+            if _row_pitch(t) is None:
+                raise ValueError("local tensors must be contiguous, or row-strided windows of a row-major buffer")
             if t.dtype != dtype:
                 raise ValueError("local tensor dtype differs from the descriptor's")
 
@@ -170,6 +193,7 @@ class SbpTensor:
             d.sbp[p] = self.sigs[p]._c()
         for r, t in enumerate(self.locals):
             d.local[r] = t.data_ptr() if t is not None else None
+            d.local_ld[r] = _row_pitch(t) if t is not None else 0
         return d
 
 
@@ -199,6 +223,26 @@ def sbp_local_shape(shape, sig, k, r: int, dtype=torch.float32):
     return tuple(out[i] for i in range(len(shape)))
 
 
+def sbp_view_b_to_s(b: SbpTensor, axis: int) -> SbpTensor:
+    """The B tensor `b` seen as S(axis) without moving anything (Table 2: B -> S costs nothing): the
+    local tensors of the result are windows into b's replicas.  The pointers and leading dimensions
+    come from the library; the torch views built here only keep the memory alive and are checked
+    against them."""
+    out = _Tensor()
+    _check(load_library().sbp_view_b_to_s(C.byref(b._c()), int(axis), C.byref(out)))
+    locs = []
+    start = 0
+    for r, t in enumerate(b.locals):
+        ln = sbp_local_shape(b.shape, S(axis), b.k, r, b.dtype)[axis]
+        v = t.narrow(axis, start, ln)
+        start += ln
+        if ln > 0 and v.numel() > 0:
+            if v.data_ptr() != out.local[r] or (_row_pitch(v) or 0) != (out.local_ld[r] if out.local_ld[r] != v.shape[-1] else 0):
+                raise RuntimeError("sbp_view_b_to_s: the library's view and the torch view disagree")
+        locs.append(v)
+    return SbpTensor(b.shape, b.dtype, S(axis), locs)
+
+
 def empty_global(shape, dtype, sig, k, device="cuda", alias_replicas: bool = False) -> SbpTensor:
     """Allocates (torch.empty) the local tensors of a global tensor (k an int, or (k0, k1))."""
     pshape = tuple(k) if isinstance(k, (tuple, list)) else None
@@ -223,6 +267,13 @@ def sbp_transfer_cost(src: Sig, dst: Sig, p1: int, p2: int, disjoint: bool, t_by
     out = C.c_uint64()
     _check(load_library().sbp_transfer_cost(src._c(), dst._c(), p1, p2, 1 if disjoint else 0, t_bytes, C.byref(out)))
     return int(out.value)
+
+
+def sbp_tensor_map_stats():
+    """(re-used, encoded) counts of the tensor-core path's copy-engine descriptors."""
+    a, b = C.c_uint64(), C.c_uint64()
+    load_library().sbp_tensor_map_stats(C.byref(a), C.byref(b))
+    return int(a.value), int(b.value)
 
 
 def sbp_launch_count() -> int:

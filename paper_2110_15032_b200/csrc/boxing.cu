@@ -31,6 +31,7 @@ struct TaskGeom {
   long long la;
   long long Na_s, aoff_s, Nb_s, boff_s;
   long long Na_d, aoff_d, Nb_d, boff_d;
+  long long Ps, Pd;           // row pitch on either side (the local Nb extent unless a leading dimension is given)
 };
 
 __device__ __forceinline__ void task_geometry(const BoxParams& p, int s, int d, int vbytes, TaskGeom* g) {
@@ -46,6 +47,8 @@ __device__ __forceinline__ void task_geometry(const BoxParams& p, int s, int d, 
   g->Nb_s = p.src_b ? lb : p.Nb;  g->boff_s = p.src_b ? 0 : b0;
   g->Na_d = p.dst_a ? la : p.Na;  g->aoff_d = p.dst_a ? 0 : a0;
   g->Nb_d = p.dst_b ? lb : p.Nb;  g->boff_d = p.dst_b ? 0 : b0;
+  g->Ps = p.src_pitch[s] ? p.src_pitch[s] : g->Nb_s;
+  g->Pd = p.dst_pitch[d] ? p.dst_pitch[d] : g->Nb_d;
 }
 
 // V: vector type moved by one thread access.  OP: BoxOp.  J: vectors per thread.
@@ -95,8 +98,8 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
       x = q / g.la;
       ia = q - x * g.la;
     }
-    so[j] = ((((x * g.Na_s + g.aoff_s + ia) * p.M + m) * g.Nb_s + g.boff_s) * cs) / (long long)sizeof(V) + col;
-    dofs[j] = ((((x * g.Na_d + g.aoff_d + ia) * p.M + m) * g.Nb_d + g.boff_d) * cs) / (long long)sizeof(V) + col;
+    so[j] = ((((x * g.Na_s + g.aoff_s + ia) * p.M + m) * g.Ps + g.boff_s) * cs) / (long long)sizeof(V) + col;
+    dofs[j] = ((((x * g.Na_d + g.aoff_d + ia) * p.M + m) * g.Pd + g.boff_d) * cs) / (long long)sizeof(V) + col;
   }
 
   SBP_PDL_WAIT();   // the previous kernel's results are visible from here on
@@ -296,6 +299,7 @@ static std::atomic<int> g_copy_engine{0};
 
 struct Plan {
   BoxParams p;
+  bool pitched;     // some local tensor has a leading dimension: only the tile kernel applies
   int op;
   int vbytes;
   int ntasks;
@@ -315,6 +319,8 @@ static int pick_vector_bytes(const BoxParams& p, const sbp_tensor* src, const sb
       }
     }
     ok = ok && (p.Nb * p.C * p.esz) % vb == 0;
+    for (int r = 0; r < k && ok; ++r)
+      ok = (p.src_pitch[r] * p.C * p.esz) % vb == 0 && (p.dst_pitch[r] * p.C * p.esz) % vb == 0;
     if (ok) return vb;
   }
   return p.esz;
@@ -411,7 +417,32 @@ static sbp_status make_plan(const sbp_tensor* src, const sbp_tensor* dst, int ds
     return v;
   };
   p.A = p.Na = p.M = p.Nb = 1;
-  if (sa < 0 && da < 0) {
+  const bool pitched = has_ld(src) || has_ld(dst);
+  pl->pitched = pitched;
+  if (pitched) {
+    // Local tensors with a leading dimension: rows are no longer back to back, so the view keeps
+    // the two tensor axes apart ([1][n0][1][n1][1]) and every segment is (a piece of) one row.
+    if (src->ndim != 2)
+      return fail(SBP_ERR_UNSUPPORTED, "local tensors with a leading dimension are boxed as 2-D tensors only");
+    if (p.mode == MODE_SCATTER_P || src->dtype != dst->dtype)
+      return fail(SBP_ERR_UNSUPPORTED, "boxing to P(sum) and the cast-fused gather take dense local tensors only");
+    p.Na = src->shape[0];
+    p.Nb = src->shape[1];
+    p.C = 1;
+    p.src_a = sa == 0;  p.dst_a = da == 0;
+    p.src_b = sa == 1;  p.dst_b = da == 1;
+    for (int r = 0; r < k; ++r) {
+      p.src_pitch[r] = local_pitch(src, r);
+      if (dst_shard < 0 || r == dst_shard) p.dst_pitch[r] = local_pitch(dst, r);
+    }
+    // a reduction reads every source at one offset, a gather / all-reduce writes every replica at one
+    for (int r = 1; r < k; ++r) {
+      if (src_p && !dst_p && p.src_pitch[r] != p.src_pitch[0])
+        return fail(SBP_ERR_UNSUPPORTED, "the partial values of a reduction must share one leading dimension");
+      if ((p.mode == MODE_GATHER || p.mode == MODE_REDUCE_B) && dst_shard < 0 && p.dst_pitch[r] != p.dst_pitch[0])
+        return fail(SBP_ERR_UNSUPPORTED, "the replicas of a B destination must share one leading dimension");
+    }
+  } else if (sa < 0 && da < 0) {
     p.C = prod(0, src->ndim);
   } else if (sa >= 0 && sa == da) {
     // Same split on both sides: shard r's local tensor is copied whole, and a local tensor
@@ -517,7 +548,7 @@ static sbp_status check_pair(const sbp_tensor* src, const sbp_tensor* dst, bool 
 }
 
 // Different shard counts on the two sides (defined in boxing_disjoint.cu).
-sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard, cudaStream_t stream);
+sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard, cudaStream_t stream, bool dry);
 
 }  // namespace sbp
 
@@ -534,10 +565,17 @@ void sbp_boxing_set_copy_engine(int32_t engine) { g_copy_engine.store(engine); }
 // axis 0 changes (valid when the unchanged axis-1 mapping commutes with the change).
 static bool is_partial(sbp_sig s) { return s.kind == SBP_PARTIAL_SUM || s.kind == SBP_PARTIAL_MAX; }
 
-static sbp_status boxing_2d(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream) {
+// dry: every check is made (descriptors, signature pair, sizes) and nothing is launched.
+static sbp_status boxing_one_axis(const sbp_tensor* src, sbp_tensor* dst, int dst_shard, void* cuda_stream, bool dry);
+
+static sbp_status boxing_2d(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream, bool dry) {
   sbp_status st = check_tensor_nd(src, "src", true);
   if (st != SBP_OK) return st;
   st = check_tensor_nd(dst, "dst", true);
+  if (st != SBP_OK) return st;
+  st = refuse_ld(src, "src", "boxing on a two-axis placement");
+  if (st != SBP_OK) return st;
+  st = refuse_ld(dst, "dst", "boxing on a two-axis placement");
   if (st != SBP_OK) return st;
   if (src->pdims != 2 || dst->pdims != 2 || src->pshape[0] != dst->pshape[0] || src->pshape[1] != dst->pshape[1])
     return fail(SBP_ERR_INVALID_ARG, "src and dst must live on the same two-axis placement");
@@ -553,6 +591,7 @@ static sbp_status boxing_2d(const sbp_tensor* src, sbp_tensor* dst, void* cuda_s
   sbp_tensor s1 = *src, d1 = *dst;
   s1.pdims = d1.pdims = 1;
   s1.pshape[1] = d1.pshape[1] = 1;
+  for (int r = 0; r < SBP_MAX_K; ++r) s1.local_ld[r] = d1.local_ld[r] = 0;
   if (!ch0) {
     // axis 1 changes (or nothing does): one boxing op inside each group, on the group's tensor
     s1.pshape[0] = d1.pshape[0] = k1;
@@ -568,7 +607,7 @@ static sbp_status boxing_2d(const sbp_tensor* src, sbp_tensor* dst, void* cuda_s
         s1.local[j] = src->local[i * k1 + j];
         d1.local[j] = dst->local[i * k1 + j];
       }
-      st = sbp_boxing(&s1, &d1, cuda_stream);
+      st = boxing_one_axis(&s1, &d1, -1, cuda_stream, dry);
       if (st != SBP_OK) return st;
     }
     return SBP_OK;
@@ -596,21 +635,21 @@ static sbp_status boxing_2d(const sbp_tensor* src, sbp_tensor* dst, void* cuda_s
       s1.local[i] = src->local[i * k1 + j];
       d1.local[i] = dst->local[i * k1 + j];
     }
-    st = sbp_boxing(&s1, &d1, cuda_stream);
+    st = boxing_one_axis(&s1, &d1, -1, cuda_stream, dry);
     if (st != SBP_OK) return st;
   }
   return SBP_OK;
 }
 
-static sbp_status boxing_one_axis(const sbp_tensor* src, sbp_tensor* dst, int dst_shard, void* cuda_stream) {
+static sbp_status boxing_one_axis(const sbp_tensor* src, sbp_tensor* dst, int dst_shard, void* cuda_stream, bool dry) {
   sbp_status st = check_pair(src, dst, true, dst_shard);
   if (st != SBP_OK) return st;
   if (placement_k(src) != placement_k(dst))
-    return boxing_disjoint(src, dst, dst_shard, static_cast<cudaStream_t>(cuda_stream));
+    return boxing_disjoint(src, dst, dst_shard, static_cast<cudaStream_t>(cuda_stream), dry);
   Plan pl;
   st = make_plan(src, dst, dst_shard, &pl);
   if (st != SBP_OK) return st;
-  if (numel(src) == 0) return SBP_OK;
+  if (dry || numel(src) == 0) return SBP_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
   bool done = false;
@@ -676,7 +715,7 @@ static sbp_status boxing_one_axis(const sbp_tensor* src, sbp_tensor* dst, int ds
   // available on request.
   const int engine = g_copy_engine.load();
   const bool want_bulk = engine == 2;
-  if (!done && pl.op == OP_COPY && want_bulk && pl.vbytes == 16)
+  if (!done && pl.op == OP_COPY && want_bulk && pl.vbytes == 16 && !pl.pitched)
     done = launch_bulk_copy(pl.p, pl.ntasks, stream);
   if (!done) {
     switch (pl.op) {
@@ -694,13 +733,18 @@ static sbp_status boxing_one_axis(const sbp_tensor* src, sbp_tensor* dst, int ds
 }
 
 sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream) {
-  if (src && dst && (src->pdims == 2 || dst->pdims == 2)) return boxing_2d(src, dst, cuda_stream);
-  return boxing_one_axis(src, dst, -1, cuda_stream);
+  if (src && dst && (src->pdims == 2 || dst->pdims == 2)) {
+    // every group's one-axis op is checked before the first of them is launched
+    sbp_status st = boxing_2d(src, dst, cuda_stream, true);
+    if (st != SBP_OK) return st;
+    return boxing_2d(src, dst, cuda_stream, false);
+  }
+  return boxing_one_axis(src, dst, -1, cuda_stream, false);
 }
 
 sbp_status sbp_boxing_shard(const sbp_tensor* src, sbp_tensor* dst, int32_t dst_shard, void* cuda_stream) {
   if (dst_shard < 0) return fail(SBP_ERR_INVALID_ARG, "dst_shard %d is negative", dst_shard);
-  return boxing_one_axis(src, dst, dst_shard, cuda_stream);
+  return boxing_one_axis(src, dst, dst_shard, cuda_stream, false);
 }
 
 static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
@@ -717,6 +761,10 @@ size_t sbp_boxing_host_workspace_bytes(const sbp_tensor* src_host, const sbp_ten
 sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, void* dev_ws, size_t dev_ws_bytes,
                            void* cuda_stream) {
   sbp_status st = check_pair(src_host, dst_host, true);
+  if (st != SBP_OK) return st;
+  st = refuse_ld(src_host, "src_host", "sbp_boxing_host");
+  if (st != SBP_OK) return st;
+  st = refuse_ld(dst_host, "dst_host", "sbp_boxing_host");
   if (st != SBP_OK) return st;
   const size_t need = sbp_boxing_host_workspace_bytes(src_host, dst_host);
   if (need > 0 && (!dev_ws || dev_ws_bytes < need))
@@ -742,6 +790,10 @@ sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, voi
       cur += align256((size_t)local_numel(dst_host, r) * esz_dst);
     }
   }
+  // the transform's own refusals (signature pair, sizes) come before the first copy is enqueued
+  if (s.pdims == 2 || d.pdims == 2) st = boxing_2d(&s, &d, cuda_stream, true);
+  else st = boxing_one_axis(&s, &d, -1, cuda_stream, true);
+  if (st != SBP_OK) return st;
   for (int r = 0; r < ks; ++r) {
     const size_t bytes = (size_t)local_numel(src_host, r) * esz;
     if (bytes) SBP_CUDA_TRY(cudaMemcpyAsync(s.local[r], src_host->local[r], bytes, cudaMemcpyHostToDevice, stream));

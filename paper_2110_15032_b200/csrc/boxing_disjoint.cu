@@ -228,7 +228,8 @@ static void launch_disjoint(const DisjointParams& p, int vbytes, long long grid,
 // src and dst have been validated by the caller (same logical shape and dtype, one-axis
 // placements, pointers present); ks != kd is the expected case but not required.
 // dst_shard >= 0: only that destination local tensor is produced (the other dst pointers may be null).
-sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard, cudaStream_t stream) {
+// dry: every check is made and nothing is launched.
+sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard, cudaStream_t stream, bool dry) {
   const int ks = placement_k(src), kd = placement_k(dst);
   const sbp_sig ss = src->sbp[0], ds = dst->sbp[0];
   const bool src_p = ss.kind == SBP_PARTIAL_SUM || ss.kind == SBP_PARTIAL_MAX;
@@ -236,6 +237,9 @@ sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard
   const int esz = elem_size(src->dtype);
   if (src->dtype != dst->dtype)
     return fail(SBP_ERR_UNSUPPORTED, "the cast-fused gather needs src and dst on the same placement");
+  sbp_status ld_st = refuse_ld(src, "src", "boxing between different placements");
+  if (ld_st == SBP_OK) ld_st = refuse_ld(dst, "dst", "boxing between different placements");
+  if (ld_st != SBP_OK) return ld_st;
 
   DisjointParams p{};
   p.ks = ks; p.kd = kd; p.esz = esz;
@@ -365,6 +369,28 @@ sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard
       for (int q = 0; q < p.n_dst; ++q) p.dst[q] = uniq[q];
   }
 
+  // tiling, sized by the largest cut any task can have
+  auto max_cut = [&](long long n, bool by_src, bool by_dst) {
+    long long m = n;
+    if (by_src) m = std::min(m, (n + ks - 1) / ks);
+    if (by_dst) m = std::min(m, (n + kd - 1) / kd);
+    return m;
+  };
+  const long long nseg_max = p.A * max_cut(p.Na, p.src_a, p.dst_a) * p.M;
+  const long long seg_vecs_max = max_cut(p.Nb, p.src_b, p.dst_b) * p.C * esz / vbytes;
+  const int tile_vecs = (op == OP_COPY ? 4 : 2) * 256;
+  int cv_log2 = 0;
+  while ((1 << cv_log2) < tile_vecs && (1LL << cv_log2) < seg_vecs_max) ++cv_log2;
+  p.cv_log2 = cv_log2;
+  p.rows_per_tile = tile_vecs >> cv_log2;
+  p.col_tiles = std::max(1LL, (seg_vecs_max + (1LL << cv_log2) - 1) >> cv_log2);
+  const long long row_tiles = std::max(1LL, (nseg_max + p.rows_per_tile - 1) / p.rows_per_tile);
+  p.tiles_per_task = p.col_tiles * row_tiles;
+  const long long grid = p.tiles_per_task * p.ntasks;
+  if (copy_needed && grid > 0x7fffffffLL) return fail(SBP_ERR_UNSUPPORTED, "tensor too large for one launch");
+  if (dry) return SBP_OK;   // every refusal lies above this line, every launch below it
+
+
   if (zero_first) {
     // The partials start as zeros.  One kernel clears all of them when they are 16-byte
     // aligned (one launch instead of up to kd memsets with their gaps); else memsets do.
@@ -391,27 +417,6 @@ sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard
     }
   }
   if (!copy_needed) return SBP_OK;
-
-  // tiling, sized by the largest cut any task can have
-  auto max_cut = [&](long long n, bool by_src, bool by_dst) {
-    long long m = n;
-    if (by_src) m = std::min(m, (n + ks - 1) / ks);
-    if (by_dst) m = std::min(m, (n + kd - 1) / kd);
-    return m;
-  };
-  const long long nseg_max = p.A * max_cut(p.Na, p.src_a, p.dst_a) * p.M;
-  const long long seg_vecs_max = max_cut(p.Nb, p.src_b, p.dst_b) * p.C * esz / vbytes;
-  const int tile_vecs = (op == OP_COPY ? 4 : 2) * 256;
-  int cv_log2 = 0;
-  while ((1 << cv_log2) < tile_vecs && (1LL << cv_log2) < seg_vecs_max) ++cv_log2;
-  p.cv_log2 = cv_log2;
-  p.rows_per_tile = tile_vecs >> cv_log2;
-  p.col_tiles = std::max(1LL, (seg_vecs_max + (1LL << cv_log2) - 1) >> cv_log2);
-  const long long row_tiles = std::max(1LL, (nseg_max + p.rows_per_tile - 1) / p.rows_per_tile);
-  p.tiles_per_task = p.col_tiles * row_tiles;
-  const long long grid = p.tiles_per_task * p.ntasks;
-  if (grid > 0x7fffffffLL) return fail(SBP_ERR_UNSUPPORTED, "tensor too large for one launch");
-
   switch (op) {
     case OP_COPY: launch_disjoint<OP_COPY>(p, vbytes, grid, stream); break;
     case OP_SUM_F32: launch_disjoint<OP_SUM_F32>(p, vbytes, grid, stream); break;

@@ -29,6 +29,9 @@ struct BoxParams {
   int ntasks;                       // tasks of the transform; tiles are dealt task-fastest
   int one_dst, dst_shard;           // one_dst: only the tasks that produce destination shard dst_shard
   long long a_base, a_rem, b_base, b_rem;   // Na / k, Na % k, Nb / k, Nb % k: the balanced split without a division
+  // Row pitch of every local tensor in units of C elements, 0 = dense (the pitch is then the local
+  // extent of the Nb axis).  Non-zero only for 2-D tensors with a leading dimension (C == 1).
+  long long src_pitch[SBP_MAX_K], dst_pitch[SBP_MAX_K];
 };
 
 // Start and length of shard r's piece of an axis whose n / k and n % k are known.

@@ -159,6 +159,86 @@ __global__ void __launch_bounds__(256, MINB) embedding_kernel(const __grid_const
   }
 }
 
+// Fused gather with a single destination per row (k = 1, or all B replicas the same buffer).
+// There the element-wise kernel above is bound by the latency of its id -> row -> store chain, not
+// by bandwidth.  This form takes the id load out of the chain.  A persistent CTA walks chunks of
+// 256 * J consecutive 16-byte pieces of the result (for 512-byte rows and J = 8: 64 consecutive
+// lookups).  The ids of a chunk sit in shared memory before its rows are asked for; the ids of the
+// CTA's next chunk are requested first (one coalesced load), then every thread puts J row loads in
+// flight at once (a warp: J whole rows), stores them, and only then parks the next ids in the other
+// half of the shared buffer -- so the id latency hides behind the rows.  The result is written with
+// streaming (evict-first) stores so that the output, which is never read back, does not push the
+// table's hot rows out of L2.  vpr (vectors per row) must be a power of two between 8 and 256 * J, so
+// that a chunk starts on a row boundary and holds at most 256 lookups (one id per thread).
+template <typename V, int ESZ, int J>
+__global__ void __launch_bounds__(256) embedding_rows_kernel(const __grid_constant__ EmbParams p) {
+  __shared__ long long ids_s[2][256];
+  const long long total = p.n_lookups * p.vpr;
+  const long long n_chunks = (total + 256 * J - 1) / (256 * J);
+
+  // first and last lookup of a chunk
+  auto span = [&](long long chunk, long long* look0, int* n_ids) {
+    const long long first = chunk * (256 * J);
+    long long last = first + 256 * J - 1;
+    if (last >= total) last = total - 1;
+    *look0 = first >> p.vpr_log2;
+    *n_ids = (int)((last >> p.vpr_log2) - *look0) + 1;
+  };
+
+  long long chunk = blockIdx.x;
+  if (chunk >= n_chunks) return;
+  int cur = 0;
+  {
+    long long look0;
+    int n_ids;
+    span(chunk, &look0, &n_ids);
+    if ((int)threadIdx.x < n_ids) ids_s[0][threadIdx.x] = __ldcs(p.ids[0] + look0 + threadIdx.x);
+  }
+  __syncthreads();
+
+  for (; chunk < n_chunks; chunk += gridDim.x) {
+    const long long cta_base = chunk * (256 * J);
+    long long look0;
+    int n_ids;
+    span(chunk, &look0, &n_ids);
+    // request the next chunk's ids; they are not touched until this chunk's rows are stored
+    const long long next = chunk + gridDim.x;
+    long long nlook0 = 0, nid = 0;
+    int nn = 0;
+    if (next < n_chunks) {
+      span(next, &nlook0, &nn);
+      if ((int)threadIdx.x < nn) nid = __ldcs(p.ids[0] + nlook0 + threadIdx.x);
+    }
+
+    V val[J];
+    bool ok[J];
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      const long long item = cta_base + j * 256 + threadIdx.x;
+      ok[j] = item < total;
+      val[j] = zero_vec<V>();
+      if (!ok[j]) continue;
+      const long long look = item >> p.vpr_log2, col = item & (p.vpr - 1);
+      const long long id = ids_s[cur][look - look0];
+      if (id < 0 || id >= p.rows) {
+        if (p.oob && col == 0) atomicAdd(p.oob, 1);
+        continue;
+      }
+      long long start;
+      const int r = owner_of_row(id, p.base, p.rem, p.big, p.narrow, &start);
+      val[j] = __ldg(reinterpret_cast<const V*>(p.table[r]) + (id - start) * p.vpr + col);
+    }
+    V* o = reinterpret_cast<V*>(p.out[0]);
+#pragma unroll
+    for (int j = 0; j < J; ++j)
+      if (ok[j]) __stcs(o + cta_base + j * 256 + threadIdx.x, p.canon_neg_zero ? canon<V, ESZ>(val[j]) : val[j]);
+
+    if ((int)threadIdx.x < nn) ids_s[cur ^ 1][threadIdx.x] = nid;
+    __syncthreads();
+    cur ^= 1;
+  }
+}
+
 // Two shapes of the same kernel.  With several destinations per row the kernel is bound by its
 // stores and runs best with four lookups per thread; with a single destination (aliased
 // replicas, k = 1) it is bound by the latency of the id -> row -> store chain and runs best
@@ -172,7 +252,22 @@ static void launch_emb(const EmbParams& p, bool fused, cudaStream_t st) {
     long long b = (total + 256LL * j - 1) / (256LL * j);
     return (unsigned)(b < 1 ? 1 : b);
   };
-  if (fused && p.n_dst == 1) {
+  if (fused && p.n_dst == 1 && p.vpr_log2 >= 3 && p.vpr_log2 <= 11) {
+    // persistent: as many CTAs as fit at once
+    static int resident = 0;
+    if (resident == 0) {
+      int dev = 0, sms = 148, per_sm = 4;
+      cudaGetDevice(&dev);
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+      if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, embedding_rows_kernel<V, ESZ, 8>, 256, 0) != cudaSuccess || per_sm < 1) {
+        cudaGetLastError();
+        per_sm = 4;
+      }
+      resident = sms * per_sm;
+    }
+    const unsigned chunks = blocks_for(8);
+    embedding_rows_kernel<V, ESZ, 8><<<dim3(chunks < (unsigned)resident ? chunks : (unsigned)resident), 256, 0, st>>>(p);
+  } else if (fused && p.n_dst == 1) {
     embedding_kernel<V, ESZ, 2, true, 8><<<dim3(blocks_for(2)), 256, 0, st>>>(p);
   } else if (fused) {
     embedding_kernel<V, ESZ, 4, true, 1><<<dim3(blocks_for(4)), 256, 0, st>>>(p);
@@ -431,6 +526,10 @@ extern "C" sbp_status sbp_embedding(const sbp_tensor* table, const sbp_tensor* i
   if (st != SBP_OK) return st;
   st = check_tensor(out, "out", true);
   if (st != SBP_OK) return st;
+  const sbp_tensor* dense_only[3] = {table, ids, out};
+  const char* dense_names[3] = {"table", "ids", "out"};
+  for (int i = 0; i < 3; ++i)
+    if ((st = refuse_ld(dense_only[i], dense_names[i], "sbp_embedding")) != SBP_OK) return st;
   if (table->ndim != 2) return fail(SBP_ERR_SHAPE, "table must be [rows, dim]");
   if (table->dtype != SBP_F32 && table->dtype != SBP_BF16) return fail(SBP_ERR_DTYPE, "table must be F32 or BF16");
   if (out->dtype != table->dtype) return fail(SBP_ERR_DTYPE, "out and table differ in dtype");
@@ -512,6 +611,10 @@ extern "C" sbp_status sbp_embedding_backward(const sbp_tensor* grad_out, const s
   if (st != SBP_OK) return st;
   st = check_tensor(grad_table, "grad_table", true);
   if (st != SBP_OK) return st;
+  const sbp_tensor* dense_only[3] = {grad_out, ids, grad_table};
+  const char* dense_names[3] = {"grad_out", "ids", "grad_table"};
+  for (int i = 0; i < 3; ++i)
+    if ((st = refuse_ld(dense_only[i], dense_names[i], "sbp_embedding_backward")) != SBP_OK) return st;
   if (grad_table->ndim != 2) return fail(SBP_ERR_SHAPE, "grad_table must be [rows, dim]");
   if (grad_table->dtype != SBP_F32 || grad_out->dtype != SBP_F32)
     return fail(SBP_ERR_DTYPE, "the embedding backward accumulates in F32: grad_out and grad_table must be F32");

@@ -23,6 +23,7 @@ sbp_status check_xent_outputs(const sbp_tensor* labels, const sbp_tensor* loss, 
                               const sbp_tensor* row_sum, long long rows, int k);
 size_t xent_finish_stage_floats(long long rows);
 size_t matmul_tc_workspace_bytes(const MatmulPlan& plan);
+void tensor_map_cache_stats(unsigned long long* hits, unsigned long long* encodes);
 
 __device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f)); }
 
@@ -209,20 +210,20 @@ static sbp_status build_plan(const sbp_tensor* x, const sbp_tensor* w, const sbp
     long long st_, ln;
     p.a[r] = x->local[r];
     p.b[r] = w->local[r];
-    // leading dimensions of the stored local tensors: their last axis, M or K for x, K or N for w
-    p.lda[r] = tx ? M : K;
-    p.ldb[r] = tw ? K : N;
+    // leading dimensions of the stored local tensors: the descriptor's, else their last local extent
+    p.lda[r] = local_pitch(x, r);
+    p.ldb[r] = local_pitch(w, r);
     p.kseg[r] = K;
-    if (is_s(xs, 1)) { range(K, r, &st_, &ln); p.kseg[r] = ln; if (!tx) p.lda[r] = ln; }
-    if (is_s(xs, 0) && tx) { range(M, r, &st_, &ln); p.lda[r] = ln; }
-    if (is_s(ws, 1) && !tw) { range(N, r, &st_, &ln); p.ldb[r] = ln; }
-    if (is_s(ws, 0) && tw) { range(K, r, &st_, &ln); p.ldb[r] = ln; }
+    if (is_s(xs, 1)) { range(K, r, &st_, &ln); p.kseg[r] = ln; }
   }
   p.nseg = k;
 
+  for (int r = 1; r < k; ++r)
+    if (is_b(ys) && local_pitch(y, r) != local_pitch(y, 0))
+      return fail(SBP_ERR_UNSUPPORTED, "the replicas of a B result must share one leading dimension");
   auto set_replicas = [&]() {   // one group, stored to every distinct B replica
     p.ngroups = 1;
-    p.m[0] = M; p.n[0] = N; p.ldy[0] = N;
+    p.m[0] = M; p.n[0] = N; p.ldy[0] = local_pitch(y, 0);
     void* uniq[SBP_MAX_K];
     int nu = 0;
     for (int r = 0; r < k; ++r) {
@@ -244,9 +245,9 @@ static sbp_status build_plan(const sbp_tensor* x, const sbp_tensor* w, const sbp
       p.ngroups = k;
       for (int g = 0; g < k; ++g) {
         long long st_, ln;
-        p.m[g] = M; p.n[g] = N; p.ldy[g] = N;
+        p.m[g] = M; p.n[g] = N; p.ldy[g] = local_pitch(y, g);
         if (is_s(natural, 0)) { range(M, g, &st_, &ln); p.m[g] = ln; }
-        if (is_s(natural, 1)) { range(N, g, &st_, &ln); p.n[g] = ln; p.ldy[g] = ln; }
+        if (is_s(natural, 1)) { range(N, g, &st_, &ln); p.n[g] = ln; }
         p.y[g] = y->local[g];
       }
     }
@@ -258,9 +259,9 @@ static sbp_status build_plan(const sbp_tensor* x, const sbp_tensor* w, const sbp
       p.ngroups = k;
       for (int g = 0; g < k; ++g) {
         long long st_, ln;
-        p.m[g] = M; p.n[g] = N; p.ldy[g] = N;
+        p.m[g] = M; p.n[g] = N; p.ldy[g] = local_pitch(y, g);
         if (ys.axis == 0) { range(M, g, &st_, &ln); p.m[g] = ln; p.row_off[g] = st_; }
-        else { range(N, g, &st_, &ln); p.n[g] = ln; p.col_off[g] = st_; p.ldy[g] = ln; }
+        else { range(N, g, &st_, &ln); p.n[g] = ln; p.col_off[g] = st_; }
         p.y[g] = y->local[g];
       }
     }
@@ -322,12 +323,12 @@ static sbp_status build_plan_2d(const sbp_tensor* x, const sbp_tensor* w, const 
                   (long long)ys[1]);
     p.a[r] = x->local[r];
     p.b[r] = w->local[r];
-    p.lda[r] = xs[1];
-    p.ldb[r] = wsz[1];
+    p.lda[r] = local_pitch(x, r);
+    p.ldb[r] = local_pitch(w, r);
     p.kseg[r] = xs[1];
     p.m[r] = xs[0];
     p.n[r] = wsz[1];
-    p.ldy[r] = wsz[1];
+    p.ldy[r] = local_pitch(y, r);
     p.y[r] = y->local[r];
   }
   return SBP_OK;
@@ -343,6 +344,13 @@ size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, cons
   MatmulPlan plan;
   if (build_plan(x, w, y, 0, false, &plan) != SBP_OK) return 0;
   return matmul_tc_workspace_bytes(plan);
+}
+
+void sbp_tensor_map_stats(uint64_t* reused, uint64_t* encoded) {
+  unsigned long long h = 0, e = 0;
+  tensor_map_cache_stats(&h, &e);
+  if (reused) *reused = h;
+  if (encoded) *encoded = e;
 }
 
 sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, uint32_t flags, void* ws,
@@ -428,8 +436,8 @@ sbp_status sbp_matmul_softmax_xent(const sbp_tensor* features, const sbp_tensor*
     split_range(N, k, r, &s0, &ln);
     plan.a[r] = features->local[r];
     plan.b[r] = weight->local[r];
-    plan.lda[r] = K;
-    plan.ldb[r] = ln;
+    plan.lda[r] = local_pitch(features, r);
+    plan.ldb[r] = local_pitch(weight, r);
     plan.kseg[r] = K;
     plan.m[r] = rows;
     plan.n[r] = ln;
@@ -492,12 +500,12 @@ sbp_status sbp_matmul_softmax_xent_backward(const sbp_tensor* features, const sb
     split_range(N, k, r, &s0, &ln);
     plan.a[r] = features->local[r];
     plan.b[r] = weight->local[r];
-    plan.lda[r] = K;
-    plan.ldb[r] = ln;
+    plan.lda[r] = local_pitch(features, r);
+    plan.ldb[r] = local_pitch(weight, r);
     plan.kseg[r] = K;
     plan.m[r] = rows;
     plan.n[r] = ln;
-    plan.ldy[r] = ln;
+    plan.ldy[r] = local_pitch(grad_logits, r);
     plan.y[r] = grad_logits->local[r];
     xf.class_start[r] = s0;
   }

@@ -601,9 +601,53 @@ static EncodeTiledFn encode_fn() {
   return fn;
 }
 
+// Tensor maps already encoded by this process, keyed by everything that goes into one.  A map holds
+// nothing but the address and the layout, so an entry stays valid for as long as its key recurs: a
+// product that is called again on the same buffers (every step of a training loop) encodes nothing.
+// Direct-mapped; used with the parameter block's lock held.
+struct MapKey {
+  const void* base;
+  long long rows, cols, ld;
+  int esz, box_rows, box_cols;
+  bool operator==(const MapKey& o) const {
+    return base == o.base && rows == o.rows && cols == o.cols && ld == o.ld && esz == o.esz && box_rows == o.box_rows &&
+           box_cols == o.box_cols;
+  }
+};
+struct MapSlot {
+  CUtensorMap map;
+  MapKey key;
+  bool used;
+};
+constexpr int kMapCacheSlots = 1024;
+static MapSlot g_map_cache[kMapCacheSlots];
+static unsigned long long g_map_hits = 0, g_map_encodes = 0;
+
+static unsigned map_slot_of(const MapKey& k) {
+  unsigned long long h = reinterpret_cast<uintptr_t>(k.base) >> 4;
+  auto mix = [&](unsigned long long v) { h = (h ^ v) * 0x9E3779B97F4A7C15ull; h ^= h >> 29; };
+  mix((unsigned long long)k.rows);
+  mix((unsigned long long)k.cols);
+  mix((unsigned long long)k.ld);
+  mix((unsigned long long)(k.esz | (k.box_rows << 8) | (k.box_cols << 20)));
+  return (unsigned)(h % kMapCacheSlots);
+}
+
+void tensor_map_cache_stats(unsigned long long* hits, unsigned long long* encodes) {
+  *hits = g_map_hits;
+  *encodes = g_map_encodes;
+}
+
 // 2-D row-major tensor [rows, cols] with leading dimension ld (elements), box [box_rows, box_cols].
 static bool make_map(CUtensorMap* map, const void* base, int esz, long long rows, long long cols, long long ld,
                      int box_rows, int box_cols) {
+  const MapKey key{base, rows, cols, ld, esz, box_rows, box_cols};
+  MapSlot& slot = g_map_cache[map_slot_of(key)];
+  if (slot.used && slot.key == key) {
+    *map = slot.map;
+    ++g_map_hits;
+    return true;
+  }
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -611,9 +655,14 @@ static bool make_map(CUtensorMap* map, const void* base, int esz, long long rows
   cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
   cuuint32_t estr[2] = {1, 1};
   CUtensorMapDataType dt = esz == 2 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
-  return fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
-            CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) ==
-         CUDA_SUCCESS;
+  if (fn(map, dt, 2, const_cast<void*>(base), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+         CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  ++g_map_encodes;
+  slot.map = *map;
+  slot.key = key;
+  slot.used = true;
+  return true;
 }
 
 size_t matmul_tc_workspace_bytes(const MatmulPlan&) { return 0; }

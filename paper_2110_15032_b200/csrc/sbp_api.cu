@@ -46,6 +46,14 @@ static sbp_status check_common(const sbp_tensor* t, const char* name, bool need_
     if (s.kind == SBP_SPLIT && (s.axis < 0 || s.axis >= t->ndim))
       return fail(SBP_ERR_SIGNATURE, "%s: split axis %d outside [0,%d)", name, s.axis, t->ndim);
   }
+  for (int r = 0; r < k; ++r) {
+    if (t->local_ld[r] == 0) continue;
+    int64_t shp[SBP_MAX_DIMS];
+    local_shape_nd(t, r, shp);
+    if (t->local_ld[r] < shp[t->ndim - 1])
+      return fail(SBP_ERR_INVALID_ARG, "%s: local_ld[%d] = %lld is below the local row length %lld", name, r,
+                  (long long)t->local_ld[r], (long long)shp[t->ndim - 1]);
+  }
   if (need_ptrs) {
     for (int r = 0; r < k; ++r) {
       if (!t->local[r] && local_numel(t, r) > 0)
@@ -86,6 +94,31 @@ int64_t local_numel(const sbp_tensor* t, int r) {
   int64_t n = 1;
   for (int d = 0; d < t->ndim; ++d) n *= shp[d];
   return n;
+}
+
+int64_t local_pitch(const sbp_tensor* t, int r) {
+  if (t->local_ld[r] != 0) return t->local_ld[r];
+  int64_t shp[SBP_MAX_DIMS];
+  local_shape_nd(t, r, shp);
+  return shp[t->ndim - 1];
+}
+
+bool has_ld(const sbp_tensor* t) {
+  if (t->ndim < 2) return false;           // a single row has no pitch
+  const int k = placement_k(t);
+  for (int r = 0; r < k; ++r) {
+    if (t->local_ld[r] == 0) continue;
+    int64_t shp[SBP_MAX_DIMS];
+    local_shape_nd(t, r, shp);
+    if (t->local_ld[r] != shp[t->ndim - 1]) return true;
+  }
+  return false;
+}
+
+sbp_status refuse_ld(const sbp_tensor* t, const char* name, const char* entry) {
+  if (t && has_ld(t))
+    return fail(SBP_ERR_UNSUPPORTED, "%s: %s takes dense local tensors only (local_ld must be 0 or the row length)", name, entry);
+  return SBP_OK;
 }
 
 // Defined next to the kernels that own the flags.
@@ -142,6 +175,40 @@ sbp_status sbp_local_shape(const sbp_tensor* t, int32_t r, int64_t out_shape[SBP
   int k = placement_k(t);
   if (r < 0 || r >= k) return fail(SBP_ERR_INVALID_ARG, "shard %d outside [0,%d)", r, k);
   local_shape_nd(t, r, out_shape);
+  return SBP_OK;
+}
+
+sbp_status sbp_view_b_to_s(const sbp_tensor* b, int32_t axis, sbp_tensor* view) {
+  sbp_status st = check_tensor(b, "b", true);
+  if (st != SBP_OK) return st;
+  if (!view) return fail(SBP_ERR_INVALID_ARG, "view is null");
+  if (b->sbp[0].kind != SBP_BROADCAST) return fail(SBP_ERR_SIGNATURE, "b must be a B tensor");
+  if (axis < 0 || axis >= b->ndim) return fail(SBP_ERR_INVALID_ARG, "axis %d outside [0,%d)", axis, b->ndim);
+  if (axis != 0 && axis != b->ndim - 1)
+    return fail(SBP_ERR_UNSUPPORTED, "a view split along an inner axis of an N-D tensor needs two strides");
+  const int k = placement_k(b);
+  const int esz = elem_size(b->dtype);
+  sbp_tensor v = *b;
+  v.sbp[0].kind = SBP_SPLIT;
+  v.sbp[0].axis = axis;
+  int64_t inner = 1;   // elements in one step of axis 0, in a replica
+  for (int d = 1; d < b->ndim; ++d) inner *= b->shape[d];
+  for (int r = 0; r < k; ++r) {
+    int64_t start, len;
+    split_range(b->shape[axis], k, r, &start, &len);
+    const int64_t pitch = local_pitch(b, r);             // row length of the replica
+    char* base = static_cast<char*>(b->local[r]);
+    if (axis == b->ndim - 1) {                            // a column block: rows stay `pitch` apart
+      v.local[r] = base ? base + start * esz : nullptr;
+      v.local_ld[r] = b->ndim >= 2 ? pitch : 0;          // a 1-D tensor is a single row: no pitch
+    } else {                                              // a block of whole rows (ndim >= 2 here)
+      const int64_t rows_per_step = inner / b->shape[b->ndim - 1];
+      v.local[r] = base ? base + start * rows_per_step * pitch * esz : nullptr;
+      v.local_ld[r] = b->local_ld[r];
+    }
+    if (len == 0) v.local[r] = b->local[r];               // an empty piece: any valid pointer
+  }
+  *view = v;
   return SBP_OK;
 }
 

@@ -62,6 +62,15 @@ inline int64_t numel(const sbp_tensor* t) {
 // Elements of shard r's local tensor.
 int64_t local_numel(const sbp_tensor* t, int r);
 
+// Row pitch of shard r's local tensor in elements: local_ld[r], or its last local extent when dense.
+int64_t local_pitch(const sbp_tensor* t, int r);
+
+// True when some local tensor of t has a leading dimension other than its row length.
+bool has_ld(const sbp_tensor* t);
+
+// SBP_ERR_UNSUPPORTED (with the entry point's name in the message) when t is not dense.
+sbp_status refuse_ld(const sbp_tensor* t, const char* name, const char* entry);
+
 sbp_status cuda_fail(cudaError_t e, const char* what);
 
 // Launch of `kernel` as a programmatic dependent of the kernel before it in the stream: if that

@@ -36,6 +36,7 @@ struct XentParams {
   float* part_s;
   float* part_t;
   long long rows, classes;
+  long long pitch[SBP_MAX_K];   // elements between consecutive rows of shard r's logits
   int k, nsplit;
   long long chunk;   // elements per chunk (kThreads * kLoadsPerThread * VEC)
   long long span;    // elements per CTA (chunk * chunks per CTA)
@@ -174,7 +175,7 @@ __global__ void __launch_bounds__(kThreads) xent_partial_kernel(const __grid_con
   long long n = c_len - c0;       // elements of this CTA's span (may be <= 0 on uneven shards)
   if (n > p.span) n = p.span;
   const int part = shard * p.nsplit + split;
-  const T* z = reinterpret_cast<const T*>(p.logits[shard]) + row * c_len + c0;
+  const T* z = reinterpret_cast<const T*>(p.logits[shard]) + row * p.pitch[shard] + c0;
   const int tid = threadIdx.x;
   // The kernel that combines the partials may be set up while this one runs; it waits for
   // this grid to finish before it reads anything.
@@ -279,7 +280,7 @@ static int pick_vec(const sbp_tensor* logits) {
   for (int r = 0; r < k; ++r) {
     int64_t st, ln;
     split_range(logits->shape[1], k, r, &st, &ln);
-    if ((ln * esz) % 16 != 0) return 1;
+    if ((ln * esz) % 16 != 0 || (local_pitch(logits, r) * esz) % 16 != 0) return 1;
     if (logits->local[r] && reinterpret_cast<uintptr_t>(logits->local[r]) % 16 != 0) return 1;
   }
   return 16 / esz;
@@ -448,6 +449,7 @@ struct XentBwdParams {
   const float* row_max;
   const float* row_sum;
   long long rows, classes;
+  long long lpitch[SBP_MAX_K], gpitch[SBP_MAX_K];   // elements between consecutive rows: logits, gradient
   int k;
 };
 
@@ -457,8 +459,8 @@ __global__ void __launch_bounds__(kThreads) xent_backward_kernel(const __grid_co
   const int shard = blockIdx.z;
   long long c_start, c_len;
   split_range(p.classes, p.k, shard, (int64_t*)&c_start, (int64_t*)&c_len);
-  const T* z = reinterpret_cast<const T*>(p.logits[shard]) + row * c_len;
-  T* g = reinterpret_cast<T*>(p.grad[shard]) + row * c_len;
+  const T* z = reinterpret_cast<const T*>(p.logits[shard]) + row * p.lpitch[shard];
+  T* g = reinterpret_cast<T*>(p.grad[shard]) + row * p.gpitch[shard];
   // softmax = 2^(z log2e - m log2e - log2 S): the division by the row sum is folded into the exponent
   const float neg = -p.row_max[row] * kLog2e - log2f(p.row_sum[row]);
   const long long y = p.labels[row] - c_start;      // label's column inside this shard, if any
@@ -526,7 +528,10 @@ sbp_status sbp_softmax_xent(const sbp_tensor* logits, const sbp_tensor* labels, 
   if (rows > 0x7fffffffLL || nsplit > 65535) return fail(SBP_ERR_UNSUPPORTED, "shape too large for one launch");
 
   XentParams p{};
-  for (int r = 0; r < k; ++r) p.logits[r] = static_cast<const char*>(logits->local[r]);
+  for (int r = 0; r < k; ++r) {
+    p.logits[r] = static_cast<const char*>(logits->local[r]);
+    p.pitch[r] = local_pitch(logits, r);
+  }
   p.labels = static_cast<const long long*>(labels->local[0]);
   p.part_m = static_cast<float*>(ws);
   p.part_s = p.part_m + (size_t)parts * rows;
@@ -654,8 +659,11 @@ extern "C" sbp_status sbp_softmax_xent_backward(const sbp_tensor* logits, const 
   for (int r = 0; r < k; ++r) {
     int64_t s0, ln;
     split_range(classes, k, r, &s0, &ln);
+    p.lpitch[r] = local_pitch(logits, r);
+    p.gpitch[r] = local_pitch(grad_logits, r);
     vec_ok = vec_ok && (ln * esz) % 16 == 0 && reinterpret_cast<uintptr_t>(logits->local[r]) % 16 == 0 &&
-             reinterpret_cast<uintptr_t>(grad_logits->local[r]) % 16 == 0;
+             reinterpret_cast<uintptr_t>(grad_logits->local[r]) % 16 == 0 && (p.lpitch[r] * esz) % 16 == 0 &&
+             (p.gpitch[r] * esz) % 16 == 0;
     p.logits[r] = static_cast<const char*>(logits->local[r]);
     p.grad[r] = static_cast<char*>(grad_logits->local[r]);
   }

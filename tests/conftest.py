@@ -12,6 +12,21 @@ def pytest_configure(config):
     config.addinivalue_line("markers", "gpu: needs a CUDA device (B200, sm_100a)")
 
 
+@pytest.fixture(autouse=True)
+def _guard_bands(request, monkeypatch):
+    """GPU tests: every buffer obtained through the package's empty_global lies between guard bands
+    (tests/helpers.py), and the bands are checked when the test ends."""
+    if request.node.get_closest_marker("gpu") is None:
+        yield
+        return
+    import helpers
+    import paper_2110_15032_b200 as sbp
+    monkeypatch.setattr(sbp, "empty_global", helpers.guarded_empty_global)
+    helpers._GUARDED.clear()
+    yield
+    helpers.check_guards(clear=True)
+
+
 GOLDEN = os.path.join(ROOT, "tests", "golden")
 
 

@@ -68,3 +68,57 @@ def assert_close(gpu: np.ndarray, ref: np.ndarray, rtol, atol, what=""):
         i = np.unravel_index(np.argmax(err - bound), err.shape)
         raise AssertionError(f"{what}: {int(bad.sum())} of {bad.size} outside tolerance; worst at {i}: "
                              f"gpu={gpu[i]!r} ref={ref[i]!r} err={err[i]:.3e} bound={bound[i]:.3e}")
+
+
+# ------------------------------------------------------------------------------ guard bands
+#
+# Every output buffer the GPU tests hand to the library sits between two bands of 256 bytes of
+# 0xAB, and its own bytes start as 0xFF (a NaN pattern for the floating types, -1 for int64).  A
+# kernel that stores outside a local tensor changes a band; one that skips an element leaves a NaN
+# behind that the comparison with the oracle then trips over.
+
+GUARD_BYTES = 256
+_GUARDED = []          # (raw uint8 buffer, payload bytes, description)
+
+
+def guarded_empty(shape, dtype, device="cuda", what=""):
+    """An uninitialised-looking tensor of `shape` whose storage is flanked by guard bands."""
+    esz = torch.empty((), dtype=dtype).element_size()
+    n = esz
+    for s in shape:
+        n *= int(s)
+    raw = torch.empty(n + 2 * GUARD_BYTES, dtype=torch.uint8, device=device)
+    raw[:GUARD_BYTES] = 0xAB
+    raw[GUARD_BYTES + n:] = 0xAB
+    raw[GUARD_BYTES:GUARD_BYTES + n] = 0xFF
+    _GUARDED.append((raw, n, f"{what} {tuple(shape)} {dtype}"))
+    return raw[GUARD_BYTES:GUARD_BYTES + n].view(dtype).view(tuple(int(s) for s in shape))
+
+
+def guarded_empty_global(shape, dtype, sig, k, device="cuda", alias_replicas=False):
+    """Same contract as the package's empty_global, every local tensor inside guard bands."""
+    pshape = tuple(k) if isinstance(k, (tuple, list)) else None
+    n = k if pshape is None else pshape[0] * pshape[1]
+    locs = []
+    for r in range(n):
+        if alias_replicas and pshape is None and sig.kind == sbp.B.kind and r > 0:
+            locs.append(locs[0])
+        else:
+            locs.append(guarded_empty(sbp.sbp_local_shape(shape, sig, k, r, dtype), dtype, device, f"shard {r} of"))
+    return sbp.SbpTensor(shape, dtype, sig, locs, pshape)
+
+
+def check_guards(clear=False):
+    """Waits for the device and asserts that no band around any guarded buffer has changed."""
+    if torch.cuda.is_available():
+        torch.cuda.synchronize()
+    bad = []
+    for raw, n, what in _GUARDED:
+        bands = torch.cat([raw[:GUARD_BYTES], raw[GUARD_BYTES + n:]]).cpu().numpy()
+        if not (bands == 0xAB).all():
+            at = int(np.flatnonzero(bands != 0xAB)[0])
+            side = "before" if at < GUARD_BYTES else "after"
+            bad.append(f"{what}: byte {at % GUARD_BYTES} of the band {side} the buffer was overwritten")
+    if clear:
+        _GUARDED.clear()
+    assert not bad, "stores outside a destination buffer: " + "; ".join(bad)

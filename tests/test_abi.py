@@ -34,10 +34,26 @@ def test_library_exports_every_declared_symbol(lib):
         assert hasattr(lib, n), f"{n} is declared in include/sbp.h but not exported"
 
 
-def test_struct_layout_matches_header(lib):
-    # ndim,dtype (8) + shape (32) + pdims (4) + pshape (8) + sbp (16) + pad (4) + local (128)
-    assert C.sizeof(binding._Tensor) == 8 + 32 + 4 + 8 + 16 + 4 + 128
+def test_struct_layout_matches_header(lib, tmp_path):
+    # ndim,dtype (8) + shape (32) + pdims (4) + pshape (8) + sbp (16) + pad (4) + local (128) + local_ld (128)
+    assert C.sizeof(binding._Tensor) == 8 + 32 + 4 + 8 + 16 + 4 + 128 + 128
     assert binding._Tensor.local.offset % 8 == 0
+    # and against the header itself, as a C compiler lays it out
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        pytest.skip("no C compiler")
+    src = tmp_path / "layout.c"
+    src.write_text('#include <stdio.h>\n#include <stddef.h>\n#include "sbp.h"\n'
+                   'int main(void) { printf("%zu %zu %zu %zu %zu %zu %zu %zu\\n", sizeof(sbp_tensor), offsetof(sbp_tensor, ndim), '
+                   'offsetof(sbp_tensor, dtype), offsetof(sbp_tensor, shape), offsetof(sbp_tensor, pdims), '
+                   'offsetof(sbp_tensor, sbp), offsetof(sbp_tensor, local), offsetof(sbp_tensor, local_ld)); return 0; }\n')
+    exe = tmp_path / "layout"
+    subprocess.run(["gcc", "-I", os.path.join(ROOT, "include"), str(src), "-o", str(exe)], check=True)
+    got = [int(v) for v in subprocess.run([str(exe)], capture_output=True, text=True, check=True).stdout.split()]
+    T = binding._Tensor
+    assert got == [C.sizeof(T), T.ndim.offset, T.dtype.offset, T.shape.offset, T.pdims.offset, T.sbp.offset,
+                   T.local.offset, T.local_ld.offset]
 
 
 def test_status_strings(lib):
@@ -229,3 +245,33 @@ def test_transfer_cost_is_table2(lib):
 
 def osig_(sig):
     return O.S(sig.axis) if sig.kind == 0 else {1: O.B, 2: O.PSUM, 3: O.PMAX}[sig.kind]
+
+
+@pytest.mark.parametrize("shape,k", [((6, 10), 3), ((7, 5), 4), ((4, 3, 8), 2), ((9,), 4), ((2, 16), 8)])
+def test_view_b_to_s_points_into_the_replicas(lib, shape, k):
+    """Host-only: the zero-copy B -> S(axis) view (Table 2: cost 0).  Every local tensor of the view is
+    the window of the replica that the oracle's split of the same tensor holds."""
+    n = 1
+    for s in shape:
+        n *= s
+    T = torch.arange(n, dtype=torch.float32).reshape(shape)
+    b = sbp.SbpTensor(shape, torch.float32, sbp.B, [T.clone() for _ in range(k)])
+    for axis in sorted({0, len(shape) - 1}):
+        v = sbp.sbp_view_b_to_s(b, axis)
+        want = O.to_locals(T.numpy(), O.S(axis), k)
+        for r in range(k):
+            assert tuple(v.locals[r].shape) == want[r].shape
+            assert (v.locals[r].numpy() == want[r]).all()
+            if v.locals[r].numel():
+                assert v.locals[r].untyped_storage().data_ptr() == b.locals[r].untyped_storage().data_ptr()
+    if len(shape) == 3:
+        with pytest.raises(sbp.SbpError) as e:
+            sbp.sbp_view_b_to_s(b, 1)
+        assert e.value.name == "SBP_ERR_UNSUPPORTED"
+    with pytest.raises(sbp.SbpError) as e:
+        sbp.sbp_view_b_to_s(sbp.SbpTensor(shape, torch.float32, sbp.S(0), list(O_split(T, k))), 0)
+    assert e.value.name == "SBP_ERR_SIGNATURE"
+
+
+def O_split(T, k):
+    return [torch.from_numpy(a.copy()) for a in O.to_locals(T.numpy(), O.S0, k)]

@@ -6,7 +6,7 @@ fp64 cross-check that is safe under cancellation.  P(max) is exact."""
 import numpy as np
 import pytest
 import torch
-from helpers import bits, make_global, np_bits, osig, split_cpu, storage_of, to_np
+from helpers import bits, check_guards, make_global, np_bits, osig, split_cpu, storage_of, to_np
 
 import paper_2110_15032_b200 as sbp
 import sbp_datagen as dg
@@ -59,6 +59,7 @@ def _run(shape, dtype, src_sig, dst_sig, k, seed=1, engine=0, alias=False, offse
         sbp.sbp_check_device_errors()
     finally:
         sbp.sbp_boxing_set_copy_engine(0)
+    check_guards()                                   # nothing was stored outside a destination shard
     assert len(want) == k
     for r in range(k):
         got = dst.locals[r]

@@ -9,7 +9,7 @@ import math
 import numpy as np
 import pytest
 import torch
-from helpers import assert_close, bits, make_global, np_bits, osig, split_cpu, to_np
+from helpers import assert_close, bits, check_guards, make_global, np_bits, osig, split_cpu, to_np
 
 import paper_2110_15032_b200 as sbp
 import sbp_datagen as dg
@@ -70,6 +70,7 @@ def _matmul_case(M, K, N, k, dtype, xs, ws, ys=None, flags=0, out_dtype=None, se
     sbp.sbp_matmul(x, w, y, flags, wsbuf)
     torch.cuda.synchronize()
     sbp.sbp_check_device_errors()
+    check_guards()
 
     y_sig, y_locals, Y = O.matmul_locals([to_np(t) for t in xl], osig(xs), [to_np(t) for t in wl], osig(ws))
     assert osig(natural) == y_sig
@@ -287,6 +288,7 @@ def _xent_case(rows, classes, k, dtype, sigma=1.0, seed=1004, alias=False, with_
     ws = torch.empty(sbp.sbp_softmax_xent_workspace_bytes(logits), dtype=torch.uint8, device="cuda")
     sbp.sbp_softmax_xent(logits, lab, loss, rmax, rsum, ws)
     torch.cuda.synchronize()
+    check_guards()
     m, Ssum, ref = O.softmax_xent_logical(to_np(Z), labels.numpy())
     for t in loss.locals:
         assert_close(to_np(t), ref, 2e-2, 1e-3, "loss")
@@ -354,6 +356,7 @@ def _emb_case(rows, dim, ids, k, dtype, fused, alias=False, table=None):
     oob = torch.zeros(1, dtype=torch.int32, device="cuda")
     sbp.sbp_embedding(tab, idt, out, oob)
     torch.cuda.synchronize()
+    check_guards()
     tnp = to_np(table)
     if fused:
         want = O.embedding_logical(tnp, ids.numpy())
@@ -506,6 +509,7 @@ def _fused_classifier_case(rows, feat, classes, k, seed, w_std=0.05, alias=False
     sbp.sbp_matmul_softmax_xent(f, w, lab, loss, rmax, rsum, ws)
     torch.cuda.synchronize()
     sbp.sbp_check_device_errors()
+    check_guards()
     Z = O.matmul_logical(to_np(Fm), to_np(W))
     m, S, ref = O.softmax_xent_logical(Z, labels.numpy())
     for t in loss.locals:
@@ -525,6 +529,7 @@ def _fused_classifier_case(rows, feat, classes, k, seed, w_std=0.05, alias=False
         sbp.sbp_matmul_softmax_xent_backward(f, w, lab, rmax, rsum, grad)
         torch.cuda.synchronize()
         sbp.sbp_check_device_errors()
+        check_guards()
         for r in range(k):
             assert tuple(grad.locals[r].shape) == tuple(want[r].shape)
             assert_close(to_np(grad.locals[r]), want[r], 2e-2, 1e-3, f"fused grad shard {r}")
@@ -664,3 +669,26 @@ def test_embedding_backward_large_batch(k, rows, dim, s, batch):
     got = O.from_locals([to_np(t).astype(np.float64) for t in gt.locals], O.S0)
     assert np.all(np.abs(got - want) <= counts * 2.0 ** -24 * mag + 1e-30)
     assert np.all(got[counts[:, 0] == 0] == 0.0)
+
+
+def test_repeated_tensor_core_product_encodes_no_new_descriptors():
+    """The copy-engine descriptors of a product are kept: calling it again on the same buffers
+    re-uses all of them (what a training loop does every step)."""
+    M, K, N, k = 256, 256, 512, 4
+    X = dg.normal(77, 0, (M, K), 0.0, 1.0, BF16)
+    W = dg.normal(77, 1, (K, N), 0.0, 0.1, BF16)
+    x = make_global([X] * k, (M, K), BF16, sbp.B)
+    w = make_global(split_cpu(W, sbp.S(1), k), (K, N), BF16, sbp.S(1))
+    y = sbp.empty_global((M, N), BF16, sbp.S(1), k)
+    ws = torch.empty(1, dtype=torch.uint8, device="cuda")
+    sbp.sbp_matmul(x, w, y, 0, ws)
+    reused0, encoded0 = sbp.sbp_tensor_map_stats()
+    assert encoded0 > 0                                   # this shape takes the tensor-core path
+    sbp.sbp_matmul(x, w, y, 0, ws)
+    reused1, encoded1 = sbp.sbp_tensor_map_stats()
+    assert encoded1 == encoded0 and reused1 >= reused0 + 3 * k
+    torch.cuda.synchronize()
+    check_guards()
+    want = O.to_locals(O.matmul_logical(to_np(X), to_np(W)), O.S1, k)
+    for r in range(k):
+        assert_close(to_np(y.locals[r]), want[r], 2e-2, 1e-3, f"shard {r}")

@@ -264,13 +264,24 @@ void sbp_boxing_set_copy_engine(int32_t engine);
  * dW = X^T dY (x = X with SBP_TRANS_X) and dX = dY W^T (w = W with SBP_TRANS_W).  Data
  * parallelism (Section 3.1: X S(0), W B) then gives dW = (S(1), S(0)) -> P(sum), and asking
  * for y as B folds the gradient all-reduce into the product.  One-axis placements only.
- * ws: scratch for the tensor-core path (see sbp_matmul_workspace_bytes; may be NULL when
- * that returns 0).
+ * ws: scratch for the tensor-core path (see below; may be NULL when the query returns 0).
+ * A result whose base or leading dimension the copy engine cannot address is written by the
+ * kernel's own stores instead; that needs no workspace.
  */
 #define SBP_EPILOGUE_GELU 1u
 #define SBP_TRANS_X 2u
 #define SBP_TRANS_W 4u
-size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y);   /* untransposed operands */
+/* Workspace: bf16 operands that the tensor-core path cannot address in place -- a local tensor whose
+ * base is not 16-byte aligned or whose leading dimension is not a multiple of 8 elements (a shard
+ * width of 333), or a fused S(i) result whose shards start on an odd column -- are first copied
+ * into `ws` in an aligned layout (one read and one write of the operand) so that the product stays
+ * on the tensor cores.  sbp_matmul_workspace_bytes_for returns the bytes that needs for the given
+ * descriptors and flags (0 when nothing has to be copied; judged from the shapes, so pass 256-byte
+ * aligned local tensors or add the operands' sizes yourself); ws must be 256-byte aligned.  Without
+ * a large enough workspace such a product runs on the FMA kernel: same results within the stated
+ * tolerance, far slower.  sbp_matmul_workspace_bytes is the same query for flags = 0. */
+size_t sbp_matmul_workspace_bytes_for(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y, uint32_t flags);
+size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y);
 
 /* The tensor-core path describes every operand and result tile layout to the copy engine with a
  * descriptor that the driver encodes on the host.  The library keeps the descriptors it has

@@ -105,6 +105,8 @@ def load_library():
     lib.sbp_selftest_wait_timeout.argtypes = [C.c_uint32, C.c_void_p]
     lib.sbp_matmul_workspace_bytes.restype = C.c_size_t
     lib.sbp_matmul_workspace_bytes.argtypes = [T, T, T]
+    lib.sbp_matmul_workspace_bytes_for.restype = C.c_size_t
+    lib.sbp_matmul_workspace_bytes_for.argtypes = [T, T, T, C.c_uint32]
     lib.sbp_matmul.argtypes = [T, T, T, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.sbp_tensor_map_stats.argtypes = [C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     lib.sbp_tensor_map_stats.restype = None
@@ -315,9 +317,9 @@ def sbp_boxing_host(src_host: SbpTensor, dst_host: SbpTensor, dev_ws: torch.Tens
                                           dev_ws.numel() * dev_ws.element_size(), _stream_ptr(stream)))
 
 
-def sbp_matmul_workspace_bytes(x: SbpTensor, w: SbpTensor, y: SbpTensor) -> int:
+def sbp_matmul_workspace_bytes(x: SbpTensor, w: SbpTensor, y: SbpTensor, flags: int = 0) -> int:
     a, b, c = x._c(), w._c(), y._c()
-    return int(load_library().sbp_matmul_workspace_bytes(C.byref(a), C.byref(b), C.byref(c)))
+    return int(load_library().sbp_matmul_workspace_bytes_for(C.byref(a), C.byref(b), C.byref(c), flags))
 
 
 def sbp_matmul(x: SbpTensor, w: SbpTensor, y: SbpTensor, flags: int = 0,

@@ -146,6 +146,186 @@ static sbp_status launch_fma(const MatmulPlan& p, cudaStream_t st) {
   return SBP_OK;
 }
 
+// ------------------------------------------------------------------ operands the copy engine cannot address
+//
+// The tensor-core kernel reads its operands through tiled bulk copies, which need a 16-byte aligned
+// base, a row pitch that is a multiple of 16 bytes and, for the operand whose contiguous index is M
+// or N, a start column that is a multiple of 8 elements.  A bf16 operand that breaks one of these
+// rules (a shard width of 333, an odd column offset of a fused S(1) result) is first copied into
+// the caller's workspace in a layout that keeps them: rows padded to a multiple of 8 elements,
+// every output group's column block starting on a multiple of 8.  The product then runs on the
+// tensor cores from the copy instead of falling to the FMA kernel (two orders of magnitude slower
+// at large sizes); the copy costs one read and one write of the operand.
+
+struct PackBlock {
+  const unsigned short* src;
+  unsigned short* dst;
+  long long rows, cols, src_ld, dst_ld;
+};
+constexpr int kPackBlocks = 64;
+struct PackList {
+  PackBlock b[kPackBlocks];
+};
+
+// One 16-byte store per thread and step: eight consecutive elements of a row, zeros past its end.
+__global__ void __launch_bounds__(256) matmul_pack_kernel(const __grid_constant__ PackList L) {
+  const PackBlock& B = L.b[blockIdx.y];
+  const long long groups = (B.cols + 7) / 8;
+  const long long total = B.rows * groups;
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < total; i += (long long)gridDim.x * 256) {
+    const long long row = i / groups, g8 = i - row * groups;
+    const unsigned short* sp = B.src + row * B.src_ld + g8 * 8;
+    unsigned short v[8];
+#pragma unroll
+    for (int e = 0; e < 8; ++e) v[e] = (g8 * 8 + e < B.cols) ? __ldg(sp + e) : (unsigned short)0;
+    uint4 o;
+    o.x = v[0] | ((unsigned)v[1] << 16);
+    o.y = v[2] | ((unsigned)v[3] << 16);
+    o.z = v[4] | ((unsigned)v[5] << 16);
+    o.w = v[6] | ((unsigned)v[7] << 16);
+    *reinterpret_cast<uint4*>(B.dst + row * B.dst_ld + g8 * 8) = o;
+  }
+}
+
+static long long pad8(long long v) { return (v + 7) / 8 * 8; }
+static size_t align256(size_t v) { return (v + 255) & ~size_t(255); }
+static bool aligned16p(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
+
+// What has to be repacked for the tensor-core kernel to take a bf16 plan, and how large the copies are.
+struct PackNeed {
+  bool a, b;              // operand x / w needs a packed copy
+  bool a_blocked, b_blocked;   // its M / N index is cut into one block per output group
+  size_t bytes;
+};
+
+static PackNeed pack_need(const MatmulPlan& p, bool with_ptrs) {
+  PackNeed n{};
+  if (p.in_dtype != SBP_BF16) return n;
+  for (int s = 0; s < p.nseg; ++s) {
+    const bool used = p.chain || s < p.ngroups;
+    if (!used || p.kseg[s] == 0) continue;
+    if (p.lda[s] % 8 != 0 || (with_ptrs && !aligned16p(p.a[s]))) n.a = true;
+    if (p.ldb[s] % 8 != 0 || (with_ptrs && !aligned16p(p.b[s]))) n.b = true;
+  }
+  for (int g = 0; g < p.ngroups; ++g) {
+    if (p.a_trans && p.row_off[g] % 8 != 0) n.a = n.a_blocked = true;
+    if (!p.b_trans && p.col_off[g] % 8 != 0) n.b = n.b_blocked = true;
+  }
+  // a packed operand whose M / N index is contiguous keeps the groups' blocks apart whenever offsets are in use
+  if (n.a && p.a_trans && p.chain && p.ngroups > 1) n.a_blocked = true;
+  if (n.b && !p.b_trans && p.chain && p.ngroups > 1) n.b_blocked = true;
+  long long rows_a = 0, cols_b = 0, blocked_a = 0, blocked_b = 0;
+  for (int g = 0; g < p.ngroups; ++g) {
+    rows_a = rows_a > p.row_off[g] + p.m[g] ? rows_a : p.row_off[g] + p.m[g];
+    cols_b = cols_b > p.col_off[g] + p.n[g] ? cols_b : p.col_off[g] + p.n[g];
+    blocked_a += pad8(p.m[g]);
+    blocked_b += pad8(p.n[g]);
+  }
+  for (int s = 0; s < p.nseg; ++s) {
+    const bool used = p.chain || s < p.ngroups;
+    if (!used || p.kseg[s] == 0) continue;
+    const long long ra = p.chain ? rows_a : p.m[s], cb = p.chain ? cols_b : p.n[s];
+    if (n.a) n.bytes += align256((size_t)(p.a_trans ? p.kseg[s] * (n.a_blocked ? blocked_a : pad8(ra)) : ra * pad8(p.kseg[s])) * 2);
+    if (n.b) n.bytes += align256((size_t)(p.b_trans ? cb * pad8(p.kseg[s]) : p.kseg[s] * (n.b_blocked ? blocked_b : pad8(cb))) * 2);
+  }
+  return n;
+}
+
+// Copies the operands named by `need` into ws and rewrites the plan to read the copies.
+static sbp_status pack_operands(MatmulPlan* plan, const PackNeed& need, void* ws, cudaStream_t st) {
+  MatmulPlan& p = *plan;
+  PackList list{};
+  int nb = 0;
+  auto flush = [&]() -> sbp_status {
+    if (nb == 0) return SBP_OK;
+    long long most = 0;
+    for (int i = 0; i < nb; ++i) {
+      const long long t = list.b[i].rows * ((list.b[i].cols + 7) / 8);
+      most = t > most ? t : most;
+    }
+    long long gx = (most + 255) / 256;
+    if (gx < 1) gx = 1;
+    if (gx > 148 * 8) gx = 148 * 8;
+    matmul_pack_kernel<<<dim3((unsigned)gx, (unsigned)nb), 256, 0, st>>>(list);
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(e, "operand repack launch");
+    count_launch();
+    nb = 0;
+    return SBP_OK;
+  };
+  auto add = [&](const void* src, void* dst, long long rows, long long cols, long long sld, long long dld) -> sbp_status {
+    if (rows == 0 || cols == 0) return SBP_OK;
+    list.b[nb++] = PackBlock{static_cast<const unsigned short*>(src), static_cast<unsigned short*>(dst), rows, cols, sld, dld};
+    return nb == kPackBlocks ? flush() : SBP_OK;
+  };
+  long long rows_a = 0, cols_b = 0, blocked_a = 0, blocked_b = 0;
+  long long new_row_off[SBP_MAX_K], new_col_off[SBP_MAX_K];
+  for (int g = 0; g < p.ngroups; ++g) {
+    rows_a = rows_a > p.row_off[g] + p.m[g] ? rows_a : p.row_off[g] + p.m[g];
+    cols_b = cols_b > p.col_off[g] + p.n[g] ? cols_b : p.col_off[g] + p.n[g];
+    new_row_off[g] = blocked_a;
+    new_col_off[g] = blocked_b;
+    blocked_a += pad8(p.m[g]);
+    blocked_b += pad8(p.n[g]);
+  }
+  char* cur = static_cast<char*>(ws);
+  sbp_status stt;
+  for (int s = 0; s < p.nseg; ++s) {
+    const bool used = p.chain || s < p.ngroups;
+    if (!used || p.kseg[s] == 0) continue;
+    const long long K = p.kseg[s];
+    const long long ra = p.chain ? rows_a : p.m[s], cb = p.chain ? cols_b : p.n[s];
+    if (need.a) {
+      const unsigned short* src = static_cast<const unsigned short*>(p.a[s]);
+      unsigned short* dst = reinterpret_cast<unsigned short*>(cur);
+      long long ld;
+      if (!p.a_trans) {                       // stored [rows, K]
+        ld = pad8(K);
+        if ((stt = add(src, dst, ra, K, p.lda[s], ld)) != SBP_OK) return stt;
+        cur += align256((size_t)ra * ld * 2);
+      } else if (!need.a_blocked) {           // stored [K, rows]
+        ld = pad8(ra);
+        if ((stt = add(src, dst, K, ra, p.lda[s], ld)) != SBP_OK) return stt;
+        cur += align256((size_t)K * ld * 2);
+      } else {                                // stored [K, rows], one column block per output group
+        ld = blocked_a;
+        for (int g = 0; g < p.ngroups; ++g)
+          if ((stt = add(src + p.row_off[g], dst + new_row_off[g], K, p.m[g], p.lda[s], ld)) != SBP_OK) return stt;
+        cur += align256((size_t)K * ld * 2);
+      }
+      p.a[s] = dst;
+      p.lda[s] = ld;
+    }
+    if (need.b) {
+      const unsigned short* src = static_cast<const unsigned short*>(p.b[s]);
+      unsigned short* dst = reinterpret_cast<unsigned short*>(cur);
+      long long ld;
+      if (p.b_trans) {                        // stored [cols, K]
+        ld = pad8(K);
+        if ((stt = add(src, dst, cb, K, p.ldb[s], ld)) != SBP_OK) return stt;
+        cur += align256((size_t)cb * ld * 2);
+      } else if (!need.b_blocked) {           // stored [K, cols]
+        ld = pad8(cb);
+        if ((stt = add(src, dst, K, cb, p.ldb[s], ld)) != SBP_OK) return stt;
+        cur += align256((size_t)K * ld * 2);
+      } else {
+        ld = blocked_b;
+        for (int g = 0; g < p.ngroups; ++g)
+          if ((stt = add(src + p.col_off[g], dst + new_col_off[g], K, p.n[g], p.ldb[s], ld)) != SBP_OK) return stt;
+        cur += align256((size_t)K * ld * 2);
+      }
+      p.b[s] = dst;
+      p.ldb[s] = ld;
+    }
+  }
+  if ((stt = flush()) != SBP_OK) return stt;
+  for (int g = 0; g < p.ngroups; ++g) {
+    if (need.a_blocked) p.row_off[g] = new_row_off[g];
+    if (need.b_blocked) p.col_off[g] = new_col_off[g];
+  }
+  return SBP_OK;
+}
+
 static bool is_s(sbp_sig s, int ax) { return s.kind == SBP_SPLIT && s.axis == ax; }
 static bool is_b(sbp_sig s) { return s.kind == SBP_BROADCAST; }
 static bool is_p(sbp_sig s) { return s.kind == SBP_PARTIAL_SUM; }
@@ -273,12 +453,12 @@ static sbp_status build_plan(const sbp_tensor* x, const sbp_tensor* w, const sbp
 // own -- e.g. (S(0),B) x (B,S(1)) -> (S(0),S(1)) and (S(0),S(1)) x (B,S(0)) -> (S(0),P(sum)) --
 // and every device multiplies its local tensors.  No fused output boxing on this path.
 static sbp_status build_plan_2d(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y, uint32_t flags,
-                                MatmulPlan* plan) {
-  sbp_status st = check_tensor_nd(x, "x", true);
+                                bool need_ptrs, MatmulPlan* plan) {
+  sbp_status st = check_tensor_nd(x, "x", need_ptrs);
   if (st != SBP_OK) return st;
-  st = check_tensor_nd(w, "w", true);
+  st = check_tensor_nd(w, "w", need_ptrs);
   if (st != SBP_OK) return st;
-  st = check_tensor_nd(y, "y", true);
+  st = check_tensor_nd(y, "y", need_ptrs);
   if (st != SBP_OK) return st;
   if (x->pdims != 2 || w->pdims != 2 || y->pdims != 2) return fail(SBP_ERR_INVALID_ARG, "x, w and y must share one two-axis placement");
   for (int p = 0; p < 2; ++p)
@@ -340,10 +520,17 @@ using namespace sbp;
 
 extern "C" {
 
-size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y) {
+size_t sbp_matmul_workspace_bytes_for(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y, uint32_t flags) {
   MatmulPlan plan;
-  if (build_plan(x, w, y, 0, false, &plan) != SBP_OK) return 0;
-  return matmul_tc_workspace_bytes(plan);
+  const bool two_axes = x && w && y && (x->pdims == 2 || w->pdims == 2 || y->pdims == 2);
+  const sbp_status st = two_axes ? build_plan_2d(x, w, y, flags, false, &plan) : build_plan(x, w, y, flags, false, &plan);
+  if (st != SBP_OK) return 0;
+  // without pointers to look at, an operand counts as misaligned only by its shape
+  return pack_need(plan, false).bytes + matmul_tc_workspace_bytes(plan);
+}
+
+size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, const sbp_tensor* y) {
+  return sbp_matmul_workspace_bytes_for(x, w, y, 0);
 }
 
 void sbp_tensor_map_stats(uint64_t* reused, uint64_t* encoded) {
@@ -357,14 +544,22 @@ sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, u
                       size_t ws_bytes, void* cuda_stream) {
   MatmulPlan plan;
   const bool two_axes = x && w && y && (x->pdims == 2 || w->pdims == 2 || y->pdims == 2);
-  sbp_status st = two_axes ? build_plan_2d(x, w, y, flags, &plan) : build_plan(x, w, y, flags, true, &plan);
+  sbp_status st = two_axes ? build_plan_2d(x, w, y, flags, true, &plan) : build_plan(x, w, y, flags, true, &plan);
   if (st != SBP_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   bool taken = false;
-  (void)ws;
-  (void)ws_bytes;
   st = launch_matmul_tc(plan, nullptr, stream, &taken);
   if (taken) return st;
+  // bf16 operands that only miss the copy engine's alignment rules: repack them into the workspace,
+  // when the caller gave one that is large enough, and stay on the tensor cores
+  const PackNeed need = pack_need(plan, true);
+  if ((need.a || need.b) && ws && ws_bytes >= need.bytes && reinterpret_cast<uintptr_t>(ws) % 256 == 0) {
+    MatmulPlan packed = plan;
+    st = pack_operands(&packed, need, ws, stream);
+    if (st != SBP_OK) return st;
+    st = launch_matmul_tc(packed, nullptr, stream, &taken);
+    if (taken) return st;
+  }
   return launch_fma(plan, stream);
 }
 

@@ -71,6 +71,12 @@ struct TcParams {
   int total_tiles;
   int xent;                     // 1: softmax partials instead of stored logits
   XentFusion xf;
+  // Results the copy engine cannot address (a base or a row pitch that is not a multiple of 16
+  // bytes): the epilogue then writes its staged slabs itself, row by row, with element-wise stores.
+  int y_direct;
+  void* y_ptr[SBP_MAX_K];
+  void* rep_ptr[SBP_MAX_K];
+  long long ldy[SBP_MAX_K];
 };
 
 // ------------------------------------------------------------------ PTX helpers
@@ -549,6 +555,33 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
                 *reinterpret_cast<uint4*>(rowp + ((c ^ (lane & 7)) << 4)) = o;
               }
             }
+            if (p.y_direct) {
+              // rows of the slab, one after the other; the lanes take consecutive elements of a row
+              __syncwarp();
+              const int n_out = (tc.g == 0 ? p.n_rep : 0) + 1;
+              for (int o = 0; o < n_out; ++o) {
+                unsigned char* yb = static_cast<unsigned char*>(o == 0 ? p.y_ptr[tc.g] : p.rep_ptr[o - 1]);
+                const long long ld = p.ldy[tc.g];
+                for (int r = 0; r < 32 && row0 + r < Mg; ++r) {
+                  const unsigned char* srow = buf + r * 128;
+                  if (p.out_f32) {
+                    const int c = lane;
+                    if (col0 + c < Ng)
+                      reinterpret_cast<float*>(yb)[(row0 + r) * ld + col0 + c] =
+                          *reinterpret_cast<const float*>(srow + ((((c >> 2) ^ (r & 7)) << 4) | ((c & 3) << 2)));
+                  } else {
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                      const int c = lane + 32 * h;
+                      if (col0 + c < Ng)
+                        reinterpret_cast<unsigned short*>(yb)[(row0 + r) * ld + col0 + c] =
+                            *reinterpret_cast<const unsigned short*>(srow + ((((c >> 3) ^ (r & 7)) << 4) | ((c & 7) << 1)));
+                    }
+                  }
+                }
+              }
+              __syncwarp();      // the buffer is rewritten two slabs from now
+            } else {
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0) {
@@ -556,6 +589,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
               if (tc.g == 0)
                 for (int r = 0; r < p.n_rep; ++r) tma_store_2d(&p.map_rep[r], col0, row0, smem_addr(buf));
               asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+            }
             }
             ++slab_iter;
           }
@@ -723,11 +757,12 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
     if (plan.lda[s] % 8 != 0 || plan.ldb[s] % 8 != 0) return SBP_ERR_UNSUPPORTED;
     if (plan.lda[s] == 0 || plan.ldb[s] == 0) return SBP_ERR_UNSUPPORTED;
   }
+  bool y_direct = false;
   long long ktotal_chain = 0;
   for (int s = 0; s < plan.nseg; ++s) ktotal_chain += plan.kseg[s];
   for (int g = 0; g < plan.ngroups; ++g) {
     if (plan.m[g] == 0 || plan.n[g] == 0) continue;
-    if (stores_y && (!aligned16(plan.y[g]) || (plan.ldy[g] * oesz) % 16 != 0)) return SBP_ERR_UNSUPPORTED;
+    if (stores_y && (!aligned16(plan.y[g]) || (plan.ldy[g] * oesz) % 16 != 0)) y_direct = true;
     if (!plan.b_trans && plan.col_off[g] % 8 != 0) return SBP_ERR_UNSUPPORTED;   // the x coordinate of a TMA load
     if (plan.a_trans && plan.row_off[g] % 8 != 0) return SBP_ERR_UNSUPPORTED;
     const long long kg = plan.chain ? ktotal_chain : plan.kseg[g];
@@ -735,7 +770,7 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
     if (plan.m[g] > 0x7fffffffLL || plan.n[g] > 0x7fffffffLL) return SBP_ERR_UNSUPPORTED;
   }
   for (int r = 0; r < plan.n_rep; ++r)
-    if (!aligned16(plan.y_rep[r])) return SBP_ERR_UNSUPPORTED;
+    if (!aligned16(plan.y_rep[r])) y_direct = true;
   if (!encode_fn()) return SBP_ERR_UNSUPPORTED;
 
   static TcParams p;          // large; filled under a lock and copied by value at launch
@@ -749,6 +784,7 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
   p.out_f32 = plan.out_dtype == SBP_F32;
   p.xent = xf ? (xf->grad ? 2 : 1) : 0;
   if (xf) p.xf = *xf;
+  p.y_direct = y_direct ? 1 : 0;
 
   for (int s = 0; s < plan.nseg; ++s) {
     p.kblocks[s] = (int)((plan.kseg[s] + BK - 1) / BK);
@@ -787,16 +823,20 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
     if (plan.m[g] > 0 && plan.n[g] > 0) {
       if (tm * tn + tiles > 0x3fffffffLL) return SBP_ERR_UNSUPPORTED;
       tiles += (int)(tm * tn);
-      if (stores_y && !make_map(&p.map_y[g], plan.y[g], oesz, plan.m[g], plan.n[g], plan.ldy[g], 32, box_cols))
+      p.y_ptr[g] = plan.y[g];
+      p.ldy[g] = plan.ldy[g];
+      if (stores_y && !y_direct && !make_map(&p.map_y[g], plan.y[g], oesz, plan.m[g], plan.n[g], plan.ldy[g], 32, box_cols))
         return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for the result of group %d", g);
     }
   }
   p.tile_begin[plan.ngroups] = tiles;
   for (int g = plan.ngroups + 1; g <= SBP_MAX_K; ++g) p.tile_begin[g] = tiles;
   p.total_tiles = tiles;
-  for (int r = 0; r < plan.n_rep; ++r)
-    if (!make_map(&p.map_rep[r], plan.y_rep[r], oesz, plan.m[0], plan.n[0], plan.ldy[0], 32, box_cols))
+  for (int r = 0; r < plan.n_rep; ++r) {
+    p.rep_ptr[r] = plan.y_rep[r];
+    if (!y_direct && !make_map(&p.map_rep[r], plan.y_rep[r], oesz, plan.m[0], plan.n[0], plan.ldy[0], 32, box_cols))
       return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for a result replica");
+  }
   *taken = true;
   if (tiles == 0) return SBP_OK;
 

@@ -41,7 +41,7 @@ def _swap(sig):
     return sbp.S(1 - sig.axis) if sig.kind == 0 else sig
 
 
-def _matmul_case(M, K, N, k, dtype, xs, ws, ys=None, flags=0, out_dtype=None, seed=1001, tx=False, tw=False):
+def _matmul_case(M, K, N, k, dtype, xs, ws, ys=None, flags=0, out_dtype=None, seed=1001, tx=False, tw=False, use_ws=True):
     """xs / ws are the signatures of the operands as they enter the product.  With tx (tw) the
     library is handed the transpose of x (w) -- stored [K,M] ([N,K]) with the swapped signature --
     together with SBP_TRANS_X (SBP_TRANS_W); the oracle sees the untransposed operands."""
@@ -65,8 +65,8 @@ def _matmul_case(M, K, N, k, dtype, xs, ws, ys=None, flags=0, out_dtype=None, se
     y = sbp.empty_global((M, N), out_dtype, ys, k)
     for t in y.locals:
         t.view(torch.uint8).fill_(0x7F)
-    nbytes = 0 if (tx or tw) else sbp.sbp_matmul_workspace_bytes(x, w, y)
-    wsbuf = torch.empty(max(nbytes, 1), dtype=torch.uint8, device="cuda")
+    nbytes = sbp.sbp_matmul_workspace_bytes(x, w, y, flags) if use_ws else 0
+    wsbuf = torch.empty(max(nbytes, 1), dtype=torch.uint8, device="cuda") if use_ws else None
     sbp.sbp_matmul(x, w, y, flags, wsbuf)
     torch.cuda.synchronize()
     sbp.sbp_check_device_errors()
@@ -692,3 +692,33 @@ def test_repeated_tensor_core_product_encodes_no_new_descriptors():
     want = O.to_locals(O.matmul_logical(to_np(X), to_np(W)), O.S1, k)
     for r in range(k):
         assert_close(to_np(y.locals[r]), want[r], 2e-2, 1e-3, f"shard {r}")
+
+
+UNALIGNED = [  # M, K, N, k: shard widths / contraction lengths that are not multiples of 8 elements
+    (130, 70, 333, 3), (96, 136, 2 * 333, 2), (257, 64, 90, 4)]
+
+
+@pytest.mark.parametrize("xs,ws,ys", [(sbp.S(0), sbp.B, None), (sbp.B, sbp.S(1), None), (sbp.S(1), sbp.S(0), None),
+                                      (sbp.S(1), sbp.S(0), sbp.B), (sbp.S(1), sbp.S(0), sbp.S(1)), (sbp.S(1), sbp.S(0), sbp.S(0)),
+                                      (sbp.P_SUM, sbp.B, None), (sbp.B, sbp.B, None)])
+@pytest.mark.parametrize("shape", UNALIGNED)
+def test_matmul_bf16_unaligned_shapes_stay_on_tensor_cores(xs, ws, ys, shape):
+    """bf16 operands whose shard widths miss the copy engine's 16-byte rules: with a workspace they
+    are repacked and multiplied on the tensor cores (descriptors get encoded), without one the FMA
+    kernel takes them; both meet the stated tolerance against the oracle."""
+    M, K, N, k = shape
+    before = sum(sbp.sbp_tensor_map_stats())
+    _matmul_case(M, K, N, k, BF16, xs, ws, ys=ys, seed=1201)
+    assert sum(sbp.sbp_tensor_map_stats()) > before, "the repacked product did not reach the tensor-core kernel"
+    before = sum(sbp.sbp_tensor_map_stats())
+    _matmul_case(M, K, N, k, BF16, xs, ws, ys=ys, seed=1201, use_ws=False)
+    assert sum(sbp.sbp_tensor_map_stats()) == before, "without a workspace the FMA kernel is the one that runs"
+
+
+@pytest.mark.parametrize("tx,tw", [(True, False), (False, True), (True, True)])
+@pytest.mark.parametrize("xs,ws,ys", [(sbp.S(0), sbp.B, None), (sbp.B, sbp.S(1), None), (sbp.S(1), sbp.S(0), sbp.S(0)),
+                                      (sbp.S(1), sbp.S(0), sbp.S(1)), (sbp.S(1), sbp.S(0), sbp.B)])
+def test_matmul_bf16_unaligned_transposed_operands(xs, ws, ys, tx, tw):
+    for M, K, N, k in UNALIGNED[:2]:
+        _matmul_case(M, K, N, k, BF16, xs, ws, ys=ys, seed=1202, tx=tx, tw=tw)
+        _matmul_case(M, K, N, k, BF16, xs, ws, ys=ys, seed=1202, tx=tx, tw=tw, out_dtype=F32)

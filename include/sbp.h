@@ -48,7 +48,9 @@ typedef enum {
   SBP_ERR_ALIGNMENT = 6,   /* a pointer is not aligned to its element size               */
   SBP_ERR_WORKSPACE = 7,   /* workspace missing or too small                             */
   SBP_ERR_CUDA = 8,        /* a CUDA runtime / driver call failed (no device, launch...) */
-  SBP_ERR_TIMEOUT = 9      /* a bounded device-side wait expired                         */
+  SBP_ERR_TIMEOUT = 9,     /* a bounded device-side wait expired                         */
+  SBP_ERR_BOUNDS = 10      /* debug-bounds build only: a kernel computed an address outside
+                              the buffers of its call (the access was skipped)           */
 } sbp_status;
 
 typedef enum { SBP_F32 = 0, SBP_BF16 = 1, SBP_I64 = 2 } sbp_dtype;
@@ -219,9 +221,27 @@ size_t sbp_boxing_host_workspace_bytes(const sbp_tensor* src_host, const sbp_ten
 sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, void* dev_ws,
                            size_t dev_ws_bytes, void* cuda_stream);
 
+/* 1 when this library was compiled as the debug-bounds build, else 0.  In that build every
+ * global-memory address a kernel computes is compared, before it is used, with the buffers of the
+ * call (every local tensor by its host-computed extent, and the workspace); an address outside
+ * them is recorded and the access skipped -- nothing traps -- and the next
+ * sbp_check_device_errors() returns SBP_ERR_BOUNDS.  It is an order of magnitude slower than the
+ * normal build and meant for small and ragged test shapes; it stands in for a memory checker where
+ * none can be run.  Build it with `python -m paper_2110_15032_b200.build --debug-bounds`
+ * (libsbp_b200_dbg.so) and select it with SBP_B200_LIBRARY=<path> before the package loads. */
+int32_t sbp_debug_bounds_enabled(void);
+
+/* Self-test of that report path, safe to run anywhere (debug-bounds build only; the normal build
+ * answers SBP_ERR_UNSUPPORTED): registers the device buffer [buf, buf + bytes) and enqueues a
+ * one-thread kernel that asks the checker about buf[0] (allowed: the byte is set to 1) and about
+ * the byte just past the end (refused: recorded, and NOT accessed).  After the stream has drained,
+ * sbp_check_device_errors() returns SBP_ERR_BOUNDS once. */
+sbp_status sbp_selftest_debug_bounds(void* buf, size_t bytes, void* cuda_stream);
+
 /* Kernels of this library bound every device-side wait.  When one expires the kernel sets a
  * device flag and returns; this call (which synchronises with the device) reads and clears
- * the flag: SBP_ERR_TIMEOUT if a wait expired since the last call, else SBP_OK. */
+ * the flag: SBP_ERR_TIMEOUT if a wait expired since the last call, else SBP_OK (debug-bounds
+ * build: SBP_ERR_BOUNDS first, if a kernel's address check failed). */
 sbp_status sbp_check_device_errors(void);
 
 /* Self-test of that path, safe to run anywhere: enqueues a one-thread kernel that waits on a
@@ -255,7 +275,10 @@ void sbp_boxing_set_copy_engine(int32_t engine);
  *   SBP_BF16 : bf16 operands, fp32 accumulation on the tensor cores, y SBP_BF16 or SBP_F32.
  * flags: SBP_EPILOGUE_GELU applies GeLU(v) = v/2 (1 + erf(v/sqrt 2)) to the fp32
  * accumulator before the store; only where Y is S or B (GeLU is not linear, so it cannot
- * be applied to partial values).
+ * be applied to partial values).  erf is evaluated to about 1.5e-7 absolute on the tensor-core
+ * path (a rational approximation) and by the fp32 library erf on the FMA path, so the same call
+ * may differ in the last bits of an fp32 result depending on which kernel its shapes select;
+ * both are far inside the stated tolerance.
  *        SBP_TRANS_X / SBP_TRANS_W: the descriptor x (w) holds the transpose of the operand,
  * i.e. x is stored as [K,M] (w as [N,K]), logically and in every local tensor, and its
  * signature refers to the stored axes.  The operand that enters Table 1 is the transpose, so a
@@ -399,7 +422,9 @@ sbp_status sbp_embedding(const sbp_tensor* table, const sbp_tensor* ids, sbp_ten
  *                           zero for rows never looked up (the whole tensor is written)
  * dim must be a multiple of 4.  The sums are accumulated with fp32 atomic adds in no fixed
  * order, so a row that many lookups hit may differ in its last bits from run to run.  Ids
- * outside [0, rows) contribute nothing (and are counted in oob_count when it is not NULL). */
+ * outside [0, rows) contribute nothing (and are counted in oob_count when it is not NULL).
+ * Two launches (zero fill, then scatter-add): every argument check comes before the first, but
+ * should the second LAUNCH itself fail (SBP_ERR_CUDA) the gradient has already been zeroed. */
 sbp_status sbp_embedding_backward(const sbp_tensor* grad_out, const sbp_tensor* ids, sbp_tensor* grad_table,
                                   int32_t* oob_count, void* cuda_stream);
 

@@ -70,7 +70,9 @@ _LIB = None
 
 
 def lib_path() -> str:
-    return os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsbp_b200.so")
+    """The library this process loads: libsbp_b200.so beside this file, or the file SBP_B200_LIBRARY
+    names (the debug-bounds build, for instance)."""
+    return os.environ.get("SBP_B200_LIBRARY") or os.path.join(os.path.dirname(os.path.abspath(__file__)), "libsbp_b200.so")
 
 
 def load_library():
@@ -89,6 +91,8 @@ def load_library():
     lib.sbp_status_string.argtypes = [C.c_int]
     lib.sbp_last_error.restype = C.c_char_p
     lib.sbp_launch_count.restype = C.c_uint64
+    lib.sbp_debug_bounds_enabled.restype = C.c_int32
+    lib.sbp_selftest_debug_bounds.argtypes = [C.c_void_p, C.c_size_t, C.c_void_p]
     lib.sbp_local_shape.argtypes = [T, C.c_int32, C.POINTER(C.c_int64)]
     lib.sbp_view_b_to_s.argtypes = [T, C.c_int32, T]
     lib.sbp_matmul_infer.argtypes = [_Sig, _Sig, C.POINTER(_Sig)]
@@ -276,6 +280,15 @@ def sbp_tensor_map_stats():
     a, b = C.c_uint64(), C.c_uint64()
     load_library().sbp_tensor_map_stats(C.byref(a), C.byref(b))
     return int(a.value), int(b.value)
+
+
+def sbp_selftest_debug_bounds(buf: torch.Tensor, stream=None) -> None:
+    _check(load_library().sbp_selftest_debug_bounds(C.c_void_p(buf.data_ptr()), buf.numel() * buf.element_size(),
+                                                    _stream_ptr(stream)))
+
+
+def sbp_debug_bounds_enabled() -> bool:
+    return bool(load_library().sbp_debug_bounds_enabled())
 
 
 def sbp_launch_count() -> int:

@@ -18,6 +18,7 @@
 #include <algorithm>
 #include <atomic>
 
+#include "bounds_check.h"
 #include "boxing_arith.h"
 #include "boxing_params.h"
 #include "sbp_internal.h"
@@ -109,7 +110,7 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
     const V* sp = reinterpret_cast<const V*>(p.src[s]);
 #pragma unroll
     for (int j = 0; j < J; ++j)
-      if (ok[j]) val[j] = ld_stream(sp + so[j]);
+      if (ok[j] && SBP_GUARD(sp + so[j], sizeof(V))) val[j] = ld_stream(sp + so[j]);
 
   } else {
     using L = typename Lanes<OP, V>::type;
@@ -120,7 +121,8 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
       for (int j = 0; j < J; ++j)
 #pragma unroll
         for (int r = 0; r < (KT ? KT : 1); ++r)
-          if (ok[j]) raw[j][r] = ld_stream(reinterpret_cast<const V*>(p.src[r]) + so[j]);
+          if (ok[j] && SBP_GUARD(reinterpret_cast<const V*>(p.src[r]) + so[j], sizeof(V)))
+            raw[j][r] = ld_stream(reinterpret_cast<const V*>(p.src[r]) + so[j]);
 #pragma unroll
       for (int j = 0; j < J; ++j) {
         if (!ok[j]) continue;
@@ -139,9 +141,11 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
       for (int j = 0; j < J; ++j) {
         if (!ok[j]) continue;
         L acc;
+        if (!SBP_GUARD(reinterpret_cast<const V*>(p.src[0]) + so[j], sizeof(V))) continue;
         acc.load(ld_stream(reinterpret_cast<const V*>(p.src[0]) + so[j]));
         for (int r = 1; r < kk; ++r) {
           L x;
+          if (!SBP_GUARD(reinterpret_cast<const V*>(p.src[r]) + so[j], sizeof(V))) continue;
           x.load(ld_stream(reinterpret_cast<const V*>(p.src[r]) + so[j]));
           combine<OP>(acc, x);
         }
@@ -155,13 +159,13 @@ __global__ void __launch_bounds__(256) box_tile_kernel(const __grid_constant__ B
       V* dp = reinterpret_cast<V*>(p.dst[r]);
 #pragma unroll
       for (int j = 0; j < J; ++j)
-        if (ok[j]) st_stream(dp + dofs[j], val[j]);
+        if (ok[j] && SBP_GUARD(dp + dofs[j], sizeof(V))) st_stream(dp + dofs[j], val[j]);
     }
   } else {
     V* dp = reinterpret_cast<V*>(p.dst[d]);
 #pragma unroll
     for (int j = 0; j < J; ++j)
-      if (ok[j]) st_stream(dp + dofs[j], val[j]);
+      if (ok[j] && SBP_GUARD(dp + dofs[j], sizeof(V))) st_stream(dp + dofs[j], val[j]);
   }
 }
 
@@ -211,12 +215,12 @@ __global__ void __launch_bounds__(256) box_scatter_kernel(const __grid_constant_
     for (int j = 0; j < kScatterJ; ++j) {
       const long long col = col0 + j * 256;
       val[j] = V{};
-      if (col >= lo && col < hi) val[j] = ld_stream(sp + row * w + (col - lo));
+      if (col >= lo && col < hi && SBP_GUARD(sp + row * w + (col - lo), sizeof(V))) val[j] = ld_stream(sp + row * w + (col - lo));
     }
 #pragma unroll
     for (int j = 0; j < kScatterJ; ++j) {
       const long long col = col0 + j * 256;
-      if (col < p.row_vecs) dp[row * p.row_vecs + col] = val[j];
+      if (col < p.row_vecs && SBP_GUARD(dp + row * p.row_vecs + col, sizeof(V))) dp[row * p.row_vecs + col] = val[j];
     }
   }
 }
@@ -225,6 +229,7 @@ template <typename V>
 static void launch_scatter_v(const ScatterParams& sp, int k, cudaStream_t st) {
   long long gx = sp.total_chunks < 148 * 6 ? sp.total_chunks : 148 * 6;
   if (gx < 1) gx = 1;
+  SBP_BOUNDS_UPLOAD(st);
   launch_dependent(box_scatter_kernel<V>, dim3((unsigned)gx, (unsigned)k), dim3(256), 0, st, sp);
 }
 
@@ -257,11 +262,11 @@ __global__ void __launch_bounds__(256) box_gather_cast_kernel(const __grid_const
     chunk_row(c, chunks_per_row, &row, &within);
     const long long col0 = within * (256 * J) + threadIdx.x;
     const float* sp = p.src[s] + (row * w) * EPV;
-    float v[J][EPV];
+    float v[J][EPV] = {};
 #pragma unroll
     for (int j = 0; j < J; ++j) {
       const long long col = col0 + j * 256;
-      if (col < w) {
+      if (col < w && SBP_GUARD(sp + col * EPV, EPV * sizeof(float))) {
         if (EPV == 8) {
           const float4 a = __ldg(reinterpret_cast<const float4*>(sp + col * 8));
           const float4 b = __ldg(reinterpret_cast<const float4*>(sp + col * 8) + 1);
@@ -284,10 +289,12 @@ __global__ void __launch_bounds__(256) box_gather_cast_kernel(const __grid_const
         h = __floats2bfloat162_rn(v[j][2], v[j][3]); o.y = *reinterpret_cast<unsigned*>(&h);
         h = __floats2bfloat162_rn(v[j][4 % EPV], v[j][5 % EPV]); o.z = *reinterpret_cast<unsigned*>(&h);
         h = __floats2bfloat162_rn(v[j][6 % EPV], v[j][7 % EPV]); o.w = *reinterpret_cast<unsigned*>(&h);
-        for (int q = 0; q < p.n_dst; ++q) reinterpret_cast<uint4*>(p.dst[q])[at] = o;
+        for (int q = 0; q < p.n_dst; ++q)
+          if (SBP_GUARD(reinterpret_cast<uint4*>(p.dst[q]) + at, 16)) reinterpret_cast<uint4*>(p.dst[q])[at] = o;
       } else {
         const __nv_bfloat16 o = __float2bfloat16_rn(v[j][0]);
-        for (int q = 0; q < p.n_dst; ++q) p.dst[q][at] = o;
+        for (int q = 0; q < p.n_dst; ++q)
+          if (SBP_GUARD(p.dst[q] + at, 2)) p.dst[q][at] = o;
       }
     }
   }
@@ -333,6 +340,7 @@ static int pick_vector_bytes(const BoxParams& p, const sbp_tensor* src, const sb
 // the launch behaves like a plain one.
 template <typename V, int OP, int J, int KT>
 static void launch_tile(const Plan& pl, cudaStream_t st) {
+  SBP_BOUNDS_UPLOAD(st);
   launch_dependent(box_tile_kernel<V, OP, J, KT>, dim3((unsigned)pl.grid), dim3(256), 0, st, pl.p);   // errors are picked up by the caller's cudaGetLastError
 }
 
@@ -651,6 +659,10 @@ static sbp_status boxing_one_axis(const sbp_tensor* src, sbp_tensor* dst, int ds
   if (st != SBP_OK) return st;
   if (dry || numel(src) == 0) return SBP_OK;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  SBP_BOUNDS_RESET();
+  SBP_BOUNDS_TENSOR(src);
+  if (dst_shard >= 0) SBP_BOUNDS_SHARD(dst, dst_shard);
+  else SBP_BOUNDS_TENSOR(dst);
 
   bool done = false;
   if (src->dtype != dst->dtype) {   // S(i) -> B with the fp32 -> bf16 cast folded in
@@ -676,6 +688,7 @@ static sbp_status boxing_one_axis(const sbp_tensor* src, sbp_tensor* dst, int ds
     gp.n_dst = b.n_dst;
     for (int q = 0; q < b.n_dst; ++q) gp.dst[q] = reinterpret_cast<__nv_bfloat16*>(b.dst[q]);
     dim3 grid(148 * 4, (unsigned)b.k);
+    SBP_BOUNDS_UPLOAD(stream);
     if (vec) launch_dependent(box_gather_cast_kernel<8>, grid, dim3(256), 0, stream, gp);
     else launch_dependent(box_gather_cast_kernel<1>, grid, dim3(256), 0, stream, gp);
     done = true;

@@ -16,6 +16,7 @@
 //             ascending r; a destination that gets nothing is zero)
 #include <algorithm>
 
+#include "bounds_check.h"
 #include "boxing_arith.h"
 #include "sbp_internal.h"
 
@@ -139,7 +140,7 @@ __global__ void __launch_bounds__(256, OP == OP_COPY ? 4 : 3) box_disjoint_kerne
     const V* sp = reinterpret_cast<const V*>(p.src[s]);
 #pragma unroll
     for (int j = 0; j < J; ++j)
-      if (ok[j]) val[j] = ld_stream(sp + so[j]);
+      if (ok[j] && SBP_GUARD(sp + so[j], sizeof(V))) val[j] = ld_stream(sp + so[j]);
   } else {
     using L = typename Lanes<OP, V>::type;
     int first = 0, stride = 1, count = p.ks;
@@ -159,7 +160,8 @@ __global__ void __launch_bounds__(256, OP == OP_COPY ? 4 : 3) box_disjoint_kerne
       for (int j = 0; j < J; ++j)
 #pragma unroll
         for (int i = 0; i < kBatch; ++i)
-          if (ok[j] && base + i < count)
+          if (ok[j] && base + i < count &&
+              SBP_GUARD(reinterpret_cast<const V*>(p.src[first + (base + i) * stride]) + so[j], sizeof(V)))
             raw[j][i] = ld_stream(reinterpret_cast<const V*>(p.src[first + (base + i) * stride]) + so[j]);
 #pragma unroll
       for (int j = 0; j < J; ++j)
@@ -184,13 +186,13 @@ __global__ void __launch_bounds__(256, OP == OP_COPY ? 4 : 3) box_disjoint_kerne
       V* dp = reinterpret_cast<V*>(p.dst[r]);
 #pragma unroll
       for (int j = 0; j < J; ++j)
-        if (ok[j]) dp[dofs[j]] = val[j];
+        if (ok[j] && SBP_GUARD(dp + dofs[j], sizeof(V))) dp[dofs[j]] = val[j];
     }
   } else {
     V* dp = reinterpret_cast<V*>(p.dst[d]);
 #pragma unroll
     for (int j = 0; j < J; ++j)
-      if (ok[j]) dp[dofs[j]] = val[j];
+      if (ok[j] && SBP_GUARD(dp + dofs[j], sizeof(V))) dp[dofs[j]] = val[j];
   }
 }
 
@@ -208,11 +210,13 @@ __global__ void __launch_bounds__(256) box_zero_kernel(const __grid_constant__ Z
   uint4* d = reinterpret_cast<uint4*>(z.dst[blockIdx.y]);
   const long long n = z.bytes / 16;
   const uint4 zero = make_uint4(0u, 0u, 0u, 0u);
-  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) d[i] = zero;
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256)
+    if (SBP_GUARD(d + i, 16)) d[i] = zero;
 }
 
 template <int OP>
 static void launch_disjoint(const DisjointParams& p, int vbytes, long long grid, cudaStream_t st) {
+  SBP_BOUNDS_UPLOAD(st);
   const dim3 g((unsigned)grid), b(256);
   switch (vbytes) {
     case 16: launch_dependent(box_disjoint_kernel<uint4, OP>, g, b, 0, st, p); break;
@@ -389,6 +393,10 @@ sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard
   const long long grid = p.tiles_per_task * p.ntasks;
   if (copy_needed && grid > 0x7fffffffLL) return fail(SBP_ERR_UNSUPPORTED, "tensor too large for one launch");
   if (dry) return SBP_OK;   // every refusal lies above this line, every launch below it
+  SBP_BOUNDS_RESET();
+  SBP_BOUNDS_TENSOR(src);
+  if (dst_shard >= 0) SBP_BOUNDS_SHARD(dst, dst_shard);
+  else SBP_BOUNDS_TENSOR(dst);
 
 
   if (zero_first) {
@@ -407,6 +415,7 @@ sbp_status boxing_disjoint(const sbp_tensor* src, sbp_tensor* dst, int dst_shard
       if (vec_ok) {
         long long zb = (z.bytes / 16 + 256 * 8 - 1) / (256 * 8);
         if (zb > 148 * 16) zb = 148 * 16;
+        SBP_BOUNDS_UPLOAD(stream);
         launch_dependent(box_zero_kernel, dim3((unsigned)zb, (unsigned)z.n), dim3(256), 0, stream, z);
         cudaError_t ze = cudaGetLastError();
         if (ze != cudaSuccess) return cuda_fail(ze, "zero fill launch");

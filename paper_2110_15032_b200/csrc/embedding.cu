@@ -11,6 +11,7 @@
 // lookups; all id loads, then all row loads, are issued before the first store.
 #include <cuda_bf16.h>
 
+#include "bounds_check.h"
 #include "sbp_internal.h"
 
 namespace sbp {
@@ -123,7 +124,7 @@ __global__ void __launch_bounds__(256, MINB) embedding_kernel(const __grid_const
     split_item(item[j], p.vpr, p.vpr_log2, &look[j], &col[j]);
   }
 #pragma unroll
-  for (int j = 0; j < J; ++j) id[j] = ok[j] ? __ldg(p.ids[shard] + look[j]) : 0;
+  for (int j = 0; j < J; ++j) id[j] = (ok[j] && SBP_GUARD(p.ids[shard] + look[j], 8)) ? __ldg(p.ids[shard] + look[j]) : -1;
 
   V val[J];
 #pragma unroll
@@ -133,13 +134,14 @@ __global__ void __launch_bounds__(256, MINB) embedding_kernel(const __grid_const
     if (!ok[j]) continue;
     const bool in_table = id[j] >= 0 && id[j] < p.rows;
     if (!in_table) {
-      if (p.oob && col[j] == 0 && shard == 0) atomicAdd(p.oob, 1);
+      if (p.oob && col[j] == 0 && shard == 0 && SBP_GUARD(p.oob, 4)) atomicAdd(p.oob, 1);
       continue;
     }
     long long start;
     const int r = owner_of_row(id[j], p.base, p.rem, p.big, p.narrow, &start);
     own[j] = r;
-    val[j] = __ldg(reinterpret_cast<const V*>(p.table[r]) + (id[j] - start) * p.vpr + col[j]);
+    const V* src = reinterpret_cast<const V*>(p.table[r]) + (id[j] - start) * p.vpr + col[j];
+    if (SBP_GUARD(src, sizeof(V))) val[j] = __ldg(src);
   }
 
   if (FUSED) {
@@ -147,14 +149,14 @@ __global__ void __launch_bounds__(256, MINB) embedding_kernel(const __grid_const
       V* o = reinterpret_cast<V*>(p.out[q]);
 #pragma unroll
       for (int j = 0; j < J; ++j)
-        if (ok[j]) o[item[j]] = p.canon_neg_zero ? canon<V, ESZ>(val[j]) : val[j];
+        if (ok[j] && SBP_GUARD(o + item[j], sizeof(V))) o[item[j]] = p.canon_neg_zero ? canon<V, ESZ>(val[j]) : val[j];
     }
   } else {
     for (int q = 0; q < p.k; ++q) {
       V* o = reinterpret_cast<V*>(p.out[q]);
 #pragma unroll
       for (int j = 0; j < J; ++j)
-        if (ok[j]) o[item[j]] = own[j] == q ? val[j] : zero_vec<V>();
+        if (ok[j] && SBP_GUARD(o + item[j], sizeof(V))) o[item[j]] = own[j] == q ? val[j] : zero_vec<V>();
     }
   }
 }
@@ -192,7 +194,8 @@ __global__ void __launch_bounds__(256) embedding_rows_kernel(const __grid_consta
     long long look0;
     int n_ids;
     span(chunk, &look0, &n_ids);
-    if ((int)threadIdx.x < n_ids) ids_s[0][threadIdx.x] = __ldcs(p.ids[0] + look0 + threadIdx.x);
+    if ((int)threadIdx.x < n_ids)
+      ids_s[0][threadIdx.x] = SBP_GUARD(p.ids[0] + look0 + threadIdx.x, 8) ? __ldcs(p.ids[0] + look0 + threadIdx.x) : -1;
   }
   __syncthreads();
 
@@ -207,7 +210,7 @@ __global__ void __launch_bounds__(256) embedding_rows_kernel(const __grid_consta
     int nn = 0;
     if (next < n_chunks) {
       span(next, &nlook0, &nn);
-      if ((int)threadIdx.x < nn) nid = __ldcs(p.ids[0] + nlook0 + threadIdx.x);
+      if ((int)threadIdx.x < nn && SBP_GUARD(p.ids[0] + nlook0 + threadIdx.x, 8)) nid = __ldcs(p.ids[0] + nlook0 + threadIdx.x);
     }
 
     V val[J];
@@ -221,17 +224,19 @@ __global__ void __launch_bounds__(256) embedding_rows_kernel(const __grid_consta
       const long long look = item >> p.vpr_log2, col = item & (p.vpr - 1);
       const long long id = ids_s[cur][look - look0];
       if (id < 0 || id >= p.rows) {
-        if (p.oob && col == 0) atomicAdd(p.oob, 1);
+        if (p.oob && col == 0 && SBP_GUARD(p.oob, 4)) atomicAdd(p.oob, 1);
         continue;
       }
       long long start;
       const int r = owner_of_row(id, p.base, p.rem, p.big, p.narrow, &start);
-      val[j] = __ldg(reinterpret_cast<const V*>(p.table[r]) + (id - start) * p.vpr + col);
+      const V* src = reinterpret_cast<const V*>(p.table[r]) + (id - start) * p.vpr + col;
+      if (SBP_GUARD(src, sizeof(V))) val[j] = __ldg(src);
     }
     V* o = reinterpret_cast<V*>(p.out[0]);
 #pragma unroll
     for (int j = 0; j < J; ++j)
-      if (ok[j]) __stcs(o + cta_base + j * 256 + threadIdx.x, p.canon_neg_zero ? canon<V, ESZ>(val[j]) : val[j]);
+      if (ok[j] && SBP_GUARD(o + cta_base + j * 256 + threadIdx.x, sizeof(V)))
+        __stcs(o + cta_base + j * 256 + threadIdx.x, p.canon_neg_zero ? canon<V, ESZ>(val[j]) : val[j]);
 
     if ((int)threadIdx.x < nn) ids_s[cur ^ 1][threadIdx.x] = nid;
     __syncthreads();
@@ -248,6 +253,7 @@ __global__ void __launch_bounds__(256) embedding_rows_kernel(const __grid_consta
 template <typename V, int ESZ>
 static void launch_emb(const EmbParams& p, bool fused, cudaStream_t st) {
   const long long total = p.n_lookups * p.vpr;
+  SBP_BOUNDS_UPLOAD(st);
   auto blocks_for = [&](int j) {
     long long b = (total + 256LL * j - 1) / (256LL * j);
     return (unsigned)(b < 1 ? 1 : b);
@@ -309,32 +315,35 @@ __global__ void __launch_bounds__(256) embedding_s1_kernel(const __grid_constant
     shard[j] = r;
   }
 #pragma unroll
-  for (int j = 0; j < J; ++j) id[j] = ok[j] ? __ldg(p.ids[FUSED ? 0 : shard[j]] + look[j]) : 0;
+  for (int j = 0; j < J; ++j)
+    id[j] = (ok[j] && SBP_GUARD(p.ids[FUSED ? 0 : shard[j]] + look[j], 8)) ? __ldg(p.ids[FUSED ? 0 : shard[j]] + look[j]) : -1;
   V val[J];
 #pragma unroll
   for (int j = 0; j < J; ++j) {
     val[j] = zero_vec<V>();
     if (!ok[j]) continue;
     if (id[j] < 0 || id[j] >= p.rows) {
-      if (p.oob && col[j] == 0) atomicAdd(p.oob, 1);
+      if (p.oob && col[j] == 0 && SBP_GUARD(p.oob, 4)) atomicAdd(p.oob, 1);
       continue;
     }
     const long long w = p.vstart[shard[j] + 1] - p.vstart[shard[j]];
-    val[j] = __ldg(reinterpret_cast<const V*>(p.table[shard[j]]) + id[j] * w + (col[j] - p.vstart[shard[j]]));
+    const V* src = reinterpret_cast<const V*>(p.table[shard[j]]) + id[j] * w + (col[j] - p.vstart[shard[j]]);
+    if (SBP_GUARD(src, sizeof(V))) val[j] = __ldg(src);
   }
   if (FUSED) {
     for (int q = 0; q < p.n_dst; ++q) {
       V* o = reinterpret_cast<V*>(p.out[q]);
 #pragma unroll
       for (int j = 0; j < J; ++j)
-        if (ok[j]) o[item[j]] = val[j];
+        if (ok[j] && SBP_GUARD(o + item[j], sizeof(V))) o[item[j]] = val[j];
     }
   } else {
 #pragma unroll
     for (int j = 0; j < J; ++j) {
       if (!ok[j]) continue;
       const long long w = p.vstart[shard[j] + 1] - p.vstart[shard[j]];
-      reinterpret_cast<V*>(p.out[shard[j]])[look[j] * w + (col[j] - p.vstart[shard[j]])] = val[j];
+      V* dstp = reinterpret_cast<V*>(p.out[shard[j]]) + look[j] * w + (col[j] - p.vstart[shard[j]]);
+      if (SBP_GUARD(dstp, sizeof(V))) *dstp = val[j];
     }
   }
 }
@@ -345,6 +354,7 @@ static void launch_emb_s1(const EmbS1Params& p, bool fused, cudaStream_t st) {
   const long long total = p.n_lookups * p.vpr_total;
   long long blocks = (total + 256LL * J - 1) / (256LL * J);
   if (blocks < 1) blocks = 1;
+  SBP_BOUNDS_UPLOAD(st);
   if (fused) embedding_s1_kernel<V, J, true><<<(unsigned)blocks, 256, 0, st>>>(p);
   else embedding_s1_kernel<V, J, false><<<(unsigned)blocks, 256, 0, st>>>(p);
 }
@@ -434,7 +444,8 @@ __global__ void __launch_bounds__(256) embedding_zero_kernel(const __grid_consta
   float4* g = reinterpret_cast<float4*>(p.grad_table[blockIdx.y]);
   const long long n = p.shard_vecs[blockIdx.y];
   const float4 z = make_float4(0.f, 0.f, 0.f, 0.f);
-  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256) g[i] = z;
+  for (long long i = (long long)blockIdx.x * 256 + threadIdx.x; i < n; i += (long long)gridDim.x * 256)
+    if (SBP_GUARD(g + i, 16)) g[i] = z;
 }
 
 // CHUNK lookups per CTA pass (256 or 1024); key = id * CHUNK + position in the chunk, all ones
@@ -454,9 +465,9 @@ __global__ void __launch_bounds__(256, 3) embedding_backward_kernel(const __grid
     for (int i = tid; i < CHUNK; i += 256) {
       unsigned long long kv = kNone;
       if (first + i < p.n_lookups) {
-        const long long id = __ldg(p.ids + first + i);
+        const long long id = SBP_GUARD(p.ids + first + i, 8) ? __ldg(p.ids + first + i) : -1;
         if (id >= 0 && id < p.rows) kv = ((unsigned long long)id << kShift) | (unsigned)i;
-        else if (p.oob) atomicAdd(p.oob, 1);
+        else if (p.oob && SBP_GUARD(p.oob, 4)) atomicAdd(p.oob, 1);
       }
       key[i] = kv;
     }
@@ -483,7 +494,8 @@ __global__ void __launch_bounds__(256, 3) embedding_backward_kernel(const __grid
         if (cur >= 0 && active) {
           long long start;
           const int r = owner_of_row(cur, p.base, p.rem, p.big, p.narrow, &start);
-          atomicAdd(reinterpret_cast<float4*>(p.grad_table[r]) + (cur - start) * p.vpr + col, acc);
+          float4* at = reinterpret_cast<float4*>(p.grad_table[r]) + (cur - start) * p.vpr + col;
+          if (SBP_GUARD(at, 16)) atomicAdd(at, acc);
         }
       };
       for (int pos = warp * kPerWarp; pos < (warp + 1) * kPerWarp; pos += kBatch) {
@@ -493,7 +505,8 @@ __global__ void __launch_bounds__(256, 3) embedding_backward_kernel(const __grid
         for (int j = 0; j < kBatch; ++j) {
           kv[j] = key[pos + j];
           gv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-          if (kv[j] != kNone && active) gv[j] = __ldg(gout + (first + (long long)(kv[j] & (CHUNK - 1))) * p.vpr + col);
+          if (kv[j] != kNone && active && SBP_GUARD(gout + (first + (long long)(kv[j] & (CHUNK - 1))) * p.vpr + col, 16))
+            gv[j] = __ldg(gout + (first + (long long)(kv[j] & (CHUNK - 1))) * p.vpr + col);
         }
 #pragma unroll
         for (int j = 0; j < kBatch; ++j) {
@@ -543,6 +556,11 @@ extern "C" sbp_status sbp_embedding(const sbp_tensor* table, const sbp_tensor* i
   if (placement_k(ids) != k || placement_k(out) != k) return fail(SBP_ERR_INVALID_ARG, "operands differ in k");
   if (table->sbp[0].kind != SBP_SPLIT) return fail(SBP_ERR_SIGNATURE, "table must be S(0) or S(1)");
   if (ids->sbp[0].kind != SBP_BROADCAST) return fail(SBP_ERR_SIGNATURE, "ids must be B");
+  SBP_BOUNDS_RESET();
+  SBP_BOUNDS_TENSOR(table);
+  SBP_BOUNDS_TENSOR(ids);
+  SBP_BOUNDS_TENSOR(out);
+  SBP_BOUNDS_ADD(oob_count, 4);
   if (table->sbp[0].axis == 1)
     return embedding_hidden_split(table, ids, out, oob_count, static_cast<cudaStream_t>(cuda_stream));
   const bool fused = out->sbp[0].kind == SBP_BROADCAST;
@@ -636,6 +654,11 @@ extern "C" sbp_status sbp_embedding_backward(const sbp_tensor* grad_out, const s
       return fail(SBP_ERR_ALIGNMENT, "grad_table shards must be 16-byte aligned");
   if (reinterpret_cast<uintptr_t>(grad_out->local[0]) % 16 != 0) return fail(SBP_ERR_ALIGNMENT, "grad_out must be 16-byte aligned");
   if (dim == 0 || grad_table->shape[0] == 0) return SBP_OK;
+  SBP_BOUNDS_RESET();
+  SBP_BOUNDS_TENSOR(grad_out);
+  SBP_BOUNDS_TENSOR(ids);
+  SBP_BOUNDS_TENSOR(grad_table);
+  SBP_BOUNDS_ADD(oob_count, 4);
 
   EmbBwdParams p{};
   p.k = k;
@@ -659,6 +682,7 @@ extern "C" sbp_status sbp_embedding_backward(const sbp_tensor* grad_out, const s
   long long zb = (max_vecs + 256 * 8 - 1) / (256 * 8);
   if (zb < 1) zb = 1;
   if (zb > 148 * 16) zb = 148 * 16;
+  SBP_BOUNDS_UPLOAD(stream);
   embedding_zero_kernel<<<dim3((unsigned)zb, (unsigned)k), 256, 0, stream>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e, "embedding backward launch");

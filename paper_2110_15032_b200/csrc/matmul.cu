@@ -7,6 +7,7 @@
 //     core kernel cannot take), fp32 accumulation with fused multiply-adds, k ascending.
 #include <cuda_bf16.h>
 
+#include "bounds_check.h"
 #include "matmul_plan.h"
 #include "sbp_internal.h"
 
@@ -70,23 +71,23 @@ __global__ void __launch_bounds__(256) matmul_fma_kernel(const __grid_constant__
       if (p.a_trans) {
         for (int e = threadIdx.x; e < BM * BK; e += 256) {
           const int c = e / BM, r = e % BM;   // consecutive threads walk the stored rows
-          As[c][r] = (m0 + r < M && k0 + c < K) ? ld_f32<TI>(A + r * a_rs + (k0 + c) * a_ks) : 0.f;
+          As[c][r] = (m0 + r < M && k0 + c < K && SBP_GUARD(A + r * a_rs + (k0 + c) * a_ks, sizeof(TI))) ? ld_f32<TI>(A + r * a_rs + (k0 + c) * a_ks) : 0.f;
         }
       } else {
         for (int e = threadIdx.x; e < BM * BK; e += 256) {
           const int r = e / BK, c = e % BK;
-          As[c][r] = (m0 + r < M && k0 + c < K) ? ld_f32<TI>(A + r * a_rs + (k0 + c) * a_ks) : 0.f;
+          As[c][r] = (m0 + r < M && k0 + c < K && SBP_GUARD(A + r * a_rs + (k0 + c) * a_ks, sizeof(TI))) ? ld_f32<TI>(A + r * a_rs + (k0 + c) * a_ks) : 0.f;
         }
       }
       if (p.b_trans) {
         for (int e = threadIdx.x; e < BK * BN; e += 256) {
           const int c = e / BK, r = e % BK;
-          Bs[r][c] = (k0 + r < K && n0 + c < N) ? ld_f32<TI>(Bm + (k0 + r) * b_ks + c * b_cs) : 0.f;
+          Bs[r][c] = (k0 + r < K && n0 + c < N && SBP_GUARD(Bm + (k0 + r) * b_ks + c * b_cs, sizeof(TI))) ? ld_f32<TI>(Bm + (k0 + r) * b_ks + c * b_cs) : 0.f;
         }
       } else {
         for (int e = threadIdx.x; e < BK * BN; e += 256) {
           const int r = e / BN, c = e % BN;
-          Bs[r][c] = (k0 + r < K && n0 + c < N) ? ld_f32<TI>(Bm + (k0 + r) * b_ks + c * b_cs) : 0.f;
+          Bs[r][c] = (k0 + r < K && n0 + c < N && SBP_GUARD(Bm + (k0 + r) * b_ks + c * b_cs, sizeof(TI))) ? ld_f32<TI>(Bm + (k0 + r) * b_ks + c * b_cs) : 0.f;
         }
       }
       __syncthreads();
@@ -115,9 +116,10 @@ __global__ void __launch_bounds__(256) matmul_fma_kernel(const __grid_constant__
       if (c >= N) continue;
       float v = acc[i][j];
       if (p.gelu) v = gelu_erf(v);
-      st_out<TO>(static_cast<TO*>(p.y[g]) + r * p.ldy[g] + c, v);
+      if (SBP_GUARD(static_cast<TO*>(p.y[g]) + r * p.ldy[g] + c, sizeof(TO))) st_out<TO>(static_cast<TO*>(p.y[g]) + r * p.ldy[g] + c, v);
       if (g == 0)
-        for (int q = 0; q < p.n_rep; ++q) st_out<TO>(static_cast<TO*>(p.y_rep[q]) + r * p.ldy[g] + c, v);
+        for (int q = 0; q < p.n_rep; ++q)
+          if (SBP_GUARD(static_cast<TO*>(p.y_rep[q]) + r * p.ldy[g] + c, sizeof(TO))) st_out<TO>(static_cast<TO*>(p.y_rep[q]) + r * p.ldy[g] + c, v);
     }
   }
 }
@@ -132,6 +134,7 @@ static sbp_status launch_fma(const MatmulPlan& p, cudaStream_t st) {
   const long long gx = (nmax + BN - 1) / BN, gy = (mmax + BM - 1) / BM;
   if (gx > 0x7fffffffLL || gy > 65535) return fail(SBP_ERR_UNSUPPORTED, "matrix too large for the FMA kernel");
   dim3 grid((unsigned)gx, (unsigned)gy, (unsigned)p.ngroups);
+  SBP_BOUNDS_UPLOAD(st);
   if (p.in_dtype == SBP_F32 && p.out_dtype == SBP_F32)
     matmul_fma_kernel<float, float><<<grid, 256, 0, st>>>(p);
   else if (p.in_dtype == SBP_BF16 && p.out_dtype == SBP_BF16)
@@ -177,13 +180,13 @@ __global__ void __launch_bounds__(256) matmul_pack_kernel(const __grid_constant_
     const unsigned short* sp = B.src + row * B.src_ld + g8 * 8;
     unsigned short v[8];
 #pragma unroll
-    for (int e = 0; e < 8; ++e) v[e] = (g8 * 8 + e < B.cols) ? __ldg(sp + e) : (unsigned short)0;
+    for (int e = 0; e < 8; ++e) v[e] = (g8 * 8 + e < B.cols && SBP_GUARD(sp + e, 2)) ? __ldg(sp + e) : (unsigned short)0;
     uint4 o;
     o.x = v[0] | ((unsigned)v[1] << 16);
     o.y = v[2] | ((unsigned)v[3] << 16);
     o.z = v[4] | ((unsigned)v[5] << 16);
     o.w = v[6] | ((unsigned)v[7] << 16);
-    *reinterpret_cast<uint4*>(B.dst + row * B.dst_ld + g8 * 8) = o;
+    if (SBP_GUARD(B.dst + row * B.dst_ld + g8 * 8, 16)) *reinterpret_cast<uint4*>(B.dst + row * B.dst_ld + g8 * 8) = o;
   }
 }
 
@@ -246,6 +249,7 @@ static sbp_status pack_operands(MatmulPlan* plan, const PackNeed& need, void* ws
     long long gx = (most + 255) / 256;
     if (gx < 1) gx = 1;
     if (gx > 148 * 8) gx = 148 * 8;
+    SBP_BOUNDS_UPLOAD(st);
     matmul_pack_kernel<<<dim3((unsigned)gx, (unsigned)nb), 256, 0, st>>>(list);
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return cuda_fail(e, "operand repack launch");
@@ -547,6 +551,11 @@ sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, u
   sbp_status st = two_axes ? build_plan_2d(x, w, y, flags, true, &plan) : build_plan(x, w, y, flags, true, &plan);
   if (st != SBP_OK) return st;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  SBP_BOUNDS_RESET();
+  SBP_BOUNDS_TENSOR(x);
+  SBP_BOUNDS_TENSOR(w);
+  SBP_BOUNDS_TENSOR(y);
+  SBP_BOUNDS_ADD(ws, ws_bytes);
   bool taken = false;
   st = launch_matmul_tc(plan, nullptr, stream, &taken);
   if (taken) return st;
@@ -647,6 +656,14 @@ sbp_status sbp_matmul_softmax_xent(const sbp_tensor* features, const sbp_tensor*
   xf.labels = static_cast<const long long*>(labels->local[0]);
   xf.rows = rows;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  SBP_BOUNDS_RESET();
+  SBP_BOUNDS_TENSOR(features);
+  SBP_BOUNDS_TENSOR(weight);
+  SBP_BOUNDS_TENSOR(labels);
+  SBP_BOUNDS_TENSOR(loss);
+  SBP_BOUNDS_TENSOR(row_max);
+  SBP_BOUNDS_TENSOR(row_sum);
+  SBP_BOUNDS_ADD(ws, need);
   bool taken = false;
   st = launch_matmul_tc(plan, &xf, stream, &taken);
   if (!taken)
@@ -709,6 +726,13 @@ sbp_status sbp_matmul_softmax_xent_backward(const sbp_tensor* features, const sb
   xf.row_max = static_cast<const float*>(row_max->local[0]);
   xf.row_sum = static_cast<const float*>(row_sum->local[0]);
   xf.rows = rows;
+  SBP_BOUNDS_RESET();
+  SBP_BOUNDS_TENSOR(features);
+  SBP_BOUNDS_TENSOR(weight);
+  SBP_BOUNDS_TENSOR(labels);
+  SBP_BOUNDS_TENSOR(row_max);
+  SBP_BOUNDS_TENSOR(row_sum);
+  SBP_BOUNDS_TENSOR(grad_logits);
   bool taken = false;
   st = launch_matmul_tc(plan, &xf, static_cast<cudaStream_t>(cuda_stream), &taken);
   if (!taken)

@@ -22,7 +22,9 @@
 // A fused "P(sum) product written as B / S(i)" plan simply chains the K-blocks of all shards'
 // operands, in rank order, into the same accumulator: the partial products are never stored.
 //
-// Every wait is bounded in time.  A wait that expires raises a flag that
+// Every barrier wait is bounded in time (the one wait that is not is the allocation of tensor memory
+// at the start, which cannot block: the shared-memory footprint keeps the kernel to one CTA per SM,
+// so the CTA is alone on its SM's tensor memory).  A wait that expires raises a flag that
 // sbp_check_device_errors() reports; the CTA then stops issuing work, waits (bounded) for the
 // loads it still has in flight, meets its partner at the closing cluster barrier, frees its
 // tensor memory and returns.
@@ -34,6 +36,7 @@
 #include <mutex>
 #include <type_traits>
 
+#include "bounds_check.h"
 #include "matmul_plan.h"
 #include "sbp_internal.h"
 
@@ -246,9 +249,10 @@ struct TileCoord {
   int g, m0, n0;
 };
 
-// Tiles of a group are walked in panels of kPanelM m-tiles, n fastest across the panel, so that
-// the CTA pairs running at the same time cover a roughly square patch of the output and share
-// both their A rows and their B columns in L2.
+// Tiles of a group are walked in panels of kPanelM m-tiles: inside a panel the m-tile index varies
+// fastest and the n-tile index steps once per column of the panel, so that the CTA pairs running at
+// the same time cover a roughly square patch of the output and share both their A rows and their B
+// columns in L2.
 constexpr int kPanelM = 8;
 
 __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
@@ -436,7 +440,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
         if (row0 < Mg && colbase < Ng) {            // warp-uniform
           float m = -INFINITY, s = 0.f, t = 0.f;
           long long want = -1;
-          if (row < Mg) want = p.xf.labels[row] - p.xf.class_start[tc.g] - colbase;
+          if (row < Mg && SBP_GUARD(p.xf.labels + row, 8)) want = p.xf.labels[row] - p.xf.class_start[tc.g] - colbase;
           for (int b = 0; b < 4; ++b) {
             const int c0 = colbase + b * 32;
             if (c0 >= Ng) break;                      // warp-uniform
@@ -487,9 +491,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
           }
           if (row < Mg) {
             const long long slot = (long long)(p.xf.part_base[tc.g] + colbase / 128) * p.xf.rows + row;
-            p.xf.part_m[slot] = m;
-            p.xf.part_s[slot] = s;
-            p.xf.part_t[slot] = t;
+            if (SBP_GUARD(p.xf.part_m + slot, 4)) p.xf.part_m[slot] = m;
+            if (SBP_GUARD(p.xf.part_s + slot, 4)) p.xf.part_s[slot] = s;
+            if (SBP_GUARD(p.xf.part_t + slot, 4)) p.xf.part_t[slot] = t;
           }
         }
       } else {
@@ -499,7 +503,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
       // softmax = 2^(z log2e - m log2e - log2 S): the division by the row sum is folded into the exponent
       float g_neg = 0.f;
       long long g_lab = -1;
-      if (p.xent == 2 && row0 + lane < Mg) {      // this thread's row constants
+      if (p.xent == 2 && row0 + lane < Mg && SBP_GUARD(p.xf.row_max + row0 + lane, 4) &&
+          SBP_GUARD(p.xf.row_sum + row0 + lane, 4) && SBP_GUARD(p.xf.labels + row0 + lane, 8)) {      // this thread's row constants
         const long long row = row0 + lane;
         g_neg = -p.xf.row_max[row] * 1.4426950408889634f - log2f(p.xf.row_sum[row]);
         g_lab = p.xf.labels[row] - p.xf.class_start[tc.g];
@@ -566,14 +571,14 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
                   const unsigned char* srow = buf + r * 128;
                   if (p.out_f32) {
                     const int c = lane;
-                    if (col0 + c < Ng)
+                    if (col0 + c < Ng && SBP_GUARD(reinterpret_cast<float*>(yb) + (row0 + r) * ld + col0 + c, 4))
                       reinterpret_cast<float*>(yb)[(row0 + r) * ld + col0 + c] =
                           *reinterpret_cast<const float*>(srow + ((((c >> 2) ^ (r & 7)) << 4) | ((c & 3) << 2)));
                   } else {
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
                       const int c = lane + 32 * h;
-                      if (col0 + c < Ng)
+                      if (col0 + c < Ng && SBP_GUARD(reinterpret_cast<unsigned short*>(yb) + (row0 + r) * ld + col0 + c, 2))
                         reinterpret_cast<unsigned short*>(yb)[(row0 + r) * ld + col0 + c] =
                             *reinterpret_cast<const unsigned short*>(srow + ((((c >> 3) ^ (r & 7)) << 4) | ((c & 7) << 1)));
                     }
@@ -736,6 +741,7 @@ static sbp_status launch_tc_form(const TcParams& p, int tiles, cudaStream_t st) 
   }
   const int max_pairs = pairs_on_device[dev];
   const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  SBP_BOUNDS_UPLOAD(st);
   matmul_tc_kernel<AT, BT><<<2 * pairs, kThreadsTc, kSmemBytes, st>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e, "tensor-core matmul launch");

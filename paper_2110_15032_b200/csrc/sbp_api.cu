@@ -2,9 +2,55 @@
 #include <atomic>
 #include <cstring>
 
+#include "bounds_check.h"
 #include "sbp_internal.h"
 
 namespace sbp {
+
+#ifdef SBP_DEBUG_BOUNDS
+static thread_local BoundsTable g_bounds_host;
+static BoundsPollFn g_bounds_polls[16];
+static int g_bounds_npolls = 0;
+
+void bounds_reset() { g_bounds_host.n = 0; }
+
+void bounds_add(const void* p, size_t bytes) {
+  if (!p || bytes == 0) return;
+  BoundsTable& t = g_bounds_host;
+  const unsigned long long lo = reinterpret_cast<uintptr_t>(p), hi = lo + bytes;
+  for (int i = 0; i < t.n; ++i)
+    if (t.lo[i] == lo && t.hi[i] >= hi) return;
+  if (t.n < kBoundsMax) {
+    t.lo[t.n] = lo;
+    t.hi[t.n] = hi;
+    ++t.n;
+  }
+}
+
+void bounds_add_tensor_shard(const sbp_tensor* t, int r) {
+  if (!t || !t->local[r]) return;
+  int64_t shp[SBP_MAX_DIMS];
+  local_shape_nd(t, r, shp);
+  int64_t rows = 1;
+  for (int d = 0; d + 1 < t->ndim; ++d) rows *= shp[d];
+  const int64_t cols = shp[t->ndim - 1];
+  if (rows == 0 || cols == 0) return;
+  const int64_t elems = (rows - 1) * local_pitch(t, r) + cols;   // the last row ends where its data ends
+  bounds_add(t->local[r], (size_t)elems * elem_size(t->dtype));
+}
+
+void bounds_add_tensor(const sbp_tensor* t) {
+  if (!t) return;
+  const int k = placement_k(t);
+  for (int r = 0; r < k && r < SBP_MAX_K; ++r) bounds_add_tensor_shard(t, r);
+}
+
+const BoundsTable& bounds_current() { return g_bounds_host; }
+
+void bounds_register_poll(BoundsPollFn fn) {
+  if (g_bounds_npolls < 16) g_bounds_polls[g_bounds_npolls++] = fn;
+}
+#endif
 
 static thread_local char g_err[512] = "";
 static std::atomic<uint64_t> g_launches{0};
@@ -121,6 +167,15 @@ sbp_status refuse_ld(const sbp_tensor* t, const char* name, const char* entry) {
   return SBP_OK;
 }
 
+#ifdef SBP_DEBUG_BOUNDS
+// Self-test of the debug-bounds report path: asks the checker about the byte just past a registered
+// buffer.  The check fails, so the store below it is skipped: nothing outside the buffer is touched.
+__global__ void bounds_selftest_kernel(unsigned char* buf, size_t bytes) {
+  if (SBP_GUARD(buf, 1)) buf[0] = 1;                 // inside: performed
+  if (SBP_GUARD(buf + bytes, 1)) buf[bytes] = 1;     // one past the end: refused and recorded
+}
+#endif
+
 // Defined next to the kernels that own the flags.
 sbp_status read_and_clear_bulk_timeout(bool* timed_out);
 sbp_status read_and_clear_tc_timeout(bool* timed_out);
@@ -144,11 +199,20 @@ const char* sbp_status_string(sbp_status s) {
     case SBP_ERR_WORKSPACE: return "SBP_ERR_WORKSPACE";
     case SBP_ERR_CUDA: return "SBP_ERR_CUDA";
     case SBP_ERR_TIMEOUT: return "SBP_ERR_TIMEOUT";
+    case SBP_ERR_BOUNDS: return "SBP_ERR_BOUNDS";
   }
   return "SBP_ERR_?";
 }
 
 const char* sbp_last_error(void) { return g_err; }
+
+int32_t sbp_debug_bounds_enabled(void) {
+#ifdef SBP_DEBUG_BOUNDS
+  return 1;
+#else
+  return 0;
+#endif
+}
 
 uint64_t sbp_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
@@ -158,9 +222,35 @@ sbp_status sbp_check_device_errors(void) {
   if (st != SBP_OK) return st;
   st = read_and_clear_tc_timeout(&tc);
   if (st != SBP_OK) return st;
+#ifdef SBP_DEBUG_BOUNDS
+  if (cudaDeviceSynchronize() != cudaSuccess) return fail(SBP_ERR_CUDA, "device synchronisation failed");
+  for (int i = 0; i < g_bounds_npolls; ++i) {
+    unsigned long long addr = 0;
+    if (g_bounds_polls[i](&addr))
+      return fail(SBP_ERR_BOUNDS, "a kernel computed the address 0x%llx, which lies in none of its call's buffers; the access was skipped", addr);
+  }
+#endif
   if (bulk) return fail(SBP_ERR_TIMEOUT, "a bulk-copy boxing kernel gave up waiting for its loads");
   if (tc) return fail(SBP_ERR_TIMEOUT, "the tensor-core matmul kernel gave up waiting on one of its barriers");
   return SBP_OK;
+}
+
+sbp_status sbp_selftest_debug_bounds(void* buf, size_t bytes, void* cuda_stream) {
+#ifdef SBP_DEBUG_BOUNDS
+  if (!buf || bytes == 0) return fail(SBP_ERR_INVALID_ARG, "a device buffer of at least one byte is needed");
+  cudaStream_t st = static_cast<cudaStream_t>(cuda_stream);
+  SBP_BOUNDS_RESET();
+  SBP_BOUNDS_ADD(buf, bytes);
+  SBP_BOUNDS_UPLOAD(st);
+  bounds_selftest_kernel<<<1, 1, 0, st>>>(static_cast<unsigned char*>(buf), bytes);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return cuda_fail(e, "bounds self-test launch");
+  count_launch();
+  return SBP_OK;
+#else
+  (void)buf; (void)bytes; (void)cuda_stream;
+  return fail(SBP_ERR_UNSUPPORTED, "this is not the debug-bounds build of the library");
+#endif
 }
 
 sbp_status sbp_selftest_wait_timeout(uint32_t limit_ms, void* cuda_stream) {

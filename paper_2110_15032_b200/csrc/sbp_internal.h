@@ -77,6 +77,14 @@ sbp_status cuda_fail(cudaError_t e, const char* what);
 // kernel releases its dependents early (SBP_PDL_RELEASE), this one's CTAs may be set up while its
 // last CTAs still run.  Such a kernel must execute SBP_PDL_WAIT before its first access to
 // global memory; after any other kind of work the launch behaves like a plain one.
+// Invariant the dependents rely on: several of them read their sources through the non-coherent
+// path (ld.global.nc / __ldg), which is only sound for data that no thread of the SAME grid writes
+// and that is complete before the grid's first read.  Both hold because every read comes after
+// SBP_PDL_WAIT (the producer grid has finished and its writes are visible) and because no kernel
+// of this library that releases its dependents early reads the buffers it writes.  A kernel that
+// reads and then writes one buffer must use plain loads.  tests/test_boxing_gpu.py
+// (test_ping_pong_between_two_buffers_without_a_host_sync) rewrites a source between two reads of
+// it with no synchronisation in between.
 template <typename... KArgs, typename... Args>
 inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
                                     Args&&... args) {

@@ -21,6 +21,7 @@
 
 #include <mutex>
 
+#include "bounds_check.h"
 #include "sbp_internal.h"
 
 namespace sbp {
@@ -83,7 +84,7 @@ struct ChunkBF16x8 {
 #pragma unroll
     for (int u = 0; u < kLoadsPerThread; ++u) {
       const long long e0 = ((long long)u * kThreads + tid) * VEC;
-      if (e0 < n) {
+      if (e0 < n && SBP_GUARD(z + e0, 16)) {
         asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
                      : "=r"(raw[u].x), "=r"(raw[u].y), "=r"(raw[u].z), "=r"(raw[u].w)
                      : "l"(z + e0));
@@ -134,7 +135,7 @@ struct ChunkGeneric {
 #pragma unroll
     for (int u = 0; u < kLoadsPerThread; ++u) {
       const long long e0 = ((long long)u * kThreads + tid) * VEC;
-      ok[u] = e0 < n;
+      ok[u] = e0 < n && SBP_GUARD(z + e0, sizeof(Pack));
       if (ok[u]) raw[u] = *reinterpret_cast<const Pack*>(z + e0);
     }
   }
@@ -215,11 +216,12 @@ __global__ void __launch_bounds__(kThreads) xent_partial_kernel(const __grid_con
 #pragma unroll
     for (int w = 1; w < kThreads / 32; ++w) merge(mm, sv, sm[w], ss[w]);
     float t = 0.f;
-    const long long y = p.labels[row] - c_start - c0;
-    if (y >= 0 && y < n) t = static_cast<float>(z[y]);
-    p.part_m[(long long)part * p.rows + row] = mm;
-    p.part_s[(long long)part * p.rows + row] = sv;
-    p.part_t[(long long)part * p.rows + row] = t;
+    const long long y = (SBP_GUARD(p.labels + row, 8) ? p.labels[row] : -1) - c_start - c0;
+    if (y >= 0 && y < n && SBP_GUARD(z + y, sizeof(T))) t = static_cast<float>(z[y]);
+    const long long at = (long long)part * p.rows + row;
+    if (SBP_GUARD(p.part_m + at, 4)) p.part_m[at] = mm;
+    if (SBP_GUARD(p.part_s + at, 4)) p.part_s[at] = sv;
+    if (SBP_GUARD(p.part_t + at, 4)) p.part_t[at] = t;
   }
 }
 
@@ -237,6 +239,7 @@ __global__ void __launch_bounds__(kCombineThreads) xent_combine_kernel(const __g
   float m = -INFINITY, S = 0.f, zy = 0.f;
   for (int q = lane; q < p.parts; q += 32) {
     const long long at = (long long)q * p.rows + row;
+    if (!SBP_GUARD(p.part_m + at, 4) || !SBP_GUARD(p.part_s + at, 4) || !SBP_GUARD(p.part_t + at, 4)) continue;
     merge(m, S, p.part_m[at], p.part_s[at]);
     zy += p.part_t[at];
   }
@@ -249,9 +252,12 @@ __global__ void __launch_bounds__(kCombineThreads) xent_combine_kernel(const __g
   }
   if (lane == 0) {
     const float loss = logf(S) + m - zy;
-    for (int j = 0; j < p.n_loss; ++j) p.loss[j][row] = loss;
-    for (int j = 0; j < p.n_max; ++j) p.row_max[j][row] = m;
-    for (int j = 0; j < p.n_sum; ++j) p.row_sum[j][row] = S;
+    for (int j = 0; j < p.n_loss; ++j)
+      if (SBP_GUARD(p.loss[j] + row, 4)) p.loss[j][row] = loss;
+    for (int j = 0; j < p.n_max; ++j)
+      if (SBP_GUARD(p.row_max[j] + row, 4)) p.row_max[j][row] = m;
+    for (int j = 0; j < p.n_sum; ++j)
+      if (SBP_GUARD(p.row_sum[j] + row, 4)) p.row_sum[j][row] = S;
   }
 }
 
@@ -341,9 +347,10 @@ __global__ void __launch_bounds__(256) xent_reduce_parts_kernel(const __grid_con
       for (int j = 0; j < 4; ++j) {
         const int qq = q + 8 * j;
         const long long at = (long long)(qq < hi ? qq : q) * p.rows + row;
-        pm[j] = p.in_m[at];
-        ps[j] = p.in_s[at];
-        pt[j] = p.in_t[at];
+        const bool in_ok = SBP_GUARD(p.in_m + at, 4) && SBP_GUARD(p.in_s + at, 4) && SBP_GUARD(p.in_t + at, 4);
+        pm[j] = in_ok ? p.in_m[at] : -INFINITY;
+        ps[j] = in_ok ? p.in_s[at] : 0.f;
+        pt[j] = in_ok ? p.in_t[at] : 0.f;
       }
 #pragma unroll
       for (int j = 0; j < 4; ++j)
@@ -365,9 +372,9 @@ __global__ void __launch_bounds__(256) xent_reduce_parts_kernel(const __grid_con
       t += st[j][tx];
     }
     const long long at = (long long)blockIdx.y * p.rows + row;
-    p.out_m[at] = m;
-    p.out_s[at] = s;
-    p.out_t[at] = t;
+    if (SBP_GUARD(p.out_m + at, 4)) p.out_m[at] = m;
+    if (SBP_GUARD(p.out_s + at, 4)) p.out_s[at] = s;
+    if (SBP_GUARD(p.out_t + at, 4)) p.out_t[at] = t;
   }
 }
 
@@ -420,6 +427,7 @@ sbp_status launch_xent_finish(float* part_m, float* part_s, float* part_t, int p
   cfg.stream = st;
   cfg.attrs = pdl;
   cfg.numAttrs = 1;
+  SBP_BOUNDS_UPLOAD(st);
   cudaError_t e = cudaLaunchKernelEx(&cfg, xent_reduce_parts_kernel, r);
   if (e != cudaSuccess) return cuda_fail(e, "softmax reduce launch");
   XentCombineParams c{};
@@ -462,11 +470,13 @@ __global__ void __launch_bounds__(kThreads) xent_backward_kernel(const __grid_co
   const T* z = reinterpret_cast<const T*>(p.logits[shard]) + row * p.lpitch[shard];
   T* g = reinterpret_cast<T*>(p.grad[shard]) + row * p.gpitch[shard];
   // softmax = 2^(z log2e - m log2e - log2 S): the division by the row sum is folded into the exponent
+  if (!SBP_GUARD(p.row_max + row, 4) || !SBP_GUARD(p.row_sum + row, 4) || !SBP_GUARD(p.labels + row, 8)) return;
   const float neg = -p.row_max[row] * kLog2e - log2f(p.row_sum[row]);
   const long long y = p.labels[row] - c_start;      // label's column inside this shard, if any
   struct alignas(sizeof(T) * VEC) Pack { T e[VEC]; };
   for (long long e0 = ((long long)blockIdx.y * kThreads + threadIdx.x) * VEC; e0 < c_len;
        e0 += (long long)gridDim.y * kThreads * VEC) {
+    if (!SBP_GUARD(z + e0, sizeof(Pack)) || !SBP_GUARD(g + e0, sizeof(Pack))) continue;
     Pack in = *reinterpret_cast<const Pack*>(z + e0), out;
     const int y_rel = (y >= e0 && y < e0 + VEC) ? (int)(y - e0) : -1;   // the label's place in this vector, if it is here
 #pragma unroll
@@ -547,6 +557,14 @@ sbp_status sbp_softmax_xent(const sbp_tensor* logits, const sbp_tensor* labels, 
 
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   dim3 grid((unsigned)rows, (unsigned)nsplit, (unsigned)k);
+  SBP_BOUNDS_RESET();
+  SBP_BOUNDS_TENSOR(logits);
+  SBP_BOUNDS_TENSOR(labels);
+  SBP_BOUNDS_TENSOR(loss);
+  SBP_BOUNDS_TENSOR(row_max);
+  SBP_BOUNDS_TENSOR(row_sum);
+  SBP_BOUNDS_ADD(ws, need);
+  SBP_BOUNDS_UPLOAD(stream);
   if (logits->dtype == SBP_BF16) {
     if (vec > 1) xent_partial_kernel<ChunkBF16x8><<<grid, kThreads, 0, stream>>>(p);
     else xent_partial_kernel<ChunkGeneric<__nv_bfloat16, 1>><<<grid, kThreads, 0, stream>>>(p);
@@ -680,6 +698,13 @@ extern "C" sbp_status sbp_softmax_xent_backward(const sbp_tensor* logits, const 
   if (gy > 65535) gy = 65535;
   dim3 grid((unsigned)rows, (unsigned)gy, (unsigned)k);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  SBP_BOUNDS_RESET();
+  SBP_BOUNDS_TENSOR(logits);
+  SBP_BOUNDS_TENSOR(labels);
+  SBP_BOUNDS_TENSOR(row_max);
+  SBP_BOUNDS_TENSOR(row_sum);
+  SBP_BOUNDS_TENSOR(grad_logits);
+  SBP_BOUNDS_UPLOAD(stream);
   if (logits->dtype == SBP_BF16) {
     if (vec > 1) xent_backward_kernel<__nv_bfloat16, 8><<<grid, kThreads, 0, stream>>>(p);
     else xent_backward_kernel<__nv_bfloat16, 1><<<grid, kThreads, 0, stream>>>(p);

@@ -25,6 +25,7 @@ def _guard_bands(request, monkeypatch):
     helpers._GUARDED.clear()
     yield
     helpers.check_guards(clear=True)
+    sbp.sbp_check_device_errors()     # an expired device wait, or (debug-bounds build) a refused address
 
 
 GOLDEN = os.path.join(ROOT, "tests", "golden")

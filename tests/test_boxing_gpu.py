@@ -235,6 +235,37 @@ def test_back_to_back_calls_keep_stream_order():
             assert torch.equal(b2.locals[r].cpu(), want_s1[id(Z)][r]), f"repeat {rep}: second chain shard {r}"
 
 
+def test_ping_pong_between_two_buffers_without_a_host_sync():
+    """X -> Y, Y -> X, X -> Y over and over on one stream with different data each round and no
+    synchronisation in between: every read of a buffer must see what the launch just before it wrote
+    there, although the kernels read through the non-coherent path and each may be set up on the GPU
+    while its predecessor still runs.  Data movement (S(0) <-> S(1)) and the reduction (P(sum) -> B)."""
+    k, shape, rounds = 4, (1024, 2048), 6
+    data = [dg.normal(41, i, shape, 0, 1, BF16) for i in range(rounds)]
+    srcs = [make_global(split_cpu(D, sbp.S(0), k), shape, BF16, sbp.S(0)) for D in data]
+    X = sbp.empty_global(shape, BF16, sbp.S(0), k)
+    Y = sbp.empty_global(shape, BF16, sbp.S(1), k)
+    outs = [sbp.empty_global(shape, BF16, sbp.S(1), k) for _ in range(rounds)]
+    parts = [[dg.normal(42, 10 * i + r, shape, 0, 1, BF16) for r in range(k)] for i in range(rounds)]
+    psrc = [make_global(p, shape, BF16, sbp.P_SUM) for p in parts]
+    P = sbp.empty_global(shape, BF16, sbp.P_SUM, k)
+    sums = [sbp.empty_global(shape, BF16, sbp.B, k, alias_replicas=True) for _ in range(rounds)]
+    for i in range(rounds):
+        sbp.sbp_boxing(srcs[i], X)      # new data into X
+        sbp.sbp_boxing(X, Y)            # X -> Y
+        sbp.sbp_boxing(Y, X)            # Y -> X (X rewritten by a kernel that has just read Y)
+        sbp.sbp_boxing(X, outs[i])      # X -> this round's result
+        sbp.sbp_boxing(psrc[i], P)      # new partial values into P
+        sbp.sbp_boxing(P, sums[i])      # reduced right behind their writer
+    torch.cuda.synchronize()
+    for i in range(rounds):
+        want = split_cpu(data[i], sbp.S(1), k)
+        for r in range(k):
+            assert torch.equal(outs[i].locals[r].cpu(), want[r]), f"round {i}, shard {r}: stale or torn data"
+        ref = O.boxing([to_np(t) for t in parts[i]], O.PSUM, O.B, "bf16")[0]
+        assert np.array_equal(bits(sums[i].locals[0]), np_bits(ref, BF16)), f"round {i}: reduction read stale partial values"
+
+
 def test_host_buffer_entry_point():
     k, shape = 4, (128, 256)
     src_cpu = [dg.normal(9, r, shape, 0, 1, BF16).pin_memory() for r in range(k)]

@@ -112,6 +112,14 @@ def test_config3_mlp_full_size_sampled_rows():
     for t in (y.locals[0], y.locals[k - 1]):
         err = np.abs(to_np(t[rows]).astype(np.float64) - want)
         assert np.all(err <= 1e-3 + 2e-2 * np.abs(want) + noise), float((err - noise).max())
+        # The bound above is a maximum over 20480 outputs and leaves room for a kernel several times
+        # noisier than it should be.  The sharp check is the size of the error as a whole: its RMS
+        # against the predicted standard deviation -- the hidden state's rounding, sigma_ij above,
+        # plus the result's own rounding to bf16 (uniform within 2^-8 |Y_ij|) -- with 50 % headroom.
+        sigma2 = (noise * 0.25) ** 2 / 3.0 + (2.0 ** -8 * np.abs(want)) ** 2 / 3.0
+        rms, predicted = float(np.sqrt(np.mean(err ** 2))), float(np.sqrt(np.mean(sigma2)))
+        assert rms <= 1.5 * predicted, (rms, predicted)
+        assert rms >= 0.2 * predicted, (rms, predicted)          # and the prediction is of the right size
     assert all(torch.equal(y.locals[0], t) for t in y.locals[1:])
     # second product on its own, seeded bf16 input in place of the hidden state: the stated
     # tolerance as it stands, for the fused (S(1),S(0)) -> B route and for fp32 partials + boxing

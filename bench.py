@@ -173,36 +173,39 @@ def run_sweep(sbp, work, events=None):
 # None = not captured for the kernel as it stands.
 NCU_TRAFFIC = {
     # profiles/box_kernels_sweep_bf16_8192x8192_k4.md (full size)
-    "P(sum)->B": 1020.4e6, "P(sum)->S(0)": 647.2e6, "P(sum)->S(1)": 644.5e6, "S(0)->B": 612.7e6,
-    "S(0)->S(1)": 218.1e6, "S(1)->S(0)": 216.3e6, "B->S(1)": 217.2e6,
+    "P(sum)->B": 1024.0e6, "P(sum)->S(0)": 647.0e6, "P(sum)->S(1)": 648.1e6, "S(0)->B": 614.1e6,
+    "S(0)->S(1)": 219.2e6, "S(1)->S(0)": 217.3e6, "B->S(1)": 217.8e6,
     # profiles/xent_partial_bf16_512x1048576_k8.md (full size)
-    "softmax-xent on bf16 logits (partial + combine)": 1077.5e6,
-    "softmax-xent backward (softmax - onehot, S(1))": 2100.3e6,
+    "softmax-xent on bf16 logits (partial + combine)": 1077.2e6,
+    "softmax-xent backward (softmax - onehot, S(1))": 2099.7e6,
     # profiles/matmul_tc_classifier_bf16_512x512x1048576_k8.md (full size)
-    "classifier GEMM (B,S(1))->S(1), bf16 logits": 2105.6e6,
-    "classifier GEMM fused with softmax-xent (no logits stored)": 1127.2e6 + 50.3e6,
-    "classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)": 2104.0e6,
+    "classifier GEMM (B,S(1))->S(1), bf16 logits": 2104.7e6,
+    "classifier GEMM fused with softmax-xent (no logits stored)": 1126.3e6 + 50.5e6,
+    "classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)": 2105.3e6,
     # profiles/matmul_tc_mlp_bf16_8192x4096x16384_k8.md (full size)
-    "MLP GEMM1 (B,S(1))->S(1) + GeLU": 975.0e6,
-    "MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials": 910.8e6,
-    "MLP GEMM2 fused (S(1),S(0))->B": 1731.9e6,
-    "DP layer backward dW = X^T dY, (S(1),S(0))->S(0) fused": 2506.1e6,
-    "DP layer backward dW = X^T dY, (S(1),S(0))->B fused (8 replicas written)": 2090.9e6,
-    "DP layer backward dX = dY W^T, (S(0),B)->S(0)": 1474.8e6,
+    "MLP GEMM1 (B,S(1))->S(1) + GeLU": 993.0e6,
+    "MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials": 911.1e6,
+    "MLP GEMM2 fused (S(1),S(0))->B": 1732.5e6,
+    "DP layer backward dW = X^T dY, (S(1),S(0))->S(0) fused": 2459.8e6,
+    "DP layer backward dW = X^T dY, (S(1),S(0))->B fused (8 replicas written)": 2091.0e6,
+    "DP layer backward dX = dY W^T, (S(0),B)->S(0)": 1502.6e6,
     # profiles/extras_bf16_8192x8192_p4_and_embedding_fp32_4194304x128_batch16384_k8.md (full size)
-    "S(0)->P(sum) bf16 [8192,8192] k=4": 615.7e6,
-    "B->P(sum) bf16 [8192,8192] k=4": 611.4e6,
-    "S(0) fp32 -> B bf16 (cast fused into the gather) [8192,8192] k=4": 748.6e6,
-    "disjoint placements: S(0)[4] -> S(0)[8] bf16 [8192,8192]": 215.0e6,
-    "disjoint placements: S(0)[4] -> S(1)[8] bf16 [8192,8192]": 214.5e6,
-    "disjoint placements: S(0)[4] -> B[8] bf16 [8192,8192]": 1169.0e6,
-    "disjoint placements: P(sum)[4] -> S(0)[8] bf16 [8192,8192]": 616.7e6,
-    "disjoint placements: P(sum)[4] -> B[2] bf16 [8192,8192]": 749.7e6,
-    "disjoint placements: S(0)[4] -> P(sum)[8] bf16 [8192,8192]": 1015.4e6 + 215.5e6,
-    # profiles/embedding_fused_fp32_4194304x128_batch16384_k8.md (quarter batch, scaled x 4)
-    "embedding fused gather -> B (8 replicas written)": 7102.8e6,
-    "embedding fused gather -> B (replicas aliased, 1 write)": 950.4e6,
+    "S(0)->P(sum) bf16 [8192,8192] k=4": 619.4e6,
+    "B->P(sum) bf16 [8192,8192] k=4": 611.7e6,
+    "S(0) fp32 -> B bf16 (cast fused into the gather) [8192,8192] k=4": 749.2e6,
+    "disjoint placements: S(0)[4] -> S(0)[8] bf16 [8192,8192]": 216.3e6,
+    "disjoint placements: S(0)[4] -> S(1)[8] bf16 [8192,8192]": 215.2e6,
+    "disjoint placements: S(0)[4] -> B[8] bf16 [8192,8192]": 1148.7e6,
+    "disjoint placements: P(sum)[4] -> S(0)[8] bf16 [8192,8192]": 616.9e6,
+    "disjoint placements: P(sum)[4] -> B[2] bf16 [8192,8192]": 752.2e6,
+    "disjoint placements: S(0)[4] -> P(sum)[8] bf16 [8192,8192]": 1015.0e6 + 216.1e6,
+    # profiles/embedding_fused_fp32_config5_full_size_and_quarter_batch.md (full size, one-pass DRAM counters)
+    "embedding fused gather -> B (8 replicas written)": 7308.8e6,
+    "embedding fused gather -> B (replicas aliased, 1 write)": 1093.3e6,
 }
+# The commit whose kernels the captures above were taken on.  A kernel that changes afterwards gets
+# its entry set to None (or recaptured) in the same commit: a stale figure is worse than none.
+NCU_TRAFFIC_CAPTURED_AT = "a61a16e"
 
 
 def ncu_traffic(name):
@@ -964,7 +967,8 @@ def main():
     dom = max(per, key=lambda p: p["ms"])
     roofline = {"bound": "hbm", "kernel": "box_tile_kernel (" + dom["transform"] + ")",
                 "achieved": dom["gbs"], "peak": peaks["hbm_gbs"], "peak_source": peaks["source"],
-                "unit": "GB/s", "frac": dom["gbs"] / peaks["hbm_gbs"], "traffic": ncu_traffic(dom["transform"])}
+                "unit": "GB/s", "frac": dom["gbs"] / peaks["hbm_gbs"], "traffic": ncu_traffic(dom["transform"]),
+                "traffic_captured_at": NCU_TRAFFIC_CAPTURED_AT}
 
     line = {
         "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps,

@@ -746,6 +746,7 @@ static sbp_status boxing_one_axis(const sbp_tensor* src, sbp_tensor* dst, int ds
 }
 
 sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream) {
+  SBP_RANGE("sbp_boxing");
   if (src && dst && (src->pdims == 2 || dst->pdims == 2)) {
     // every group's one-axis op is checked before the first of them is launched
     sbp_status st = boxing_2d(src, dst, cuda_stream, true);
@@ -756,6 +757,7 @@ sbp_status sbp_boxing(const sbp_tensor* src, sbp_tensor* dst, void* cuda_stream)
 }
 
 sbp_status sbp_boxing_shard(const sbp_tensor* src, sbp_tensor* dst, int32_t dst_shard, void* cuda_stream) {
+  SBP_RANGE("sbp_boxing_shard");
   if (dst_shard < 0) return fail(SBP_ERR_INVALID_ARG, "dst_shard %d is negative", dst_shard);
   return boxing_one_axis(src, dst, dst_shard, cuda_stream, false);
 }
@@ -773,6 +775,7 @@ size_t sbp_boxing_host_workspace_bytes(const sbp_tensor* src_host, const sbp_ten
 
 sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, void* dev_ws, size_t dev_ws_bytes,
                            void* cuda_stream) {
+  SBP_RANGE("sbp_boxing_host");
   sbp_status st = check_pair(src_host, dst_host, true);
   if (st != SBP_OK) return st;
   st = refuse_ld(src_host, "src_host", "sbp_boxing_host");

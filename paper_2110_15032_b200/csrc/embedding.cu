@@ -533,6 +533,7 @@ using namespace sbp;
 
 extern "C" sbp_status sbp_embedding(const sbp_tensor* table, const sbp_tensor* ids, sbp_tensor* out,
                                     int32_t* oob_count, void* cuda_stream) {
+  SBP_RANGE("sbp_embedding");
   sbp_status st = check_tensor(table, "table", true);
   if (st != SBP_OK) return st;
   st = check_tensor(ids, "ids", true);
@@ -623,6 +624,7 @@ extern "C" sbp_status sbp_embedding(const sbp_tensor* table, const sbp_tensor* i
 
 extern "C" sbp_status sbp_embedding_backward(const sbp_tensor* grad_out, const sbp_tensor* ids, sbp_tensor* grad_table,
                                              int32_t* oob_count, void* cuda_stream) {
+  SBP_RANGE("sbp_embedding_backward");
   sbp_status st = check_tensor(grad_out, "grad_out", true);
   if (st != SBP_OK) return st;
   st = check_tensor(ids, "ids", true);

@@ -546,6 +546,7 @@ void sbp_tensor_map_stats(uint64_t* reused, uint64_t* encoded) {
 
 sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, uint32_t flags, void* ws,
                       size_t ws_bytes, void* cuda_stream) {
+  SBP_RANGE("sbp_matmul");
   MatmulPlan plan;
   const bool two_axes = x && w && y && (x->pdims == 2 || w->pdims == 2 || y->pdims == 2);
   sbp_status st = two_axes ? build_plan_2d(x, w, y, flags, true, &plan) : build_plan(x, w, y, flags, true, &plan);
@@ -617,6 +618,7 @@ size_t sbp_matmul_softmax_xent_workspace_bytes(const sbp_tensor* features, const
 sbp_status sbp_matmul_softmax_xent(const sbp_tensor* features, const sbp_tensor* weight, const sbp_tensor* labels,
                                    sbp_tensor* loss, sbp_tensor* row_max, sbp_tensor* row_sum, void* ws,
                                    size_t ws_bytes, void* cuda_stream) {
+  SBP_RANGE("sbp_matmul_softmax_xent");
   sbp_status st = check_classifier(features, weight, true);
   if (st != SBP_OK) return st;
   const int k = placement_k(features);
@@ -677,6 +679,7 @@ sbp_status sbp_matmul_softmax_xent(const sbp_tensor* features, const sbp_tensor*
 sbp_status sbp_matmul_softmax_xent_backward(const sbp_tensor* features, const sbp_tensor* weight,
                                             const sbp_tensor* labels, const sbp_tensor* row_max,
                                             const sbp_tensor* row_sum, sbp_tensor* grad_logits, void* cuda_stream) {
+  SBP_RANGE("sbp_matmul_softmax_xent_backward");
   sbp_status st = check_classifier(features, weight, true);
   if (st != SBP_OK) return st;
   const int k = placement_k(features);

@@ -69,6 +69,8 @@ struct TcParams {
   int tile_begin[SBP_MAX_K + 1];   // prefix sum of tiles per group
   int tiles_m[SBP_MAX_K];
   int tiles_n[SBP_MAX_K];
+  int mt_begin[SBP_MAX_K + 1];     // stacked == 1: prefix sum of m-tiles per group; == 2: of n-tiles
+  int stacked;                     // the groups are row (1) / column (2) blocks of one result and are walked as one grid
   int ngroups, nseg, chain, gelu, n_rep;
   int out_f32;
   int total_tiles;
@@ -256,6 +258,31 @@ struct TileCoord {
 constexpr int kPanelM = 8;
 
 __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
+  if (p.stacked == 2) {
+    // The same for a fused product written as S(1): column blocks of one result, which share every
+    // A row block; the n-tiles of all groups form one list.
+    const int tm = p.tiles_m[0], tn = p.mt_begin[p.ngroups];
+    const int panel = tile / (kPanelM * tn);
+    const int rem = tile - panel * (kPanelM * tn);
+    const int pm = min(kPanelM, tm - panel * kPanelM);
+    const int nt = rem / pm, mt = panel * kPanelM + (rem - nt * pm);
+    int g = 0;
+    while (g + 1 < p.ngroups && nt >= p.mt_begin[g + 1]) ++g;
+    return TileCoord{g, mt * BM, (nt - p.mt_begin[g]) * BN};
+  }
+  if (p.stacked) {
+    // A fused product written as S(0): the groups are the row blocks of ONE result and share every
+    // B column block.  Walking them one after the other would stream the whole B operand once per
+    // group; instead the m-tiles of all groups form one list and the panel walk runs over that.
+    const int tm = p.mt_begin[p.ngroups], tn = p.tiles_n[0];
+    const int panel = tile / (kPanelM * tn);
+    const int rem = tile - panel * (kPanelM * tn);
+    const int pm = min(kPanelM, tm - panel * kPanelM);
+    const int nt = rem / pm, mt = panel * kPanelM + (rem - nt * pm);
+    int g = 0;
+    while (g + 1 < p.ngroups && mt >= p.mt_begin[g + 1]) ++g;
+    return TileCoord{g, (mt - p.mt_begin[g]) * BM, nt * BN};
+  }
   int g = 0;
   while (g + 1 < p.ngroups && tile >= p.tile_begin[g + 1]) ++g;
   const int local = tile - p.tile_begin[g];
@@ -834,6 +861,18 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
       if (stores_y && !y_direct && !make_map(&p.map_y[g], plan.y[g], oesz, plan.m[g], plan.n[g], plan.ldy[g], 32, box_cols))
         return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for the result of group %d", g);
     }
+  }
+  // row-block (or column-block) groups of one fused result: one grid for the walk
+  bool rows_stack = plan.chain && plan.ngroups > 1, cols_stack = rows_stack;
+  for (int g = 0; g < plan.ngroups; ++g) {
+    if (plan.n[g] != plan.n[0] || plan.col_off[g] != 0 || plan.n[g] == 0) rows_stack = false;
+    if (plan.m[g] != plan.m[0] || plan.row_off[g] != 0 || plan.m[g] == 0) cols_stack = false;
+  }
+  p.stacked = rows_stack ? 1 : (cols_stack ? 2 : 0);
+  p.mt_begin[0] = 0;
+  for (int g = 0; g < plan.ngroups; ++g) {
+    const bool live = plan.m[g] > 0 && plan.n[g] > 0;
+    p.mt_begin[g + 1] = p.mt_begin[g] + (live ? (p.stacked == 2 ? p.tiles_n[g] : p.tiles_m[g]) : 0);
   }
   p.tile_begin[plan.ngroups] = tiles;
   for (int g = plan.ngroups + 1; g <= SBP_MAX_K; ++g) p.tile_begin[g] = tiles;

@@ -2,6 +2,7 @@
 #pragma once
 
 #include <cuda_runtime.h>
+#include <nvtx3/nvToolsExt.h>
 
 #include <cstdarg>
 #include <cstdint>
@@ -10,6 +11,16 @@
 #include "sbp.h"
 
 namespace sbp {
+
+// A named range around an entry point for tools that show NVTX ranges on a timeline (the header-only
+// NVTX costs a null-pointer test per call when no tool is attached).
+struct NvtxRange {
+  explicit NvtxRange(const char* name) { nvtxRangePushA(name); }
+  ~NvtxRange() { nvtxRangePop(); }
+  NvtxRange(const NvtxRange&) = delete;
+  NvtxRange& operator=(const NvtxRange&) = delete;
+};
+#define SBP_RANGE(name) ::sbp::NvtxRange sbp_range_guard_(name)
 
 // Records the detail string returned by sbp_last_error() and passes the status through.
 sbp_status fail(sbp_status s, const char* fmt, ...);

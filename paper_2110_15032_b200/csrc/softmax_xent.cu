@@ -508,6 +508,7 @@ size_t sbp_softmax_xent_workspace_bytes(const sbp_tensor* logits) {
 sbp_status sbp_softmax_xent(const sbp_tensor* logits, const sbp_tensor* labels, sbp_tensor* loss,
                             sbp_tensor* row_max, sbp_tensor* row_sum, void* ws, size_t ws_bytes,
                             void* cuda_stream) {
+  SBP_RANGE("sbp_softmax_xent");
   sbp_status st = check_tensor(logits, "logits", true);
   if (st != SBP_OK) return st;
   st = check_tensor(labels, "labels", true);
@@ -616,6 +617,7 @@ constexpr int kMaxDevices = 64;
 
 extern "C" sbp_status sbp_softmax_xent_static(const sbp_tensor* logits, const sbp_tensor* labels, sbp_tensor* loss,
                                               sbp_tensor* row_max, sbp_tensor* row_sum, void* cuda_stream) {
+  SBP_RANGE("sbp_softmax_xent_static");
   // Size check first, so that an oversized request is refused before anything else happens.
   sbp_status st = check_tensor(logits, "logits", true);
   if (st != SBP_OK) return st;
@@ -651,6 +653,7 @@ extern "C" sbp_status sbp_softmax_xent_static(const sbp_tensor* logits, const sb
 extern "C" sbp_status sbp_softmax_xent_backward(const sbp_tensor* logits, const sbp_tensor* labels,
                                                 const sbp_tensor* row_max, const sbp_tensor* row_sum,
                                                 sbp_tensor* grad_logits, void* cuda_stream) {
+  SBP_RANGE("sbp_softmax_xent_backward");
   sbp_status st = check_tensor(logits, "logits", true);
   if (st != SBP_OK) return st;
   st = check_tensor(grad_logits, "grad_logits", true);

@@ -722,3 +722,16 @@ def test_matmul_bf16_unaligned_transposed_operands(xs, ws, ys, tx, tw):
     for M, K, N, k in UNALIGNED[:2]:
         _matmul_case(M, K, N, k, BF16, xs, ws, ys=ys, seed=1202, tx=tx, tw=tw)
         _matmul_case(M, K, N, k, BF16, xs, ws, ys=ys, seed=1202, tx=tx, tw=tw, out_dtype=F32)
+
+
+@pytest.mark.parametrize("tx", [False, True])
+def test_matmul_fused_split_results_walk_their_groups_as_one_grid(tx):
+    """A P(sum) product written as S(0) / S(1): the row (column) blocks of the result are separate
+    output groups that the tensor-core kernel walks as one grid, panels of eight m-tiles running
+    across group boundaries.  Several tiles per group, ragged groups, more tiles than CTA pairs,
+    groups of one row and empty groups."""
+    _matmul_case(2600, 192, 1100, 3, BF16, sbp.S(1), sbp.S(0), ys=sbp.S(0), seed=2101, tx=tx)
+    _matmul_case(700, 192, 2600, 3, BF16, sbp.S(1), sbp.S(0), ys=sbp.S(1), seed=2102, tx=tx)
+    _matmul_case(5, 128, 520, 8, BF16, sbp.S(1), sbp.S(0), ys=sbp.S(0), seed=2103, tx=tx)
+    _matmul_case(520, 128, 5, 8, BF16, sbp.S(1), sbp.S(0), ys=sbp.S(1), seed=2104, tx=tx, out_dtype=F32)
+    _matmul_case(4096, 64, 4864, 8, BF16, sbp.P_SUM, sbp.B, ys=sbp.S(0), seed=2105)

@@ -415,6 +415,16 @@ def section_mlp(sbp, device, peaks, opts):
     res.append(_hbm_entry("MLP P(sum)->B of the bf16 partials", 2 * k * M * H * 2, avg, best, peaks))
     avg, best = time_op(lambda: sbp.sbp_matmul(h, w2, y_b, 0, ws), device, iters=5)
     res.append(_tensor_entry("MLP GEMM2 fused (S(1),S(0))->B", flops, avg, best, peaks))
+    # The same two products with the weights kept in memory as their transposes ([N,K], SBP_TRANS_W):
+    # both operands of the MMA are then K-major, the form the tensor pipe runs fastest.
+    w1t = sbp.SbpTensor((F, H), bf16, sbp.S(0), [t.t().contiguous() for t in w1.locals])      # stored S(0) = S(1) of W1
+    avg, best = time_op(lambda: sbp.sbp_matmul(x, w1t, h, sbp.SBP_EPILOGUE_GELU | sbp.SBP_TRANS_W, ws), device, iters=5)
+    res.append(_tensor_entry("MLP GEMM1 with W1 stored transposed (SBP_TRANS_W) + GeLU", flops, avg, best, peaks))
+    del w1t
+    w2t = sbp.SbpTensor((H, F), bf16, sbp.S(1), [t.t().contiguous() for t in w2.locals])      # stored S(1) = S(0) of W2
+    avg, best = time_op(lambda: sbp.sbp_matmul(h, w2t, y_b, sbp.SBP_TRANS_W, ws), device, iters=5)
+    res.append(_tensor_entry("MLP GEMM2 fused (S(1),S(0))->B with W2 stored transposed (SBP_TRANS_W)", flops, avg, best, peaks))
+    del w2t
     del h, y_p, y_b, w1, w2, x
     # Backward products of a data-parallel layer of the same size (tokens S(0), weight B), taken
     # from the stored operands with the transpose flags: dW = X^T dY is (S(1),S(0)) -> P(sum),

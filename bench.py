@@ -581,7 +581,7 @@ def section_cliffs(sbp, device, peaks, opts):
     return res
 
 
-# BASELINE config each operator section belongs to (None: beyond the five configs)
+# workload configuration (1-5) each operator section belongs to (None: beyond the five)
 SECTION_CONFIG = {"softmax": 4, "classifier": 4, "mlp": 3, "embedding": 5, "extras": None, "cliffs": None}
 
 # kernel behind an HBM-bound line, by the start of its name (tensor-bound lines: matmul_tc_kernel)

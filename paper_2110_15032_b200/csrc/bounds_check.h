@@ -9,7 +9,7 @@
 // dereferenced, so the device stays usable; sbp_check_device_errors() reports SBP_ERR_BOUNDS.
 // Accesses made by the copy engine are not covered: the tiled copies of the tensor-core kernel are
 // clipped by the hardware to the extents of their descriptors (built from the same host-computed
-// shapes), and the bulk-copy boxing engine is simply not selected in this build.
+// shapes), and the bulk-copy boxing engine is simply not selected in the debug-bounds build.
 #pragma once
 
 #include <cuda_runtime.h>

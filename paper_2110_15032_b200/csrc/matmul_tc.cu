@@ -33,6 +33,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <cstdlib>
 #include <mutex>
 #include <type_traits>
 
@@ -53,6 +54,21 @@ constexpr int kSlabBytes = 32 * 128;              // one epilogue slab: 32 rows 
 constexpr int kEpiBufs = 2;                       // staging slabs per epilogue warp
 constexpr int kEpiBytes = kEpiWarps * kEpiBufs * kSlabBytes;
 constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024;   // + alignment slack
+// The tall form (MH = 2): a CTA pair owns a 512 x 256 tile -- two m-halves of 256 rows that share
+// every B slice -- with BOTH 256-column accumulators in use at once.  A 64-deep K-block then brings
+// 48 KiB per CTA into shared memory for 2 x 4 MMAs (1024 clocks) instead of 32 KiB for 4 MMAs
+// (512 clocks): a quarter less operand traffic per MMA clock, both from L2 and through shared
+// memory.  At the square form's rate the shared-memory data path has to carry one 128-byte
+// wavefront every clock (TMA writes + MMA reads) and the tensor pipe reaches 76 %; with the
+// slack the tall form leaves it runs the main loop at full rate.  The price is that the
+// epilogue of a tile no longer overlaps the next tile's MMAs in full (the second accumulator is
+// not a spare any more), which a long contraction repays many times over and a short one does not:
+// the host picks the form per product.
+constexpr int kStagesTall = 4;
+constexpr int kStageBytesTall = 2 * kStageA + kStageB;     // 48 KiB per CTA
+constexpr int kEpiBufsTall = 1;
+constexpr int kSmemBytesTall = kStagesTall * kStageBytesTall + kEpiWarps * kEpiBufsTall * kSlabBytes + 1024;
+constexpr int kMaxStages = kStages > kStagesTall ? kStages : kStagesTall;
 constexpr int kThreadsTc = 32 * (2 + kEpiWarps);
 constexpr int kTmemCols = 512;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -74,6 +90,9 @@ struct TcParams {
   int ngroups, nseg, chain, gelu, n_rep;
   int out_f32;
   int total_tiles;
+  int walk_m;                   // rows of a walked tile: 256, or 512 (tall form and the square remainder of a mixed run)
+  int tile_first;               // index of the first walked tile of this launch
+  int half_split;               // square form over 512-row walked tiles: launch tile 2t + h is m-half h of walked tile t
   int xent;                     // 1: softmax partials instead of stored logits
   XentFusion xf;
   // Results the copy engine cannot address (a base or a row pitch that is not a multiple of 16
@@ -258,6 +277,12 @@ struct TileCoord {
 constexpr int kPanelM = 8;
 
 __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
+  int half_m = 0;
+  if (p.half_split) {
+    half_m = (tile & 1) * BM;
+    tile >>= 1;
+  }
+  tile += p.tile_first;
   if (p.stacked == 2) {
     // The same for a fused product written as S(1): column blocks of one result, which share every
     // A row block; the n-tiles of all groups form one list.
@@ -268,7 +293,7 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
     const int nt = rem / pm, mt = panel * kPanelM + (rem - nt * pm);
     int g = 0;
     while (g + 1 < p.ngroups && nt >= p.mt_begin[g + 1]) ++g;
-    return TileCoord{g, mt * BM, (nt - p.mt_begin[g]) * BN};
+    return TileCoord{g, mt * p.walk_m + half_m, (nt - p.mt_begin[g]) * BN};
   }
   if (p.stacked) {
     // A fused product written as S(0): the groups are the row blocks of ONE result and share every
@@ -281,7 +306,7 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
     const int nt = rem / pm, mt = panel * kPanelM + (rem - nt * pm);
     int g = 0;
     while (g + 1 < p.ngroups && mt >= p.mt_begin[g + 1]) ++g;
-    return TileCoord{g, (mt - p.mt_begin[g]) * BM, nt * BN};
+    return TileCoord{g, (mt - p.mt_begin[g]) * p.walk_m + half_m, nt * BN};
   }
   int g = 0;
   while (g + 1 < p.ngroups && tile >= p.tile_begin[g + 1]) ++g;
@@ -291,7 +316,7 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
   const int rem = local - panel * (kPanelM * tn);
   const int pm = min(kPanelM, tm - panel * kPanelM);   // m-tiles in this (possibly last) panel
   const int nt = rem / pm, mt = panel * kPanelM + (rem - nt * pm);
-  return TileCoord{g, mt * BM, nt * BN};
+  return TileCoord{g, mt * p.walk_m + half_m, nt * BN};
 }
 
 // ------------------------------------------------------------------ the kernel
@@ -299,23 +324,28 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
 // AT / BT: operand A / B is stored transposed.  They are compile-time so that the usual
 // (untransposed) form carries no trace of the other three: as run-time switches they cost the
 // MMA-issuing thread and the producer enough to slow every product by 6 %.
-template <int AT, int BT>
+// MH: m-halves of 256 rows per pair tile (1 = square form, 2 = tall form, see kStageBytesTall).
+template <int AT, int BT, int MH>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
     matmul_tc_kernel(const __grid_constant__ TcParams p) {
+  constexpr int kSt = MH == 2 ? kStagesTall : kStages;                  // ring depth
+  constexpr int kStA = MH * kStageA;                                    // bytes of A per ring slot
+  constexpr int kStBytes = kStA + kStageB;
+  constexpr int kEB = MH == 2 ? kEpiBufsTall : kEpiBufs;                // staging slabs per epilogue warp
   extern __shared__ unsigned char smem_raw[];
-  __shared__ __align__(8) unsigned long long bar_full[kStages], bar_empty[kStages], bar_acc_full[2], bar_acc_empty[2];
+  __shared__ __align__(8) unsigned long long bar_full[kMaxStages], bar_empty[kMaxStages], bar_acc_full[2], bar_acc_empty[2];
   __shared__ unsigned tmem_base_slot;
   __shared__ int abort_flag_s;
   volatile int* abort_flag = &abort_flag_s;
 
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  unsigned char* epi = smem + kStages * kStageBytes;
+  unsigned char* epi = smem + kSt * kStBytes;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const unsigned rank = cluster_ctarank();     // 0 = the CTA that issues the pair's MMAs
 
   if (threadIdx.x == 0) {
     abort_flag_s = 0;
-    for (int i = 0; i < kStages; ++i) {
+    for (int i = 0; i < kSt; ++i) {
       mbar_init(smem_addr(&bar_full[i]), 1);      // used in CTA 0 only: one arrive + both CTAs' bytes
       mbar_init(smem_addr(&bar_empty[i]), 1);     // one commit per use, delivered to both CTAs
     }
@@ -352,21 +382,25 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
         const int s_lo = p.chain ? 0 : tc.g, s_hi = p.chain ? p.nseg : tc.g + 1;
         for (int s = s_lo; s < s_hi; ++s) {
           for (int kb = 0; kb < p.kblocks[s]; ++kb, ++kb_iter) {
-            const int slot = (int)(kb_iter % kStages);
-            const unsigned parity = (unsigned)(((kb_iter / kStages) & 1) ^ 1);
+            const int slot = (int)(kb_iter % kSt);
+            const unsigned parity = (unsigned)(((kb_iter / kSt) & 1) ^ 1);
             if (!mbar_wait(smem_addr(&bar_empty[slot]), parity, abort_flag)) goto producer_done;
             const unsigned full0 = map_to_cta(smem_addr(&bar_full[slot]), 0);
-            if (rank == 0) mbar_expect_tx(smem_addr(&bar_full[slot]), 2 * kStageBytes);
-            unsigned char* sa = smem + slot * kStageBytes;
-            unsigned char* sb = sa + kStageA;
-            const int arow = (int)p.row_off[tc.g] + tc.m0 + (int)rank * BMH;
+            if (rank == 0) mbar_expect_tx(smem_addr(&bar_full[slot]), 2 * kStBytes);
+            unsigned char* sa0 = smem + slot * kStBytes;
+            unsigned char* sb = sa0 + kStA;
             const int bcol = (int)p.col_off[tc.g] + tc.n0 + (int)rank * BNH;
-            if constexpr (!AT) {   // [rows, K] in memory: one box of 128 rows x 64 K
-              tma_load_2d(smem_addr(sa), &p.map_a[s], kb * BK, arow, full0);
-            } else {            // [K, rows] in memory: two boxes of 64 K x 64 rows
 #pragma unroll
-              for (int c = 0; c < BMH / 64; ++c)
-                tma_load_2d(smem_addr(sa + c * (BK * 128)), &p.map_a[s], arow + c * 64, kb * BK, full0);
+            for (int h = 0; h < MH; ++h) {       // this CTA's 128 rows of every m-half
+              unsigned char* sa = sa0 + h * kStageA;
+              const int arow = (int)p.row_off[tc.g] + tc.m0 + h * BM + (int)rank * BMH;
+              if constexpr (!AT) {   // [rows, K] in memory: one box of 128 rows x 64 K
+                tma_load_2d(smem_addr(sa), &p.map_a[s], kb * BK, arow, full0);
+              } else {            // [K, rows] in memory: two boxes of 64 K x 64 rows
+#pragma unroll
+                for (int c = 0; c < BMH / 64; ++c)
+                  tma_load_2d(smem_addr(sa + c * (BK * 128)), &p.map_a[s], arow + c * 64, kb * BK, full0);
+              }
             }
             if constexpr (!BT) {   // [K, cols] in memory: two boxes of 64 K x 64 columns
 #pragma unroll
@@ -382,9 +416,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
       if (*abort_flag && rank == 0) {
         // give the loads still in flight a bounded chance to land before the CTA goes away
         const long long issued = kb_iter;
-        for (long long i = issued > kStages ? issued - kStages : 0; i < issued; ++i) {
+        for (long long i = issued > kSt ? issued - kSt : 0; i < issued; ++i) {
           const unsigned long long t0 = now_ns();
-          while (!mbar_try(smem_addr(&bar_full[i % kStages]), (unsigned)((i / kStages) & 1)) && now_ns() - t0 < 100000000ull) {
+          while (!mbar_try(smem_addr(&bar_full[i % kSt]), (unsigned)((i / kSt) & 1)) && now_ns() - t0 < 100000000ull) {
           }
         }
       }
@@ -397,23 +431,37 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
       constexpr unsigned idesc = make_idesc(AT, BT);
       for (int tile = first; tile < p.total_tiles && !*abort_flag; tile += stride, ++tile_iter) {
         const TileCoord tc = tile_coord(p, tile);
-        const int acc = tile_iter & 1;
-        if (!mbar_wait(smem_addr(&bar_acc_empty[acc]), (unsigned)(((tile_iter >> 1) & 1) ^ 1), abort_flag)) break;
+        // Square form: the two accumulators take turns, so a tile's MMAs run while the tile before
+        // it is drained.  Tall form: accumulator h belongs to m-half h of every tile; the first
+        // m-half may start as soon as ITS accumulator has been drained, the second waits for its own.
+        const int acc = MH == 2 ? 0 : (tile_iter & 1);
+        const unsigned empty_parity = MH == 2 ? (unsigned)((tile_iter & 1) ^ 1) : (unsigned)(((tile_iter >> 1) & 1) ^ 1);
+        if (!mbar_wait(smem_addr(&bar_acc_empty[acc]), empty_parity, abort_flag)) break;
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-        const unsigned d_tmem = tmem_base + acc * BN;
         const int s_lo = p.chain ? 0 : tc.g, s_hi = p.chain ? p.nseg : tc.g + 1;
         unsigned accumulate = 0;
         bool ok = true;
         for (int s = s_lo; s < s_hi && ok; ++s) {
           for (int kb = 0; kb < p.kblocks[s]; ++kb, ++kb_iter) {
-            const int slot = (int)(kb_iter % kStages);
-            if (!mbar_wait(smem_addr(&bar_full[slot]), (unsigned)((kb_iter / kStages) & 1), abort_flag)) {
+            const int slot = (int)(kb_iter % kSt);
+            if (!mbar_wait(smem_addr(&bar_full[slot]), (unsigned)((kb_iter / kSt) & 1), abort_flag)) {
               ok = false;
               break;
             }
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            const unsigned sa = smem_addr(smem + slot * kStageBytes);
-            const unsigned sb = sa + kStageA;
+            const unsigned sa0 = smem_addr(smem + slot * kStBytes);
+            const unsigned sb = sa0 + kStA;
+#pragma unroll
+            for (int h = 0; h < MH; ++h) {
+            if (MH == 2 && h == 1 && accumulate == 0) {      // first K-block of the tile: the second accumulator must be free too
+              if (!mbar_wait(smem_addr(&bar_acc_empty[1]), empty_parity, abort_flag)) {
+                ok = false;
+                break;
+              }
+              asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            }
+            const unsigned sa = sa0 + h * kStageA;
+            const unsigned d_tmem = tmem_base + (MH == 2 ? h : acc) * BN;
 #pragma unroll
             for (int kk = 0; kk < BK / 16; ++kk) {
               // K-major tile (A as given, B transposed): rows of 128 bytes = 64 K-elements, 8-row
@@ -425,21 +473,23 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
                   AT ? smem_desc(sa + kk * 2048, BK * 128, 1024) : smem_desc(sa + kk * 32, 16, 1024);
               const unsigned long long db =
                   BT ? smem_desc(sb + kk * 32, 16, 1024) : smem_desc(sb + kk * 2048, BK * 128, 1024);
-              umma_bf16(d_tmem, da, db, idesc, accumulate);
-              accumulate = 1;
+              umma_bf16(d_tmem, da, db, idesc, kk == 0 ? accumulate : 1u);
             }
+            }
+            if (!ok) break;
+            accumulate = 1;
             umma_commit_pair(smem_addr(&bar_empty[slot]));   // slot reusable in both CTAs
           }
         }
         if (!ok) break;
-        umma_commit_pair(smem_addr(&bar_acc_full[acc]));      // accumulator complete in both CTAs
+        umma_commit_pair(smem_addr(&bar_acc_full[acc]));      // accumulator(s) complete in both CTAs
       }
     }
   } else {
     // ------------------------------------------------ epilogue (warps 2..9, both CTAs)
     const int q = warp & 3;                       // the 32 tensor-memory lanes this warp may read
     const int half = (warp - 2) >> 2;             // which 128 of the 256 columns
-    unsigned char* my_epi = epi + (warp - 2) * kEpiBufs * kSlabBytes;
+    unsigned char* my_epi = epi + (warp - 2) * kEB * kSlabBytes;
     const int cols_per_slab = p.out_f32 ? 32 : 64;
     const int nslabs = (BN / 2) / cols_per_slab;
     const unsigned acc_empty0[2] = {map_to_cta(smem_addr(&bar_acc_empty[0]), 0), map_to_cta(smem_addr(&bar_acc_empty[1]), 0)};
@@ -448,14 +498,19 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
     for (int tile = first; tile < p.total_tiles; tile += stride, ++tile_iter) {
       if (*abort_flag) break;
       const TileCoord tc = tile_coord(p, tile);
-      const int acc = tile_iter & 1;
+      const int facc = MH == 2 ? 0 : (tile_iter & 1);
       bool ok = true;
-      if (lane == 0) ok = mbar_wait(smem_addr(&bar_acc_full[acc]), (unsigned)((tile_iter >> 1) & 1), abort_flag);
+      if (lane == 0)
+        ok = mbar_wait(smem_addr(&bar_acc_full[facc]), MH == 2 ? (unsigned)(tile_iter & 1) : (unsigned)((tile_iter >> 1) & 1), abort_flag);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) break;
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const long long Mg = p.m[tc.g], Ng = p.n[tc.g];
-      const int row0 = tc.m0 + (int)rank * BMH + q * 32;
+      // tall form: the accumulator of the first m-half is drained (and handed back) before the second
+#pragma unroll 1
+      for (int h = 0; h < MH; ++h) {
+      const int acc = MH == 2 ? h : facc;
+      const int row0 = tc.m0 + h * BM + (int)rank * BMH + q * 32;
       const unsigned taddr = tmem_base + ((unsigned)(q * 32) << 16) + acc * BN + half * (BN / 2);
       if (p.xent == 1) {
         // Softmax partials of this warp's 32 rows x 128 columns; one thread owns one row, so
@@ -559,9 +614,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
             tmem_ld32(taddr + sl * cols_per_slab, v);
             if (!p.out_f32) tmem_ld32(taddr + sl * cols_per_slab + 32, v + 32);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-            unsigned char* buf = my_epi + (slab_iter % kEpiBufs) * kSlabBytes;
+            unsigned char* buf = my_epi + (slab_iter % kEB) * kSlabBytes;
             // the store that last used this buffer must have finished reading it
-            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kEpiBufs - 1) : "memory");
+            if (lane == 0) asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(kEB - 1) : "memory");
             __syncwarp();
             unsigned char* rowp = buf + lane * 128;
             if (p.out_f32) {
@@ -634,6 +689,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
       asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive_cluster(acc_empty0[acc]);   // tells CTA 0's MMA thread
+      }
     }
     if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
   }
@@ -670,7 +726,7 @@ static EncodeTiledFn encode_fn() {
 // Tensor maps already encoded by this process, keyed by everything that goes into one.  A map holds
 // nothing but the address and the layout, so an entry stays valid for as long as its key recurs: a
 // product that is called again on the same buffers (every step of a training loop) encodes nothing.
-// Direct-mapped; used with the parameter block's lock held.
+// Two-way set-associative; used with the parameter block's lock held.
 struct MapKey {
   const void* base;
   long long rows, cols, ld;
@@ -685,8 +741,9 @@ struct MapSlot {
   MapKey key;
   bool used;
 };
-constexpr int kMapCacheSlots = 1024;
-static MapSlot g_map_cache[kMapCacheSlots];
+constexpr int kMapCacheSets = 2048, kMapCacheWays = 2;
+static MapSlot g_map_cache[kMapCacheSets][kMapCacheWays];
+static unsigned char g_map_victim[kMapCacheSets];
 static unsigned long long g_map_hits = 0, g_map_encodes = 0;
 
 static unsigned map_slot_of(const MapKey& k) {
@@ -696,7 +753,7 @@ static unsigned map_slot_of(const MapKey& k) {
   mix((unsigned long long)k.cols);
   mix((unsigned long long)k.ld);
   mix((unsigned long long)(k.esz | (k.box_rows << 8) | (k.box_cols << 20)));
-  return (unsigned)(h % kMapCacheSlots);
+  return (unsigned)(h % kMapCacheSets);
 }
 
 void tensor_map_cache_stats(unsigned long long* hits, unsigned long long* encodes) {
@@ -708,12 +765,20 @@ void tensor_map_cache_stats(unsigned long long* hits, unsigned long long* encode
 static bool make_map(CUtensorMap* map, const void* base, int esz, long long rows, long long cols, long long ld,
                      int box_rows, int box_cols) {
   const MapKey key{base, rows, cols, ld, esz, box_rows, box_cols};
-  MapSlot& slot = g_map_cache[map_slot_of(key)];
-  if (slot.used && slot.key == key) {
-    *map = slot.map;
-    ++g_map_hits;
-    return true;
+  const unsigned set = map_slot_of(key);
+  for (int w = 0; w < kMapCacheWays; ++w) {
+    const MapSlot& hit = g_map_cache[set][w];
+    if (hit.used && hit.key == key) {
+      *map = hit.map;
+      ++g_map_hits;
+      return true;
+    }
   }
+  int way = (g_map_victim[set] + 1) % kMapCacheWays;      // the way not written last ...
+  for (int w = kMapCacheWays - 1; w >= 0; --w)
+    if (!g_map_cache[set][w].used) way = w;                 // ... unless one is still unused
+  g_map_victim[set] = (unsigned char)way;
+  MapSlot& slot = g_map_cache[set][way];
   EncodeTiledFn fn = encode_fn();
   if (!fn) return false;
   cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -735,23 +800,25 @@ size_t matmul_tc_workspace_bytes(const MatmulPlan&) { return 0; }
 
 static bool aligned16(const void* p) { return reinterpret_cast<uintptr_t>(p) % 16 == 0; }
 
-// Launch of one compiled form of the kernel (called with the parameter block's lock held).
-template <int AT, int BT>
-static sbp_status launch_tc_form(const TcParams& p, int tiles, cudaStream_t st) {
+// Launch of one compiled form of the kernel (called with the parameter block's lock held), or,
+// with p == nullptr, only the number of CTA pairs of that form the device holds at once.
+template <int AT, int BT, int MH>
+static sbp_status launch_tc_form(const TcParams* p, cudaStream_t st, int* capacity) {
+  constexpr int kSmem = MH == 2 ? kSmemBytesTall : kSmemBytes;
   // per device: the kernel's shared-memory opt-in and the number of CTA pairs that fit at once
   static int pairs_on_device[64] = {};
   int dev = 0;
   SBP_CUDA_TRY(cudaGetDevice(&dev));
   if (dev < 0 || dev >= 64) return fail(SBP_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
   if (pairs_on_device[dev] == 0) {
-    SBP_CUDA_TRY(cudaFuncSetAttribute(matmul_tc_kernel<AT, BT>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes));
+    SBP_CUDA_TRY(cudaFuncSetAttribute(matmul_tc_kernel<AT, BT, MH>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem));
     int sms = 0;
     SBP_CUDA_TRY(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
     // how many CTA pairs the device can hold at once (pairs must sit in one GPC)
     cudaLaunchConfig_t probe = {};
     probe.gridDim = dim3((unsigned)(2 * (sms / 2)));
     probe.blockDim = dim3(kThreadsTc);
-    probe.dynamicSmemBytes = kSmemBytes;
+    probe.dynamicSmemBytes = kSmem;
     cudaLaunchAttribute attr;
     attr.id = cudaLaunchAttributeClusterDimension;
     attr.val.clusterDim.x = 2;
@@ -760,20 +827,73 @@ static sbp_status launch_tc_form(const TcParams& p, int tiles, cudaStream_t st) 
     probe.attrs = &attr;
     probe.numAttrs = 1;
     int clusters = 0;
-    if (cudaOccupancyMaxActiveClusters(&clusters, matmul_tc_kernel<AT, BT>, &probe) != cudaSuccess || clusters < 1) {
+    if (cudaOccupancyMaxActiveClusters(&clusters, matmul_tc_kernel<AT, BT, MH>, &probe) != cudaSuccess || clusters < 1) {
       cudaGetLastError();
       clusters = sms / 2;
     }
     pairs_on_device[dev] = clusters;
   }
   const int max_pairs = pairs_on_device[dev];
-  const int pairs = tiles < max_pairs ? tiles : max_pairs;
+  if (capacity) *capacity = max_pairs;
+  if (!p) return SBP_OK;
+  const int pairs = p->total_tiles < max_pairs ? p->total_tiles : max_pairs;
   SBP_BOUNDS_UPLOAD(st);
-  matmul_tc_kernel<AT, BT><<<2 * pairs, kThreadsTc, kSmemBytes, st>>>(p);
+  matmul_tc_kernel<AT, BT, MH><<<2 * pairs, kThreadsTc, kSmem, st>>>(*p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e, "tensor-core matmul launch");
   count_launch();
   return SBP_OK;
+}
+
+static sbp_status launch_tc(bool tall, bool a_trans, bool b_trans, const TcParams* p, cudaStream_t st, int* capacity) {
+  switch ((tall ? 4 : 0) | (a_trans ? 2 : 0) | (b_trans ? 1 : 0)) {
+    case 0: return launch_tc_form<0, 0, 1>(p, st, capacity);
+    case 1: return launch_tc_form<0, 1, 1>(p, st, capacity);
+    case 2: return launch_tc_form<1, 0, 1>(p, st, capacity);
+    case 3: return launch_tc_form<1, 1, 1>(p, st, capacity);
+    case 4: return launch_tc_form<0, 0, 2>(p, st, capacity);
+    case 5: return launch_tc_form<0, 1, 2>(p, st, capacity);
+    case 6: return launch_tc_form<1, 0, 2>(p, st, capacity);
+    default: return launch_tc_form<1, 1, 2>(p, st, capacity);
+  }
+}
+
+// Which form runs a product.  Times in microseconds per wave (one tile on every CTA pair), fitted
+// to this kernel's measured times on B200 under its power cap (the clock settles lower the busier
+// the tensor pipe is, which is why these are not clock counts):
+//   square form  0.428 per 64-deep K-block; the epilogue is hidden unless it is store-bound;
+//   tall form    0.69 per K-block for twice the rows, plus an exposed epilogue of about 9.
+// A run may be mixed: `tall_waves` full waves of tall tiles, then the rest of the walk in the
+// square form (two 256-row halves per walked tile) -- a last wave that only half fills the device
+// costs a whole tall wave otherwise.
+struct FormChoice {
+  bool walk_tall;      // tiles are walked 512 rows at a time
+  int tall_tiles;      // the first so many walked tiles run in the tall form
+};
+
+static FormChoice choose_form(long long tiles_sq, long long tiles_tall, long long kb, int cap_sq, int cap_tall, bool gelu, int n_rep,
+                              bool out_f32, int forced) {
+  const double wave_sq = 0.428 * kb + 0.5 + (gelu ? 1.0 : 0.0) + 1.5 * n_rep + (out_f32 ? 1.0 : 0.0);
+  const double wave_tall = 0.69 * kb + 9.0 + (gelu ? 6.0 : 0.0) + 3.0 * n_rep + (out_f32 ? 4.0 : 0.0);
+  const double kRelaunch = 3.0;
+  auto waves = [](long long tiles, int cap) { return (double)((tiles + cap - 1) / cap); };
+  const double cost_sq = waves(tiles_sq, cap_sq) * wave_sq;
+  const double cost_tall = waves(tiles_tall, cap_tall) * wave_tall;
+  const long long full = tiles_tall / cap_tall * cap_tall;       // tall tiles in whole waves
+  const double cost_mixed = full == 0 || full == tiles_tall
+                                ? 1e30
+                                : (double)(full / cap_tall) * wave_tall + waves(2 * (tiles_tall - full), cap_sq) * wave_sq + kRelaunch;
+  int pick;      // 0 square, 1 tall, 2 mixed
+  if (forced) pick = forced - 1;
+  else {
+    pick = 0;
+    double best = cost_sq * 0.98;                                // ties go to the square form
+    if (cost_tall < best) { best = cost_tall; pick = 1; }
+    if (cost_mixed < best) { best = cost_mixed; pick = 2; }
+  }
+  if (pick == 2 && (full == 0 || full == tiles_tall)) pick = full == 0 ? 0 : 1;
+  if (pick == 0) return FormChoice{false, 0};
+  return FormChoice{true, (int)(pick == 1 ? tiles_tall : full)};
 }
 
 sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaStream_t st, bool* taken) {
@@ -842,6 +962,34 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
                                    : make_map(&p.map_b[s], plan.b[s], 2, plan.kseg[s], cols_b, plan.ldb[s], BK, 64);
     if (!ok_b) return fail(SBP_ERR_CUDA, "cuTensorMapEncodeTiled failed for operand w of shard %d", s);
   }
+  // Which form (see choose_form).  The softmax epilogues are written for the square form, and so is
+  // the element-wise store of a result the copy engine cannot address.
+  long long kb_tile = 0, tiles_sq = 0, tiles_tall = 0;
+  for (int s = 0; s < plan.nseg; ++s)
+    if (plan.chain || s < plan.ngroups) kb_tile = plan.chain ? kb_tile + p.kblocks[s] : std::max<long long>(kb_tile, p.kblocks[s]);
+  for (int g = 0; g < plan.ngroups; ++g) {
+    if (plan.m[g] <= 0 || plan.n[g] <= 0) continue;
+    const long long tn = (plan.n[g] + BN - 1) / BN;
+    tiles_sq += (plan.m[g] + BM - 1) / BM * tn;
+    tiles_tall += (plan.m[g] + 2 * BM - 1) / (2 * BM) * tn;
+  }
+  static const int forced_env = [] {
+    const char* e = getenv("SBP_TC_FORM");     // "square" / "tall" / "mixed": for measurements; the default chooses
+    return e ? (e[0] == 's' ? 1 : (e[0] == 't' ? 2 : (e[0] == 'm' ? 3 : 0))) : 0;
+  }();
+  FormChoice form{false, 0};
+  if (!xf && !y_direct && tiles_tall > 0 && tiles_sq <= 0x1fffffffLL) {
+    int cap_sq = 0, cap_tall = 0;
+    sbp_status qs = launch_tc(false, plan.a_trans, plan.b_trans, nullptr, st, &cap_sq);
+    if (qs == SBP_OK) qs = launch_tc(true, plan.a_trans, plan.b_trans, nullptr, st, &cap_tall);
+    if (qs != SBP_OK) return qs;
+    form = choose_form(tiles_sq, tiles_tall, kb_tile, cap_sq, cap_tall, plan.gelu != 0, plan.n_rep, plan.out_dtype == SBP_F32, forced_env);
+  }
+  const int tile_m = form.walk_tall ? 2 * BM : BM;
+  p.walk_m = tile_m;
+  p.tile_first = 0;
+  p.half_split = 0;
+
   int tiles = 0;
   const int box_cols = p.out_f32 ? 32 : 64;
   for (int g = 0; g < plan.ngroups; ++g) {
@@ -850,7 +998,7 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
     p.row_off[g] = plan.row_off[g];
     p.col_off[g] = plan.col_off[g];
     p.tile_begin[g] = tiles;
-    const long long tm = (plan.m[g] + BM - 1) / BM, tn = (plan.n[g] + BN - 1) / BN;
+    const long long tm = (plan.m[g] + tile_m - 1) / tile_m, tn = (plan.n[g] + BN - 1) / BN;
     p.tiles_m[g] = (int)std::max(1LL, tm);
     p.tiles_n[g] = (int)std::max(1LL, tn);
     if (plan.m[g] > 0 && plan.n[g] > 0) {
@@ -885,12 +1033,16 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
   *taken = true;
   if (tiles == 0) return SBP_OK;
 
-  switch ((plan.a_trans ? 2 : 0) | (plan.b_trans ? 1 : 0)) {
-    case 0: return launch_tc_form<0, 0>(p, tiles, st);
-    case 1: return launch_tc_form<0, 1>(p, tiles, st);
-    case 2: return launch_tc_form<1, 0>(p, tiles, st);
-    default: return launch_tc_form<1, 1>(p, tiles, st);
-  }
+  if (!form.walk_tall) return launch_tc(false, plan.a_trans, plan.b_trans, &p, st, nullptr);
+  // tall form over the first walked tiles, then (mixed run) the square form over the halves of the rest
+  const int tall_tiles = std::min(form.tall_tiles, tiles);
+  p.total_tiles = tall_tiles;
+  sbp_status rs = launch_tc(true, plan.a_trans, plan.b_trans, &p, st, nullptr);
+  if (rs != SBP_OK || tall_tiles == tiles) return rs;
+  p.tile_first = tall_tiles;
+  p.half_split = 1;
+  p.total_tiles = 2 * (tiles - tall_tiles);
+  return launch_tc(false, plan.a_trans, plan.b_trans, &p, st, nullptr);
 }
 
 sbp_status read_and_clear_tc_timeout(bool* timed_out) {

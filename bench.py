@@ -311,6 +311,16 @@ def time_op(fn, device, iters=10, warmup=3):
     return sum(ms) / len(ms), min(ms)
 
 
+def time_mm(sbp, fn, device, iters=5):
+    """time_op for a tensor-core product, plus the form(s) of the kernel that one call launches."""
+    before = sbp.sbp_matmul_form_stats()
+    fn()
+    d = [a - b for a, b in zip(sbp.sbp_matmul_form_stats(), before)]
+    form = "mixed" if d[2] else ("tall" if d[1] else ("square" if d[0] else "none"))
+    avg, best = time_op(fn, device, iters=iters)
+    return avg, best, {"form": form}
+
+
 def _hbm_entry(name, nbytes, avg, best, peaks, extra=None, config=None, kernel=None):
     """One HBM-bound line.  `achieved` counts the ALGORITHMIC bytes; where an ncu capture of the kernel
     as it stands exists, `achieved_dram` is that capture's DRAM bytes per launch over the same time."""
@@ -407,23 +417,23 @@ def section_mlp(sbp, device, peaks, opts):
                      dtype=torch.uint8, device=device)
     flops = 2.0 * M * H * F
     res = []
-    avg, best = time_op(lambda: sbp.sbp_matmul(x, w1, h, sbp.SBP_EPILOGUE_GELU, ws), device, iters=5)
-    res.append(_tensor_entry("MLP GEMM1 (B,S(1))->S(1) + GeLU", flops, avg, best, peaks))
-    avg, best = time_op(lambda: sbp.sbp_matmul(h, w2, y_p, 0, ws), device, iters=5)
-    res.append(_tensor_entry("MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials", flops, avg, best, peaks))
+    avg, best, form = time_mm(sbp, lambda: sbp.sbp_matmul(x, w1, h, sbp.SBP_EPILOGUE_GELU, ws), device)
+    res.append(_tensor_entry("MLP GEMM1 (B,S(1))->S(1) + GeLU", flops, avg, best, peaks, form))
+    avg, best, form = time_mm(sbp, lambda: sbp.sbp_matmul(h, w2, y_p, 0, ws), device)
+    res.append(_tensor_entry("MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials", flops, avg, best, peaks, form))
     avg, best = time_op(lambda: sbp.sbp_boxing(y_p, y_b), device)
     res.append(_hbm_entry("MLP P(sum)->B of the bf16 partials", 2 * k * M * H * 2, avg, best, peaks))
-    avg, best = time_op(lambda: sbp.sbp_matmul(h, w2, y_b, 0, ws), device, iters=5)
-    res.append(_tensor_entry("MLP GEMM2 fused (S(1),S(0))->B", flops, avg, best, peaks))
+    avg, best, form = time_mm(sbp, lambda: sbp.sbp_matmul(h, w2, y_b, 0, ws), device)
+    res.append(_tensor_entry("MLP GEMM2 fused (S(1),S(0))->B", flops, avg, best, peaks, form))
     # The same two products with the weights kept in memory as their transposes ([N,K], SBP_TRANS_W):
     # both operands of the MMA are then K-major, the form the tensor pipe runs fastest.
     w1t = sbp.SbpTensor((F, H), bf16, sbp.S(0), [t.t().contiguous() for t in w1.locals])      # stored S(0) = S(1) of W1
-    avg, best = time_op(lambda: sbp.sbp_matmul(x, w1t, h, sbp.SBP_EPILOGUE_GELU | sbp.SBP_TRANS_W, ws), device, iters=5)
-    res.append(_tensor_entry("MLP GEMM1 with W1 stored transposed (SBP_TRANS_W) + GeLU", flops, avg, best, peaks))
+    avg, best, form = time_mm(sbp, lambda: sbp.sbp_matmul(x, w1t, h, sbp.SBP_EPILOGUE_GELU | sbp.SBP_TRANS_W, ws), device)
+    res.append(_tensor_entry("MLP GEMM1 with W1 stored transposed (SBP_TRANS_W) + GeLU", flops, avg, best, peaks, form))
     del w1t
     w2t = sbp.SbpTensor((H, F), bf16, sbp.S(1), [t.t().contiguous() for t in w2.locals])      # stored S(1) = S(0) of W2
-    avg, best = time_op(lambda: sbp.sbp_matmul(h, w2t, y_b, sbp.SBP_TRANS_W, ws), device, iters=5)
-    res.append(_tensor_entry("MLP GEMM2 fused (S(1),S(0))->B with W2 stored transposed (SBP_TRANS_W)", flops, avg, best, peaks))
+    avg, best, form = time_mm(sbp, lambda: sbp.sbp_matmul(h, w2t, y_b, sbp.SBP_TRANS_W, ws), device)
+    res.append(_tensor_entry("MLP GEMM2 fused (S(1),S(0))->B with W2 stored transposed (SBP_TRANS_W)", flops, avg, best, peaks, form))
     del w2t
     del h, y_p, y_b, w1, w2, x
     # Backward products of a data-parallel layer of the same size (tokens S(0), weight B), taken
@@ -435,15 +445,15 @@ def section_mlp(sbp, device, peaks, opts):
     Wb = dg.normal(1003, 70, (H, F), 0.0, 0.02, bf16, device)
     wb = sbp.SbpTensor((H, F), bf16, sbp.B, [Wb] * k)
     dw_s = sbp.empty_global((H, F), bf16, sbp.S(0), k, device=device)
-    avg, best = time_op(lambda: sbp.sbp_matmul(xs, dy, dw_s, sbp.SBP_TRANS_X), device, iters=5)
-    res.append(_tensor_entry("DP layer backward dW = X^T dY, (S(1),S(0))->S(0) fused", flops, avg, best, peaks))
+    avg, best, form = time_mm(sbp, lambda: sbp.sbp_matmul(xs, dy, dw_s, sbp.SBP_TRANS_X), device)
+    res.append(_tensor_entry("DP layer backward dW = X^T dY, (S(1),S(0))->S(0) fused", flops, avg, best, peaks, form))
     dw_b = sbp.empty_global((H, F), bf16, sbp.B, k, device=device)
-    avg, best = time_op(lambda: sbp.sbp_matmul(xs, dy, dw_b, sbp.SBP_TRANS_X), device, iters=5)
-    res.append(_tensor_entry("DP layer backward dW = X^T dY, (S(1),S(0))->B fused (8 replicas written)", flops, avg, best, peaks))
+    avg, best, form = time_mm(sbp, lambda: sbp.sbp_matmul(xs, dy, dw_b, sbp.SBP_TRANS_X), device)
+    res.append(_tensor_entry("DP layer backward dW = X^T dY, (S(1),S(0))->B fused (8 replicas written)", flops, avg, best, peaks, form))
     del dw_b
     dx = sbp.empty_global((M, H), bf16, sbp.S(0), k, device=device)
-    avg, best = time_op(lambda: sbp.sbp_matmul(dy, wb, dx, sbp.SBP_TRANS_W), device, iters=5)
-    res.append(_tensor_entry("DP layer backward dX = dY W^T, (S(0),B)->S(0)", flops, avg, best, peaks))
+    avg, best, form = time_mm(sbp, lambda: sbp.sbp_matmul(dy, wb, dx, sbp.SBP_TRANS_W), device)
+    res.append(_tensor_entry("DP layer backward dX = dY W^T, (S(0),B)->S(0)", flops, avg, best, peaks, form))
     return res
 
 
@@ -457,8 +467,8 @@ def section_classifier_gemm(sbp, device, peaks, opts):
                       [dg.normal(1004, 40 + r, (feat, classes // k), 0.0, 0.01, bf16, device) for r in range(k)])
     z = sbp.empty_global((rows, classes), bf16, sbp.S(1), k, device=device)
     ws = torch.empty(max(1, sbp.sbp_matmul_workspace_bytes(f, w, z)), dtype=torch.uint8, device=device)
-    avg, best = time_op(lambda: sbp.sbp_matmul(f, w, z, 0, ws), device, iters=5)
-    e = _tensor_entry("classifier GEMM (B,S(1))->S(1), bf16 logits", 2.0 * rows * feat * classes, avg, best, peaks)
+    avg, best, form = time_mm(sbp, lambda: sbp.sbp_matmul(f, w, z, 0, ws), device)
+    e = _tensor_entry("classifier GEMM (B,S(1))->S(1), bf16 logits", 2.0 * rows * feat * classes, avg, best, peaks, form)
     nbytes = feat * classes * 2 + rows * classes * 2 + rows * feat * 2
     e["hbm_gbs"] = nbytes / (avg * 1e-3) / 1e9
     e["hbm_frac_measured"] = e["hbm_gbs"] / peaks["hbm_gbs"]
@@ -468,9 +478,9 @@ def section_classifier_gemm(sbp, device, peaks, opts):
     loss = sbp.empty_global((rows,), torch.float32, sbp.B, k, device=device)
     del z
     ws2 = torch.empty(sbp.sbp_matmul_softmax_xent_workspace_bytes(f, w), dtype=torch.uint8, device=device)
-    avg, best = time_op(lambda: sbp.sbp_matmul_softmax_xent(f, w, lab, loss, None, None, ws2), device, iters=5)
+    avg, best, form = time_mm(sbp, lambda: sbp.sbp_matmul_softmax_xent(f, w, lab, loss, None, None, ws2), device)
     e2 = _tensor_entry("classifier GEMM fused with softmax-xent (no logits stored)", 2.0 * rows * feat * classes,
-                       avg, best, peaks, {"loss_mean": float(loss.locals[0].mean().item())})
+                       avg, best, peaks, dict(form, loss_mean=float(loss.locals[0].mean().item())))
     nbytes2 = feat * classes * 2 + rows * feat * 2
     e2["hbm_gbs"] = nbytes2 / (avg * 1e-3) / 1e9
     e2["hbm_frac_measured"] = e2["hbm_gbs"] / peaks["hbm_gbs"]
@@ -479,9 +489,9 @@ def section_classifier_gemm(sbp, device, peaks, opts):
     rsum = sbp.empty_global((rows,), torch.float32, sbp.B, k, device=device)
     sbp.sbp_matmul_softmax_xent(f, w, lab, loss, rmax, rsum, ws2)
     grad = sbp.empty_global((rows, classes), bf16, sbp.S(1), k, device=device)
-    avg, best = time_op(lambda: sbp.sbp_matmul_softmax_xent_backward(f, w, lab, rmax, rsum, grad), device, iters=5)
+    avg, best, form = time_mm(sbp, lambda: sbp.sbp_matmul_softmax_xent_backward(f, w, lab, rmax, rsum, grad), device)
     e3 = _tensor_entry("classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)",
-                       2.0 * rows * feat * classes, avg, best, peaks)
+                       2.0 * rows * feat * classes, avg, best, peaks, form)
     e3["hbm_gbs"] = nbytes / (avg * 1e-3) / 1e9
     e3["hbm_frac_measured"] = e3["hbm_gbs"] / peaks["hbm_gbs"]
     return [e, e2, e3]
@@ -562,10 +572,10 @@ def section_cliffs(sbp, device, peaks, opts):
         w = sbp.SbpTensor((K, N), bf16, sbp.S(1), [dg.normal(1003, 80 + r, (K, width), 0.0, 0.02, bf16, device) for r in range(k)])
         y = sbp.empty_global((M, N), bf16, sbp.S(1), k, device=device)
         ws = torch.empty(max(1, sbp.sbp_matmul_workspace_bytes(x, w, y)), dtype=torch.uint8, device=device)
-        avg, best = time_op(lambda: sbp.sbp_matmul(x, w, y, 0, ws), device, iters=5)
+        avg, best, form = time_mm(sbp, lambda: sbp.sbp_matmul(x, w, y, 0, ws), device)
         res.append(_tensor_entry(f"bf16 product (B,S(1))->S(1), [8192,4096] x [4096,{N}], shard width {width}"
                                  + ("" if width % 8 == 0 else " (not a multiple of 8)"),
-                                 2.0 * M * K * N, avg, best, peaks, kernel=None))
+                                 2.0 * M * K * N, avg, best, peaks, form, kernel=None))
         del w, y, ws
     del x, X
     torch.cuda.empty_cache()

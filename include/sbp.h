@@ -312,6 +312,27 @@ size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, cons
  * same buffers.  This reports how many were re-used and how many encoded since the library was
  * loaded (process-wide), so that a harness can check that a steady-state call encodes nothing. */
 void sbp_tensor_map_stats(uint64_t* reused, uint64_t* encoded);
+/* The tensor-core kernel has two compiled forms: CTA pairs that own 256 x 256 tiles of the result
+ * with a spare accumulator, so that a tile's epilogue runs under the next tile's MMAs ("square"),
+ * and pairs that own 512 x 256 tiles with both accumulators in use ("tall": less operand traffic per
+ * MMA, the epilogue exposed).  The library picks per product, from the tile count, the length of
+ * the contraction and the epilogue, one of: square; tall; or a mixed run -- whole waves of tall
+ * tiles, then the rest of the result in the square form as a second launch.  The results do not
+ * depend on the choice (same accumulation order per element).  This reports the launches since the
+ * library was loaded (process-wide): [0] square, [1] tall, [2] the square launch that ends a mixed run.
+ * sbp_matmul_set_form overrides the choice for tests and measurements (process-wide, not a tuning
+ * knob): form 0 = the library chooses, 1 = square, 2 = tall, 3 = mixed (where a product cannot run
+ * the forced form -- softmax epilogues, results written element-wise, fewer tiles than one wave
+ * for "mixed" -- it runs the nearest one that it can); max_pairs > 0 caps the CTA pairs of a
+ * launch (0 = all the device holds), which makes small products run many waves.  Until it is
+ * called, the environment variables SBP_TC_FORM = square | tall | mixed and SBP_TC_PAIRS, read
+ * once, give the same two values. */
+#define SBP_TC_FORM_AUTO 0
+#define SBP_TC_FORM_SQUARE 1
+#define SBP_TC_FORM_TALL 2
+#define SBP_TC_FORM_MIXED 3
+void sbp_matmul_set_form(int32_t form, int32_t max_pairs);
+void sbp_matmul_form_stats(uint64_t launches[3]);
 sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, uint32_t flags,
                       void* ws, size_t ws_bytes, void* cuda_stream);
 

@@ -114,6 +114,10 @@ def load_library():
     lib.sbp_matmul.argtypes = [T, T, T, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.sbp_tensor_map_stats.argtypes = [C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     lib.sbp_tensor_map_stats.restype = None
+    lib.sbp_matmul_set_form.argtypes = [C.c_int32, C.c_int32]
+    lib.sbp_matmul_set_form.restype = None
+    lib.sbp_matmul_form_stats.argtypes = [C.POINTER(C.c_uint64)]
+    lib.sbp_matmul_form_stats.restype = None
     lib.sbp_softmax_xent_workspace_bytes.restype = C.c_size_t
     lib.sbp_softmax_xent_workspace_bytes.argtypes = [T]
     lib.sbp_softmax_xent.argtypes = [T, T, T, T, T, C.c_void_p, C.c_size_t, C.c_void_p]
@@ -280,6 +284,21 @@ def sbp_tensor_map_stats():
     a, b = C.c_uint64(), C.c_uint64()
     load_library().sbp_tensor_map_stats(C.byref(a), C.byref(b))
     return int(a.value), int(b.value)
+
+
+SBP_TC_FORM_AUTO, SBP_TC_FORM_SQUARE, SBP_TC_FORM_TALL, SBP_TC_FORM_MIXED = 0, 1, 2, 3
+
+
+def sbp_matmul_set_form(form: int = 0, max_pairs: int = 0) -> None:
+    """Test and measurement override of the tensor-core kernel's form and CTA-pair count."""
+    load_library().sbp_matmul_set_form(int(form), int(max_pairs))
+
+
+def sbp_matmul_form_stats():
+    """Launches of the tensor-core kernel by form: (square, tall, square part of a mixed run)."""
+    v = (C.c_uint64 * 3)()
+    load_library().sbp_matmul_form_stats(v)
+    return int(v[0]), int(v[1]), int(v[2])
 
 
 def sbp_selftest_debug_bounds(buf: torch.Tensor, stream=None) -> None:

@@ -25,6 +25,8 @@ sbp_status check_xent_outputs(const sbp_tensor* labels, const sbp_tensor* loss, 
 size_t xent_finish_stage_floats(long long rows);
 size_t matmul_tc_workspace_bytes(const MatmulPlan& plan);
 void tensor_map_cache_stats(unsigned long long* hits, unsigned long long* encodes);
+void tc_form_stats(unsigned long long out[3]);
+void tc_set_form(int form, int max_pairs);
 
 __device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f)); }
 
@@ -542,6 +544,15 @@ void sbp_tensor_map_stats(uint64_t* reused, uint64_t* encoded) {
   tensor_map_cache_stats(&h, &e);
   if (reused) *reused = h;
   if (encoded) *encoded = e;
+}
+
+void sbp_matmul_set_form(int32_t form, int32_t max_pairs) { tc_set_form(form, max_pairs); }
+
+void sbp_matmul_form_stats(uint64_t launches[3]) {
+  unsigned long long v[3] = {0, 0, 0};
+  tc_form_stats(v);
+  if (launches)
+    for (int i = 0; i < 3; ++i) launches[i] = v[i];
 }
 
 sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, uint32_t flags, void* ws,

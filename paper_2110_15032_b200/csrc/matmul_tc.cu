@@ -33,6 +33,7 @@
 #include <cuda_runtime.h>
 
 #include <algorithm>
+#include <atomic>
 #include <cstdlib>
 #include <mutex>
 #include <type_traits>
@@ -761,6 +762,42 @@ void tensor_map_cache_stats(unsigned long long* hits, unsigned long long* encode
   *encodes = g_map_encodes;
 }
 
+// launches of the kernel by form: square, tall, square over the halves that a mixed run leaves
+static std::atomic<unsigned long long> g_form_launches[3];
+
+// Overrides of the form choice and of the CTA pairs a launch may use (tests and measurements):
+// set by tc_set_form, else taken once from SBP_TC_FORM (square | tall | mixed) and SBP_TC_PAIRS.
+static std::atomic<int> g_forced_form{-1}, g_pair_cap{-1};
+
+static int forced_form() {
+  int v = g_forced_form.load();
+  if (v < 0) {
+    const char* e = getenv("SBP_TC_FORM");
+    v = e ? (e[0] == 's' ? 1 : (e[0] == 't' ? 2 : (e[0] == 'm' ? 3 : 0))) : 0;
+    g_forced_form.store(v);
+  }
+  return v;
+}
+
+static int pair_cap() {
+  int v = g_pair_cap.load();
+  if (v < 0) {
+    const char* e = getenv("SBP_TC_PAIRS");
+    v = e ? std::max(0, atoi(e)) : 0;
+    g_pair_cap.store(v);
+  }
+  return v;
+}
+
+void tc_set_form(int form, int max_pairs) {
+  g_forced_form.store(form >= 0 && form <= 3 ? form : 0);
+  g_pair_cap.store(max_pairs > 0 ? max_pairs : 0);
+}
+
+void tc_form_stats(unsigned long long out[3]) {
+  for (int i = 0; i < 3; ++i) out[i] = g_form_launches[i].load();
+}
+
 // 2-D row-major tensor [rows, cols] with leading dimension ld (elements), box [box_rows, box_cols].
 static bool make_map(CUtensorMap* map, const void* base, int esz, long long rows, long long cols, long long ld,
                      int box_rows, int box_cols) {
@@ -833,7 +870,10 @@ static sbp_status launch_tc_form(const TcParams* p, cudaStream_t st, int* capaci
     }
     pairs_on_device[dev] = clusters;
   }
-  const int max_pairs = pairs_on_device[dev];
+  // a cap on the pairs (test and measurement switch): a small one makes small products run many
+  // waves, and so take the mixed route
+  const int cap = pair_cap();
+  const int max_pairs = cap > 0 && cap < pairs_on_device[dev] ? cap : pairs_on_device[dev];
   if (capacity) *capacity = max_pairs;
   if (!p) return SBP_OK;
   const int pairs = p->total_tiles < max_pairs ? p->total_tiles : max_pairs;
@@ -842,6 +882,7 @@ static sbp_status launch_tc_form(const TcParams* p, cudaStream_t st, int* capaci
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return cuda_fail(e, "tensor-core matmul launch");
   count_launch();
+  g_form_launches[MH == 2 ? 1 : (p->half_split ? 2 : 0)]++;
   return SBP_OK;
 }
 
@@ -860,12 +901,13 @@ static sbp_status launch_tc(bool tall, bool a_trans, bool b_trans, const TcParam
 
 // Which form runs a product.  Times in microseconds per wave (one tile on every CTA pair), fitted
 // to this kernel's measured times on B200 under its power cap (the clock settles lower the busier
-// the tensor pipe is, which is why these are not clock counts):
-//   square form  0.428 per 64-deep K-block; the epilogue is hidden unless it is store-bound;
-//   tall form    0.69 per K-block for twice the rows, plus an exposed epilogue of about 9.
-// A run may be mixed: `tall_waves` full waves of tall tiles, then the rest of the walk in the
-// square form (two 256-row halves per walked tile) -- a last wave that only half fills the device
-// costs a whole tall wave otherwise.
+// the tensor pipe is -- about 1.6 GHz in the square form, 1.4 GHz in the tall one -- which is why
+// these are times and not clock counts):
+//   square form  0.427 per 64-deep K-block (680 clocks); the epilogue is hidden unless it is store-bound;
+//   tall form    0.727 per K-block (1024 clocks) for twice the rows, plus an exposed epilogue of about 3.5.
+// A run may be mixed: whole waves of tall tiles, then the rest of the walk in the square form (two
+// 256-row halves per walked tile) -- a last wave that only half fills the device costs a whole
+// tall wave otherwise.
 struct FormChoice {
   bool walk_tall;      // tiles are walked 512 rows at a time
   int tall_tiles;      // the first so many walked tiles run in the tall form
@@ -873,8 +915,8 @@ struct FormChoice {
 
 static FormChoice choose_form(long long tiles_sq, long long tiles_tall, long long kb, int cap_sq, int cap_tall, bool gelu, int n_rep,
                               bool out_f32, int forced) {
-  const double wave_sq = 0.428 * kb + 0.5 + (gelu ? 1.0 : 0.0) + 1.5 * n_rep + (out_f32 ? 1.0 : 0.0);
-  const double wave_tall = 0.69 * kb + 9.0 + (gelu ? 6.0 : 0.0) + 3.0 * n_rep + (out_f32 ? 4.0 : 0.0);
+  const double wave_sq = 0.427 * kb + (gelu ? 1.0 : 0.0) + 1.1 * n_rep + (out_f32 ? 1.0 : 0.0);
+  const double wave_tall = 0.727 * kb + 3.5 + (gelu ? 8.5 : 0.0) + 2.2 * n_rep + (out_f32 ? 3.0 : 0.0);
   const double kRelaunch = 3.0;
   auto waves = [](long long tiles, int cap) { return (double)((tiles + cap - 1) / cap); };
   const double cost_sq = waves(tiles_sq, cap_sq) * wave_sq;
@@ -973,17 +1015,13 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
     tiles_sq += (plan.m[g] + BM - 1) / BM * tn;
     tiles_tall += (plan.m[g] + 2 * BM - 1) / (2 * BM) * tn;
   }
-  static const int forced_env = [] {
-    const char* e = getenv("SBP_TC_FORM");     // "square" / "tall" / "mixed": for measurements; the default chooses
-    return e ? (e[0] == 's' ? 1 : (e[0] == 't' ? 2 : (e[0] == 'm' ? 3 : 0))) : 0;
-  }();
   FormChoice form{false, 0};
   if (!xf && !y_direct && tiles_tall > 0 && tiles_sq <= 0x1fffffffLL) {
     int cap_sq = 0, cap_tall = 0;
     sbp_status qs = launch_tc(false, plan.a_trans, plan.b_trans, nullptr, st, &cap_sq);
     if (qs == SBP_OK) qs = launch_tc(true, plan.a_trans, plan.b_trans, nullptr, st, &cap_tall);
     if (qs != SBP_OK) return qs;
-    form = choose_form(tiles_sq, tiles_tall, kb_tile, cap_sq, cap_tall, plan.gelu != 0, plan.n_rep, plan.out_dtype == SBP_F32, forced_env);
+    form = choose_form(tiles_sq, tiles_tall, kb_tile, cap_sq, cap_tall, plan.gelu != 0, plan.n_rep, plan.out_dtype == SBP_F32, forced_form());
   }
   const int tile_m = form.walk_tall ? 2 * BM : BM;
   p.walk_m = tile_m;

@@ -312,12 +312,12 @@ def time_op(fn, device, iters=10, warmup=3):
 
 
 def time_mm(sbp, fn, device, iters=5):
-    """time_op for a tensor-core product, plus the form(s) of the kernel that one call launches."""
+    """time_op for a tensor-core product, plus the route the library takes for it (which compiled
+    form(s) of the kernel its calls launched, from the library's own launch counters)."""
     before = sbp.sbp_matmul_form_stats()
-    fn()
+    avg, best = time_op(fn, device, iters=iters)
     d = [a - b for a, b in zip(sbp.sbp_matmul_form_stats(), before)]
     form = "mixed" if d[2] else ("tall" if d[1] else ("square" if d[0] else "none"))
-    avg, best = time_op(fn, device, iters=iters)
     return avg, best, {"form": form}
 
 

@@ -180,15 +180,17 @@ NCU_TRAFFIC = {
     "softmax-xent backward (softmax - onehot, S(1))": 2099.7e6,
     # profiles/matmul_tc_classifier_bf16_512x512x1048576_k8.md (full size)
     "classifier GEMM (B,S(1))->S(1), bf16 logits": 2104.7e6,
-    "classifier GEMM fused with softmax-xent (no logits stored)": 1126.3e6 + 50.5e6,
-    "classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)": 2105.3e6,
-    # profiles/matmul_tc_mlp_bf16_8192x4096x16384_k8.md (full size)
-    "MLP GEMM1 (B,S(1))->S(1) + GeLU": 993.0e6,
-    "MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials": 911.1e6,
-    "MLP GEMM2 fused (S(1),S(0))->B": 1732.5e6,
-    "DP layer backward dW = X^T dY, (S(1),S(0))->S(0) fused": 2459.8e6,
-    "DP layer backward dW = X^T dY, (S(1),S(0))->B fused (8 replicas written)": 2091.0e6,
-    "DP layer backward dX = dY W^T, (S(0),B)->S(0)": 1502.6e6,
+    "classifier GEMM fused with softmax-xent (no logits stored)": 1126.9e6 + 50.5e6,
+    "classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)": 2104.2e6,
+    # profiles/matmul_tc_mlp_bf16_8192x4096x16384_k8.md (full size; a mixed run is the sum of its two launches)
+    "MLP GEMM1 (B,S(1))->S(1) + GeLU": 990.1e6,
+    "MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials": 1002.4e6,
+    "MLP GEMM2 fused (S(1),S(0))->B": 1196.7e6 + 193.2e6,
+    "MLP GEMM1 with W1 stored transposed (SBP_TRANS_W) + GeLU": 992.9e6,
+    "MLP GEMM2 fused (S(1),S(0))->B with W2 stored transposed (SBP_TRANS_W)": 1196.6e6 + 193.2e6,
+    "DP layer backward dW = X^T dY, (S(1),S(0))->S(0) fused": 875.0e6,
+    "DP layer backward dW = X^T dY, (S(1),S(0))->B fused (8 replicas written)": 1777.2e6,
+    "DP layer backward dX = dY W^T, (S(0),B)->S(0)": 748.2e6 + 205.0e6,
     # profiles/extras_bf16_8192x8192_p4_and_embedding_fp32_4194304x128_batch16384_k8.md (full size)
     "S(0)->P(sum) bf16 [8192,8192] k=4": 619.4e6,
     "B->P(sum) bf16 [8192,8192] k=4": 611.7e6,
@@ -203,9 +205,11 @@ NCU_TRAFFIC = {
     "embedding fused gather -> B (8 replicas written)": 7308.8e6,
     "embedding fused gather -> B (replicas aliased, 1 write)": 1093.3e6,
 }
-# The commit whose kernels the captures above were taken on.  A kernel that changes afterwards gets
-# its entry set to None (or recaptured) in the same commit: a stale figure is worse than none.
-NCU_TRAFFIC_CAPTURED_AT = "a61a16e"
+# The commits whose kernels the captures above were taken on (the tensor-core MatMul lines were
+# taken again after the kernel got its tall and mixed forms; the other kernels have not changed
+# since the first).  A kernel that changes afterwards gets its entry set to None (or recaptured)
+# in the same commit: a stale figure is worse than none.
+NCU_TRAFFIC_CAPTURED_AT = "a61a16e (boxing, softmax, embedding); ce7b3e3 (matmul_tc_kernel)"
 
 
 def ncu_traffic(name):

@@ -233,8 +233,9 @@ def e2e_sweep(sbp, src, work, device, steps, dist):
         hd = sbp.SbpTensor(d.shape, d.dtype, d.sig,
                            [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in d.locals])
         jobs.append((hs, hd))
-        h2d += sum(t.numel() * t.element_size() for t in hs.locals)
-        d2h += sum(t.numel() * t.element_size() for t in hd.locals)
+        a, b = sbp.sbp_boxing_host_copy_bytes(hs, hd)      # what the call really copies (B -> S(i): one block per replica)
+        h2d += a
+        d2h += b
         ws_bytes = max(ws_bytes, sbp.sbp_boxing_host_workspace_bytes(hs, hd))
     # Four streams, each with its own device workspace: consecutive transforms go round them, so
     # the device->host copies of some overlap the host->device copies of others (measured: 55 ms a

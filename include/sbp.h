@@ -216,8 +216,15 @@ sbp_status sbp_boxing_shard(const sbp_tensor* src, sbp_tensor* dst, int32_t dst_
 /* Same transform, but every local[] pointer of src_host and dst_host is a HOST pointer
  * (pinned memory recommended).  The source local tensors are copied to the device
  * workspace, transformed there and the destination local tensors copied back, all
- * enqueued on cuda_stream.  dev_ws must hold sbp_boxing_host_workspace_bytes() bytes. */
+ * enqueued on cuda_stream.  dev_ws must hold sbp_boxing_host_workspace_bytes() bytes.
+ * Only what the transform reads crosses to the device: for B -> S(i) on equal placements that is,
+ * of source replica r, the block that becomes shard r (Table 2: B -> S moves no data between
+ * devices); every other transform reads all of every source local tensor.  Destination replicas
+ * that share one host pointer are copied back once.  sbp_boxing_host_copy_bytes reports the bytes a
+ * call copies in each direction (host pointers are only compared, never dereferenced). */
 size_t sbp_boxing_host_workspace_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_host);
+sbp_status sbp_boxing_host_copy_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_host, uint64_t* h2d_bytes,
+                                      uint64_t* d2h_bytes);
 sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, void* dev_ws,
                            size_t dev_ws_bytes, void* cuda_stream);
 

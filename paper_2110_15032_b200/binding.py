@@ -103,6 +103,7 @@ def load_library():
     lib.sbp_boxing_host_workspace_bytes.restype = C.c_size_t
     lib.sbp_boxing_host_workspace_bytes.argtypes = [T, T]
     lib.sbp_boxing_host.argtypes = [T, T, C.c_void_p, C.c_size_t, C.c_void_p]
+    lib.sbp_boxing_host_copy_bytes.argtypes = [T, T, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
     lib.sbp_boxing_set_copy_engine.argtypes = [C.c_int32]
     lib.sbp_boxing_set_copy_engine.restype = None
     lib.sbp_check_device_errors.argtypes = []
@@ -341,6 +342,14 @@ def sbp_boxing_shard(src: SbpTensor, dst: SbpTensor, dst_shard: int, stream=None
 def sbp_boxing_host_workspace_bytes(src_host: SbpTensor, dst_host: SbpTensor) -> int:
     a, b = src_host._c(), dst_host._c()
     return int(load_library().sbp_boxing_host_workspace_bytes(C.byref(a), C.byref(b)))
+
+
+def sbp_boxing_host_copy_bytes(src_host: SbpTensor, dst_host: SbpTensor):
+    """(host->device, device->host) bytes that one sbp_boxing_host call copies."""
+    a, b = src_host._c(), dst_host._c()
+    h2d, d2h = C.c_uint64(), C.c_uint64()
+    _check(load_library().sbp_boxing_host_copy_bytes(C.byref(a), C.byref(b), C.byref(h2d), C.byref(d2h)))
+    return int(h2d.value), int(d2h.value)
 
 
 def sbp_boxing_host(src_host: SbpTensor, dst_host: SbpTensor, dev_ws: torch.Tensor, stream=None) -> None:

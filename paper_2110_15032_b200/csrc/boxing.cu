@@ -773,6 +773,51 @@ size_t sbp_boxing_host_workspace_bytes(const sbp_tensor* src_host, const sbp_ten
   return total;
 }
 
+// B -> S(axis) on equal one-axis placements reads, of source replica r, only the block that becomes
+// destination shard r: the host path copies that block alone.  Geometry of replica r's block as a
+// pitched 2-D copy: `outer` rows of `width` bytes, `pitch` bytes apart, starting at byte `offset`.
+struct HostBlock {
+  size_t offset, pitch, width, outer;
+};
+
+static bool host_copy_is_diagonal(const sbp_tensor* src, const sbp_tensor* dst) {
+  return src->pdims <= 1 && dst->pdims <= 1 && placement_k(src) == placement_k(dst) && src->dtype == dst->dtype &&
+         src->sbp[0].kind == SBP_BROADCAST && dst->sbp[0].kind == SBP_SPLIT;
+}
+
+static HostBlock host_diagonal_block(const sbp_tensor* src, int axis, int r) {
+  int64_t start = 0, len = 0;
+  split_range(src->shape[axis], placement_k(src), r, &start, &len);
+  size_t outer = 1, inner = (size_t)elem_size(src->dtype);
+  for (int d = 0; d < axis; ++d) outer *= (size_t)src->shape[d];
+  for (int d = axis + 1; d < src->ndim; ++d) inner *= (size_t)src->shape[d];
+  return HostBlock{(size_t)start * inner, (size_t)src->shape[axis] * inner, (size_t)len * inner, outer};
+}
+
+sbp_status sbp_boxing_host_copy_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_host, uint64_t* h2d, uint64_t* d2h) {
+  sbp_status st = check_pair(src_host, dst_host, false);
+  if (st != SBP_OK) return st;
+  const int ks = placement_k(src_host), kd = placement_k(dst_host);
+  uint64_t in = 0, out = 0;
+  const bool diag = host_copy_is_diagonal(src_host, dst_host);
+  for (int r = 0; r < ks; ++r) {
+    if (diag) {
+      const HostBlock b = host_diagonal_block(src_host, dst_host->sbp[0].axis, r);
+      in += (uint64_t)b.width * b.outer;
+    } else {
+      in += (uint64_t)local_numel(src_host, r) * elem_size(src_host->dtype);
+    }
+  }
+  for (int r = 0; r < kd; ++r) {
+    bool dup = false;
+    for (int q = 0; q < r; ++q) dup = dup || dst_host->local[q] == dst_host->local[r];
+    if (!dup) out += (uint64_t)local_numel(dst_host, r) * elem_size(dst_host->dtype);
+  }
+  if (h2d) *h2d = in;
+  if (d2h) *d2h = out;
+  return SBP_OK;
+}
+
 sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, void* dev_ws, size_t dev_ws_bytes,
                            void* cuda_stream) {
   SBP_RANGE("sbp_boxing_host");
@@ -810,7 +855,17 @@ sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, voi
   if (s.pdims == 2 || d.pdims == 2) st = boxing_2d(&s, &d, cuda_stream, true);
   else st = boxing_one_axis(&s, &d, -1, cuda_stream, true);
   if (st != SBP_OK) return st;
+  const bool diag = host_copy_is_diagonal(src_host, dst_host);
   for (int r = 0; r < ks; ++r) {
+    if (diag) {
+      // the rest of this replica's device copy stays unwritten: the transform never reads it
+      const HostBlock b = host_diagonal_block(src_host, dst_host->sbp[0].axis, r);
+      if (b.width && b.outer)
+        SBP_CUDA_TRY(cudaMemcpy2DAsync(static_cast<char*>(s.local[r]) + b.offset, b.pitch,
+                                       static_cast<const char*>(src_host->local[r]) + b.offset, b.pitch, b.width, b.outer,
+                                       cudaMemcpyHostToDevice, stream));
+      continue;
+    }
     const size_t bytes = (size_t)local_numel(src_host, r) * esz;
     if (bytes) SBP_CUDA_TRY(cudaMemcpyAsync(s.local[r], src_host->local[r], bytes, cudaMemcpyHostToDevice, stream));
   }

@@ -285,6 +285,41 @@ def test_host_buffer_entry_point():
     assert e.value.name == "SBP_ERR_WORKSPACE"
 
 
+@pytest.mark.parametrize("shape,axis", [((130, 96), 0), ((128, 250), 1), ((6, 50, 10), 1), ((5, 7, 64), 2)])
+def test_host_entry_point_copies_only_the_blocks_b_to_s_reads(shape, axis):
+    """B -> S(axis) takes block r from replica r.  The host path sends only those blocks to the
+    device: everything outside replica r's own block is poisoned here (a different value in every
+    replica), so a result that matches the logical tensor shows that nothing else was read, and the
+    reported byte count is that of one tensor, not of k."""
+    k = 4
+    T = dg.normal(11, 0, shape, 0, 1, BF16)
+    want = split_cpu(T, sbp.S(axis), k)
+    src_cpu = []
+    for r in range(k):
+        rep = torch.full(shape, float(100 + r), dtype=BF16)
+        lo = sum(w.shape[axis] for w in want[:r])
+        idx = [slice(None)] * len(shape)
+        idx[axis] = slice(lo, lo + want[r].shape[axis])
+        rep[tuple(idx)] = T[tuple(idx)]
+        src_cpu.append(rep.pin_memory())
+    src = sbp.SbpTensor(shape, BF16, sbp.B, src_cpu)
+    dst_cpu = [torch.empty(w.shape, dtype=BF16).pin_memory() for w in want]
+    dst = sbp.SbpTensor(shape, BF16, sbp.S(axis), dst_cpu)
+    h2d, d2h = sbp.sbp_boxing_host_copy_bytes(src, dst)
+    assert h2d == T.numel() * 2 and d2h == T.numel() * 2
+    ws = torch.empty(sbp.sbp_boxing_host_workspace_bytes(src, dst), dtype=torch.uint8, device="cuda")
+    ws.fill_(0x5A)
+    sbp.sbp_boxing_host(src, dst, ws)
+    torch.cuda.synchronize()
+    for r in range(k):
+        assert torch.equal(dst_cpu[r], want[r]), f"shard {r}"
+    # every other transform still copies all of its sources, and aliased destination replicas go back once
+    psrc = sbp.SbpTensor(shape, BF16, sbp.P_SUM, src_cpu)
+    one = torch.empty(shape, dtype=BF16).pin_memory()
+    h2d, d2h = sbp.sbp_boxing_host_copy_bytes(psrc, sbp.SbpTensor(shape, BF16, sbp.B, [one] * k))
+    assert h2d == k * T.numel() * 2 and d2h == T.numel() * 2
+
+
 def test_expired_device_wait_is_reported_and_the_device_stays_usable():
     """A bounded wait that runs out (a barrier nothing signals) ends the kernel normally and is
     reported once as SBP_ERR_TIMEOUT; nothing faults and later launches work."""

@@ -91,6 +91,7 @@ struct TcParams {
   int ngroups, nseg, chain, gelu, n_rep;
   int out_f32;
   int total_tiles;
+  unsigned panel_magic[SBP_MAX_K];   // floor(2^32 / (kPanelM * n-tiles)) of the group (stacked walks: entry 0, of the whole list)
   int walk_m;                   // rows of a walked tile: 256, or 512 (tall form and the square remainder of a mixed run)
   int tile_first;               // index of the first walked tile of this launch
   int half_split;               // square form over 512-row walked tiles: launch tile 2t + h is m-half h of walked tile t
@@ -228,14 +229,16 @@ __device__ __forceinline__ void tmem_ld32(unsigned taddr, float* v) {
       : "memory");
 }
 
-// Shared-memory matrix descriptor, 128-byte swizzle.  lbo / sbo in bytes.
-__device__ __forceinline__ unsigned long long smem_desc(unsigned addr, unsigned lbo, unsigned sbo) {
-  unsigned long long d = 0;
-  d |= (unsigned long long)((addr & 0x3FFFF) >> 4);
-  d |= (unsigned long long)(lbo >> 4) << 16;
-  d |= (unsigned long long)(sbo >> 4) << 32;
-  d |= 1ull << 46;   // descriptor version of this architecture
-  d |= 2ull << 61;   // 128-byte swizzle
+// Shared-memory matrix descriptor, 128-byte swizzle (lbo / sbo in bytes): bits 0-13 start address
+// >> 4, bits 16-29 lbo >> 4, bits 32-45 sbo >> 4, bit 46 the descriptor version of this architecture,
+// bits 61-63 = 2 the 128-byte swizzle.  It is handled in two parts: what never changes (the high
+// word, and the leading-dimension field of the low word) and the start-address field, so that the
+// MMA-issuing thread builds a descriptor with one add and one register pair.
+__host__ __device__ constexpr unsigned desc_lo_fixed(unsigned lbo) { return (lbo >> 4) << 16; }
+__host__ __device__ constexpr unsigned desc_hi_fixed(unsigned sbo) { return (sbo >> 4) | (1u << 14) | (2u << 29); }
+__device__ __forceinline__ unsigned long long desc_pack(unsigned lo, unsigned hi) {
+  unsigned long long d;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(d) : "r"(lo), "r"(hi));
   return d;
 }
 
@@ -277,6 +280,19 @@ struct TileCoord {
 // columns in L2.
 constexpr int kPanelM = 8;
 
+// n / d for 0 <= n < 2^31 and d >= 2 with magic = floor(2^32 / d): the high product is short of the
+// quotient by at most one or two, which the loop makes up.  (The tile walk divides twice per tile
+// in each of three roles; the generic division is a few hundred clocks of the one thread that
+// issues the MMAs.)
+__device__ __forceinline__ int div_by(int n, int d, unsigned magic) {
+  int q = (int)__umulhi((unsigned)n, magic);
+  while (n - q * d >= d) ++q;
+  return q;
+}
+
+// position inside a panel of pm m-tiles: pm is kPanelM everywhere but in a group's last panel
+__device__ __forceinline__ int div_panel(int rem, int pm) { return pm == kPanelM ? rem / kPanelM : rem / pm; }
+
 __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
   int half_m = 0;
   if (p.half_split) {
@@ -288,10 +304,10 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
     // The same for a fused product written as S(1): column blocks of one result, which share every
     // A row block; the n-tiles of all groups form one list.
     const int tm = p.tiles_m[0], tn = p.mt_begin[p.ngroups];
-    const int panel = tile / (kPanelM * tn);
+    const int panel = div_by(tile, kPanelM * tn, p.panel_magic[0]);
     const int rem = tile - panel * (kPanelM * tn);
     const int pm = min(kPanelM, tm - panel * kPanelM);
-    const int nt = rem / pm, mt = panel * kPanelM + (rem - nt * pm);
+    const int nt = div_panel(rem, pm), mt = panel * kPanelM + (rem - nt * pm);
     int g = 0;
     while (g + 1 < p.ngroups && nt >= p.mt_begin[g + 1]) ++g;
     return TileCoord{g, mt * p.walk_m + half_m, (nt - p.mt_begin[g]) * BN};
@@ -301,10 +317,10 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
     // B column block.  Walking them one after the other would stream the whole B operand once per
     // group; instead the m-tiles of all groups form one list and the panel walk runs over that.
     const int tm = p.mt_begin[p.ngroups], tn = p.tiles_n[0];
-    const int panel = tile / (kPanelM * tn);
+    const int panel = div_by(tile, kPanelM * tn, p.panel_magic[0]);
     const int rem = tile - panel * (kPanelM * tn);
     const int pm = min(kPanelM, tm - panel * kPanelM);
-    const int nt = rem / pm, mt = panel * kPanelM + (rem - nt * pm);
+    const int nt = div_panel(rem, pm), mt = panel * kPanelM + (rem - nt * pm);
     int g = 0;
     while (g + 1 < p.ngroups && mt >= p.mt_begin[g + 1]) ++g;
     return TileCoord{g, (mt - p.mt_begin[g]) * p.walk_m + half_m, nt * BN};
@@ -313,10 +329,10 @@ __device__ __forceinline__ TileCoord tile_coord(const TcParams& p, int tile) {
   while (g + 1 < p.ngroups && tile >= p.tile_begin[g + 1]) ++g;
   const int local = tile - p.tile_begin[g];
   const int tm = p.tiles_m[g], tn = p.tiles_n[g];
-  const int panel = local / (kPanelM * tn);
+  const int panel = div_by(local, kPanelM * tn, p.panel_magic[g]);
   const int rem = local - panel * (kPanelM * tn);
   const int pm = min(kPanelM, tm - panel * kPanelM);   // m-tiles in this (possibly last) panel
-  const int nt = rem / pm, mt = panel * kPanelM + (rem - nt * pm);
+  const int nt = div_panel(rem, pm), mt = panel * kPanelM + (rem - nt * pm);
   return TileCoord{g, mt * p.walk_m + half_m, nt * BN};
 }
 
@@ -377,14 +393,18 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
   if (warp == 0) {
     // ------------------------------------------------ producer (both CTAs)
     if (lane == 0) {
+      // ring position kept as (slot, round parity) and stepped, not divided out of a running count:
+      // with five slots the division is a long instruction sequence, once per K-block
       long long kb_iter = 0;
+      int slot = 0;
+      unsigned round = 0;
       for (int tile = first; tile < p.total_tiles && !*abort_flag; tile += stride) {
         const TileCoord tc = tile_coord(p, tile);
         const int s_lo = p.chain ? 0 : tc.g, s_hi = p.chain ? p.nseg : tc.g + 1;
         for (int s = s_lo; s < s_hi; ++s) {
-          for (int kb = 0; kb < p.kblocks[s]; ++kb, ++kb_iter) {
-            const int slot = (int)(kb_iter % kSt);
-            const unsigned parity = (unsigned)(((kb_iter / kSt) & 1) ^ 1);
+          const int nkb = p.kblocks[s];
+          for (int kb = 0; kb < nkb; ++kb, ++kb_iter, slot = slot + 1 == kSt ? 0 : slot + 1, round ^= (slot == 0)) {
+            const unsigned parity = round ^ 1;
             if (!mbar_wait(smem_addr(&bar_empty[slot]), parity, abort_flag)) goto producer_done;
             const unsigned full0 = map_to_cta(smem_addr(&bar_full[slot]), 0);
             if (rank == 0) mbar_expect_tx(smem_addr(&bar_full[slot]), 2 * kStBytes);
@@ -427,7 +447,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
   } else if (warp == 1) {
     // ------------------------------------------------ MMA issuer (first CTA of the pair only)
     if (lane == 0 && rank == 0) {
-      long long kb_iter = 0;
+      int slot = 0;
+      unsigned round = 0;
       int tile_iter = 0;
       constexpr unsigned idesc = make_idesc(AT, BT);
       for (int tile = first; tile < p.total_tiles && !*abort_flag; tile += stride, ++tile_iter) {
@@ -443,9 +464,9 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
         unsigned accumulate = 0;
         bool ok = true;
         for (int s = s_lo; s < s_hi && ok; ++s) {
-          for (int kb = 0; kb < p.kblocks[s]; ++kb, ++kb_iter) {
-            const int slot = (int)(kb_iter % kSt);
-            if (!mbar_wait(smem_addr(&bar_full[slot]), (unsigned)((kb_iter / kSt) & 1), abort_flag)) {
+          const int nkb = p.kblocks[s];
+          for (int kb = 0; kb < nkb; ++kb, slot = slot + 1 == kSt ? 0 : slot + 1, round ^= (slot == 0)) {
+            if (!mbar_wait(smem_addr(&bar_full[slot]), round, abort_flag)) {
               ok = false;
               break;
             }
@@ -470,10 +491,12 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
               // MN-major tile (B as given, A transposed): 64-element chunks of the M / N index
               //    BK*128 bytes apart, 8-row K groups 1024 bytes apart; 16 K-rows = 2048 bytes.
               // Each CTA holds its 128 of the pair's 256 rows (A) or columns (B).
-              const unsigned long long da =
-                  AT ? smem_desc(sa + kk * 2048, BK * 128, 1024) : smem_desc(sa + kk * 32, 16, 1024);
-              const unsigned long long db =
-                  BT ? smem_desc(sb + kk * 32, 16, 1024) : smem_desc(sb + kk * 2048, BK * 128, 1024);
+              // (shared-memory addresses are below 256 KiB and the tiles 1024-byte aligned, so the
+              //  start-address field is address >> 4 and stepping it cannot carry out of the field)
+              constexpr unsigned a_lo = desc_lo_fixed(AT ? BK * 128 : 16), b_lo = desc_lo_fixed(BT ? 16 : BK * 128);
+              constexpr unsigned hi = desc_hi_fixed(1024);
+              const unsigned long long da = desc_pack(a_lo + (sa >> 4) + kk * (AT ? 128 : 2), hi);
+              const unsigned long long db = desc_pack(b_lo + (sb >> 4) + kk * (BT ? 2 : 128), hi);
               umma_bf16(d_tmem, da, db, idesc, kk == 0 ? accumulate : 1u);
             }
             }
@@ -1059,6 +1082,10 @@ sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaSt
   for (int g = 0; g < plan.ngroups; ++g) {
     const bool live = plan.m[g] > 0 && plan.n[g] > 0;
     p.mt_begin[g + 1] = p.mt_begin[g] + (live ? (p.stacked == 2 ? p.tiles_n[g] : p.tiles_m[g]) : 0);
+  }
+  for (int g = 0; g < plan.ngroups; ++g) {
+    const long long tn_walk = p.stacked == 2 ? p.mt_begin[plan.ngroups] : (p.stacked ? p.tiles_n[0] : p.tiles_n[g]);
+    p.panel_magic[g] = (unsigned)((1ull << 32) / (unsigned long long)(kPanelM * std::max(1LL, tn_walk)));
   }
   p.tile_begin[plan.ngroups] = tiles;
   for (int g = plan.ngroups + 1; g <= SBP_MAX_K; ++g) p.tile_begin[g] = tiles;

@@ -90,11 +90,12 @@ def test_library_choice_takes_each_form_on_a_whole_device():
     sbp.sbp_matmul_set_form(sbp.SBP_TC_FORM_AUTO, 0)
     # 2 x 3 square tiles: far less than a wave
     _sampled_product(600, 512, 520, 2001, (1, 0, 0))
-    # 48 tall tiles (one wave) against 96 square ones (two), long contraction
-    _sampled_product(3072, 6144, 2048, 2002, (0, 1, 0))
-    # 80 tall tiles: one whole wave, the other 6 as 12 halves in the square form
-    y = _sampled_product(4096, 8192, 2560, 2003, (0, 1, 1))
+    # 74 tall tiles (exactly one wave) against 148 square ones (two), 256 K-blocks per tile
+    _sampled_product(1024, 16384, 9472, 2002, (0, 1, 0))
+    # 240 tall tiles: three whole waves, the other 18 as 36 halves in the square form (against seven
+    # square waves, or four tall ones)
+    y = _sampled_product(8192, 16384, 3840, 2003, (0, 1, 1))
     # the same product as one square run: identical bits
     sbp.sbp_matmul_set_form(sbp.SBP_TC_FORM_SQUARE, 0)
-    y2 = _sampled_product(4096, 8192, 2560, 2003, (1, 0, 0))
+    y2 = _sampled_product(8192, 16384, 3840, 2003, (1, 0, 0))
     assert torch.equal(y.locals[0].view(torch.uint8), y2.locals[0].view(torch.uint8))

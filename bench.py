@@ -179,18 +179,18 @@ NCU_TRAFFIC = {
     "softmax-xent on bf16 logits (partial + combine)": 1077.2e6,
     "softmax-xent backward (softmax - onehot, S(1))": 2099.7e6,
     # profiles/matmul_tc_classifier_bf16_512x512x1048576_k8.md (full size)
-    "classifier GEMM (B,S(1))->S(1), bf16 logits": 2104.7e6,
-    "classifier GEMM fused with softmax-xent (no logits stored)": 1126.9e6 + 50.5e6,
-    "classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)": 2104.2e6,
+    "classifier GEMM (B,S(1))->S(1), bf16 logits": 2105.0e6,
+    "classifier GEMM fused with softmax-xent (no logits stored)": 1126.7e6 + 50.5e6,
+    "classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)": 2103.8e6,
     # profiles/matmul_tc_mlp_bf16_8192x4096x16384_k8.md (full size; a mixed run is the sum of its two launches)
-    "MLP GEMM1 (B,S(1))->S(1) + GeLU": 990.1e6,
-    "MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials": 1002.4e6,
-    "MLP GEMM2 fused (S(1),S(0))->B": 1196.7e6 + 193.2e6,
-    "MLP GEMM1 with W1 stored transposed (SBP_TRANS_W) + GeLU": 992.9e6,
-    "MLP GEMM2 fused (S(1),S(0))->B with W2 stored transposed (SBP_TRANS_W)": 1196.6e6 + 193.2e6,
-    "DP layer backward dW = X^T dY, (S(1),S(0))->S(0) fused": 875.0e6,
-    "DP layer backward dW = X^T dY, (S(1),S(0))->B fused (8 replicas written)": 1777.2e6,
-    "DP layer backward dX = dY W^T, (S(0),B)->S(0)": 748.2e6 + 205.0e6,
+    "MLP GEMM1 (B,S(1))->S(1) + GeLU": 972.7e6,
+    "MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials": 912.0e6,
+    "MLP GEMM2 fused (S(1),S(0))->B": 1196.3e6 + 193.5e6,
+    "MLP GEMM1 with W1 stored transposed (SBP_TRANS_W) + GeLU": 972.5e6,
+    "MLP GEMM2 fused (S(1),S(0))->B with W2 stored transposed (SBP_TRANS_W)": 1197.1e6 + 194.0e6,
+    "DP layer backward dW = X^T dY, (S(1),S(0))->S(0) fused": 874.6e6,
+    "DP layer backward dW = X^T dY, (S(1),S(0))->B fused (8 replicas written)": 1776.5e6,
+    "DP layer backward dX = dY W^T, (S(0),B)->S(0)": 748.5e6 + 205.5e6,
     # profiles/extras_bf16_8192x8192_p4_and_embedding_fp32_4194304x128_batch16384_k8.md (full size)
     "S(0)->P(sum) bf16 [8192,8192] k=4": 619.4e6,
     "B->P(sum) bf16 [8192,8192] k=4": 611.7e6,
@@ -209,7 +209,7 @@ NCU_TRAFFIC = {
 # taken again after the kernel got its tall and mixed forms; the other kernels have not changed
 # since the first).  A kernel that changes afterwards gets its entry set to None (or recaptured)
 # in the same commit: a stale figure is worse than none.
-NCU_TRAFFIC_CAPTURED_AT = "a61a16e (boxing, softmax, embedding); ce7b3e3 (matmul_tc_kernel)"
+NCU_TRAFFIC_CAPTURED_AT = "a61a16e (boxing, softmax, embedding); 4256f79 (matmul_tc_kernel)"
 
 
 def ncu_traffic(name):
@@ -238,8 +238,8 @@ def e2e_sweep(sbp, src, work, device, steps, dist):
         d2h += b
         ws_bytes = max(ws_bytes, sbp.sbp_boxing_host_workspace_bytes(hs, hd))
     # Four streams, each with its own device workspace: consecutive transforms go round them, so
-    # the device->host copies of some overlap the host->device copies of others (measured: 55 ms a
-    # step against 62 ms with two streams; the host->device direction, 2.55 GB a step, is the bound).
+    # the device->host copies of some overlap the host->device copies of others (measured: 44 ms a
+    # step with four streams or more; the host->device direction, 2.15 GB a step at 49 GB/s, is the bound).
     n_streams = int(os.environ.get("SBP_E2E_STREAMS", "4"))
     streams = [torch.cuda.Stream(device=device) for _ in range(n_streams)]
     wss = [torch.empty(ws_bytes, dtype=torch.uint8, device=device) for _ in streams]

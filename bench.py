@@ -656,7 +656,7 @@ def roofline_configs(per, ops):
         e = {"config": o["config"], "line": o["op"], "kernel": o.get("kernel"), "bound": o["bound"], "ms": o["ms"],
              "work": o.get("bytes", o.get("flops")), "achieved": o["achieved"], "unit": o["unit"],
              "frac": o["frac_measured"]}
-        for key in ("traffic", "achieved_dram", "frac_dram", "hbm_gbs", "hbm_frac_measured", "frac_sustained"):
+        for key in ("traffic", "achieved_dram", "frac_dram", "hbm_gbs", "hbm_frac_measured", "frac_sustained", "form"):
             if o.get(key) is not None:
                 e[key] = o[key]
         out.append(e)

@@ -174,7 +174,19 @@ __global__ void __launch_bounds__(256, MINB) embedding_kernel(const __grid_const
 // that a chunk starts on a row boundary and holds at most 256 lookups (one id per thread).
 template <typename V, int ESZ, int J>
 __global__ void __launch_bounds__(256) embedding_rows_kernel(const __grid_constant__ EmbParams p) {
-  __shared__ long long ids_s[2][256];
+  // Per lookup of the chunk: where its table row starts (null for an id outside the table).  The
+  // owner of an id -- a division by the shard size -- is worked out once per lookup by the thread
+  // that stages it, a chunk ahead, not by each of the row's 16-byte vectors on its way to the load.
+  __shared__ const char* rows_s[2][256];
+  auto resolve = [&](long long id) -> const char* {
+    if (id < 0 || id >= p.rows) {
+      if (p.oob && SBP_GUARD(p.oob, 4)) atomicAdd(p.oob, 1);
+      return nullptr;
+    }
+    long long start;
+    const int r = owner_of_row(id, p.base, p.rem, p.big, p.narrow, &start);
+    return p.table[r] + (id - start) * p.vpr * (long long)sizeof(V);
+  };
   const long long total = p.n_lookups * p.vpr;
   const long long n_chunks = (total + 256 * J - 1) / (256 * J);
 
@@ -195,7 +207,7 @@ __global__ void __launch_bounds__(256) embedding_rows_kernel(const __grid_consta
     int n_ids;
     span(chunk, &look0, &n_ids);
     if ((int)threadIdx.x < n_ids)
-      ids_s[0][threadIdx.x] = SBP_GUARD(p.ids[0] + look0 + threadIdx.x, 8) ? __ldcs(p.ids[0] + look0 + threadIdx.x) : -1;
+      rows_s[0][threadIdx.x] = resolve(SBP_GUARD(p.ids[0] + look0 + threadIdx.x, 8) ? __ldcs(p.ids[0] + look0 + threadIdx.x) : -1);
   }
   __syncthreads();
 
@@ -222,14 +234,9 @@ __global__ void __launch_bounds__(256) embedding_rows_kernel(const __grid_consta
       val[j] = zero_vec<V>();
       if (!ok[j]) continue;
       const long long look = item >> p.vpr_log2, col = item & (p.vpr - 1);
-      const long long id = ids_s[cur][look - look0];
-      if (id < 0 || id >= p.rows) {
-        if (p.oob && col == 0 && SBP_GUARD(p.oob, 4)) atomicAdd(p.oob, 1);
-        continue;
-      }
-      long long start;
-      const int r = owner_of_row(id, p.base, p.rem, p.big, p.narrow, &start);
-      const V* src = reinterpret_cast<const V*>(p.table[r]) + (id - start) * p.vpr + col;
+      const char* row = rows_s[cur][look - look0];
+      if (!row) continue;
+      const V* src = reinterpret_cast<const V*>(row) + col;
       if (SBP_GUARD(src, sizeof(V))) val[j] = __ldg(src);
     }
     V* o = reinterpret_cast<V*>(p.out[0]);
@@ -238,7 +245,7 @@ __global__ void __launch_bounds__(256) embedding_rows_kernel(const __grid_consta
       if (ok[j] && SBP_GUARD(o + cta_base + j * 256 + threadIdx.x, sizeof(V)))
         __stcs(o + cta_base + j * 256 + threadIdx.x, p.canon_neg_zero ? canon<V, ESZ>(val[j]) : val[j]);
 
-    if ((int)threadIdx.x < nn) ids_s[cur ^ 1][threadIdx.x] = nid;
+    if ((int)threadIdx.x < nn) rows_s[cur ^ 1][threadIdx.x] = resolve(nid);
     __syncthreads();
     cur ^= 1;
   }

@@ -626,7 +626,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
           if constexpr (MODE == 2) {
             float e;
             asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(x, 1.4426950408889634f, g_neg)));
-            return idx == lab_rel ? e - 1.0f : e;
+            return e;          // the label's column gets its -1 below, outside the per-element path
           } else if constexpr (MODE == 1) {
             return gelu_erf_tc(x);
           } else {
@@ -669,6 +669,29 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
                 h = __floats2bfloat162_rn(f[6], f[7]); o.w = *reinterpret_cast<unsigned*>(&h);
                 *reinterpret_cast<uint4*>(rowp + ((c ^ (lane & 7)) << 4)) = o;
               }
+            }
+            if constexpr (MODE == 2) {
+              // softmax - onehot: a row's label falls into this slab once in 2^14 slabs, so the -1 is
+              // not a compare and a select on every element but a rare fix-up: the column is read
+              // again from tensor memory (one row at a time, so the load stays warp-uniform) and the
+              // staged element rewritten with exp - 1 computed in fp32 as before.
+              unsigned hits = __ballot_sync(0xffffffffu, lab_rel >= 0);
+              while (hits) {
+                const int src_lane = __ffs(hits) - 1;
+                hits &= hits - 1;
+                const int col = __shfl_sync(0xffffffffu, lab_rel, src_lane);
+                unsigned bitsv;
+                asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];" : "=r"(bitsv) : "r"(taddr + sl * cols_per_slab + col) : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (lane == src_lane) {
+                  float e;
+                  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(fmaf(__uint_as_float(bitsv), 1.4426950408889634f, g_neg)));
+                  e -= 1.0f;
+                  if (p.out_f32) *reinterpret_cast<float*>(rowp + (((col >> 2) ^ (lane & 7)) << 4) + ((col & 3) << 2)) = e;
+                  else *reinterpret_cast<__nv_bfloat16*>(rowp + (((col >> 3) ^ (lane & 7)) << 4) + ((col & 7) << 1)) = __float2bfloat16_rn(e);
+                }
+              }
+              __syncwarp();
             }
             if (p.y_direct) {
               // rows of the slab, one after the other; the lanes take consecutive elements of a row

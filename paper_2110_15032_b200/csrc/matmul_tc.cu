@@ -953,8 +953,8 @@ static sbp_status launch_tc(bool tall, bool a_trans, bool b_trans, const TcParam
 // to this kernel's measured times on B200 under its power cap (the clock settles lower the busier
 // the tensor pipe is -- about 1.6 GHz in the square form, 1.4 GHz in the tall one -- which is why
 // these are times and not clock counts):
-//   square form  0.40 per 64-deep K-block (about 640 clocks); the epilogue is hidden unless it is store-bound;
-//   tall form    0.727 per K-block (1024 clocks) for twice the rows, plus an exposed epilogue of about 3.5.
+//   square form  0.388 per 64-deep K-block (about 590 clocks); the epilogue is hidden unless it is store-bound;
+//   tall form    0.70 per K-block (1024 clocks) for twice the rows, plus an exposed epilogue of about 2.6.
 // A run may be mixed: whole waves of tall tiles, then the rest of the walk in the square form (two
 // 256-row halves per walked tile) -- a last wave that only half fills the device costs a whole
 // tall wave otherwise.
@@ -965,8 +965,8 @@ struct FormChoice {
 
 static FormChoice choose_form(long long tiles_sq, long long tiles_tall, long long kb, int cap_sq, int cap_tall, bool gelu, int n_rep,
                               bool out_f32, int forced) {
-  const double wave_sq = 0.40 * kb + (gelu ? 0.6 : 0.0) + 1.1 * n_rep + (out_f32 ? 1.0 : 0.0);
-  const double wave_tall = 0.727 * kb + 3.5 + (gelu ? 8.5 : 0.0) + 2.2 * n_rep + (out_f32 ? 3.0 : 0.0);
+  const double wave_sq = 0.388 * kb + (gelu ? 1.3 : 0.0) + 1.2 * n_rep + (out_f32 ? 1.0 : 0.0);
+  const double wave_tall = 0.70 * kb + 2.6 + (gelu ? 8.6 : 0.0) + 2.5 * n_rep + (out_f32 ? 3.0 : 0.0);
   const double kRelaunch = 3.0;
   auto waves = [](long long tiles, int cap) { return (double)((tiles + cap - 1) / cap); };
   const double cost_sq = waves(tiles_sq, cap_sq) * wave_sq;

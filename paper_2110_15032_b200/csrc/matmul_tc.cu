@@ -967,7 +967,7 @@ static FormChoice choose_form(long long tiles_sq, long long tiles_tall, long lon
                               bool out_f32, int forced) {
   const double wave_sq = 0.388 * kb + (gelu ? 1.3 : 0.0) + 1.2 * n_rep + (out_f32 ? 1.0 : 0.0);
   const double wave_tall = 0.70 * kb + 2.6 + (gelu ? 8.6 : 0.0) + 2.5 * n_rep + (out_f32 ? 3.0 : 0.0);
-  const double kRelaunch = 3.0;
+  const double kRelaunch = 5.0;
   auto waves = [](long long tiles, int cap) { return (double)((tiles + cap - 1) / cap); };
   const double cost_sq = waves(tiles_sq, cap_sq) * wave_sq;
   const double cost_tall = waves(tiles_tall, cap_tall) * wave_tall;

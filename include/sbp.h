@@ -339,6 +339,14 @@ void sbp_tensor_map_stats(uint64_t* reused, uint64_t* encoded);
 #define SBP_TC_FORM_TALL 2
 #define SBP_TC_FORM_MIXED 3
 void sbp_matmul_set_form(int32_t form, int32_t max_pairs);
+/* The route the library's cost model picks for ONE bf16 output group of m x n with a contraction of
+ * k on a device that holds `pairs` CTA pairs at once (74 on a B200), written to `replicas` >= 1
+ * destinations: returns 0 square, 1 tall, 2 mixed (then *tall_tiles = the 512 x 256 tiles that run
+ * in the tall form; 0 for square), -1 for arguments out of range.  Host arithmetic only: no
+ * device is touched, overrides set with sbp_matmul_set_form are not applied, and products that
+ * cannot leave the square form (softmax epilogues, element-wise stores) are not modelled. */
+int32_t sbp_matmul_route(int64_t m, int64_t n, int64_t k, int32_t pairs, uint32_t flags, int32_t replicas, int32_t out_f32,
+                         int64_t* tall_tiles);
 void sbp_matmul_form_stats(uint64_t launches[3]);
 sbp_status sbp_matmul(const sbp_tensor* x, const sbp_tensor* w, sbp_tensor* y, uint32_t flags,
                       void* ws, size_t ws_bytes, void* cuda_stream);

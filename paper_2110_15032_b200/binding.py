@@ -118,6 +118,8 @@ def load_library():
     lib.sbp_matmul_set_form.argtypes = [C.c_int32, C.c_int32]
     lib.sbp_matmul_set_form.restype = None
     lib.sbp_matmul_form_stats.argtypes = [C.POINTER(C.c_uint64)]
+    lib.sbp_matmul_route.argtypes = [C.c_int64, C.c_int64, C.c_int64, C.c_int32, C.c_uint32, C.c_int32, C.c_int32, C.POINTER(C.c_int64)]
+    lib.sbp_matmul_route.restype = C.c_int32
     lib.sbp_matmul_form_stats.restype = None
     lib.sbp_softmax_xent_workspace_bytes.restype = C.c_size_t
     lib.sbp_softmax_xent_workspace_bytes.argtypes = [T]
@@ -293,6 +295,14 @@ SBP_TC_FORM_AUTO, SBP_TC_FORM_SQUARE, SBP_TC_FORM_TALL, SBP_TC_FORM_MIXED = 0, 1
 def sbp_matmul_set_form(form: int = 0, max_pairs: int = 0) -> None:
     """Test and measurement override of the tensor-core kernel's form and CTA-pair count."""
     load_library().sbp_matmul_set_form(int(form), int(max_pairs))
+
+
+def sbp_matmul_route(m: int, n: int, k: int, pairs: int = 74, flags: int = 0, replicas: int = 1, out_f32: bool = False):
+    """(route, tall tiles) the library's cost model picks for one m x n x k bf16 product: route 0
+    square, 1 tall, 2 mixed (host arithmetic only)."""
+    t = C.c_int64()
+    r = load_library().sbp_matmul_route(m, n, k, pairs, flags, replicas, 1 if out_f32 else 0, C.byref(t))
+    return int(r), int(t.value)
 
 
 def sbp_matmul_form_stats():

@@ -27,6 +27,8 @@ size_t matmul_tc_workspace_bytes(const MatmulPlan& plan);
 void tensor_map_cache_stats(unsigned long long* hits, unsigned long long* encodes);
 void tc_form_stats(unsigned long long out[3]);
 void tc_set_form(int form, int max_pairs);
+int tc_route(long long tiles_sq, long long tiles_tall, long long kb, int pairs, bool gelu, int n_rep, bool out_f32, int forced,
+             long long* tall_tiles);
 
 __device__ __forceinline__ float gelu_erf(float v) { return 0.5f * v * (1.0f + erff(v * 0.70710678118654752440f)); }
 
@@ -547,6 +549,17 @@ void sbp_tensor_map_stats(uint64_t* reused, uint64_t* encoded) {
 }
 
 void sbp_matmul_set_form(int32_t form, int32_t max_pairs) { tc_set_form(form, max_pairs); }
+
+int32_t sbp_matmul_route(int64_t m, int64_t n, int64_t k, int32_t pairs, uint32_t flags, int32_t replicas, int32_t out_f32,
+                         int64_t* tall_tiles) {
+  if (m <= 0 || n <= 0 || k <= 0 || pairs <= 0 || replicas < 1) {
+    if (tall_tiles) *tall_tiles = 0;
+    return -1;
+  }
+  const long long tn = (n + 255) / 256;
+  return tc_route((m + 255) / 256 * tn, (m + 511) / 512 * tn, (k + 63) / 64, pairs, (flags & SBP_EPILOGUE_GELU) != 0, replicas - 1,
+                  out_f32 != 0, 0, reinterpret_cast<long long*>(tall_tiles));
+}
 
 void sbp_matmul_form_stats(uint64_t launches[3]) {
   unsigned long long v[3] = {0, 0, 0};

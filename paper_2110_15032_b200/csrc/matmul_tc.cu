@@ -988,6 +988,14 @@ static FormChoice choose_form(long long tiles_sq, long long tiles_tall, long lon
   return FormChoice{true, (int)(pick == 1 ? tiles_tall : full)};
 }
 
+// choose_form for callers outside this file (the C ABI's planning query): 0 square, 1 tall, 2 mixed.
+int tc_route(long long tiles_sq, long long tiles_tall, long long kb, int pairs, bool gelu, int n_rep, bool out_f32, int forced,
+             long long* tall_tiles) {
+  const FormChoice f = choose_form(tiles_sq, tiles_tall, kb, pairs, pairs, gelu, n_rep, out_f32, forced);
+  if (tall_tiles) *tall_tiles = f.walk_tall ? f.tall_tiles : 0;
+  return !f.walk_tall ? 0 : (f.tall_tiles == tiles_tall ? 1 : 2);
+}
+
 sbp_status launch_matmul_tc(const MatmulPlan& plan, const XentFusion* xf, cudaStream_t st, bool* taken) {
   *taken = false;
   if (plan.in_dtype != SBP_BF16) return SBP_ERR_UNSUPPORTED;

@@ -275,3 +275,35 @@ def test_view_b_to_s_points_into_the_replicas(lib, shape, k):
 
 def O_split(T, k):
     return [torch.from_numpy(a.copy()) for a in O.to_locals(T.numpy(), O.S0, k)]
+
+
+def test_matmul_route_model_on_the_host():
+    """The route choice is host arithmetic (no device): sanity of its decisions and invariants."""
+    import paper_2110_15032_b200 as sbp
+    # far less than a wave of tiles: square
+    assert sbp.sbp_matmul_route(512, 512, 4096) == (0, 0)
+    # one full wave of tall tiles against two square waves, long contraction: tall
+    r, t = sbp.sbp_matmul_route(1024, 37 * 256, 16384)
+    assert (r, t) == (1, 74)
+    # 256 tall tiles on 74 pairs, K = 16384: three whole tall waves, the rest square
+    r, t = sbp.sbp_matmul_route(8192, 4096, 16384)
+    assert (r, t) == (2, 222)
+    # the same with a short contraction: the exposed epilogue of the tall form does not pay
+    assert sbp.sbp_matmul_route(8192, 4096, 512)[0] == 0
+    # GeLU in the epilogue keeps a 4096-deep product square
+    assert sbp.sbp_matmul_route(8192, 16384, 4096, flags=sbp.SBP_EPILOGUE_GELU)[0] == 0
+    # invariants over a sweep: the tall part is whole waves (mixed) or everything (tall), never more than there is
+    for m in (256, 700, 3000, 8192, 20000):
+        for n in (256, 1000, 4096, 9000):
+            for k in (64, 512, 4096, 32768):
+                for pairs in (3, 74):
+                    r, t = sbp.sbp_matmul_route(m, n, k, pairs)
+                    tall = -(-m // 512) * -(-n // 256)
+                    assert r in (0, 1, 2) and 0 <= t <= tall
+                    if r == 0:
+                        assert t == 0
+                    elif r == 1:
+                        assert t == tall
+                    else:
+                        assert t % pairs == 0 and 0 < t < tall
+    assert sbp.sbp_matmul_route(0, 4, 4)[0] == -1

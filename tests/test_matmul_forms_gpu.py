@@ -99,3 +99,25 @@ def test_library_choice_takes_each_form_on_a_whole_device():
     sbp.sbp_matmul_set_form(sbp.SBP_TC_FORM_SQUARE, 0)
     y2 = _sampled_product(8192, 16384, 3840, 2003, (1, 0, 0))
     assert torch.equal(y.locals[0].view(torch.uint8), y2.locals[0].view(torch.uint8))
+
+
+@pytest.mark.parametrize("form,pairs", [("mixed", 5), ("tall", 9)])
+def test_operator_parity_tests_pass_with_the_form_forced_on_a_few_pairs(form, pairs):
+    """Every MatMul parity test of the suite once more, in a child process whose library is told to
+    take the given route with only a handful of CTA pairs: small products then run many waves, so
+    the tall kernel, the half-tile walk of a mixed run's square launch and the hand-over between the
+    two are exercised on all signatures, fused outputs, transposed and unaligned operands."""
+    import os
+    import subprocess
+    import sys
+    from conftest import ROOT
+    env = dict(os.environ, SBP_TC_FORM=form, SBP_TC_PAIRS=str(pairs))
+    r = subprocess.run([sys.executable, "-m", "pytest", "tests/test_ops_gpu.py", "tests/test_strided_views_gpu.py",
+                        "tests/test_two_axis_gpu.py", "-x", "-q", "-m", "gpu", "-p", "no:cacheprovider",
+                        "-k", "matmul or tensor or mlp or classifier or view or data_parallel or two_axis"],
+                       cwd=ROOT, env=env, capture_output=True, text=True, timeout=1500)
+    tail = r.stdout[-3000:] + r.stderr[-2000:]
+    assert r.returncode == 0, tail
+    last = r.stdout.strip().splitlines()[-1]
+    assert " passed" in last and "failed" not in last, tail
+    assert int(last.split(" passed")[0].split()[-1]) >= 100, last

@@ -806,7 +806,7 @@ def parse():
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-steps", type=int, default=6)
     ap.add_argument("--no-ops", action="store_true", help="skip the sharded-operator sections (N = 1 only)")
     ap.add_argument("--ops", default="softmax,classifier,mlp,embedding,extras,cliffs",
                     help="comma-separated operator sections to run: softmax, classifier, mlp, embedding, extras, cliffs")

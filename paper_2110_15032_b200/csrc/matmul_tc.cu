@@ -46,13 +46,13 @@ namespace sbp {
 
 constexpr int BM = 256, BN = 256, BK = 64;      // tile of a CTA pair
 constexpr int BMH = BM / 2, BNH = BN / 2;       // what one CTA of the pair loads
-constexpr int kStages = 5;
+constexpr int kStages = 6;                        // 6 slots + 1 staging slab per warp beat 5 + 2 once the hand-back of an accumulator was cheap
 constexpr int kStageA = BMH * BK * 2;             // 16 KiB
 constexpr int kStageB = BK * BNH * 2;             // 16 KiB
 constexpr int kStageBytes = kStageA + kStageB;    // 32 KiB per CTA
 constexpr int kEpiWarps = 8;
 constexpr int kSlabBytes = 32 * 128;              // one epilogue slab: 32 rows x 128 bytes
-constexpr int kEpiBufs = 2;                       // staging slabs per epilogue warp
+constexpr int kEpiBufs = 1;                       // staging slabs per epilogue warp
 constexpr int kEpiBytes = kEpiWarps * kEpiBufs * kSlabBytes;
 constexpr int kSmemBytes = kStages * kStageBytes + kEpiBytes + 1024;   // + alignment slack
 // The tall form (MH = 2): a CTA pair owns a 512 x 256 tile -- two m-halves of 256 rows that share
@@ -398,7 +398,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreadsTc, 1)
     // ------------------------------------------------ producer (both CTAs)
     if (lane == 0) {
       // ring position kept as (slot, round parity) and stepped, not divided out of a running count:
-      // with five slots the division is a long instruction sequence, once per K-block
+      // with a slot count that is not a power of two the division is a long instruction sequence,
+      // once per K-block
       long long kb_iter = 0;
       int slot = 0;
       unsigned round = 0;

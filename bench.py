@@ -179,18 +179,18 @@ NCU_TRAFFIC = {
     "softmax-xent on bf16 logits (partial + combine)": 1077.2e6,
     "softmax-xent backward (softmax - onehot, S(1))": 2099.7e6,
     # profiles/matmul_tc_classifier_bf16_512x512x1048576_k8.md (full size)
-    "classifier GEMM (B,S(1))->S(1), bf16 logits": 2106.6e6,
-    "classifier GEMM fused with softmax-xent (no logits stored)": 1132.6e6 + 50.5e6,
-    "classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)": 2104.9e6,
+    "classifier GEMM (B,S(1))->S(1), bf16 logits": 2104.3e6,
+    "classifier GEMM fused with softmax-xent (no logits stored)": 1127.8e6 + 50.5e6,
+    "classifier GEMM fused with the softmax-xent backward (grad S(1), no logits stored)": 2103.8e6,
     # profiles/matmul_tc_mlp_bf16_8192x4096x16384_k8.md (full size; a mixed run is the sum of its two launches)
-    "MLP GEMM1 (B,S(1))->S(1) + GeLU": 1002.9e6,
-    "MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials": 911.6e6,
-    "MLP GEMM2 fused (S(1),S(0))->B": 1200.8e6 + 193.9e6,
-    "MLP GEMM1 with W1 stored transposed (SBP_TRANS_W) + GeLU": 998.5e6,
-    "MLP GEMM2 fused (S(1),S(0))->B with W2 stored transposed (SBP_TRANS_W)": 1200.9e6 + 194.7e6,
-    "DP layer backward dW = X^T dY, (S(1),S(0))->S(0) fused": 890.7e6,
-    "DP layer backward dW = X^T dY, (S(1),S(0))->B fused (8 replicas written)": 1783.1e6,
-    "DP layer backward dX = dY W^T, (S(0),B)->S(0)": 756.6e6 + 205.9e6,
+    "MLP GEMM1 (B,S(1))->S(1) + GeLU": 1003.3e6,
+    "MLP GEMM2 (S(1),S(0))->P(sum), bf16 partials": 914.0e6,
+    "MLP GEMM2 fused (S(1),S(0))->B": 1195.4e6 + 194.6e6,
+    "MLP GEMM1 with W1 stored transposed (SBP_TRANS_W) + GeLU": 1003.4e6,
+    "MLP GEMM2 fused (S(1),S(0))->B with W2 stored transposed (SBP_TRANS_W)": 1195.2e6 + 194.4e6,
+    "DP layer backward dW = X^T dY, (S(1),S(0))->S(0) fused": 872.6e6,
+    "DP layer backward dW = X^T dY, (S(1),S(0))->B fused (8 replicas written)": 1774.9e6,
+    "DP layer backward dX = dY W^T, (S(0),B)->S(0)": 747.1e6 + 206.0e6,
     # profiles/extras_bf16_8192x8192_p4_and_embedding_fp32_4194304x128_batch16384_k8.md (full size)
     "S(0)->P(sum) bf16 [8192,8192] k=4": 619.4e6,
     "B->P(sum) bf16 [8192,8192] k=4": 611.7e6,
@@ -209,7 +209,7 @@ NCU_TRAFFIC = {
 # taken again after the kernel got its tall and mixed forms; the other kernels have not changed
 # since the first).  A kernel that changes afterwards gets its entry set to None (or recaptured)
 # in the same commit: a stale figure is worse than none.
-NCU_TRAFFIC_CAPTURED_AT = "a61a16e (boxing, softmax, embedding to several replicas); 86d3a9b (matmul_tc_kernel); 68937c6 (embedding_rows_kernel)"
+NCU_TRAFFIC_CAPTURED_AT = "a61a16e (boxing, softmax, embedding to several replicas); 073ea77 (matmul_tc_kernel); 68937c6 (embedding_rows_kernel)"
 
 
 def ncu_traffic(name):

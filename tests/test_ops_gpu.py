@@ -395,6 +395,14 @@ def test_embedding_closed_forms_and_edges():
     _, oob = _emb_case(rows, dim, bad, k, F32, False)
     assert oob == 3
     _emb_case(rows, dim, ids1, k, F32, True, alias=True)
+    # single destination (aliased replicas): the kernel that resolves a lookup's row address once, a
+    # chunk ahead -- out-of-range ids give zero rows and are counted once each, also across chunks
+    _, oob = _emb_case(rows, dim, bad, k, F32, True, alias=True)
+    assert oob == 3
+    many = dg.integers(77, 0, (4096, 3), 0, rows).cpu()
+    many[5, 1], many[700, 0], many[2049, 2], many[4095, 2] = -7, rows, 1 << 33, rows + 1
+    _, oob = _emb_case(rows, dim, many, k, F32, True, alias=True)
+    assert oob == 4
     _emb_case(3, 16, torch.tensor([0, 1, 2, 2, 0]), 8, F32, False)                   # k > rows
     _emb_case(3, 16, torch.tensor([0, 1, 2, 2, 0]), 8, F32, True)
 

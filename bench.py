@@ -219,34 +219,35 @@ def ncu_traffic(name):
 # ------------------------------------------------------------------------------ end to end
 
 def e2e_sweep(sbp, src, work, device, steps, dist):
-    """The sweep through sbp_boxing_host: pinned host buffers in, pinned host buffers out,
-    host->device and device->host copies inside the timed region."""
+    """The sweep through the host entry point: pinned host buffers in, pinned host buffers out,
+    host->device and device->host copies inside the timed region.  The transforms of a step that
+    read the same source go into one sbp_boxing_host_multi call, so every source crosses once."""
     host_src = {}
     for key, g in src.items():
         host_src[key] = sbp.SbpTensor(g.shape, g.dtype, g.sig, [t.cpu().pin_memory() for t in g.locals])
-    jobs = []
-    h2d = d2h = 0
-    ws_bytes = 0
     key_of = {id(g): key for key, g in src.items()}
-    for name, s, d, _ in work:
-        hs = host_src[key_of[id(s)]]
+    groups = {}      # source key -> host destinations, in the order of the sweep
+    host_dst_of = {}
+    for name, s_, d, _ in work:
         hd = sbp.SbpTensor(d.shape, d.dtype, d.sig,
                            [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in d.locals])
-        jobs.append((hs, hd))
-        a, b = sbp.sbp_boxing_host_copy_bytes(hs, hd)      # what the call really copies (B -> S(i): one block per replica)
+        groups.setdefault(key_of[id(s_)], []).append(hd)
+        host_dst_of[name] = hd
+    jobs = [(host_src[key], dsts) for key, dsts in groups.items()]
+    h2d = d2h = 0
+    for hs, dsts in jobs:
+        a, b = sbp.sbp_boxing_host_multi_copy_bytes(hs, dsts)      # what the call really copies
         h2d += a
         d2h += b
-        ws_bytes = max(ws_bytes, sbp.sbp_boxing_host_workspace_bytes(hs, hd))
-    # Four streams, each with its own device workspace: consecutive transforms go round them, so
-    # the device->host copies of some overlap the host->device copies of others (measured: 44 ms a
-    # step with four streams or more; the host->device direction, 2.15 GB a step at 49 GB/s, is the bound).
-    n_streams = int(os.environ.get("SBP_E2E_STREAMS", "4"))
-    streams = [torch.cuda.Stream(device=device) for _ in range(n_streams)]
-    wss = [torch.empty(ws_bytes, dtype=torch.uint8, device=device) for _ in streams]
+    # One stream and one device workspace per source: the device->host copies of one group overlap
+    # the host->device copy of the next (PCIe is full duplex; the device->host direction, 1.74 GB a
+    # step, is the bound once every source is sent once).
+    streams = [torch.cuda.Stream(device=device) for _ in jobs]
+    wss = [torch.empty(sbp.sbp_boxing_host_multi_workspace_bytes(hs, dsts), dtype=torch.uint8, device=device) for hs, dsts in jobs]
 
     def one_step():
-        for i, (hs, hd) in enumerate(jobs):
-            sbp.sbp_boxing_host(hs, hd, wss[i % n_streams], stream=streams[i % n_streams])
+        for i, (hs, dsts) in enumerate(jobs):
+            sbp.sbp_boxing_host_multi(hs, dsts, wss[i], stream=streams[i])
 
     one_step()
     torch.cuda.synchronize()
@@ -271,7 +272,7 @@ def e2e_sweep(sbp, src, work, device, steps, dist):
     ms = max_over_ranks(max(start.elapsed_time(end), wall * 1e3), dist, device) / steps
     # spot check: the last transform's result on the host equals the device-resident run
     ref = work[-1][2].locals[0].cpu()
-    if not torch.equal(ref, jobs[-1][1].locals[0]):
+    if not torch.equal(ref, host_dst_of[work[-1][0]].locals[0]):
         raise RuntimeError("end-to-end result differs from the device-resident result")
     return {"value": step_bytes() / (ms * 1e-3) / 1e9, "unit": "GB/s", "ms_per_step": ms, "steps": steps,
             "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}

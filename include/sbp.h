@@ -225,6 +225,19 @@ sbp_status sbp_boxing_shard(const sbp_tensor* src, sbp_tensor* dst, int32_t dst_
 size_t sbp_boxing_host_workspace_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_host);
 sbp_status sbp_boxing_host_copy_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_host, uint64_t* h2d_bytes,
                                       uint64_t* d2h_bytes);
+/* One source, n destinations (1 <= n <= 64; dst_hosts is an array of n descriptors): the source is
+ * copied to the device once and boxed into every destination there, each result copied back as
+ * soon as its transform is enqueued -- what a caller does who needs one host tensor under several
+ * signatures (the P(sum) result of a product as B for one consumer and as S(0) for another).  Same
+ * rules as sbp_boxing_host for every (src, dst[i]) pair; all n pairs are validated before the
+ * first copy is enqueued; only the diagonal blocks of a B source are sent when every destination is
+ * an S of the same axis.  The workspace holds the source and all n results at once.
+ * sbp_boxing_host is this call with n = 1. */
+size_t sbp_boxing_host_multi_workspace_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_hosts, int32_t n);
+sbp_status sbp_boxing_host_multi_copy_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_hosts, int32_t n,
+                                            uint64_t* h2d_bytes, uint64_t* d2h_bytes);
+sbp_status sbp_boxing_host_multi(const sbp_tensor* src_host, sbp_tensor* dst_hosts, int32_t n, void* dev_ws,
+                                 size_t dev_ws_bytes, void* cuda_stream);
 sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, void* dev_ws,
                            size_t dev_ws_bytes, void* cuda_stream);
 

@@ -104,6 +104,10 @@ def load_library():
     lib.sbp_boxing_host_workspace_bytes.argtypes = [T, T]
     lib.sbp_boxing_host.argtypes = [T, T, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.sbp_boxing_host_copy_bytes.argtypes = [T, T, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+    lib.sbp_boxing_host_multi_workspace_bytes.restype = C.c_size_t
+    lib.sbp_boxing_host_multi_workspace_bytes.argtypes = [T, T, C.c_int32]
+    lib.sbp_boxing_host_multi_copy_bytes.argtypes = [T, T, C.c_int32, C.POINTER(C.c_uint64), C.POINTER(C.c_uint64)]
+    lib.sbp_boxing_host_multi.argtypes = [T, T, C.c_int32, C.c_void_p, C.c_size_t, C.c_void_p]
     lib.sbp_boxing_set_copy_engine.argtypes = [C.c_int32]
     lib.sbp_boxing_set_copy_engine.restype = None
     lib.sbp_check_device_errors.argtypes = []
@@ -360,6 +364,33 @@ def sbp_boxing_host_copy_bytes(src_host: SbpTensor, dst_host: SbpTensor):
     h2d, d2h = C.c_uint64(), C.c_uint64()
     _check(load_library().sbp_boxing_host_copy_bytes(C.byref(a), C.byref(b), C.byref(h2d), C.byref(d2h)))
     return int(h2d.value), int(d2h.value)
+
+
+def _c_array(tensors):
+    arr = (_Tensor * len(tensors))()
+    for i, t in enumerate(tensors):
+        arr[i] = t._c()
+    return arr
+
+
+def sbp_boxing_host_multi_workspace_bytes(src_host: SbpTensor, dst_hosts) -> int:
+    a, arr = src_host._c(), _c_array(dst_hosts)
+    return int(load_library().sbp_boxing_host_multi_workspace_bytes(C.byref(a), arr, len(dst_hosts)))
+
+
+def sbp_boxing_host_multi_copy_bytes(src_host: SbpTensor, dst_hosts):
+    """(host->device, device->host) bytes that one sbp_boxing_host_multi call copies."""
+    a, arr = src_host._c(), _c_array(dst_hosts)
+    h2d, d2h = C.c_uint64(), C.c_uint64()
+    _check(load_library().sbp_boxing_host_multi_copy_bytes(C.byref(a), arr, len(dst_hosts), C.byref(h2d), C.byref(d2h)))
+    return int(h2d.value), int(d2h.value)
+
+
+def sbp_boxing_host_multi(src_host: SbpTensor, dst_hosts, dev_ws: torch.Tensor, stream=None) -> None:
+    """One host source boxed into several host destinations: one upload, len(dst_hosts) transforms."""
+    a, arr = src_host._c(), _c_array(dst_hosts)
+    _check(load_library().sbp_boxing_host_multi(C.byref(a), arr, len(dst_hosts), C.c_void_p(dev_ws.data_ptr()),
+                                                dev_ws.numel() * dev_ws.element_size(), _stream_ptr(stream)))
 
 
 def sbp_boxing_host(src_host: SbpTensor, dst_host: SbpTensor, dev_ws: torch.Tensor, stream=None) -> None:

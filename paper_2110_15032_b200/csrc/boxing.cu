@@ -794,72 +794,124 @@ static HostBlock host_diagonal_block(const sbp_tensor* src, int axis, int r) {
   return HostBlock{(size_t)start * inner, (size_t)src->shape[axis] * inner, (size_t)len * inner, outer};
 }
 
-sbp_status sbp_boxing_host_copy_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_host, uint64_t* h2d, uint64_t* d2h) {
-  sbp_status st = check_pair(src_host, dst_host, false);
-  if (st != SBP_OK) return st;
-  const int ks = placement_k(src_host), kd = placement_k(dst_host);
-  uint64_t in = 0, out = 0;
-  const bool diag = host_copy_is_diagonal(src_host, dst_host);
-  for (int r = 0; r < ks; ++r) {
+// One source, n destinations: the source crosses to the device once and every transform reads it
+// there.  Only the diagonal blocks are sent when EVERY destination is a B -> S(axis) of the same
+// axis on an equal placement.
+static bool host_multi_is_diagonal(const sbp_tensor* src, const sbp_tensor* dsts, int n) {
+  for (int i = 0; i < n; ++i)
+    if (!host_copy_is_diagonal(src, &dsts[i]) || dsts[i].sbp[0].axis != dsts[0].sbp[0].axis) return false;
+  return n > 0;
+}
+
+static sbp_status host_multi_check(const sbp_tensor* src, const sbp_tensor* dsts, int n, bool need_pointers) {
+  if (!src || !dsts) return fail(SBP_ERR_INVALID_ARG, "null descriptor");
+  if (n < 1 || n > 64) return fail(SBP_ERR_INVALID_ARG, "between 1 and 64 destinations, not %d", n);
+  for (int i = 0; i < n; ++i) {
+    sbp_status st = check_pair(src, &dsts[i], need_pointers);
+    if (st != SBP_OK) return st;
+  }
+  return SBP_OK;
+}
+
+static uint64_t host_source_bytes(const sbp_tensor* src, const sbp_tensor* dsts, int n) {
+  const bool diag = host_multi_is_diagonal(src, dsts, n);
+  uint64_t in = 0;
+  for (int r = 0; r < placement_k(src); ++r) {
     if (diag) {
-      const HostBlock b = host_diagonal_block(src_host, dst_host->sbp[0].axis, r);
+      const HostBlock b = host_diagonal_block(src, dsts[0].sbp[0].axis, r);
       in += (uint64_t)b.width * b.outer;
     } else {
-      in += (uint64_t)local_numel(src_host, r) * elem_size(src_host->dtype);
+      in += (uint64_t)local_numel(src, r) * elem_size(src->dtype);
     }
   }
-  for (int r = 0; r < kd; ++r) {
+  return in;
+}
+
+static uint64_t host_result_bytes(const sbp_tensor* dst) {
+  uint64_t out = 0;
+  for (int r = 0; r < placement_k(dst); ++r) {
     bool dup = false;
-    for (int q = 0; q < r; ++q) dup = dup || dst_host->local[q] == dst_host->local[r];
-    if (!dup) out += (uint64_t)local_numel(dst_host, r) * elem_size(dst_host->dtype);
+    for (int q = 0; q < r; ++q) dup = dup || dst->local[q] == dst->local[r];
+    if (!dup) out += (uint64_t)local_numel(dst, r) * elem_size(dst->dtype);
   }
-  if (h2d) *h2d = in;
+  return out;
+}
+
+sbp_status sbp_boxing_host_multi_copy_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_hosts, int32_t n, uint64_t* h2d,
+                                            uint64_t* d2h) {
+  sbp_status st = host_multi_check(src_host, dst_hosts, n, false);
+  if (st != SBP_OK) return st;
+  uint64_t out = 0;
+  for (int i = 0; i < n; ++i) out += host_result_bytes(&dst_hosts[i]);
+  if (h2d) *h2d = host_source_bytes(src_host, dst_hosts, n);
   if (d2h) *d2h = out;
   return SBP_OK;
 }
 
-sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, void* dev_ws, size_t dev_ws_bytes,
-                           void* cuda_stream) {
+sbp_status sbp_boxing_host_copy_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_host, uint64_t* h2d, uint64_t* d2h) {
+  return sbp_boxing_host_multi_copy_bytes(src_host, dst_host, 1, h2d, d2h);
+}
+
+size_t sbp_boxing_host_multi_workspace_bytes(const sbp_tensor* src_host, const sbp_tensor* dst_hosts, int32_t n) {
+  if (host_multi_check(src_host, dst_hosts, n, false) != SBP_OK) return 0;
+  size_t total = 0;
+  for (int r = 0; r < placement_k(src_host); ++r) total += align256((size_t)local_numel(src_host, r) * elem_size(src_host->dtype));
+  for (int i = 0; i < n; ++i)
+    for (int r = 0; r < placement_k(&dst_hosts[i]); ++r)
+      total += align256((size_t)local_numel(&dst_hosts[i], r) * elem_size(dst_hosts[i].dtype));
+  return total;
+}
+
+sbp_status sbp_boxing_host_multi(const sbp_tensor* src_host, sbp_tensor* dst_hosts, int32_t n, void* dev_ws, size_t dev_ws_bytes,
+                                 void* cuda_stream) {
   SBP_RANGE("sbp_boxing_host");
-  sbp_status st = check_pair(src_host, dst_host, true);
+  sbp_status st = host_multi_check(src_host, dst_hosts, n, true);
   if (st != SBP_OK) return st;
   st = refuse_ld(src_host, "src_host", "sbp_boxing_host");
   if (st != SBP_OK) return st;
-  st = refuse_ld(dst_host, "dst_host", "sbp_boxing_host");
-  if (st != SBP_OK) return st;
-  const size_t need = sbp_boxing_host_workspace_bytes(src_host, dst_host);
+  for (int i = 0; i < n; ++i) {
+    st = refuse_ld(&dst_hosts[i], "dst_host", "sbp_boxing_host");
+    if (st != SBP_OK) return st;
+  }
+  const size_t need = sbp_boxing_host_multi_workspace_bytes(src_host, dst_hosts, n);
   if (need > 0 && (!dev_ws || dev_ws_bytes < need))
     return fail(SBP_ERR_WORKSPACE, "device workspace of %zu bytes needed, %zu given", need, dev_ws_bytes);
   if (reinterpret_cast<uintptr_t>(dev_ws) % 256 != 0)
     return fail(SBP_ERR_ALIGNMENT, "device workspace must be 256-byte aligned");
-  const int ks = placement_k(src_host), kd = placement_k(dst_host);
+  const int ks = placement_k(src_host);
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  sbp_tensor s = *src_host, d = *dst_host;
+  sbp_tensor s = *src_host;
+  static thread_local sbp_tensor d[64];
   char* cur = static_cast<char*>(dev_ws);
-  const int esz = elem_size(src_host->dtype), esz_dst = elem_size(dst_host->dtype);
+  const int esz = elem_size(src_host->dtype);
   for (int r = 0; r < ks; ++r) {
     s.local[r] = cur;
     cur += align256((size_t)local_numel(src_host, r) * esz);
   }
-  // Destination replicas that alias on the host alias on the device as well.
-  for (int r = 0; r < kd; ++r) {
-    d.local[r] = nullptr;
-    for (int q = 0; q < r; ++q)
-      if (dst_host->local[q] == dst_host->local[r]) d.local[r] = d.local[q];
-    if (!d.local[r]) {
-      d.local[r] = cur;
-      cur += align256((size_t)local_numel(dst_host, r) * esz_dst);
+  for (int i = 0; i < n; ++i) {
+    d[i] = dst_hosts[i];
+    // Destination replicas that alias on the host alias on the device as well.
+    for (int r = 0; r < placement_k(&d[i]); ++r) {
+      d[i].local[r] = nullptr;
+      for (int q = 0; q < r; ++q)
+        if (dst_hosts[i].local[q] == dst_hosts[i].local[r]) d[i].local[r] = d[i].local[q];
+      if (!d[i].local[r]) {
+        d[i].local[r] = cur;
+        cur += align256((size_t)local_numel(&dst_hosts[i], r) * elem_size(dst_hosts[i].dtype));
+      }
     }
   }
-  // the transform's own refusals (signature pair, sizes) come before the first copy is enqueued
-  if (s.pdims == 2 || d.pdims == 2) st = boxing_2d(&s, &d, cuda_stream, true);
-  else st = boxing_one_axis(&s, &d, -1, cuda_stream, true);
-  if (st != SBP_OK) return st;
-  const bool diag = host_copy_is_diagonal(src_host, dst_host);
+  // every transform's own refusals (signature pair, sizes) come before the first copy is enqueued
+  for (int i = 0; i < n; ++i) {
+    if (s.pdims == 2 || d[i].pdims == 2) st = boxing_2d(&s, &d[i], cuda_stream, true);
+    else st = boxing_one_axis(&s, &d[i], -1, cuda_stream, true);
+    if (st != SBP_OK) return st;
+  }
+  const bool diag = host_multi_is_diagonal(src_host, dst_hosts, n);
   for (int r = 0; r < ks; ++r) {
     if (diag) {
-      // the rest of this replica's device copy stays unwritten: the transform never reads it
-      const HostBlock b = host_diagonal_block(src_host, dst_host->sbp[0].axis, r);
+      // the rest of this replica's device copy stays unwritten: the transforms never read it
+      const HostBlock b = host_diagonal_block(src_host, dst_hosts[0].sbp[0].axis, r);
       if (b.width && b.outer)
         SBP_CUDA_TRY(cudaMemcpy2DAsync(static_cast<char*>(s.local[r]) + b.offset, b.pitch,
                                        static_cast<const char*>(src_host->local[r]) + b.offset, b.pitch, b.width, b.outer,
@@ -869,16 +921,23 @@ sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, voi
     const size_t bytes = (size_t)local_numel(src_host, r) * esz;
     if (bytes) SBP_CUDA_TRY(cudaMemcpyAsync(s.local[r], src_host->local[r], bytes, cudaMemcpyHostToDevice, stream));
   }
-  st = sbp_boxing(&s, &d, cuda_stream);
-  if (st != SBP_OK) return st;
-  for (int r = 0; r < kd; ++r) {
-    bool dup = false;
-    for (int q = 0; q < r; ++q) dup = dup || dst_host->local[q] == dst_host->local[r];
-    const size_t bytes = (size_t)local_numel(dst_host, r) * esz_dst;
-    if (!dup && bytes)
-      SBP_CUDA_TRY(cudaMemcpyAsync(dst_host->local[r], d.local[r], bytes, cudaMemcpyDeviceToHost, stream));
+  for (int i = 0; i < n; ++i) {
+    st = sbp_boxing(&s, &d[i], cuda_stream);
+    if (st != SBP_OK) return st;
+    for (int r = 0; r < placement_k(&d[i]); ++r) {
+      bool dup = false;
+      for (int q = 0; q < r; ++q) dup = dup || dst_hosts[i].local[q] == dst_hosts[i].local[r];
+      const size_t bytes = (size_t)local_numel(&dst_hosts[i], r) * elem_size(dst_hosts[i].dtype);
+      if (!dup && bytes)
+        SBP_CUDA_TRY(cudaMemcpyAsync(dst_hosts[i].local[r], d[i].local[r], bytes, cudaMemcpyDeviceToHost, stream));
+    }
   }
   return SBP_OK;
+}
+
+sbp_status sbp_boxing_host(const sbp_tensor* src_host, sbp_tensor* dst_host, void* dev_ws, size_t dev_ws_bytes,
+                           void* cuda_stream) {
+  return sbp_boxing_host_multi(src_host, dst_host, 1, dev_ws, dev_ws_bytes, cuda_stream);
 }
 
 }  // extern "C"

@@ -320,6 +320,55 @@ def test_host_entry_point_copies_only_the_blocks_b_to_s_reads(shape, axis):
     assert h2d == k * T.numel() * 2 and d2h == T.numel() * 2
 
 
+def test_host_entry_point_with_one_source_and_several_destinations():
+    """sbp_boxing_host_multi: the source crosses to the device once, every transform reads it there;
+    each result equals the oracle's; a refused pair leaves every host destination untouched."""
+    k, shape = 4, (130, 250)
+    parts = [dg.normal(21, r, shape, 0, 1, BF16).pin_memory() for r in range(k)]
+    src = sbp.SbpTensor(shape, BF16, sbp.P_SUM, parts)
+    sigs = [sbp.B, sbp.S(0), sbp.S(1)]
+    dsts = []
+    for sig in sigs:
+        locs = [torch.full(sbp.sbp_local_shape(shape, sig, k, r, BF16), 7.0, dtype=BF16).pin_memory() for r in range(k)]
+        dsts.append(sbp.SbpTensor(shape, BF16, sig, locs))
+    numel = shape[0] * shape[1]
+    h2d, d2h = sbp.sbp_boxing_host_multi_copy_bytes(src, dsts)
+    assert h2d == k * numel * 2 and d2h == (k + 1 + 1) * numel * 2        # one upload; B to k replicas, S(0), S(1)
+    need = sbp.sbp_boxing_host_multi_workspace_bytes(src, dsts)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    sbp.sbp_boxing_host_multi(src, dsts, ws)
+    torch.cuda.synchronize()
+    for sig, d in zip(sigs, dsts):
+        want = O.boxing([to_np(t) for t in parts], O.PSUM, osig(sig), "bf16")
+        for r in range(k):
+            assert np.array_equal(bits(d.locals[r]), np_bits(want[r], BF16)), (sig, r)
+    # B source into S(1) twice: the diagonal blocks only; into S(0) and S(1): the whole of every replica
+    T = dg.normal(22, 0, shape, 0, 1, BF16)
+    bsrc = sbp.SbpTensor(shape, BF16, sbp.B, [T.clone().pin_memory() for _ in range(k)])
+    mk = lambda sig: sbp.SbpTensor(shape, BF16, sig, [torch.empty(sbp.sbp_local_shape(shape, sig, k, r, BF16), dtype=BF16).pin_memory()
+                                                        for r in range(k)])
+    two = [mk(sbp.S(1)), mk(sbp.S(1))]
+    assert sbp.sbp_boxing_host_multi_copy_bytes(bsrc, two) == (numel * 2, 2 * numel * 2)
+    mixed = [mk(sbp.S(0)), mk(sbp.S(1))]
+    assert sbp.sbp_boxing_host_multi_copy_bytes(bsrc, mixed) == (k * numel * 2, 2 * numel * 2)
+    for group in (two, mixed):
+        ws = torch.empty(sbp.sbp_boxing_host_multi_workspace_bytes(bsrc, group), dtype=torch.uint8, device="cuda")
+        sbp.sbp_boxing_host_multi(bsrc, group, ws)
+        torch.cuda.synchronize()
+        for d in group:
+            want = split_cpu(T, d.sig, k)
+            assert all(torch.equal(a, b) for a, b in zip(d.locals, want))
+    # one pair of the call is refused (P(sum) -> P(max) has no meaning): nothing is copied or written
+    bad = [dsts[0], sbp.SbpTensor(shape, BF16, sbp.P_MAX, [torch.full(shape, 7.0, dtype=BF16).pin_memory() for _ in range(k)])]
+    for t in dsts[0].locals:
+        t.fill_(7.0)
+    ws = torch.empty(sbp.sbp_boxing_host_multi_workspace_bytes(src, dsts) * 2, dtype=torch.uint8, device="cuda")
+    with pytest.raises(sbp.SbpError):
+        sbp.sbp_boxing_host_multi(src, bad, ws)
+    torch.cuda.synchronize()
+    assert all(bool((t == 7.0).all()) for d in bad for t in d.locals)
+
+
 def test_expired_device_wait_is_reported_and_the_device_stays_usable():
     """A bounded wait that runs out (a barrier nothing signals) ends the kernel normally and is
     reported once as SBP_ERR_TIMEOUT; nothing faults and later launches work."""

@@ -228,7 +228,8 @@ sbp_status sbp_boxing_host_copy_bytes(const sbp_tensor* src_host, const sbp_tens
 /* One source, n destinations (1 <= n <= 64; dst_hosts is an array of n descriptors): the source is
  * copied to the device once and boxed into every destination there, each result copied back as
  * soon as its transform is enqueued -- what a caller does who needs one host tensor under several
- * signatures (the P(sum) result of a product as B for one consumer and as S(0) for another).  Same
+ * signatures (Section 3.2: one boxing op per consumer whose signature differs from the producer's;
+ * e.g. the P(sum) result of a product as B for one consumer and as S(0) for another).  Same
  * rules as sbp_boxing_host for every (src, dst[i]) pair; all n pairs are validated before the
  * first copy is enqueued; only the diagonal blocks of a B source are sent when every destination is
  * an S of the same axis.  The workspace holds the source and all n results at once.
@@ -332,7 +333,7 @@ size_t sbp_matmul_workspace_bytes(const sbp_tensor* x, const sbp_tensor* w, cons
  * same buffers.  This reports how many were re-used and how many encoded since the library was
  * loaded (process-wide), so that a harness can check that a steady-state call encodes nothing. */
 void sbp_tensor_map_stats(uint64_t* reused, uint64_t* encoded);
-/* The tensor-core kernel has two compiled forms: CTA pairs that own 256 x 256 tiles of the result
+/* (No counterpart in the paper either.)  The tensor-core kernel has two compiled forms: CTA pairs that own 256 x 256 tiles of the result
  * with a spare accumulator, so that a tile's epilogue runs under the next tile's MMAs ("square"),
  * and pairs that own 512 x 256 tiles with both accumulators in use ("tall": less operand traffic per
  * MMA, the epilogue exposed).  The library picks per product, from the tile count, the length of
@@ -352,7 +353,8 @@ void sbp_tensor_map_stats(uint64_t* reused, uint64_t* encoded);
 #define SBP_TC_FORM_TALL 2
 #define SBP_TC_FORM_MIXED 3
 void sbp_matmul_set_form(int32_t form, int32_t max_pairs);
-/* The route the library's cost model picks for ONE bf16 output group of m x n with a contraction of
+/* (The paper has no counterpart: this is about how THIS library runs a Table 1 product.)
+ * The route the library's cost model picks for ONE bf16 output group of m x n with a contraction of
  * k on a device that holds `pairs` CTA pairs at once (74 on a B200), written to `replicas` >= 1
  * destinations: returns 0 square, 1 tall, 2 mixed (then *tall_tiles = the 512 x 256 tiles that run
  * in the tall form; 0 for square), -1 for arguments out of range.  Host arithmetic only: no

@@ -2,6 +2,7 @@
 and three ways to run a product: square, tall, or mixed (whole waves of tall tiles, the rest as a
 second launch in the square form).  Every element is accumulated over K in the same order in all of
 them, so the results must agree bit for bit; each is also checked against the CPU oracle."""
+import numpy as np
 import pytest
 import torch
 from helpers import assert_close, to_np
@@ -121,3 +122,32 @@ def test_operator_parity_tests_pass_with_the_form_forced_on_a_few_pairs(form, pa
     last = r.stdout.strip().splitlines()[-1]
     assert " passed" in last and "failed" not in last, tail
     assert int(last.split(" passed")[0].split()[-1]) >= 100, last
+
+
+@pytest.mark.parametrize("form", [sbp.SBP_TC_FORM_SQUARE, sbp.SBP_TC_FORM_TALL, sbp.SBP_TC_FORM_MIXED])
+def test_results_are_bit_stable_across_repeated_launches(form):
+    """The same product launched again and again gives the same bits: the ring, the hand-back of the
+    accumulators between the MMA thread and the epilogue warps and the walk of a mixed run leave no
+    room for an ordering that changes a result (a race here would show as an occasional difference).
+    Short contraction and many tiles, so that the hand-backs dominate."""
+    dev = torch.device("cuda")
+    M, K, N, k = 4096, 512, 8192, 4
+    X = dg.normal(3001, 0, (M, K), 0.0, 1.0, BF16, dev)
+    x = sbp.SbpTensor((M, K), BF16, sbp.B, [X] * k)
+    w = sbp.SbpTensor((K, N), BF16, sbp.S(1), [dg.normal(3001, 10 + r, (K, N // k), 0.0, 0.05, BF16, dev) for r in range(k)])
+    y = sbp.empty_global((M, N), BF16, sbp.S(1), k)
+    sbp.sbp_matmul_set_form(form, 0)
+    sbp.sbp_matmul(x, w, y)
+    torch.cuda.synchronize()
+    ref = [t.clone() for t in y.locals]
+    rows = [0, 255, 256, 2047, 4095]
+    want = O.matmul_logical(to_np(X[rows]), np.concatenate([to_np(t) for t in w.locals], axis=1))
+    got = np.concatenate([to_np(t[rows]) for t in ref], axis=1)
+    assert_close(got, want, 2e-2, 1e-3, "first launch")
+    for i in range(40):
+        for t in y.locals:
+            t.zero_()
+        sbp.sbp_matmul(x, w, y)
+        torch.cuda.synchronize()
+        assert all(torch.equal(a, b) for a, b in zip(ref, y.locals)), f"launch {i + 2} differs from the first"
+    sbp.sbp_check_device_errors()

@@ -307,3 +307,31 @@ def test_matmul_route_model_on_the_host():
                     else:
                         assert t % pairs == 0 and 0 < t < tall
     assert sbp.sbp_matmul_route(0, 4, 4)[0] == -1
+
+
+def test_host_path_byte_counts_on_the_host():
+    """What sbp_boxing_host[_multi] would copy is host arithmetic over the descriptors (pointers are
+    compared, never followed), so it can be pinned without a device."""
+    import torch
+    import paper_2110_15032_b200 as sbp
+    k, shape, bf16 = 4, (130, 250), torch.bfloat16
+    numel = shape[0] * shape[1]
+
+    def host(sig, alias=False):
+        if alias:
+            one = torch.empty(sbp.sbp_local_shape(shape, sig, k, 0, bf16), dtype=bf16)
+            return sbp.SbpTensor(shape, bf16, sig, [one] * k)
+        return sbp.SbpTensor(shape, bf16, sig, [torch.empty(sbp.sbp_local_shape(shape, sig, k, r, bf16), dtype=bf16) for r in range(k)])
+
+    p, b = host(sbp.P_SUM), host(sbp.B)
+    # one transform: all of every source local tensor, except B -> S(i): one block per replica
+    assert sbp.sbp_boxing_host_copy_bytes(p, host(sbp.B)) == (k * numel * 2, k * numel * 2)
+    assert sbp.sbp_boxing_host_copy_bytes(p, host(sbp.B, alias=True)) == (k * numel * 2, numel * 2)
+    assert sbp.sbp_boxing_host_copy_bytes(b, host(sbp.S(0))) == (numel * 2, numel * 2)
+    assert sbp.sbp_boxing_host_copy_bytes(b, host(sbp.S(1))) == (numel * 2, numel * 2)
+    assert sbp.sbp_boxing_host_copy_bytes(host(sbp.S(0)), host(sbp.S(1))) == (numel * 2, numel * 2)
+    # several destinations: the source once; the blocks only if every destination is an S of one axis
+    assert sbp.sbp_boxing_host_multi_copy_bytes(p, [host(sbp.B), host(sbp.S(0)), host(sbp.S(1))]) == (k * numel * 2, (k + 2) * numel * 2)
+    assert sbp.sbp_boxing_host_multi_copy_bytes(b, [host(sbp.S(1)), host(sbp.S(1))]) == (numel * 2, 2 * numel * 2)
+    assert sbp.sbp_boxing_host_multi_copy_bytes(b, [host(sbp.S(0)), host(sbp.S(1))]) == (k * numel * 2, 2 * numel * 2)
+    assert sbp.sbp_boxing_host_multi_workspace_bytes(p, [host(sbp.B), host(sbp.S(0))]) >= (2 * k + 1) * numel * 2
